@@ -1,0 +1,276 @@
+"""Pipelined Backpropagation, one tick at a time, on the CPU (test
+infrastructure; float64 unless another dtype is asked for).
+
+Follows Appendix "Pipelined Backpropagation": S stages, batch size one, each
+stage does one forward and one backward transformation per time step; a sample
+entering at tick i is forwarded by stage s at tick i+s, reaches the loss at
+tick i+S-1 and is back-propagated by stage s at tick i+2(S-1)-s, so it takes
+2S-1 steps and stage s sees D_s = 2(S-1-s) updates between its forward and
+its backward on the same sample (Eq. F_i: forward weights w^s_{i-2(S-1-s)}).
+The gradient is G(x_i; F_i, W_i): forward with the (predicted) weights of the
+forward tick, backward with the weights current at the backward tick.  Every
+stage is updated separately with its own delay (Section "Methods").
+
+The program is written per sample: everything a stage produces is stored
+under the key (stage, sample id), so a stage can only ever read what an
+earlier tick wrote for that sample.
+"""
+import numpy as np
+
+from . import layers as L
+from .optimizer import StageOptimizer
+
+# Operation codes of the layer list (the library's public enumeration).
+OP_FC, OP_CONV2D, OP_GROUPNORM, OP_RELU, OP_MAXPOOL, OP_AVGPOOL_GLOBAL, \
+    OP_ADD_SKIP, OP_SOFTMAX_CE = range(8)
+
+FLAG_SC, FLAG_LWP, FLAG_LWP_WFORM = 1, 2, 4
+
+
+class _Stage:
+    """One pipeline stage: FC or CONV2D head plus what rides with it."""
+
+    def __init__(self, index):
+        self.index = index
+        self.head = None          # the FC / CONV2D layer record
+        self.gn_groups = 0
+        self.skip = None          # (source stage, mode)
+        self.relu = False
+        self.maxpool = None       # (k, stride, pad)
+        self.avgpool = False
+        self.loss = False
+        self.src = -1             # stage whose output is the input (-1: network input)
+        self.in_shape = None
+        self.z_shape = None       # shape after head (+GN, skip, ReLU)
+        self.out_shape = None
+        self.n_params = 0
+
+    # parameter views into one flat vector, in layer order
+    def split(self, theta):
+        h = self.head
+        if h.op == OP_FC:
+            nw = h.c_in * h.c_out
+            return theta[:nw].reshape(h.c_out, h.c_in), theta[nw:nw + h.c_out], None, None
+        nw = h.c_out * h.c_in * h.k * h.k
+        W = theta[:nw].reshape(h.c_out, h.c_in, h.k, h.k)
+        if self.gn_groups:
+            return W, None, theta[nw:nw + h.c_out], theta[nw + h.c_out:nw + 2 * h.c_out]
+        return W, None, None, None
+
+    def forward(self, theta_hat, x, skip_in):
+        h = self.head
+        W, b, gamma, beta = self.split(theta_hat)
+        st = {"x": x}
+        if h.op == OP_FC:
+            n = L.fc_forward(W, b, x.ravel()).reshape(-1, 1, 1)
+        else:
+            n = L.conv2d_forward(W, x, h.stride, h.pad)
+            if self.gn_groups:
+                n, st["zhat"], st["rstd"] = L.groupnorm_forward(gamma, beta, n, self.gn_groups)
+        if self.skip is not None:
+            n = n + L.skip_forward(skip_in, self.skip[1], n.shape)
+        st["pre"] = n
+        a = L.relu_forward(n) if self.relu else n
+        if self.maxpool is not None:
+            a, st["arg"] = L.maxpool_forward(a, *self.maxpool)
+        if self.avgpool:
+            a = L.avgpool_forward(a)
+        return a, st
+
+    def backward(self, theta, st, dy, need_dx, skip_shape):
+        """Returns (g flat like theta, dx or None, dskip or None)."""
+        h = self.head
+        W, b, gamma, beta = self.split(theta)
+        pre = st["pre"]
+        d = dy.reshape(self.out_shape)
+        if self.avgpool:
+            d = L.avgpool_backward(d, pre.shape[1:])
+        if self.maxpool is not None:
+            d = L.maxpool_backward(st["arg"], d, pre.shape[1:])
+        if self.relu:
+            d = L.relu_backward(pre, d)
+        dskip = None
+        if self.skip is not None:
+            dskip = L.skip_backward(d, self.skip[1], skip_shape)
+        g = np.zeros_like(theta)
+        if h.op == OP_FC:
+            dx, gW, gb = L.fc_backward(W, st["x"].ravel(), d.ravel())
+            nw = gW.size
+            g[:nw] = gW.ravel()
+            g[nw:] = gb
+            dx = dx.reshape(st["x"].shape) if need_dx else None
+        else:
+            nw = W.size
+            if self.gn_groups:
+                d, gg, gbeta = L.groupnorm_backward(gamma, st["zhat"], st["rstd"], d, self.gn_groups)
+                g[nw:nw + h.c_out] = gg
+                g[nw + h.c_out:] = gbeta
+            dx, gW = L.conv2d_backward(W, st["x"], d, h.stride, h.pad)
+            g[:nw] = gW.ravel()
+            if not need_dx:
+                dx = None
+        return g, dx, dskip
+
+
+def build_stages(layer_list, stage_of_layer, in_shape):
+    """Group the layer list into stages and infer every shape."""
+    stages = []
+    for lay, s in zip(layer_list, stage_of_layer):
+        op = int(lay.op)
+        if op in (OP_FC, OP_CONV2D):
+            if s != len(stages):
+                raise ValueError("a stage must start with its FC/CONV2D layer")
+            st = _Stage(s)
+            st.head = lay
+            st.src = lay.src if lay.src >= 0 else s - 1
+            src_shape = tuple(in_shape) if st.src < 0 else stages[st.src].out_shape
+            st.in_shape = src_shape
+            if op == OP_FC:
+                if int(np.prod(src_shape)) != lay.c_in:
+                    raise ValueError("FC input size mismatch at stage %d" % s)
+                st.z_shape = (lay.c_out, 1, 1)
+                st.n_params = lay.c_in * lay.c_out + lay.c_out
+            else:
+                if src_shape[0] != lay.c_in:
+                    raise ValueError("conv channel mismatch at stage %d" % s)
+                oh = L.conv_out_size(src_shape[1], lay.k, lay.stride, lay.pad)
+                ow = L.conv_out_size(src_shape[2], lay.k, lay.stride, lay.pad)
+                st.z_shape = (lay.c_out, oh, ow)
+                st.n_params = lay.c_out * lay.c_in * lay.k * lay.k
+            st.out_shape = st.z_shape
+            stages.append(st)
+            continue
+        st = stages[s]
+        if op == OP_GROUPNORM:
+            st.gn_groups = lay.groups
+            st.n_params += 2 * st.head.c_out
+        elif op == OP_ADD_SKIP:
+            st.skip = (lay.src, lay.skip_mode)
+        elif op == OP_RELU:
+            st.relu = True
+        elif op == OP_MAXPOOL:
+            st.maxpool = (lay.k, lay.stride, lay.pad)
+            c, h, w = st.z_shape
+            st.out_shape = (c, L.conv_out_size(h, lay.k, lay.stride, lay.pad),
+                            L.conv_out_size(w, lay.k, lay.stride, lay.pad))
+        elif op == OP_AVGPOOL_GLOBAL:
+            st.avgpool = True
+            st.out_shape = (st.z_shape[0], 1, 1)
+        elif op == OP_SOFTMAX_CE:
+            st.loss = True
+        else:
+            raise ValueError("unknown op %d" % op)
+    return stages
+
+
+class PBOracle:
+    """PB + SC + LWP on a layer list; `tick` advances the pipeline one step."""
+
+    def __init__(self, layer_list, stage_of_layer, in_shape, n_classes, lr,
+                 momentum, flags=FLAG_SC | FLAG_LWP, dtype=np.float64,
+                 sc_delay_scale=1, horizon_scale=1, record=False):
+        self.dtype = dtype
+        self.stages = build_stages(layer_list, stage_of_layer, in_shape)
+        self.S = len(self.stages)
+        if not self.stages[-1].loss:
+            raise ValueError("the last stage must end in SOFTMAX_CE")
+        self.in_shape = tuple(in_shape)
+        self.lr, self.m, self.flags = lr, momentum, flags
+        self.sc_delay_scale, self.horizon_scale = sc_delay_scale, horizon_scale
+        self.n_params = sum(st.n_params for st in self.stages)
+        self.opt = None
+        self.t = 0
+        self.out, self.stash, self.dsum, self.labels = {}, {}, {}, {}
+        self.record = record
+        self.fwd_version, self.bwd_version, self.grads = {}, {}, {}
+        self.history = [[] for _ in self.stages]   # (w, v) after each version
+
+    def delay(self, s):
+        """D_s = 2 (S - 1 - s): updates between stage s's forward and backward."""
+        return 2 * (self.S - 1 - s)
+
+    def set_weights(self, flat):
+        flat = np.asarray(flat)
+        assert flat.size == self.n_params
+        self.opt, off = [], 0
+        for st in self.stages:
+            D = self.delay(st.index)
+            self.opt.append(StageOptimizer(
+                flat[off:off + st.n_params], self.lr, self.m, D,
+                use_sc=bool(self.flags & FLAG_SC), use_lwp=bool(self.flags & FLAG_LWP),
+                w_form=bool(self.flags & FLAG_LWP_WFORM),
+                sc_delay=self.sc_delay_scale * D, horizon=self.horizon_scale * D,
+                dtype=self.dtype))
+            off += st.n_params
+            if self.record:
+                self.history[st.index].append((self.opt[-1].w.copy(), self.opt[-1].v.copy()))
+
+    def get_weights(self):
+        return np.concatenate([o.w for o in self.opt])
+
+    def get_velocity(self):
+        return np.concatenate([o.v for o in self.opt])
+
+    def tick(self, x, label):
+        """One time step with new sample (x, label).  Returns the loss the
+        last stage computed this tick (sample t-(S-1)), NaN while filling."""
+        S, t = self.S, self.t
+        self.out[(-1, t)] = np.asarray(x, dtype=self.dtype).reshape(self.in_shape)
+        self.labels[t] = int(label)
+
+        # 1. predicted weights from the state left by the previous tick
+        theta_hat = [o.predicted() for o in self.opt]
+
+        # 2. forward of sample t-s at stage s
+        for st in self.stages:
+            s, i = st.index, t - st.index
+            if i < 0:
+                continue
+            skip_in = self.out[(st.skip[0], i)] if st.skip is not None else None
+            y, stash = st.forward(theta_hat[s], self.out[(st.src, i)], skip_in)
+            self.out[(s, i)], self.stash[(s, i)] = y, stash
+            if self.record:
+                self.fwd_version[(s, i)] = self.opt[s].version
+
+        # 3. loss and its gradient at the last stage (same tick: delay 0)
+        loss = float("nan")
+        i = t - (S - 1)
+        if i >= 0:
+            loss, delta = L.softmax_ce(self.out[(S - 1, i)].ravel(), self.labels.pop(i))
+            self.dsum[(S - 1, i)] = delta.reshape(-1, 1, 1)
+
+        # 4. backward of sample t-2(S-1)+s at stage s, with the current weights
+        grads = {}
+        for st in self.stages:
+            s, j = st.index, t - 2 * (S - 1) + st.index
+            if j < 0:
+                continue
+            dy = self.dsum.pop((s, j))
+            skip_shape = self.stages[st.skip[0]].out_shape if st.skip is not None else None
+            g, dx, dskip = st.backward(self.opt[s].w, self.stash.pop((s, j)), dy,
+                                       st.src >= 0, skip_shape)
+            if dx is not None:
+                self._accumulate((st.src, j), dx)
+            if dskip is not None:
+                self._accumulate((st.skip[0], j), dskip)
+            grads[s] = g
+            del self.out[(s, j)]
+            if s == 0:
+                del self.out[(-1, j)]
+            if self.record:
+                self.bwd_version[(s, j)] = self.opt[s].version
+                self.grads[(s, j)] = g.copy()
+
+        # 5. update every stage that received a gradient
+        for s, g in grads.items():
+            self.opt[s].update(g)
+            if self.record:
+                self.history[s].append((self.opt[s].w.copy(), self.opt[s].v.copy()))
+        self.t += 1
+        return loss
+
+    def _accumulate(self, key, d):
+        if key in self.dsum:
+            self.dsum[key] = self.dsum[key] + d
+        else:
+            self.dsum[key] = d
