@@ -1,0 +1,250 @@
+"""Throughput of Pipelined Backpropagation ticks (samples/s at batch 1).
+
+One step is one tick: every stage's forward and backward on its current
+samples plus the SC+LWP update of every stage.  Workload: the deep MLP
+(16 FC stages of width 2048), whose weights and velocities (504 MB) exceed
+the L2 cache, so every tick streams them from HBM.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+With N > 1 (under torch.distributed.run) each rank runs an independent replica
+of the pipeline on its own GPU: the tick has no data-parallel form at update
+size one, so the job scales by replicas and no collective is on the data path.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOAD = "mlp16x2048"
+METRIC = "PB ticks/sec (samples/sec, batch 1)"
+UNIT = "ticks/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f).get("hbm_gbs", 6650.0), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while timing."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def time_oracle(wl, budget_s=20.0, max_ticks=None):
+    """Times the CPU checker as it stands on steady-state ticks of `wl`."""
+    from oracle import PBOracle
+    from pb_workloads import he_normal_weights, make_inputs
+    S = wl.n_stages
+    fill = 2 * (S - 1)
+    o = PBOracle(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, wl.lr, wl.momentum, wl.flags & 7)
+    o.set_weights(he_normal_weights(wl.seed, wl))
+    cap = fill + (max_ticks if max_ticks else 64)
+    x, y = make_inputs(wl.seed, cap, wl.sample_elems, wl.n_classes)
+    with np.errstate(all="ignore"):
+        for t in range(fill):
+            o.tick(x[t], y[t])
+        n, w0, c0 = 0, time.perf_counter(), time.process_time()
+        while n < cap - fill and (n == 0 or time.perf_counter() - w0 < budget_s):
+            o.tick(x[fill + n], y[fill + n])
+            n += 1
+        wall, cpu = time.perf_counter() - w0, time.process_time() - c0
+    cores = max(1, int(round(cpu / wall)))
+    return {"value": n / wall, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d steady-state ticks (ticks %d..%d) of %s, numpy float64, %d host cores visible"
+                      % (n, fill, fill + n - 1, wl.name, os.cpu_count())}, wall / n
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    from pb_workloads import workload
+    wl = workload(WORKLOAD)
+    base, s_per_tick = time_oracle(wl, budget_s=25.0, max_ticks=max(1, min(args.steps, 16)))
+    line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * s_per_tick, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "stages": wl.n_stages, "note": "CPU checker on host cores"},
+            "cpu_baseline": base,
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4096)
+    ap.add_argument("--warmup", type=int, default=64)
+    ap.add_argument("--impl", default="b200")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2003_11666_b200 import build as pbuild
+    if local_rank == 0:
+        pbuild.build()
+    import paper_2003_11666_b200 as pbm
+    from pb_workloads import he_normal_weights, make_inputs, workload
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    wl = workload(WORKLOAD)
+    K, W = args.steps, max(args.warmup, 3)
+    S = wl.n_stages
+    seed = wl.seed + 1000 * rank            # replicas see different sample streams
+    x, y = make_inputs(seed, K + W, wl.sample_elems, wl.n_classes)
+    stream = torch.cuda.current_stream()
+    eng = pbm.PB(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, wl.lr, wl.momentum,
+                 wl.flags, stream=stream.cuda_stream)
+    eng.set_weights(he_normal_weights(wl.seed, wl))
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    losses = torch.zeros(K + W, device="cuda")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing: W warm-up ticks (fills the pipeline), then K ticks
+    eng.run(xd[:W], yd[:W], W, losses[:W])
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    eng.run(xd[W:], yd[W:], K, losses[W:])
+    e1.record(stream)
+    barrier()
+    launches = eng.last_launch_count
+    ms = max_over_ranks(e0.elapsed_time(e1))
+    clocks = sampler.stop() if rank == 0 else None
+    value = world * K / (ms * 1e-3)
+
+    # ---- per-kernel durations (CUDA events on the engine's stream, separate pass)
+    eng.profile_enable(True)
+    kp = min(K, 512)
+    eng.run(xd[W:W + kp], yd[W:W + kp], kp, losses[W:W + kp])
+    eng.sync()
+    k_ms, k_n = eng.profile_ms(0)
+    eng.profile_enable(False)
+    P = eng.num_params
+    p_last = wl.layers[-2].c_in * wl.layers[-2].c_out + wl.layers[-2].c_out
+    alg_bytes = 16.0 * (P - p_last)          # one read and one write of (w, v) per updated parameter
+    peak, peak_kind = measured_peaks()
+    achieved = alg_bytes / (k_ms / k_n * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "fc_tick_kernel(phase 0)", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_source": peak_kind,
+                "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": k_ms / k_n, "launches_timed": k_n}
+
+    # ---- end to end through the host-buffer entry point (pinned memory, copies timed)
+    eng.set_weights(he_normal_weights(wl.seed, wl))
+    hx = torch.from_numpy(x).pin_memory()
+    hy = torch.from_numpy(y).pin_memory()
+    hl = torch.zeros(K + W).pin_memory()
+    eng.run_host(hx[:W], hy[:W], W, hl[:W])
+    barrier()
+    t0 = time.perf_counter()
+    eng.run_host(hx[W:], hy[W:], K, hl[W:])
+    torch.cuda.synchronize()
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
+    e2e = {"value": world * K / (e2e_ms * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": wl.sample_elems * 4 + 4, "d2h_bytes_per_step": 4}
+    finite_ticks = int(np.isfinite(hl[W:].numpy()).sum())
+    eng.destroy()
+
+    if rank == 0:
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            cpu, _ = time_oracle(wl, budget_s=15.0, max_ticks=8)
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic",
+                "config": {"workload": WORKLOAD, "stages": S, "params": P, "batch": 1,
+                           "parallelism": "replicas x%d" % world if world > 1 else "1 gpu",
+                           "l2": "weights+velocity %.0f MB stream from HBM every tick (> 126 MB L2), no flush needed" % (8e-6 * P),
+                           "note": "literal lr 0.005 diverges (losses finite on %d of %d timed ticks); "
+                                   "kernel work does not depend on the values" % (finite_ticks, K)},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+                "roofline": roofline, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

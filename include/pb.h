@@ -1,0 +1,155 @@
+/*
+ * pb.h - C interface of the B200 Pipelined Backpropagation engine.
+ *
+ * One handle simulates fine-grained Pipelined Backpropagation (PB) at batch
+ * size one on a single GPU: the network is cut into S stages; at every tick
+ * each stage runs a forward on the sample that has reached it and a backward
+ * on the sample whose gradient has come back to it, then updates its own
+ * weights with SGD-momentum, Spike Compensation (SC) and Linear Weight
+ * Prediction (LWP), each with that stage's delay D_s = 2 (S - 1 - s)
+ * (paper: Appendix "Pipelined Backpropagation", Eqs. W_i / F_i; Section
+ * "Methods", SC_D coefficients, LWP velocity form, "Combined Mitigation").
+ *
+ * Conventions
+ *   - Every function returns PB_OK (0) or a negative pb_status; nothing throws
+ *     or aborts across this boundary.  pb_last_error() gives the text of the
+ *     last failure on a handle (or of pb_create when given NULL).
+ *   - "host" pointers are ordinary CPU memory, "dev" pointers are CUDA device
+ *     memory on the device that was current at pb_create.  The caller owns
+ *     every buffer it passes; the library owns all state behind the handle.
+ *   - All work is issued on the stream given to pb_create (a cudaStream_t cast
+ *     to void*, NULL = the default stream).  Calls taking host output
+ *     pointers synchronise that stream; the others do not.
+ *   - Tensors of one sample are [C, H, W], float32.  Parameters are one flat
+ *     float32 vector in layer-list order: FC -> weight [out, in] then bias
+ *     [out]; CONV2D -> weight [c_out, c_in, k, k]; GROUPNORM -> scale [c] then
+ *     shift [c].
+ */
+#ifndef PB_B200_H
+#define PB_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pb_handle pb_handle; /* opaque */
+
+typedef enum {
+    PB_OK = 0,
+    PB_E_ARG = -1,      /* NULL pointer, bad size, bad flag                     */
+    PB_E_SHAPE = -2,    /* layer list does not chain (channel/size mismatch)    */
+    PB_E_ALLOC = -3,    /* device or host allocation failed                     */
+    PB_E_CUDA = -4,     /* a CUDA call or kernel launch reported an error       */
+    PB_E_DEVICE = -5,   /* a kernel set the device error word (index check)     */
+    PB_E_UNSUPPORTED = -6
+} pb_status;
+
+/* Layer kinds.  A stage begins with PB_FC or PB_CONV2D (the layer that owns
+ * the weights); the others ride in the stage of the layer before them, in the
+ * order conv -> groupnorm -> add_skip -> relu -> maxpool | avgpool_global,
+ * or fc -> relu, or fc -> softmax_ce (last stage only).  Grouping convolution,
+ * normalisation and activation into one stage follows Section 2.1. */
+typedef enum {
+    PB_FC = 0, PB_CONV2D = 1, PB_GROUPNORM = 2, PB_RELU = 3, PB_MAXPOOL = 4,
+    PB_AVGPOOL_GLOBAL = 5, PB_ADD_SKIP = 6, PB_SOFTMAX_CE = 7
+} pb_op;
+
+typedef struct {
+    int32_t op;        /* pb_op                                                  */
+    int32_t c_in;      /* FC: flattened input size; CONV2D/GROUPNORM: channels   */
+    int32_t c_out;     /* FC: outputs; CONV2D: output channels                   */
+    int32_t k;         /* CONV2D / MAXPOOL window                                */
+    int32_t stride;    /* CONV2D / MAXPOOL                                       */
+    int32_t pad;       /* CONV2D / MAXPOOL                                       */
+    int32_t groups;    /* GROUPNORM                                              */
+    int32_t src;       /* FC/CONV2D: stage whose output is read (-1: the stage
+                          before, or the network input for stage 0);
+                          ADD_SKIP: stage whose output is added                  */
+    int32_t skip_mode; /* ADD_SKIP: 0 identity, 1 every second pixel + zero
+                          channels appended up to c_out                          */
+} pb_layer;
+
+/* Mitigation switches (Section "Methods").  PB_SC: a = m^D, b = (1-m^D)/(1-m),
+ * else a = 1, b = 0.  PB_LWP: forward weights w_hat = w - lr*T*v with T = D,
+ * else T = 0.  PB_CONV_BF16: convolutions multiply bf16 operands with fp32
+ * accumulation; master weights, velocity and everything else stay fp32. */
+enum { PB_SC = 1, PB_LWP = 2, PB_LWP_WFORM = 4, PB_CONV_BF16 = 8 };
+
+/* Builds the engine.  layers/stage_of_layer: host arrays of n_layers entries,
+ * stage indices non-decreasing from 0.  (in_c, in_h, in_w): shape of one
+ * sample.  The last stage must end in PB_SOFTMAX_CE over n_classes outputs.
+ * stream: cudaStream_t as void*.  All device memory is allocated here, once
+ * (weights, velocity, activation rings of D_s + 1 slots per stage, gradient
+ * hand-off buffers); ticks allocate nothing.  Weights start at zero: call
+ * pb_set_weights.  On failure *out is NULL. */
+int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_layer,
+              int in_c, int in_h, int in_w, int n_classes,
+              float lr, float momentum, unsigned flags, void* stream,
+              pb_handle** out);
+
+/* Copies n = pb_num_params() floats from host memory into the master weights,
+ * zeroes the velocity and restarts the pipeline at tick 0. */
+int pb_set_weights(pb_handle* h, const float* host_w, size_t n);
+
+/* One tick.  dev_x: the new sample (in_c*in_h*in_w floats, device memory; it
+ * is copied into the engine's input ring, so it may be reused after the call
+ * returns in stream order).  label in [0, n_classes).  If host_loss is not
+ * NULL the stream is synchronised and *host_loss receives the loss the last
+ * stage computed in this tick, which belongs to the sample fed S-1 ticks
+ * earlier (a sample needs 2S-1 steps, Appendix "Pipelined Backpropagation");
+ * it is NaN during the first S-1 ticks. */
+int pb_tick(pb_handle* h, const float* dev_x, int label, float* host_loss);
+
+/* n_ticks ticks without host synchronisation.  dev_xs: [n_ticks, sample]
+ * floats, dev_labels: [n_ticks] int32, both device memory that must stay
+ * valid and unchanged until the stream has run the ticks AND for the next
+ * 2(S-1) ticks' worth of calls (stage 0 re-reads a sample at its backward);
+ * dev_losses: [n_ticks] floats (device) or NULL.  Continues from the current
+ * tick; may be called repeatedly with consecutive batches only if the earlier
+ * batches stay alive as stated. */
+int pb_run(pb_handle* h, const float* dev_xs, const int32_t* dev_labels,
+           int n_ticks, float* dev_losses);
+
+/* Same as pb_run but every pointer is host memory: the call copies the inputs
+ * to the device, runs the ticks, copies the losses back and synchronises. */
+int pb_run_host(pb_handle* h, const float* host_xs, const int32_t* host_labels,
+                int n_ticks, float* host_losses);
+
+/* Master weights / velocities to host memory (n must equal pb_num_params);
+ * synchronises the stream. */
+int pb_get_weights(pb_handle* h, float* host_w, size_t n);
+int pb_get_velocity(pb_handle* h, float* host_v, size_t n);
+
+/* Waits for the stream and reports a set device error word as PB_E_DEVICE. */
+int pb_sync(pb_handle* h);
+
+size_t pb_num_params(const pb_handle* h);
+int pb_num_stages(const pb_handle* h);
+/* D_s = 2 (S - 1 - s); negative status for a bad stage index. */
+int pb_stage_delay(const pb_handle* h, int s);
+/* Ticks run since the last pb_set_weights. */
+long long pb_tick_count(const pb_handle* h);
+/* Kernel launches issued by the last pb_tick/pb_run/pb_run_host call. */
+long long pb_last_launch_count(const pb_handle* h);
+/* Bytes of device memory the handle holds. */
+size_t pb_device_bytes(const pb_handle* h);
+
+/* Timing hooks for benchmarks: device time in milliseconds that the kernel
+ * class `which` (0 = FC tick kernel, 1 = last-stage loss/backward kernel,
+ * 2 = update kernel, 3 = conv kernels) took over the last pb_run, measured
+ * with CUDA events on the engine's stream when enabled (enable != 0 costs a
+ * pair of event records per launch).  Returns a negative value when disabled
+ * or never run; *launches receives the number of launches timed. */
+int pb_profile_enable(pb_handle* h, int enable);
+double pb_profile_ms(pb_handle* h, int which, long long* launches);
+
+const char* pb_last_error(const pb_handle* h);
+void pb_destroy(pb_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PB_B200_H */

@@ -184,6 +184,7 @@ class PBOracle:
         self.record = record
         self.fwd_version, self.bwd_version, self.grads = {}, {}, {}
         self.history = [[] for _ in self.stages]   # (w, v) after each version
+        self.last_logits = None   # logits behind the most recent loss (for error scaling in tests)
 
     def delay(self, s):
         """D_s = 2 (S - 1 - s): updates between stage s's forward and backward."""
@@ -236,6 +237,7 @@ class PBOracle:
         loss = float("nan")
         i = t - (S - 1)
         if i >= 0:
+            self.last_logits = self.out[(S - 1, i)].ravel().copy()
             loss, delta = L.softmax_ce(self.out[(S - 1, i)].ravel(), self.labels.pop(i))
             self.dsum[(S - 1, i)] = delta.reshape(-1, 1, 1)
 

@@ -1,0 +1,325 @@
+// Fully connected stages of a Pipelined Backpropagation tick.
+//
+// For an FC stage everything a tick needs from the weights can be served by
+// ONE pass over (w, v): the forward of the sample that has just arrived uses
+// the predicted weights w_hat = w - lr*T*v (LWP, velocity form), the backward
+// of the sample whose gradient has come back uses w itself, and the update
+// v <- m v + g, w <- w - lr (a v + b g) (combined SC + LWP step) needs only the
+// rank-1 gradient g = delta x^T, which is formed on the fly.  So the kernel
+// reads w and v once, writes them once (16 bytes per parameter) and never
+// materialises w_hat or g.
+//
+// Work split: a thread block owns a band of rows [row0, row1) of one stage.
+// Each warp owns a set of 128-column chunks ("column group") and a subset of
+// the band's rows ("row split").  Row sums (the forward GEMV) are reduced with
+// warp shuffles and a small shared-memory table; column sums (the data
+// gradient W^T delta) stay in registers across the band and leave as one
+// partial row per band that the consumer adds up in a fixed order, so results
+// do not depend on scheduling.
+#pragma once
+#include "pb_internal.h"
+
+namespace pb {
+
+template <int VEC> struct VecT;
+template <> struct VecT<4> { using type = float4; };
+template <> struct VecT<1> { using type = float; };
+
+template <int VEC> __device__ __forceinline__ void vload(float (&r)[VEC], const float* p);
+template <> __device__ __forceinline__ void vload<4>(float (&r)[4], const float* p) {
+    float4 q = *reinterpret_cast<const float4*>(p);
+    r[0] = q.x; r[1] = q.y; r[2] = q.z; r[3] = q.w;
+}
+template <> __device__ __forceinline__ void vload<1>(float (&r)[1], const float* p) { r[0] = *p; }
+
+// streaming load: the weights are touched once per tick
+template <int VEC> __device__ __forceinline__ void vload_stream(float (&r)[VEC], const float* p);
+template <> __device__ __forceinline__ void vload_stream<4>(float (&r)[4], const float* p) {
+    float4 q = __ldcs(reinterpret_cast<const float4*>(p));
+    r[0] = q.x; r[1] = q.y; r[2] = q.z; r[3] = q.w;
+}
+template <> __device__ __forceinline__ void vload_stream<1>(float (&r)[1], const float* p) { r[0] = __ldcs(p); }
+
+template <int VEC> __device__ __forceinline__ void vstore(float* p, const float (&r)[VEC]);
+template <> __device__ __forceinline__ void vstore<4>(float* p, const float (&r)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(r[0], r[1], r[2], r[3]);
+}
+template <> __device__ __forceinline__ void vstore<1>(float* p, const float (&r)[1]) { *p = r[0]; }
+
+__device__ __forceinline__ int ring_slot(long long sample, int slots) {
+    return (int)(sample % slots);
+}
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// Sum of four per-lane values over the warp with 6 shuffles instead of 20:
+// after the exchange steps lane l holds the total of value (l>>3)&3... every
+// lane ends with the total of value q = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1).
+__device__ __forceinline__ float warp_sum4(float a0, float a1, float a2, float a3, int lane) {
+    const bool hi16 = lane & 16;
+    float keep0 = hi16 ? a2 : a0, send0 = hi16 ? a0 : a2;
+    float keep1 = hi16 ? a3 : a1, send1 = hi16 ? a1 : a3;
+    keep0 += __shfl_xor_sync(0xffffffffu, send0, 16);
+    keep1 += __shfl_xor_sync(0xffffffffu, send1, 16);
+    const bool hi8 = lane & 8;
+    float keep = hi8 ? keep1 : keep0, send = hi8 ? keep0 : keep1;
+    keep += __shfl_xor_sync(0xffffffffu, send, 8);
+    keep += __shfl_xor_sync(0xffffffffu, keep, 4);
+    keep += __shfl_xor_sync(0xffffffffu, keep, 2);
+    keep += __shfl_xor_sync(0xffffffffu, keep, 1);
+    return keep;
+}
+
+struct FcShared {
+    float rowpart[kFcWarps][kFcMaxSegRows];               // forward partial sums per column group
+    float delta[kFcMaxSegRows];                           // gradient w.r.t. the band's pre-activations
+    float colpart[kFcWarps][kFcChunksPerSweep * 128];     // column partials across row splits
+    float red[kFcWarps];
+    int redi[kFcWarps];
+    float bcast[2];
+};
+
+// Gradient of the loss w.r.t. the pre-activation of row `r` for the backward
+// sample: sum of the consumers' partial rows, gated by the ReLU that followed.
+__device__ __forceinline__ float gather_delta(const FcStage& st, int r, long long j) {
+    float d = 0.f;
+    for (int q = 0; q < st.n_dsrc; ++q) {
+        const DeltaSrc& ds = st.dsrc[q];
+        const float* p = ds.ptr + ((size_t)ring_slot(j, ds.slots) * ds.nparts) * st.out_dim + r;
+        for (int k = 0; k < ds.nparts; ++k) d += p[(size_t)k * st.out_dim];
+    }
+    if (st.relu) {
+        const float y = st.out[(size_t)ring_slot(j, st.out_slots) * st.out_dim + r];
+        d = y > 0.f ? d : 0.f;
+    }
+    return d;
+}
+
+// phase 0: every stage's forward, and backward + update of every stage but the
+//          last (whose gradient only exists once its own forward is done);
+// phase 1: the last stage's loss, backward and update.
+template <int VEC>
+__device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int S, int phase,
+                           const int* __restrict__ label_ring, float* __restrict__ loss_out,
+                           FcShared& sh, TickState* ts) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long i = t - st.s;                        // forward sample
+    const long long j = t - 2LL * (S - 1) + st.s;        // backward sample
+    const bool do_fwd = phase == 0 && i >= 0;
+    const bool do_bwd = j >= 0 && (st.is_last ? phase == 1 : phase == 0);
+    if (phase == 1 && seg.row0 == 0 && tid == 0 && j < 0 && loss_out) *loss_out = __int_as_float(0x7fc00000);
+    if (!do_fwd && !do_bwd) return;
+    const int rows = seg.row1 - seg.row0;
+    if (rows > kFcMaxSegRows || rows <= 0) {
+        if (tid == 0) { ts->error = kErrSegRows; ts->error_info = seg.stage; }
+        return;
+    }
+    const int in = st.in_dim, out = st.out_dim;
+    const float* __restrict__ xf = st.xin + (size_t)ring_slot(i < 0 ? 0 : i, st.xin_slots) * in;
+    const float* __restrict__ xb = st.xin + (size_t)ring_slot(j < 0 ? 0 : j, st.xin_slots) * in;
+
+    // ---- gradient w.r.t. this band's pre-activations
+    __syncthreads();   // shared memory may still be in use by the previous segment
+    if (do_bwd) {
+        if (st.is_last) {
+            // softmax over all logits (every block repeats it; n_classes is small).
+            // The term of the first maximum (exp(0) = 1) is kept out of the sum so
+            // that a confident prediction's loss, log1p(rest), keeps its digits.
+            const float* lg = st.out + (size_t)ring_slot(j, st.out_slots) * out;
+            float mx = -INFINITY;
+            int amx = 0x7fffffff;
+            for (int k = tid; k < out; k += kFcThreads) {
+                const float x = lg[k];
+                if (x > mx) { mx = x; amx = k; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float om = __shfl_xor_sync(0xffffffffu, mx, o);
+                const int oa = __shfl_xor_sync(0xffffffffu, amx, o);
+                if (om > mx || (om == mx && oa < amx)) { mx = om; amx = oa; }
+            }
+            if (lane == 0) { sh.red[warp] = mx; sh.redi[warp] = amx; }
+            __syncthreads();
+            mx = sh.red[0]; amx = sh.redi[0];
+            for (int k = 1; k < kFcWarps; ++k)
+                if (sh.red[k] > mx || (sh.red[k] == mx && sh.redi[k] < amx)) { mx = sh.red[k]; amx = sh.redi[k]; }
+            __syncthreads();
+            float rest = 0.f;
+            for (int k = tid; k < out; k += kFcThreads) rest += (k == amx) ? 0.f : expf(lg[k] - mx);
+            rest = warp_sum(rest);
+            if (lane == 0) sh.red[warp] = rest;
+            __syncthreads();
+            rest = 0.f;
+            for (int k = 0; k < kFcWarps; ++k) rest += sh.red[k];
+            const float sum = 1.f + rest;
+            int label = label_ring[ring_slot(j, S)];
+            if (label < 0 || label >= out) {
+                if (tid == 0) { ts->error = kErrLabel; ts->error_info = label; }
+                label = 0;
+            }
+            if (seg.row0 == 0 && tid == 0 && loss_out) *loss_out = log1pf(rest) - (lg[label] - mx);
+            const float inv = 1.f / sum;
+            for (int r = tid; r < rows; r += kFcThreads) {
+                const int row = seg.row0 + r;
+                sh.delta[r] = expf(lg[row] - mx) * inv - (row == label ? 1.f : 0.f);
+            }
+        } else {
+            for (int r = tid; r < rows; r += kFcThreads) sh.delta[r] = gather_delta(st, seg.row0 + r, j);
+        }
+    }
+    __syncthreads();
+
+    // ---- warp roles
+    constexpr int CW = 32 * VEC;                          // columns per chunk
+    const int nchunks = ceil_div(in, CW);
+    int ncg = 1;
+    while (ncg * 2 <= nchunks && ncg * 2 <= kFcWarps) ncg *= 2;
+    const int nrs = kFcWarps / ncg;
+    const int cg = warp % ncg, rs = warp / ncg;
+    const float nlT = st.neg_lr_T, m = st.m, nla = st.neg_lr_a, nlb = st.neg_lr_b;
+    const bool want_dx = do_bwd && st.need_dx;
+
+    for (int c0 = 0; c0 < nchunks; c0 += ncg * kFcChunksPerSweep) {
+        int col[kFcChunksPerSweep];
+        bool cok[kFcChunksPerSweep];
+        float xfr[kFcChunksPerSweep][VEC], xbr[kFcChunksPerSweep][VEC], cacc[kFcChunksPerSweep][VEC];
+#pragma unroll
+        for (int c = 0; c < kFcChunksPerSweep; ++c) {
+            col[c] = (c0 + cg + c * ncg) * CW + lane * VEC;
+            cok[c] = col[c] < in;            // in % VEC == 0, so a vector is all in or all out
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) { xfr[c][e] = 0.f; xbr[c][e] = 0.f; cacc[c][e] = 0.f; }
+            if (cok[c]) {
+                if (do_fwd) vload<VEC>(xfr[c], xf + col[c]);
+                if (do_bwd) vload<VEC>(xbr[c], xb + col[c]);
+            }
+        }
+        // rows of this row split, four at a time
+        for (int r0 = rs * 4; r0 < rows; r0 += nrs * 4) {
+            float wv[4][kFcChunksPerSweep][VEC], vv[4][kFcChunksPerSweep][VEC];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int r = r0 + u;
+#pragma unroll
+                for (int c = 0; c < kFcChunksPerSweep; ++c) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) { wv[u][c][e] = 0.f; vv[u][c][e] = 0.f; }
+                    if (r < rows && cok[c]) {
+                        const size_t off = (size_t)(seg.row0 + r) * in + col[c];
+                        vload_stream<VEC>(wv[u][c], st.w + off);
+                        if (do_bwd) vload_stream<VEC>(vv[u][c], st.v + off);
+                    }
+                }
+            }
+            float facc[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int r = r0 + u;
+                facc[u] = 0.f;
+                const float d = (do_bwd && r < rows) ? sh.delta[r] : 0.f;
+#pragma unroll
+                for (int c = 0; c < kFcChunksPerSweep; ++c) {
+                    float wn[VEC], vn[VEC];
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) {
+                        const float w = wv[u][c][e], v = vv[u][c][e];
+                        const float what = fmaf(nlT, v, w);          // w_hat = w - lr T v
+                        facc[u] = fmaf(what, xfr[c][e], facc[u]);     // forward  (W_hat x)
+                        cacc[c][e] = fmaf(w, d, cacc[c][e]);          // backward (W^T delta)
+                        const float g = d * xbr[c][e];                // rank-1 gradient
+                        vn[e] = fmaf(m, v, g);                        // v <- m v + g
+                        wn[e] = fmaf(nla, vn[e], fmaf(nlb, g, w));    // w <- w - lr (a v + b g)
+                    }
+                    if (do_bwd && r < rows && cok[c]) {
+                        const size_t off = (size_t)(seg.row0 + r) * in + col[c];
+                        vstore<VEC>(st.w + off, wn);
+                        vstore<VEC>(st.v + off, vn);
+                    }
+                }
+            }
+            if (do_fwd) {
+                const float tot = warp_sum4(facc[0], facc[1], facc[2], facc[3], lane);
+                const int q = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
+                if ((lane & 7) == 0 && r0 + q < rows) {
+                    float* slot = &sh.rowpart[cg][r0 + q];
+                    *slot = (c0 == 0 ? 0.f : *slot) + tot;
+                }
+            }
+        }
+        // column partials: combine the row splits in a fixed order, then store
+        if (want_dx) {
+            if (nrs > 1) {
+#pragma unroll
+                for (int c = 0; c < kFcChunksPerSweep; ++c)
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) sh.colpart[warp][c * 128 + lane * VEC + e] = cacc[c][e];
+                __syncthreads();
+                if (rs == 0) {
+#pragma unroll
+                    for (int c = 0; c < kFcChunksPerSweep; ++c)
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) {
+                            float a = cacc[c][e];
+                            for (int k = 1; k < nrs; ++k) a += sh.colpart[k * ncg + cg][c * 128 + lane * VEC + e];
+                            cacc[c][e] = a;
+                        }
+                }
+                __syncthreads();
+            }
+            if (rs == 0) {
+                float* dst = st.dx + ((size_t)ring_slot(j, st.dx_slots) * st.dx_nparts + seg.part) * in;
+#pragma unroll
+                for (int c = 0; c < kFcChunksPerSweep; ++c)
+                    if (cok[c]) vstore<VEC>(dst + col[c], cacc[c]);
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- finish rows: bias, activation, bias update
+    float* bias = st.w + (size_t)out * in;
+    float* vbias = st.v + (size_t)out * in;
+    for (int r = tid; r < rows; r += kFcThreads) {
+        const int row = seg.row0 + r;
+        const float b = bias[row];
+        const float vb = do_bwd ? vbias[row] : 0.f;
+        if (do_fwd) {
+            float y = 0.f;
+            for (int k = 0; k < ncg; ++k) y += sh.rowpart[k][r];
+            y += fmaf(nlT, vb, b);
+            if (st.relu) y = fmaxf(y, 0.f);
+            st.out[(size_t)ring_slot(i, st.out_slots) * out + row] = y;
+        }
+        if (do_bwd) {
+            const float g = sh.delta[r];
+            const float vn = fmaf(m, vb, g);
+            vbias[row] = vn;
+            bias[row] = fmaf(nla, vn, fmaf(nlb, g, b));
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kFcThreads, 2)
+fc_tick_kernel(const FcStage* __restrict__ stages, const FcSeg* __restrict__ segs,
+               const int* __restrict__ cta_seg_begin, TickState* ts, int S, int phase,
+               const int* __restrict__ label_ring, float* __restrict__ losses, long long t_base) {
+    __shared__ FcShared sh;
+    const long long t = ts->tick;
+    float* loss_out = losses ? losses + (t - t_base) : nullptr;
+    for (int q = cta_seg_begin[blockIdx.x]; q < cta_seg_begin[blockIdx.x + 1]; ++q) {
+        const FcSeg seg = segs[q];
+        const FcStage& st = stages[seg.stage];
+        if (st.vec == 4) fc_segment<4>(st, seg, t, S, phase, label_ring, loss_out, sh, ts);
+        else fc_segment<1>(st, seg, t, S, phase, label_ring, loss_out, sh, ts);
+    }
+    // the last kernel of a tick publishes the next tick number
+    if (phase == 1 && blockIdx.x == 0 && threadIdx.x == 0) {
+        ts->next = t + 1;
+    }
+}
+
+}  // namespace pb

@@ -1,0 +1,484 @@
+// C interface of the Pipelined Backpropagation engine: layer-list parsing,
+// stage schedule constants, device memory layout and the per-tick launches.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "fc_kernels.cuh"
+#include "pb_engine.h"
+
+using namespace pb;
+
+namespace {
+
+std::string g_create_error;
+
+int fail(pb_handle* h, int code, const std::string& msg) {
+    if (h) h->err = msg; else g_create_error = msg;
+    return code;
+}
+
+#define PB_CUDA(h, call)                                                              \
+    do {                                                                              \
+        cudaError_t e_ = (call);                                                      \
+        if (e_ != cudaSuccess)                                                        \
+            return fail(h, PB_E_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); \
+    } while (0)
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int conv_out(int n, int k, int stride, int pad) { return (n + 2 * pad - k) / stride + 1; }
+
+// ---------------------------------------------------------------- parsing
+int parse_layers(pb_handle* h, const pb_layer* layers, int n_layers, const int32_t* stage_of) {
+    std::vector<StageHost>& st = h->stages;
+    size_t user_off = 0;
+    for (int q = 0; q < n_layers; ++q) {
+        const pb_layer& L = layers[q];
+        const int s = stage_of[q];
+        if (L.op == PB_FC || L.op == PB_CONV2D) {
+            if (s != (int)st.size()) return fail(nullptr, PB_E_ARG, "a stage must start with its FC/CONV2D layer and stages must be numbered 0,1,2,...");
+            StageHost x;
+            x.index = s;
+            x.head_op = L.op;
+            x.head = L;
+            x.src = L.src >= 0 ? L.src : s - 1;
+            if (x.src >= s) return fail(nullptr, PB_E_ARG, "a stage may only read an earlier stage");
+            x.in = x.src < 0 ? h->in_shape : st[x.src].out;
+            if (L.op == PB_FC) {
+                if (L.c_in <= 0 || L.c_out <= 0 || x.in.elems() != L.c_in)
+                    return fail(nullptr, PB_E_SHAPE, "FC input size does not match its source at stage " + std::to_string(s));
+                x.z = Shape{L.c_out, 1, 1};
+                x.n_params = (size_t)L.c_in * L.c_out + L.c_out;
+            } else {
+                if (L.c_in <= 0 || L.c_out <= 0 || L.k <= 0 || L.stride <= 0 || L.pad < 0 || x.in.c != L.c_in)
+                    return fail(nullptr, PB_E_SHAPE, "CONV2D channels do not match its source at stage " + std::to_string(s));
+                x.z = Shape{L.c_out, conv_out(x.in.h, L.k, L.stride, L.pad), conv_out(x.in.w, L.k, L.stride, L.pad)};
+                if (x.z.h <= 0 || x.z.w <= 0) return fail(nullptr, PB_E_SHAPE, "CONV2D output is empty");
+                x.n_params = (size_t)L.c_out * L.c_in * L.k * L.k;
+            }
+            x.out = x.z;
+            x.user_off = user_off;
+            st.push_back(x);
+            user_off += x.n_params;
+            continue;
+        }
+        if (st.empty() || s != (int)st.size() - 1) return fail(nullptr, PB_E_ARG, "layer " + std::to_string(q) + " does not follow the head of its stage");
+        StageHost& x = st.back();
+        switch (L.op) {
+            case PB_GROUPNORM:
+                if (x.head_op != PB_CONV2D || L.groups <= 0 || x.z.c % L.groups) return fail(nullptr, PB_E_SHAPE, "bad GROUPNORM");
+                x.gn_groups = L.groups;
+                x.n_params += 2 * (size_t)x.z.c;
+                user_off += 2 * (size_t)x.z.c;
+                break;
+            case PB_ADD_SKIP:
+                if (L.src < 0 || L.src >= s) return fail(nullptr, PB_E_ARG, "ADD_SKIP needs an earlier stage");
+                x.has_skip = true; x.skip_src = L.src; x.skip_mode = L.skip_mode;
+                {
+                    const Shape& sk = st[L.src].out;
+                    bool ok = L.skip_mode == 0 ? (sk.c == x.z.c && sk.h == x.z.h && sk.w == x.z.w)
+                                               : (sk.c <= x.z.c && (sk.h + 1) / 2 == x.z.h && (sk.w + 1) / 2 == x.z.w);
+                    if (!ok) return fail(nullptr, PB_E_SHAPE, "ADD_SKIP shapes do not match at stage " + std::to_string(s));
+                }
+                break;
+            case PB_RELU: x.relu = true; break;
+            case PB_MAXPOOL:
+                if (L.k <= 0 || L.stride <= 0 || L.pad < 0 || 2 * L.pad > L.k) return fail(nullptr, PB_E_ARG, "bad MAXPOOL");
+                x.has_pool = true; x.pool_k = L.k; x.pool_stride = L.stride; x.pool_pad = L.pad;
+                x.out = Shape{x.z.c, conv_out(x.z.h, L.k, L.stride, L.pad), conv_out(x.z.w, L.k, L.stride, L.pad)};
+                break;
+            case PB_AVGPOOL_GLOBAL: x.avgpool = true; x.out = Shape{x.z.c, 1, 1}; break;
+            case PB_SOFTMAX_CE: x.loss = true; break;
+            default: return fail(nullptr, PB_E_ARG, "unknown op");
+        }
+    }
+    if (st.empty()) return fail(nullptr, PB_E_ARG, "empty layer list");
+    if (!st.back().loss || st.back().head_op != PB_FC || st.back().relu)
+        return fail(nullptr, PB_E_ARG, "the last stage must be FC + SOFTMAX_CE");
+    if (st.back().out.elems() != h->n_classes) return fail(nullptr, PB_E_SHAPE, "n_classes does not match the last FC");
+    for (size_t s = 0; s + 1 < st.size(); ++s)
+        if (st[s].loss) return fail(nullptr, PB_E_ARG, "SOFTMAX_CE before the last stage");
+    h->S = (int)st.size();
+    h->n_params = user_off;
+    return PB_OK;
+}
+
+// Per-stage constants: delay (Eq. F_i), SC_D coefficients, LWP horizon.
+void schedule_constants(pb_handle* h) {
+    const int S = h->S;
+    const double m = h->momentum;
+    size_t dev_off = 0;
+    h->all_fc = true;
+    for (StageHost& x : h->stages) {
+        x.delay = 2 * (S - 1 - x.index);
+        double a = 1.0, b = 0.0;
+        if (h->flags & PB_SC) {
+            a = std::pow(m, (double)x.delay);
+            b = (m == 1.0) ? (double)x.delay : (1.0 - a) / (1.0 - m);
+        }
+        x.a = (float)a; x.b = (float)b;
+        x.T = (h->flags & PB_LWP) ? (float)x.delay : 0.f;
+        x.dev_off = dev_off;
+        dev_off += align_up(x.n_params, 64);
+        if (x.head_op != PB_FC) h->all_fc = false;
+        if (x.src >= 0) h->stages[x.src].consumers_main.push_back(x.index);
+        if (x.has_skip) h->stages[x.skip_src].consumers_skip.push_back(x.index);
+    }
+    h->dev_params = dev_off;
+}
+
+// Split FC stages into row bands, one or more per thread block, of about equal bytes.
+void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSeg>& segs,
+                  std::vector<int>& cta_begin, std::vector<int>& nparts) {
+    double total = 0;
+    for (int f : fc_ids) total += (double)h->h_fc[f].out_dim * h->h_fc[f].in_dim * 8.0;
+    const double target = 2.0 * h->num_sms;
+    double budget = total / target;
+    if (budget < 48.0 * 1024) budget = 48.0 * 1024;
+    segs.clear(); cta_begin.clear();
+    cta_begin.push_back(0);
+    double rem = budget;
+    for (int f : fc_ids) {
+        const FcStage& st = h->h_fc[f];
+        const double row_bytes = st.in_dim * 8.0;
+        int r = 0, part = 0;
+        while (r < st.out_dim) {
+            int n = (int)(rem / row_bytes);
+            if (n < 1) n = 1;
+            if (n > kFcMaxSegRows) n = kFcMaxSegRows;
+            if (n > st.out_dim - r) n = st.out_dim - r;
+            segs.push_back(FcSeg{f, r, r + n, part++});
+            r += n;
+            rem -= n * row_bytes;
+            if (rem < row_bytes * 0.5) { cta_begin.push_back((int)segs.size()); rem = budget; }
+        }
+        nparts[f] = part;
+    }
+    if (cta_begin.back() != (int)segs.size()) cta_begin.push_back((int)segs.size());
+}
+
+__global__ void ingest_kernel(TickState* ts, const float* __restrict__ xs, const int* __restrict__ labels,
+                              int label_value, float* __restrict__ in_ring, int in_slots, int elems,
+                              int* __restrict__ label_ring, int S, long long t_base) {
+    const long long t = ts->next;
+    const float* src = xs + (size_t)(t - t_base) * elems;
+    float* dst = in_ring + (size_t)(t % in_slots) * elems;
+    for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < elems; k += gridDim.x * blockDim.x) dst[k] = src[k];
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        label_ring[t % S] = labels ? labels[t - t_base] : label_value;
+        ts->tick = t;
+    }
+}
+
+// ---------------------------------------------------------------- memory layout
+struct Carver {
+    char* base; size_t off = 0;
+    template <class T> T* take(size_t n) {
+        T* p = reinterpret_cast<T*>(base + off);
+        off += align_up(n * sizeof(T), 256);
+        return p;
+    }
+};
+
+size_t layout(pb_handle* h, char* base, size_t* zero_from) {
+    Carver c{base};
+    h->d_ts = c.take<TickState>(1);
+    h->d_fc = c.take<FcStage>(h->h_fc.size() + 1);
+    h->d_segA = c.take<FcSeg>(h->h_segA.size() + 1);
+    h->d_segB = c.take<FcSeg>(h->h_segB.size() + 1);
+    h->d_ctaA = c.take<int>(h->h_ctaA.size() + 1);
+    h->d_ctaB = c.take<int>(h->h_ctaB.size() + 1);
+    h->d_w = c.take<float>(h->dev_params);
+    *zero_from = c.off;
+    h->d_v = c.take<float>(h->dev_params);
+    h->in_slots = 2 * (h->S - 1) + 1;
+    h->in_ring = c.take<float>((size_t)h->in_slots * h->in_shape.elems());
+    h->label_ring = c.take<int>(h->S);
+    h->d_loss1 = c.take<float>(1);
+    for (StageHost& x : h->stages) {
+        x.out_slots = x.delay + 1;
+        x.out_ring = c.take<float>((size_t)x.out_slots * x.out.elems());
+        if (x.src >= 0) {
+            x.dx_slots = x.index - x.src + 1;
+            x.dx = c.take<float>((size_t)x.dx_slots * x.dx_nparts * x.in.elems());
+        }
+        if (x.has_skip) {
+            x.dskip_slots = x.index - x.skip_src + 1;
+            x.dskip = c.take<float>((size_t)x.dskip_slots * h->stages[x.skip_src].out.elems());
+        }
+    }
+    return c.off;
+}
+
+void fill_fc_tables(pb_handle* h) {
+    for (FcStage& f : h->h_fc) {
+        const StageHost& x = h->stages[f.s];
+        f.w = h->d_w + x.dev_off;
+        f.v = h->d_v + x.dev_off;
+        if (x.src < 0) { f.xin = h->in_ring; f.xin_slots = h->in_slots; }
+        else { f.xin = h->stages[x.src].out_ring; f.xin_slots = h->stages[x.src].out_slots; }
+        f.out = x.out_ring; f.out_slots = x.out_slots;
+        f.dx = x.dx; f.dx_slots = x.dx_slots; f.dx_nparts = x.dx_nparts;
+        f.n_dsrc = 0;
+        for (int c : x.consumers_main) {
+            const StageHost& y = h->stages[c];
+            f.dsrc[f.n_dsrc++] = DeltaSrc{y.dx, y.dx_slots, y.dx_nparts};
+        }
+        for (int c : x.consumers_skip) {
+            const StageHost& y = h->stages[c];
+            f.dsrc[f.n_dsrc++] = DeltaSrc{y.dskip, y.dskip_slots, 1};
+        }
+    }
+}
+
+// ---------------------------------------------------------------- profiling helpers
+void prof_begin(pb_handle* h, int cls) {
+    if (!h->profile) return;
+    if (h->ev_used + 2 > h->ev_pool.size()) {
+        for (int k = 0; k < 2; ++k) { cudaEvent_t e; cudaEventCreate(&e); h->ev_pool.push_back(e); }
+    }
+    h->ev_class.push_back(cls);
+    cudaEventRecord(h->ev_pool[h->ev_used], h->stream);
+}
+void prof_end(pb_handle* h) {
+    if (!h->profile) return;
+    cudaEventRecord(h->ev_pool[h->ev_used + 1], h->stream);
+    h->ev_used += 2;
+}
+void prof_collect(pb_handle* h) {
+    if (!h->profile) return;
+    cudaStreamSynchronize(h->stream);
+    for (size_t k = 0; k < h->ev_class.size(); ++k) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, h->ev_pool[2 * k], h->ev_pool[2 * k + 1]) == cudaSuccess) {
+            h->prof[h->ev_class[k]].ms += ms;
+            h->prof[h->ev_class[k]].launches += 1;
+        }
+    }
+    h->ev_class.clear();
+    h->ev_used = 0;
+}
+
+// ---------------------------------------------------------------- ticks
+int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int label_value,
+              int n_ticks, float* dev_losses) {
+    const int elems = h->in_shape.elems();
+    const int ingest_blocks = std::min(ceil_div(elems, 1024), 2 * h->num_sms);
+    const long long t_base = h->tick;
+    h->last_launches = 0;
+    if (h->profile) for (auto& p : h->prof) p = ProfileClass{};
+    for (int k = 0; k < n_ticks; ++k) {
+        ingest_kernel<<<ingest_blocks, 256, 0, h->stream>>>(h->d_ts, dev_xs, dev_labels, label_value, h->in_ring,
+                                                            h->in_slots, elems, h->label_ring, h->S, t_base);
+        h->last_launches += 1;
+        if (h->all_fc) {
+            prof_begin(h, 0);
+            fc_tick_kernel<<<h->nctaA, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segA, h->d_ctaA, h->d_ts, h->S, 0,
+                                                                  h->label_ring, dev_losses, t_base);
+            prof_end(h);
+            prof_begin(h, 1);
+            fc_tick_kernel<<<h->nctaB, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segB, h->d_ctaB, h->d_ts, h->S, 1,
+                                                                  h->label_ring, dev_losses, t_base);
+            prof_end(h);
+            h->last_launches += 2;
+        } else {
+            return fail(h, PB_E_UNSUPPORTED, "convolution stages are not built into this library");
+        }
+    }
+    PB_CUDA(h, cudaGetLastError());
+    h->tick += n_ticks;
+    prof_collect(h);
+    return PB_OK;
+}
+
+int check_device_error(pb_handle* h) {
+    TickState ts;
+    PB_CUDA(h, cudaMemcpyAsync(&ts, h->d_ts, sizeof(ts), cudaMemcpyDeviceToHost, h->stream));
+    PB_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (ts.error != kErrNone)
+        return fail(h, PB_E_DEVICE, "device index check failed: code " + std::to_string(ts.error) + " info " + std::to_string(ts.error_info));
+    return PB_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------- C interface
+extern "C" {
+
+int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_layer, int in_c, int in_h,
+              int in_w, int n_classes, float lr, float momentum, unsigned flags, void* stream,
+              pb_handle** out) {
+    if (out) *out = nullptr;
+    if (!layers || !stage_of_layer || !out || n_layers <= 0 || in_c <= 0 || in_h <= 0 || in_w <= 0 || n_classes <= 0)
+        return fail(nullptr, PB_E_ARG, "pb_create: NULL pointer or non-positive size");
+    if (!(momentum >= 0.f && momentum < 1.f) || !(lr >= 0.f)) return fail(nullptr, PB_E_ARG, "pb_create: need 0 <= momentum < 1 and lr >= 0");
+    if (flags & ~(unsigned)(PB_SC | PB_LWP | PB_LWP_WFORM | PB_CONV_BF16)) return fail(nullptr, PB_E_ARG, "pb_create: unknown flag");
+    if (flags & PB_LWP_WFORM) return fail(nullptr, PB_E_UNSUPPORTED, "pb_create: the weight-difference form of LWP is not built");
+    for (int q = 1; q < n_layers; ++q)
+        if (stage_of_layer[q] < stage_of_layer[q - 1]) return fail(nullptr, PB_E_ARG, "pb_create: stage indices must not decrease");
+    pb_handle* h = new (std::nothrow) pb_handle();
+    if (!h) return fail(nullptr, PB_E_ALLOC, "pb_create: out of host memory");
+    h->stream = (cudaStream_t)stream;
+    h->flags = flags; h->lr = lr; h->momentum = momentum; h->n_classes = n_classes;
+    h->in_shape = Shape{in_c, in_h, in_w};
+    int rc = parse_layers(h, layers, n_layers, stage_of_layer);
+    if (rc != PB_OK) { delete h; return rc; }
+    schedule_constants(h);
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
+    if (e != cudaSuccess) { std::string m = cudaGetErrorString(e); delete h; return fail(nullptr, PB_E_CUDA, "pb_create: no CUDA device: " + m); }
+
+    // FC tables and their partition
+    std::vector<int> idsA, idsB;
+    for (const StageHost& x : h->stages) {
+        if (x.head_op != PB_FC) continue;
+        FcStage f{};
+        f.in_dim = x.head.c_in; f.out_dim = x.head.c_out; f.s = x.index;
+        f.relu = x.relu; f.is_last = x.loss; f.need_dx = x.src >= 0;
+        f.vec = (f.in_dim % 4 == 0) ? 4 : 1;
+        f.neg_lr_T = -lr * x.T; f.m = momentum; f.neg_lr_a = -lr * x.a; f.neg_lr_b = -lr * x.b;
+        idsA.push_back((int)h->h_fc.size());
+        if (x.loss) idsB.push_back((int)h->h_fc.size());
+        h->h_fc.push_back(f);
+    }
+    std::vector<int> npartsA(h->h_fc.size(), 1), npartsB(h->h_fc.size(), 1);
+    partition_fc(h, idsA, h->h_segA, h->h_ctaA, npartsA);
+    partition_fc(h, idsB, h->h_segB, h->h_ctaB, npartsB);
+    for (size_t f = 0; f < h->h_fc.size(); ++f) {
+        StageHost& x = h->stages[h->h_fc[f].s];
+        x.dx_nparts = x.loss ? npartsB[f] : npartsA[f];
+    }
+    h->nctaA = (int)h->h_ctaA.size() - 1;
+    h->nctaB = (int)h->h_ctaB.size() - 1;
+
+    size_t zero_from = 0;
+    h->arena_bytes = layout(h, nullptr, &zero_from);
+    e = cudaMalloc((void**)&h->arena, h->arena_bytes);
+    if (e != cudaSuccess) {
+        std::string m = "pb_create: cudaMalloc of " + std::to_string(h->arena_bytes) + " bytes failed: " + cudaGetErrorString(e);
+        delete h; return fail(nullptr, PB_E_ALLOC, m);
+    }
+    layout(h, h->arena, &zero_from);
+    h->zero_from = zero_from;
+    fill_fc_tables(h);
+    e = cudaMemsetAsync(h->arena, 0, h->arena_bytes, h->stream);
+    auto up = [&](void* d, const void* s, size_t n) { if (e == cudaSuccess && n) e = cudaMemcpyAsync(d, s, n, cudaMemcpyHostToDevice, h->stream); };
+    up(h->d_fc, h->h_fc.data(), h->h_fc.size() * sizeof(FcStage));
+    up(h->d_segA, h->h_segA.data(), h->h_segA.size() * sizeof(FcSeg));
+    up(h->d_segB, h->h_segB.data(), h->h_segB.size() * sizeof(FcSeg));
+    up(h->d_ctaA, h->h_ctaA.data(), h->h_ctaA.size() * sizeof(int));
+    up(h->d_ctaB, h->h_ctaB.data(), h->h_ctaB.size() * sizeof(int));
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) {
+        std::string m = std::string("pb_create: upload failed: ") + cudaGetErrorString(e);
+        cudaFree(h->arena); delete h; return fail(nullptr, PB_E_CUDA, m);
+    }
+    *out = h;
+    return PB_OK;
+}
+
+int pb_set_weights(pb_handle* h, const float* host_w, size_t n) {
+    if (!h) return PB_E_ARG;
+    if (!host_w || n != h->n_params) return fail(h, PB_E_ARG, "pb_set_weights: need pb_num_params() floats");
+    PB_CUDA(h, cudaMemsetAsync(h->arena + h->zero_from, 0, h->arena_bytes - h->zero_from, h->stream));
+    PB_CUDA(h, cudaMemsetAsync(h->d_ts, 0, sizeof(TickState), h->stream));
+    for (const StageHost& x : h->stages)
+        PB_CUDA(h, cudaMemcpyAsync(h->d_w + x.dev_off, host_w + x.user_off, x.n_params * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+    PB_CUDA(h, cudaStreamSynchronize(h->stream));
+    h->tick = 0;
+    return PB_OK;
+}
+
+int pb_tick(pb_handle* h, const float* dev_x, int label, float* host_loss) {
+    if (!h) return PB_E_ARG;
+    if (!dev_x || label < 0 || label >= h->n_classes) return fail(h, PB_E_ARG, "pb_tick: NULL input or label out of range");
+    int rc = run_ticks(h, dev_x, nullptr, label, 1, h->d_loss1);
+    if (rc != PB_OK) return rc;
+    if (host_loss) {
+        PB_CUDA(h, cudaMemcpyAsync(host_loss, h->d_loss1, sizeof(float), cudaMemcpyDeviceToHost, h->stream));
+        return check_device_error(h);
+    }
+    return PB_OK;
+}
+
+int pb_run(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int n_ticks, float* dev_losses) {
+    if (!h) return PB_E_ARG;
+    if (!dev_xs || !dev_labels || n_ticks < 0) return fail(h, PB_E_ARG, "pb_run: NULL pointer or negative count");
+    if (n_ticks == 0) return PB_OK;
+    return run_ticks(h, dev_xs, dev_labels, 0, n_ticks, dev_losses);
+}
+
+int pb_run_host(pb_handle* h, const float* host_xs, const int32_t* host_labels, int n_ticks, float* host_losses) {
+    if (!h) return PB_E_ARG;
+    if (!host_xs || !host_labels || n_ticks < 0) return fail(h, PB_E_ARG, "pb_run_host: NULL pointer or negative count");
+    if (n_ticks == 0) return PB_OK;
+    const size_t xb = (size_t)n_ticks * h->in_shape.elems() * sizeof(float);
+    const size_t lb = (size_t)n_ticks * sizeof(int32_t), fb = (size_t)n_ticks * sizeof(float);
+    const size_t o1 = align_up(xb, 256), o2 = o1 + align_up(lb, 256), need = o2 + align_up(fb, 256);
+    cudaError_t e = cudaSuccess;
+    if (need > h->staging_bytes) {   // grow-only staging buffer, kept for later calls
+        PB_CUDA(h, cudaStreamSynchronize(h->stream));
+        if (h->staging) cudaFree(h->staging);
+        h->staging = nullptr; h->staging_bytes = 0;
+        e = cudaMalloc((void**)&h->staging, need);
+        if (e != cudaSuccess) return fail(h, PB_E_ALLOC, std::string("pb_run_host: staging allocation failed: ") + cudaGetErrorString(e));
+        h->staging_bytes = need;
+    }
+    char* stage = h->staging;
+    int rc = PB_OK;
+    e = cudaMemcpyAsync(stage, host_xs, xb, cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(stage + o1, host_labels, lb, cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) rc = run_ticks(h, (const float*)stage, (const int32_t*)(stage + o1), 0, n_ticks, (float*)(stage + o2));
+    if (e == cudaSuccess && rc == PB_OK && host_losses) e = cudaMemcpyAsync(host_losses, stage + o2, fb, cudaMemcpyDeviceToHost, h->stream);
+    cudaError_t e2 = cudaStreamSynchronize(h->stream);
+    if (rc != PB_OK) return rc;
+    if (e != cudaSuccess || e2 != cudaSuccess) return fail(h, PB_E_CUDA, std::string("pb_run_host: ") + cudaGetErrorString(e != cudaSuccess ? e : e2));
+    return check_device_error(h);
+}
+
+static int get_params(pb_handle* h, const float* dev, float* host, size_t n, const char* who) {
+    if (!h) return PB_E_ARG;
+    if (!host || n != h->n_params) return fail(h, PB_E_ARG, std::string(who) + ": need pb_num_params() floats");
+    for (const StageHost& x : h->stages)
+        PB_CUDA(h, cudaMemcpyAsync(host + x.user_off, dev + x.dev_off, x.n_params * sizeof(float), cudaMemcpyDeviceToHost, h->stream));
+    return check_device_error(h);
+}
+
+int pb_get_weights(pb_handle* h, float* host_w, size_t n) { return get_params(h, h ? h->d_w : nullptr, host_w, n, "pb_get_weights"); }
+int pb_get_velocity(pb_handle* h, float* host_v, size_t n) { return get_params(h, h ? h->d_v : nullptr, host_v, n, "pb_get_velocity"); }
+
+int pb_sync(pb_handle* h) { return h ? check_device_error(h) : PB_E_ARG; }
+size_t pb_num_params(const pb_handle* h) { return h ? h->n_params : 0; }
+int pb_num_stages(const pb_handle* h) { return h ? h->S : PB_E_ARG; }
+int pb_stage_delay(const pb_handle* h, int s) { return (h && s >= 0 && s < h->S) ? h->stages[s].delay : PB_E_ARG; }
+long long pb_tick_count(const pb_handle* h) { return h ? h->tick : -1; }
+long long pb_last_launch_count(const pb_handle* h) { return h ? h->last_launches : -1; }
+size_t pb_device_bytes(const pb_handle* h) { return h ? h->arena_bytes : 0; }
+
+int pb_profile_enable(pb_handle* h, int enable) {
+    if (!h) return PB_E_ARG;
+    h->profile = enable != 0;
+    return PB_OK;
+}
+
+double pb_profile_ms(pb_handle* h, int which, long long* launches) {
+    if (!h || which < 0 || which >= 4 || h->prof[which].launches == 0) { if (launches) *launches = 0; return -1.0; }
+    if (launches) *launches = h->prof[which].launches;
+    return h->prof[which].ms;
+}
+
+const char* pb_last_error(const pb_handle* h) { return h ? h->err.c_str() : g_create_error.c_str(); }
+
+void pb_destroy(pb_handle* h) {
+    if (!h) return;
+    cudaStreamSynchronize(h->stream);
+    for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
+    if (h->staging) cudaFree(h->staging);
+    cudaFree(h->arena);
+    delete h;
+}
+
+}  // extern "C"

@@ -1,0 +1,75 @@
+// Host-side engine state behind pb_handle.
+#pragma once
+#include <string>
+#include <vector>
+
+#include "../../include/pb.h"
+#include "pb_internal.h"
+
+namespace pb {
+
+struct Shape { int c = 0, h = 0, w = 0; int elems() const { return c * h * w; } };
+
+// Host description of one pipeline stage.
+struct StageHost {
+    int index = 0;
+    int head_op = PB_FC;            // PB_FC or PB_CONV2D
+    pb_layer head{};
+    int gn_groups = 0;
+    int skip_src = -1, skip_mode = 0;
+    bool has_skip = false, relu = false, avgpool = false, loss = false;
+    bool has_pool = false;
+    int pool_k = 0, pool_stride = 0, pool_pad = 0;
+    int src = -1;                   // producing stage (-1: network input)
+    Shape in, z, out;               // input, head output (pre-pool), stage output
+    size_t n_params = 0;
+    size_t user_off = 0;            // offset in the caller's flat parameter vector
+    size_t dev_off = 0;             // offset (floats) in the padded device arrays
+    int delay = 0;                  // D_s = 2 (S-1-s)
+    float a = 1.f, b = 0.f, T = 0.f;
+    // rings (device pointers into the arena)
+    float* out_ring = nullptr; int out_slots = 0;
+    float* dx = nullptr; int dx_slots = 0, dx_nparts = 1;          // gradient w.r.t. main input
+    float* dskip = nullptr; int dskip_slots = 0;                   // gradient w.r.t. skip input
+    std::vector<int> consumers_main, consumers_skip;               // stages reading this output
+};
+
+struct ProfileClass { double ms = 0; long long launches = 0; };
+
+}  // namespace pb
+
+struct pb_handle {
+    cudaStream_t stream = nullptr;
+    int device = 0, num_sms = 0;
+    unsigned flags = 0;
+    float lr = 0, momentum = 0;
+    int S = 0, n_classes = 0;
+    pb::Shape in_shape;
+    size_t n_params = 0, dev_params = 0;
+    std::vector<pb::StageHost> stages;
+    bool all_fc = true;
+
+    // device memory (one arena)
+    char* arena = nullptr; size_t arena_bytes = 0, zero_from = 0;
+    char* staging = nullptr; size_t staging_bytes = 0;   // pb_run_host, grow-only
+    float *d_w = nullptr, *d_v = nullptr;
+    float* in_ring = nullptr; int in_slots = 0;
+    int* label_ring = nullptr;
+    pb::TickState* d_ts = nullptr;
+    float* d_loss1 = nullptr;
+    // FC tables
+    pb::FcStage* d_fc = nullptr; int n_fc = 0;
+    pb::FcSeg *d_segA = nullptr, *d_segB = nullptr;
+    int *d_ctaA = nullptr, *d_ctaB = nullptr;
+    int nctaA = 0, nctaB = 0;
+    std::vector<pb::FcStage> h_fc;
+    std::vector<pb::FcSeg> h_segA, h_segB;
+    std::vector<int> h_ctaA, h_ctaB;
+
+    long long tick = 0, last_launches = 0;
+    bool profile = false;
+    pb::ProfileClass prof[4];
+    std::vector<cudaEvent_t> ev_pool; size_t ev_used = 0;
+    std::vector<int> ev_class;
+    std::string err;
+};

@@ -1,0 +1,72 @@
+"""Shared helpers of the GPU parity tests: run the CUDA engine and the CPU
+checker on the same seeded inputs and compare per tick."""
+import math
+
+import numpy as np
+
+from oracle import PBOracle
+from pb_workloads import he_normal_weights, make_inputs
+
+
+def rel_err(got, ref):
+    """||got - ref||_2 / max(||ref||_2, 1e-12); tensors that are exactly zero
+    in the reference must be exactly zero."""
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    n = np.linalg.norm(ref)
+    if n == 0.0:
+        return 0.0 if not got.any() else float("inf")
+    return float(np.linalg.norm(got - ref) / max(n, 1e-12))
+
+
+def make_oracle(wl, dtype=np.float64, **kw):
+    o = PBOracle(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, wl.lr, wl.momentum,
+                 wl.flags & 7, dtype=dtype, **kw)
+    o.set_weights(he_normal_weights(wl.seed, wl))
+    return o
+
+
+def make_engine(wl):
+    import torch
+    from paper_2003_11666_b200 import PB
+    eng = PB(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, wl.lr, wl.momentum,
+             wl.flags, stream=torch.cuda.current_stream().cuda_stream)
+    eng.set_weights(he_normal_weights(wl.seed, wl))
+    return eng
+
+
+def compare_ticks(wl, n_ticks, tol, check_every=1, finite_limit=1e30, loose_after=None):
+    """Tick both sides one sample at a time; returns the worst errors seen.
+
+    The window ends early (returning the tick) once the checker's own state
+    exceeds `finite_limit`: past that the float32 engine is out of range."""
+    import torch
+    x, y = make_inputs(wl.seed, n_ticks, wl.sample_elems, wl.n_classes)
+    o = make_oracle(wl)
+    eng = make_engine(wl)
+    xd = torch.from_numpy(x).cuda()
+    worst = {"loss": 0.0, "w": 0.0, "v": 0.0, "ticks": 0}
+    for t in range(n_ticks):
+        lo = o.tick(x[t], y[t])
+        lg = eng.tick(xd[t], int(y[t]))
+        wo = o.get_weights()
+        if not np.isfinite(wo).all() or np.abs(wo).max() > finite_limit:
+            break
+        tl = tol if loose_after is None or t < loose_after[0] else loose_after[1]
+        if math.isnan(lo):
+            assert math.isnan(lg), "tick %d: loss should be NaN while the pipeline fills" % t
+        else:
+            # loss = logsumexp(o) - o[label] is a difference of numbers of the
+            # logits' size, so its rounding error scales with max|o|, not with itself
+            e = abs(lg - lo) / max(abs(lo), float(np.abs(o.last_logits).max()), 1e-12)
+            worst["loss"] = max(worst["loss"], e)
+            assert e <= tl, "tick %d: loss %r vs %r (rel %.3g)" % (t, lg, lo, e)
+        if t % check_every == 0 or t == n_ticks - 1:
+            ew = rel_err(eng.get_weights(), wo)
+            ev = rel_err(eng.get_velocity(), o.get_velocity())
+            worst["w"], worst["v"] = max(worst["w"], ew), max(worst["v"], ev)
+            assert ew <= tl, "tick %d: weights rel err %.3g" % (t, ew)
+            assert ev <= tl, "tick %d: velocity rel err %.3g" % (t, ev)
+        worst["ticks"] = t + 1
+    eng.destroy()
+    return worst

@@ -1,0 +1,97 @@
+"""CUDA engine vs CPU checker on fully connected pipelines (through the C ABI)."""
+import numpy as np
+import pytest
+
+from pb_workloads import mlp, workload, make_inputs, he_normal_weights
+from tests.parity import compare_ticks, make_engine, make_oracle, rel_err
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-4      # relative, float32 path
+
+
+@pytest.mark.parametrize("sizes", [[12, 7], [20, 16, 5], [33, 17, 9, 4], [784, 256, 256, 256, 10],
+                                   [130, 260, 131, 70, 3], [512, 300, 10]])
+@pytest.mark.parametrize("flags", [3, 0, 1, 2])
+def test_small_mlps_match_checker(sizes, flags):
+    # odd widths reach the scalar path, ragged chunks and rows that are not a multiple of 4
+    wl = mlp(sizes, lr=0.002, seed=21, flags=flags)
+    S = wl.n_stages
+    w = compare_ticks(wl, 2 * (S - 1) + 24, TOL)
+    assert w["ticks"] == 2 * (S - 1) + 24
+
+
+def test_mlp4_first_64_ticks():
+    # literal benchmark hyper-parameters; these dynamics are diverging, and from
+    # tick ~54 on even float32 evaluation of the checker itself drifts past 1e-4
+    # from float64, so the strict bound is held on ticks < 48 and a 2e-3 bound after.
+    wl = workload("mlp4")
+    w = compare_ticks(wl, 64, TOL, loose_after=(48, 2e-3))
+    assert w["ticks"] == 64
+
+
+def test_mlp4_stable_learning_rate_64_ticks():
+    wl = workload("mlp4")
+    wl.lr = 0.001
+    w = compare_ticks(wl, 64, TOL)
+    assert w["ticks"] == 64
+
+
+def test_run_matches_tick_by_tick_and_loss_is_delayed():
+    import torch
+    wl = mlp([64, 48, 32, 6], lr=0.003, seed=5)
+    n = 40
+    x, y = make_inputs(wl.seed, n, wl.sample_elems, wl.n_classes)
+    a, b = make_engine(wl), make_engine(wl)
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    losses = torch.zeros(n, device="cuda")
+    a.run(xd, yd, n, losses)
+    a.sync()
+    one = [b.tick(xd[t], int(y[t])) for t in range(n)]
+    got = losses.cpu().numpy()
+    S = wl.n_stages
+    assert np.isnan(got[:S - 1]).all() and np.isfinite(got[S - 1:]).all()
+    np.testing.assert_array_equal(got[S - 1:], np.array(one[S - 1:], dtype=np.float32))
+    np.testing.assert_array_equal(a.get_weights(), b.get_weights())
+    assert a.tick_count == n and a.last_launch_count == 3 * n
+    # host-buffer entry point gives the same numbers
+    c = make_engine(wl)
+    hl = np.zeros(n, dtype=np.float32)
+    c.run_host(x, y, n, hl)
+    np.testing.assert_array_equal(hl[S - 1:], got[S - 1:])
+    np.testing.assert_array_equal(c.get_weights(), a.get_weights())
+    for e in (a, b, c):
+        e.destroy()
+
+
+def test_set_weights_restarts_the_pipeline():
+    import torch
+    wl = mlp([32, 16, 4], lr=0.01, seed=6)
+    x, y = make_inputs(wl.seed, 12, wl.sample_elems, wl.n_classes)
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    e = make_engine(wl)
+    l1 = torch.zeros(12, device="cuda")
+    e.run(xd, yd, 12, l1)
+    w1 = e.get_weights()
+    e.set_weights(he_normal_weights(wl.seed, wl))
+    assert e.tick_count == 0 and not e.get_velocity().any()
+    l2 = torch.zeros(12, device="cuda")
+    e.run(xd, yd, 12, l2)
+    np.testing.assert_array_equal(w1, e.get_weights())
+    np.testing.assert_array_equal(l1.cpu().numpy()[2:], l2.cpu().numpy()[2:])
+    e.destroy()
+
+
+def test_bad_arguments_are_reported_not_thrown_across_the_abi():
+    from paper_2003_11666_b200 import PB, PBError
+    wl = mlp([8, 4])
+    with pytest.raises(PBError):
+        PB(wl.layers, wl.stage_of_layer, (9, 1, 1), 4, 0.1, 0.9)      # FC size mismatch
+    with pytest.raises(PBError):
+        PB(wl.layers, wl.stage_of_layer, wl.in_shape, 4, 0.1, 1.5)    # momentum out of range
+    e = make_engine(wl)
+    with pytest.raises(PBError):
+        e.set_weights(np.zeros(3, np.float32))
+    with pytest.raises(PBError):
+        e.tick(0, 99)
+    e.destroy()
