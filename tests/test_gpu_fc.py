@@ -37,6 +37,24 @@ def test_mlp4_stable_learning_rate_64_ticks():
     assert w["ticks"] == 64
 
 
+def test_deep_mlp_full_size_until_float32_range_ends():
+    # Full benchmark size (63 M parameters, 16 stages), literal hyper-parameters.
+    # lr*|x|^2 is about 10 here, so the run diverges: the checker's weights pass
+    # 1e30 near tick 34, where float32 overflows; the comparison covers every tick
+    # up to there (all 16 stages have updated by tick 30).  The weights are compared
+    # on every third tick to keep the float64 norms affordable.
+    wl = workload("mlp16x2048")
+    w = compare_ticks(wl, 64, TOL, check_every=3, finite_limit=1e24)
+    assert 31 <= w["ticks"] <= 36, w
+
+
+def test_deep_mlp_narrow_stable_64_ticks():
+    # same depth (16 stages, delays 30..0) at width 256 with a stable step: all 64 ticks
+    wl = mlp([256] * 16 + [10], lr=0.0005, seed=1)
+    w = compare_ticks(wl, 2 * 15 + 34, TOL)
+    assert w["ticks"] == 64
+
+
 def test_run_matches_tick_by_tick_and_loss_is_delayed():
     import torch
     wl = mlp([64, 48, 32, 6], lr=0.003, seed=5)
