@@ -36,8 +36,21 @@ def conv_out_size(n, k, stride, pad):
     return (n + 2 * pad - k) // stride + 1
 
 
-def conv2d_forward(W, x, stride, pad):
-    """z[o, p, q] = sum_{c, r, s} W[o, c, r, s] * xpad[c, p*stride + r, q*stride + s]."""
+def round_bf16(x):
+    """Round to the nearest bfloat16 (ties to even) and return in x's dtype:
+    the value is first taken to float32, whose upper 16 bits are a bfloat16."""
+    b = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = ((b >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
+    b = (b + r) & np.uint32(0xFFFF0000)
+    return b.view(np.float32).astype(x.dtype)
+
+
+def conv2d_forward(W, x, stride, pad, rnd=None):
+    """z[o, p, q] = sum_{c, r, s} W[o, c, r, s] * xpad[c, p*stride + r, q*stride + s].
+    `rnd`, if given, is applied to both operands first (reduced-precision
+    multiplicands with exact products and wide accumulation)."""
+    if rnd is not None:
+        W, x = rnd(W), rnd(x)
     co, ci, k, _ = W.shape
     oh = conv_out_size(x.shape[1], k, stride, pad)
     ow = conv_out_size(x.shape[2], k, stride, pad)
@@ -50,8 +63,10 @@ def conv2d_forward(W, x, stride, pad):
     return z
 
 
-def conv2d_backward(W, x, dz, stride, pad):
-    """Returns (dx, gW) of conv2d_forward."""
+def conv2d_backward(W, x, dz, stride, pad, rnd=None):
+    """Returns (dx, gW) of conv2d_forward; `rnd` as there, on W, x and dz."""
+    if rnd is not None:
+        W, x, dz = rnd(W), rnd(x), rnd(dz)
     co, ci, k, _ = W.shape
     oh, ow = dz.shape[1], dz.shape[2]
     xp = _pad(x, pad)
@@ -106,14 +121,17 @@ def relu_backward(x_pre, dy):
     return np.where(x_pre > 0, dy, dy.dtype.type(0))
 
 
-def maxpool_forward(x, k, stride, pad):
+def maxpool_forward(x, k, stride, pad, want_gap=False):
     """Returns (y, arg) where arg[c, p, q] is the flat index (row*W + col in
     the unpadded input) of the first maximum in row-major window order;
-    padding never wins."""
+    padding never wins.  With want_gap also returns the smallest distance
+    between the largest and second largest entry over windows whose maximum
+    is positive (how close any window came to choosing differently)."""
     c, h, w = x.shape
     oh = conv_out_size(h, k, stride, pad)
     ow = conv_out_size(w, k, stride, pad)
     y = np.full((c, oh, ow), -np.inf, dtype=x.dtype)
+    second = np.full((c, oh, ow), -np.inf, dtype=x.dtype)
     arg = np.full((c, oh, ow), -1, dtype=np.int64)
     for p in range(oh):
         for q in range(ow):
@@ -121,9 +139,15 @@ def maxpool_forward(x, k, stride, pad):
                 for s in range(k):
                     ih, iw = p * stride + r - pad, q * stride + s - pad
                     if 0 <= ih < h and 0 <= iw < w:
-                        better = x[:, ih, iw] > y[:, p, q]
-                        y[better, p, q] = x[better, ih, iw]
+                        v = x[:, ih, iw]
+                        better = v > y[:, p, q]
+                        second[:, p, q] = np.where(better, y[:, p, q], np.maximum(second[:, p, q], v))
+                        y[better, p, q] = v[better]
                         arg[better, p, q] = ih * w + iw
+    if want_gap:
+        pos = y > 0
+        gap = float((y - second)[pos].min()) if pos.any() else float("inf")
+        return y, arg, gap
     return y, arg
 
 

@@ -57,6 +57,9 @@ class _Stage:
             return W, None, theta[nw:nw + h.c_out], theta[nw + h.c_out:nw + 2 * h.c_out]
         return W, None, None, None
 
+    rnd = None                # operand rounding of the convolutions (None or a function)
+    margins = False           # record how close the ReLU / max-pool decisions were
+
     def forward(self, theta_hat, x, skip_in):
         h = self.head
         W, b, gamma, beta = self.split(theta_hat)
@@ -64,15 +67,24 @@ class _Stage:
         if h.op == OP_FC:
             n = L.fc_forward(W, b, x.ravel()).reshape(-1, 1, 1)
         else:
-            n = L.conv2d_forward(W, x, h.stride, h.pad)
+            n = L.conv2d_forward(W, x, h.stride, h.pad, self.rnd)
             if self.gn_groups:
                 n, st["zhat"], st["rstd"] = L.groupnorm_forward(gamma, beta, n, self.gn_groups)
         if self.skip is not None:
             n = n + L.skip_forward(skip_in, self.skip[1], n.shape)
         st["pre"] = n
         a = L.relu_forward(n) if self.relu else n
+        if self.margins:
+            # smallest distance of any decision from flipping, relative to the tensor's rms
+            rms = float(np.sqrt(np.mean(n * n))) or 1.0
+            nz = np.abs(n[n != 0])
+            st["margin"] = float(nz.min()) / rms if (self.relu and nz.size) else float("inf")
         if self.maxpool is not None:
-            a, st["arg"] = L.maxpool_forward(a, *self.maxpool)
+            if self.margins:
+                a, st["arg"], gap = L.maxpool_forward(a, *self.maxpool, want_gap=True)
+                st["margin"] = min(st["margin"], gap / rms)
+            else:
+                a, st["arg"] = L.maxpool_forward(a, *self.maxpool)
         if self.avgpool:
             a = L.avgpool_forward(a)
         return a, st
@@ -105,7 +117,7 @@ class _Stage:
                 d, gg, gbeta = L.groupnorm_backward(gamma, st["zhat"], st["rstd"], d, self.gn_groups)
                 g[nw:nw + h.c_out] = gg
                 g[nw + h.c_out:] = gbeta
-            dx, gW = L.conv2d_backward(W, st["x"], d, h.stride, h.pad)
+            dx, gW = L.conv2d_backward(W, st["x"], d, h.stride, h.pad, self.rnd)
             g[:nw] = gW.ravel()
             if not need_dx:
                 dx = None
@@ -168,9 +180,19 @@ class PBOracle:
 
     def __init__(self, layer_list, stage_of_layer, in_shape, n_classes, lr,
                  momentum, flags=FLAG_SC | FLAG_LWP, dtype=np.float64,
-                 sc_delay_scale=1, horizon_scale=1, record=False):
+                 sc_delay_scale=1, horizon_scale=1, record=False, conv_operands=None,
+                 margins=False):
+        """conv_operands: None, or "bf16" to round both operands of every
+        convolution product (forward, data gradient, weight gradient) to
+        bfloat16 while accumulating in `dtype`.  margins: log in
+        `self.min_margin[(stage, sample)]` how close that forward's ReLU /
+        max-pool decisions came to flipping (relative to the tensor's rms)."""
         self.dtype = dtype
         self.stages = build_stages(layer_list, stage_of_layer, in_shape)
+        for st in self.stages:
+            st.rnd = L.round_bf16 if conv_operands == "bf16" else None
+            st.margins = margins
+        self.min_margin = {}
         self.S = len(self.stages)
         if not self.stages[-1].loss:
             raise ValueError("the last stage must end in SOFTMAX_CE")
@@ -230,6 +252,8 @@ class PBOracle:
             skip_in = self.out[(st.skip[0], i)] if st.skip is not None else None
             y, stash = st.forward(theta_hat[s], self.out[(st.src, i)], skip_in)
             self.out[(s, i)], self.stash[(s, i)] = y, stash
+            if st.margins:
+                self.min_margin[(s, i)] = stash["margin"]
             if self.record:
                 self.fwd_version[(s, i)] = self.opt[s].version
 

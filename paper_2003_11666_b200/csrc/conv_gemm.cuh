@@ -1,0 +1,172 @@
+// Grouped implicit-GEMM kernel for the float32 convolution path.
+//
+// One launch covers the forward convolutions of every stage (fprop), or the
+// data gradients (dgrad), or the weight gradients (wgrad): a tile table maps
+// each thread block to (problem, tile, K-slice).  Operands are gathered
+// straight from the activation rings / gradient scratch (no im2col buffer) into
+// shared memory; 256 threads each own a 4x4 patch of a 64x64 tile.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "conv_types.h"
+
+namespace pb {
+
+__device__ __forceinline__ float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+template <int KS> struct KDiv {
+    __device__ __forceinline__ static void split(int kk, int k, int& c, int& r, int& s) {
+        c = kk / (KS * KS); const int rs = kk - c * (KS * KS); r = rs / KS; s = rs - r * KS;
+    }
+};
+template <> struct KDiv<0> {
+    __device__ __forceinline__ static void split(int kk, int k, int& c, int& r, int& s) {
+        const int k2 = k * k; c = kk / k2; const int rs = kk - c * k2; r = rs / k; s = rs - r * k;
+    }
+};
+
+template <int KS>
+__device__ void gemm_tile(const ConvGemm& G, const GemmTile& tl, long long smp,
+                          float (&As)[kBK][kBM + 4], float (&Bs)[kBK][kBN + 4]) {
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int M = G.M, N = G.N;
+    const int kb = tl.split * G.k_per_split;
+    const int ke = min(G.K, kb + G.k_per_split);
+    const float* __restrict__ A = G.a;
+    const float* __restrict__ B = G.b + (size_t)(smp % G.b_slots) * G.b_elems;
+    float* __restrict__ Cp = G.c + ((size_t)(smp % G.c_slots) * G.nsplit + tl.split) * ((size_t)M * N);
+    const int ksz = G.k, st = G.stride, pad = G.pad, ih = G.ih, iw = G.iw, oh = G.oh, ow = G.ow;
+    const bool bf = G.bf16 != 0;
+
+    float acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+
+    // per-thread invariants of the loaders
+    const int lo16 = tid & 15, hi16 = tid >> 4;      // 0..15 each
+    const int lo64 = tid & 63, hi4 = tid >> 6;       // 0..63, 0..3
+    int n_p = 0, n_q = 0;                            // fprop/dgrad: pixel of column n = n0 + lo64
+    bool n_ok = false;
+    int wc[4], wr[4], ws[4];                         // wgrad: (ci, r, s) of columns n0 + hi16 + 16 q
+    bool w_ok[4];
+    if (G.mode == kFprop) {
+        const int n = tl.n0 + lo64; n_ok = n < N; n_p = n / ow; n_q = n - n_p * ow;
+    } else if (G.mode == kDgrad) {
+        const int n = tl.n0 + lo64; n_ok = n < N; n_p = n / iw; n_q = n - n_p * iw;
+    } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int n = tl.n0 + hi16 + 16 * q;
+            w_ok[q] = n < N;
+            KDiv<KS>::split(n, ksz, wc[q], wr[q], ws[q]);
+        }
+    }
+
+    for (int k0 = kb; k0 < ke; k0 += kBK) {
+        float ra[4], rb[4];
+        if (G.mode == kFprop) {
+            // A[m, kk] = w_hat[m*K + kk]: 16 consecutive kk per row
+            const int kk = k0 + lo16;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int m = tl.m0 + hi16 + 16 * q;
+                ra[q] = (m < M && kk < ke) ? A[(size_t)m * G.K + kk] : 0.f;
+            }
+            // B[kk, n] = x[ci, p*st + r - pad, q*st + s - pad]
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int kq = k0 + hi4 + 4 * q;
+                int c, r, s;
+                KDiv<KS>::split(kq, ksz, c, r, s);
+                const int y = n_p * st + r - pad, x = n_q * st + s - pad;
+                rb[q] = (n_ok && kq < ke && y >= 0 && y < ih && x >= 0 && x < iw) ? B[((size_t)c * ih + y) * iw + x] : 0.f;
+            }
+        } else if (G.mode == kDgrad) {
+            // A[m = ci, kk = (co, r, s)] = w[co, ci, r, s];  B[kk, n = (y, x)] = dz[co, (y+pad-r)/st, (x+pad-s)/st]
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int kq = k0 + hi4 + 4 * q;
+                int c, r, s;
+                KDiv<KS>::split(kq, ksz, c, r, s);
+                const int m = tl.m0 + lo64;
+                ra[q] = (m < M && kq < ke) ? A[(((size_t)c * G.ci + m) * ksz + r) * ksz + s] : 0.f;
+                const int ty_ = n_p + pad - r, tx_ = n_q + pad - s;
+                float v = 0.f;
+                if (n_ok && kq < ke && ty_ >= 0 && tx_ >= 0) {
+                    const int p = ty_ / st, qq = tx_ / st;
+                    if (p * st == ty_ && qq * st == tx_ && p < oh && qq < ow) v = B[((size_t)c * oh + p) * ow + qq];
+                }
+                rb[q] = v;
+            }
+        } else {
+            // A[m = co, kk = pixel] = dz[m*K + kk];  B[kk = (p, q), n = (ci, r, s)] = x[ci, p*st+r-pad, q*st+s-pad]
+            const int kk = k0 + lo16;
+            const int p = kk / ow, qq = kk - p * ow;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int m = tl.m0 + hi16 + 16 * q;
+                ra[q] = (m < M && kk < ke) ? A[(size_t)m * G.K + kk] : 0.f;
+                const int y = p * st + wr[q] - pad, x = qq * st + ws[q] - pad;
+                rb[q] = (w_ok[q] && kk < ke && y >= 0 && y < ih && x >= 0 && x < iw) ? B[((size_t)wc[q] * ih + y) * iw + x] : 0.f;
+            }
+        }
+        if (bf) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { ra[q] = round_bf16(ra[q]); rb[q] = round_bf16(rb[q]); }
+        }
+        __syncthreads();
+        if (G.mode == kDgrad) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { As[hi4 + 4 * q][lo64] = ra[q]; Bs[hi4 + 4 * q][lo64] = rb[q]; }
+        } else if (G.mode == kFprop) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { As[lo16][hi16 + 16 * q] = ra[q]; Bs[hi4 + 4 * q][lo64] = rb[q]; }
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { As[lo16][hi16 + 16 * q] = ra[q]; Bs[lo16][hi16 + 16 * q] = rb[q]; }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < kBK; ++kk) {
+            const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+            const float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+            const float av[4] = {a4.x, a4.y, a4.z, a4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int m = tl.m0 + ty * 4 + a;
+        if (m >= M) continue;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int n = tl.n0 + tx * 4 + b;
+            if (n < N) Cp[(size_t)m * N + n] = acc[a][b];
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kGemmThreads)
+conv_gemm_kernel(const ConvGemm* __restrict__ gemms, const GemmTile* __restrict__ tiles,
+                 const TickState* __restrict__ ts, int S) {
+    __shared__ __align__(16) float As[kBK][kBM + 4];
+    __shared__ __align__(16) float Bs[kBK][kBN + 4];
+    const GemmTile tl = tiles[blockIdx.x];
+    const ConvGemm& G = gemms[tl.gemm];
+    const long long t = ts->tick;
+    const long long smp = (G.mode == kFprop) ? t - G.s : t - 2LL * (S - 1) + G.s;
+    if (smp < 0) return;
+    switch (G.k) {
+        case 1: gemm_tile<1>(G, tl, smp, As, Bs); break;
+        case 3: gemm_tile<3>(G, tl, smp, As, Bs); break;
+        case 7: gemm_tile<7>(G, tl, smp, As, Bs); break;
+        default: gemm_tile<0>(G, tl, smp, As, Bs); break;
+    }
+}
+
+}  // namespace pb

@@ -1,0 +1,75 @@
+// Device-side descriptors of convolution stages.
+#pragma once
+#include "pb_internal.h"
+
+namespace pb {
+
+constexpr int kGemmThreads = 256;
+constexpr int kBM = 64, kBN = 64, kBK = 16;
+constexpr int kGroupThreads = 256;
+constexpr int kMaxGroupChannels = 64;      // channels per normalisation group
+
+enum GemmMode { kFprop = 0, kDgrad = 1, kWgrad = 2 };
+
+// One implicit GEMM  C[M,N] = sum_k A[m,k] B[k,n]  of a convolution stage.
+//   fprop: M = c_out, N = out pixels, K = c_in*k*k    A = predicted weights, B = im2col(x_fwd)
+//   dgrad: M = c_in,  N = in pixels,  K = c_out*k*k   A = weights (transposed view), B = scattered dz
+//   wgrad: M = c_out, N = c_in*k*k,   K = out pixels  A = dz, B = im2col(x_bwd)^T
+// K is cut into nsplit slices; slice q writes its own partial result
+// c + q*M*N, and the reader adds the slices in order (deterministic split-K).
+struct ConvGemm {
+    int mode, M, N, K;
+    int ci, co, k, stride, pad, ih, iw, oh, ow;
+    int s;                       // stage index (for the tick arithmetic)
+    int bf16;                    // round both operands to bfloat16 before multiplying
+    int nsplit, k_per_split;
+    const float* a;              // fprop: w_hat; dgrad: w; wgrad: dz
+    const float* b;              // fprop/wgrad: ring of the input activations; dgrad: dz
+    int b_slots, b_elems;        // ring geometry of b (1 slot for dz)
+    float* c;                    // [c_slots][nsplit][M*N]
+    int c_slots;
+};
+
+struct GemmTile { int gemm, m0, n0, split; };
+
+// Everything the normalisation / activation / pooling kernels need for one stage.
+struct ConvStage {
+    int s;
+    int co, oh, ow;              // conv output (z) shape
+    int groups, cpg;             // GroupNorm groups, channels per group
+    int relu, avgpool;
+    int pool_k, pool_stride, pool_pad;   // pool_k == 0: no max-pool
+    int out_h, out_w;            // stage output spatial shape (after pooling)
+    // forward
+    const float* zpart; int z_nsplit;    // fprop partial sums [nsplit][co*oh*ow]
+    float* z_ring;               // [slots][co*oh*ow] conv output, kept for the backward
+    float* stat_ring;            // [slots][2*groups] mean, rstd
+    unsigned char* code_ring;    // [slots][co*oh*ow] bit0: ReLU passed
+    unsigned char* arg_ring;     // [slots][co*out_h*out_w] max-pool winner position in its window
+    float* out_ring;             // [slots][co*out_h*out_w]
+    int slots;                   // D_s + 1 (all the rings above)
+    const float* wh;             // predicted parameters: weights, then gamma, then beta
+    const float* w;              // current parameters
+    float* g;                    // gradient buffer, same layout
+    int nw;                      // number of conv weights (offset of gamma)
+    // skip input
+    const float* skip_ring; int skip_slots, skip_mode, skip_c, skip_h, skip_w;   // skip_ring == nullptr: none
+    float* dskip; int dskip_slots;       // gradient handed to the skip source [slots][skip elems]
+    // backward
+    int n_dsrc; DeltaSrc dsrc[kMaxDeltaSrc];
+    float* dz;                   // scratch [co*oh*ow]
+};
+
+// A range of parameters updated together: v <- m v + g, w <- w - lr (a v + b g),
+// w_hat <- w - lr T v, with g the sum of nparts partial gradients.
+struct UpdRange {
+    float *w, *v, *wh;
+    const float* g; int nparts; long long part_stride;
+    int n;
+    int s;
+    float neg_lr_T, m, neg_lr_a, neg_lr_b;
+};
+struct UpdChunk { int range, start; };
+constexpr int kUpdChunk = 4096;
+
+}  // namespace pb

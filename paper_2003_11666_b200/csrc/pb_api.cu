@@ -6,6 +6,8 @@
 #include <cstring>
 #include <new>
 
+#include "conv_gemm.cuh"
+#include "conv_stage.cuh"
 #include "fc_kernels.cuh"
 #include "pb_engine.h"
 
@@ -160,6 +162,117 @@ void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSe
     if (cta_begin.back() != (int)segs.size()) cta_begin.push_back((int)segs.size());
 }
 
+// ---------------------------------------------------------------- convolution planning
+void choose_split(int M, int N, int K, int num_sms, int& nsplit, int& kps) {
+    const int tiles = ceil_div(M, kBM) * ceil_div(N, kBN);
+    int want = ceil_div(num_sms, tiles);
+    int by_k = K / 64;
+    if (by_k < 1) by_k = 1;
+    nsplit = std::max(1, std::min(std::min(want, by_k), 32));
+    kps = ceil_div(ceil_div(K, nsplit), kBK) * kBK;
+    nsplit = ceil_div(K, kps);
+}
+
+void plan_conv(pb_handle* h) {
+    for (StageHost& x : h->stages) {
+        if (x.head_op != PB_CONV2D) continue;
+        const int k2 = x.head.k * x.head.k;
+        choose_split(x.head.c_out, x.z.h * x.z.w, x.head.c_in * k2, h->num_sms, x.split_f, x.kps_f);
+        choose_split(x.head.c_in, x.in.h * x.in.w, x.head.c_out * k2, h->num_sms, x.split_d, x.kps_d);
+        choose_split(x.head.c_out, x.head.c_in * k2, x.z.h * x.z.w, h->num_sms, x.split_w, x.kps_w);
+        x.dx_nparts = x.split_d;
+    }
+}
+
+void add_tiles(std::vector<GemmTile>& tiles, int gemm, int M, int N, int nsplit) {
+    for (int q = 0; q < nsplit; ++q)
+        for (int m0 = 0; m0 < M; m0 += kBM)
+            for (int n0 = 0; n0 < N; n0 += kBN) tiles.push_back(GemmTile{gemm, m0, n0, q});
+}
+
+void fill_conv_tables(pb_handle* h) {
+    h->h_gemms.clear(); h->h_cs.clear(); h->h_map.clear(); h->h_upd.clear(); h->h_chunks.clear();
+    for (auto& t : h->h_tiles) t.clear();
+    const int bf = (h->flags & PB_CONV_BF16) ? 1 : 0;
+    for (const StageHost& x : h->stages) {
+        if (x.head_op != PB_CONV2D) continue;
+        const pb_layer& L = x.head;
+        const int k2 = L.k * L.k, opix = x.z.h * x.z.w, ipix = x.in.h * x.in.w, nw = L.c_out * L.c_in * k2;
+        const float* xin = x.src < 0 ? h->in_ring : h->stages[x.src].out_ring;
+        const int xin_slots = x.src < 0 ? h->in_slots : h->stages[x.src].out_slots;
+        ConvGemm g{};
+        g.ci = L.c_in; g.co = L.c_out; g.k = L.k; g.stride = L.stride; g.pad = L.pad;
+        g.ih = x.in.h; g.iw = x.in.w; g.oh = x.z.h; g.ow = x.z.w; g.s = x.index; g.bf16 = bf;
+        // fprop
+        g.mode = kFprop; g.M = L.c_out; g.N = opix; g.K = L.c_in * k2; g.nsplit = x.split_f; g.k_per_split = x.kps_f;
+        g.a = h->d_wh + x.dev_off; g.b = xin; g.b_slots = xin_slots; g.b_elems = x.in.elems();
+        g.c = x.zpart; g.c_slots = 1;
+        add_tiles(h->h_tiles[0], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
+        h->h_gemms.push_back(g);
+        // dgrad (not for the first stage: nobody needs the gradient of the input)
+        if (x.src >= 0) {
+            g.mode = kDgrad; g.M = L.c_in; g.N = ipix; g.K = L.c_out * k2; g.nsplit = x.split_d; g.k_per_split = x.kps_d;
+            g.a = h->d_w + x.dev_off; g.b = x.dz; g.b_slots = 1; g.b_elems = x.z.elems();
+            g.c = x.dx; g.c_slots = x.dx_slots;
+            add_tiles(h->h_tiles[1], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
+            h->h_gemms.push_back(g);
+        }
+        // wgrad
+        g.mode = kWgrad; g.M = L.c_out; g.N = L.c_in * k2; g.K = opix; g.nsplit = x.split_w; g.k_per_split = x.kps_w;
+        g.a = x.dz; g.b = xin; g.b_slots = xin_slots; g.b_elems = x.in.elems();
+        g.c = x.gpart; g.c_slots = 1;
+        add_tiles(h->h_tiles[2], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
+        h->h_gemms.push_back(g);
+
+        ConvStage c{};
+        c.s = x.index; c.co = L.c_out; c.oh = x.z.h; c.ow = x.z.w;
+        c.groups = x.gn_groups; c.cpg = L.c_out / x.gn_groups;
+        c.relu = x.relu; c.avgpool = x.avgpool;
+        c.pool_k = x.has_pool ? x.pool_k : 0; c.pool_stride = x.pool_stride; c.pool_pad = x.pool_pad;
+        c.out_h = x.out.h; c.out_w = x.out.w;
+        c.zpart = x.zpart; c.z_nsplit = x.split_f;
+        c.z_ring = x.z_ring; c.stat_ring = x.stat_ring; c.code_ring = x.code_ring; c.arg_ring = x.arg_ring;
+        c.out_ring = x.out_ring; c.slots = x.out_slots;
+        c.wh = h->d_wh + x.dev_off; c.w = h->d_w + x.dev_off; c.g = h->d_g + x.dev_off; c.nw = nw;
+        if (x.has_skip) {
+            const StageHost& y = h->stages[x.skip_src];
+            c.skip_ring = y.out_ring; c.skip_slots = y.out_slots; c.skip_mode = x.skip_mode;
+            c.skip_c = y.out.c; c.skip_h = y.out.h; c.skip_w = y.out.w;
+            c.dskip = x.dskip; c.dskip_slots = x.dskip_slots;
+        }
+        c.n_dsrc = 0;
+        for (int q : x.consumers_main) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dx, y.dx_slots, y.dx_nparts}; }
+        for (int q : x.consumers_skip) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dskip, y.dskip_slots, 1}; }
+        c.dz = x.dz;
+        for (int gq = 0; gq < x.gn_groups; ++gq) h->h_map.push_back(make_int2((int)h->h_cs.size(), gq));
+        h->h_cs.push_back(c);
+
+        UpdRange r{};
+        r.s = x.index; r.neg_lr_T = -h->lr * x.T; r.m = h->momentum; r.neg_lr_a = -h->lr * x.a; r.neg_lr_b = -h->lr * x.b;
+        r.w = h->d_w + x.dev_off; r.v = h->d_v + x.dev_off; r.wh = h->d_wh + x.dev_off;
+        r.g = x.gpart; r.nparts = x.split_w; r.part_stride = nw; r.n = nw;
+        for (int st = 0; st < r.n; st += kUpdChunk) h->h_chunks.push_back(UpdChunk{(int)h->h_upd.size(), st});
+        h->h_upd.push_back(r);
+        r.w += nw; r.v += nw; r.wh += nw;
+        r.g = h->d_g + x.dev_off + nw; r.nparts = 1; r.part_stride = 0; r.n = 2 * L.c_out;
+        for (int st = 0; st < r.n; st += kUpdChunk) h->h_chunks.push_back(UpdChunk{(int)h->h_upd.size(), st});
+        h->h_upd.push_back(r);
+    }
+}
+
+int validate_conv(pb_handle* h) {
+    for (const StageHost& x : h->stages) {
+        if (x.head_op != PB_CONV2D) continue;
+        if (x.gn_groups <= 0) return fail(nullptr, PB_E_UNSUPPORTED, "a CONV2D stage needs a GROUPNORM layer");
+        if (x.head.c_out / x.gn_groups > kMaxGroupChannels) return fail(nullptr, PB_E_UNSUPPORTED, "more than 64 channels per normalisation group");
+        if (x.has_pool && x.avgpool) return fail(nullptr, PB_E_UNSUPPORTED, "max-pool and average pool in one stage");
+        if ((int)(x.consumers_main.size() + x.consumers_skip.size()) > kMaxDeltaSrc) return fail(nullptr, PB_E_UNSUPPORTED, "too many consumers of one stage");
+    }
+    for (const StageHost& x : h->stages)
+        if (x.head_op == PB_FC && (x.has_skip || x.has_pool || x.avgpool || x.gn_groups)) return fail(nullptr, PB_E_UNSUPPORTED, "FC stages take only RELU or SOFTMAX_CE");
+    return PB_OK;
+}
+
 __global__ void ingest_kernel(TickState* ts, const float* __restrict__ xs, const int* __restrict__ labels,
                               int label_value, float* __restrict__ in_ring, int in_slots, int elems,
                               int* __restrict__ label_ring, int S, long long t_base) {
@@ -191,9 +304,17 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     h->d_segB = c.take<FcSeg>(h->h_segB.size() + 1);
     h->d_ctaA = c.take<int>(h->h_ctaA.size() + 1);
     h->d_ctaB = c.take<int>(h->h_ctaB.size() + 1);
+    h->d_gemms = c.take<ConvGemm>(h->h_gemms.size() + 1);
+    for (int q = 0; q < 3; ++q) h->d_tiles[q] = c.take<GemmTile>(h->h_tiles[q].size() + 1);
+    h->d_cs = c.take<ConvStage>(h->h_cs.size() + 1);
+    h->d_map = c.take<int2>(h->h_map.size() + 1);
+    h->d_upd = c.take<UpdRange>(h->h_upd.size() + 1);
+    h->d_chunks = c.take<UpdChunk>(h->h_chunks.size() + 1);
     h->d_w = c.take<float>(h->dev_params);
+    if (!h->all_fc) h->d_wh = c.take<float>(h->dev_params);
     *zero_from = c.off;
     h->d_v = c.take<float>(h->dev_params);
+    if (!h->all_fc) h->d_g = c.take<float>(h->dev_params);
     h->in_slots = 2 * (h->S - 1) + 1;
     h->in_ring = c.take<float>((size_t)h->in_slots * h->in_shape.elems());
     h->label_ring = c.take<int>(h->S);
@@ -208,6 +329,16 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
         if (x.has_skip) {
             x.dskip_slots = x.index - x.skip_src + 1;
             x.dskip = c.take<float>((size_t)x.dskip_slots * h->stages[x.skip_src].out.elems());
+        }
+        if (x.head_op == PB_CONV2D) {
+            const size_t ze = x.z.elems(), nw = (size_t)x.head.c_out * x.head.c_in * x.head.k * x.head.k;
+            x.z_ring = c.take<float>((size_t)x.out_slots * ze);
+            x.stat_ring = c.take<float>((size_t)x.out_slots * 2 * x.gn_groups);
+            x.code_ring = c.take<unsigned char>((size_t)x.out_slots * ze);
+            x.arg_ring = x.has_pool ? c.take<unsigned char>((size_t)x.out_slots * x.out.elems()) : nullptr;
+            x.zpart = c.take<float>((size_t)x.split_f * ze);
+            x.dz = c.take<float>(ze);
+            x.gpart = c.take<float>((size_t)x.split_w * nw);
         }
     }
     return c.off;
@@ -285,7 +416,28 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             prof_end(h);
             h->last_launches += 2;
         } else {
-            return fail(h, PB_E_UNSUPPORTED, "convolution stages are not built into this library");
+            // forward chain: convolutions -> normalise/activate/pool; FC forward
+            prof_begin(h, 3);
+            conv_gemm_kernel<<<(int)h->h_tiles[0].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[0], h->d_ts, h->S);
+            conv_post_fwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts);
+            // backward chain: through pool/ReLU/GroupNorm -> data and weight gradients
+            conv_post_bwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts, h->S);
+            if (!h->h_tiles[1].empty())
+                conv_gemm_kernel<<<(int)h->h_tiles[1].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[1], h->d_ts, h->S);
+            conv_gemm_kernel<<<(int)h->h_tiles[2].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[2], h->d_ts, h->S);
+            prof_end(h);
+            prof_begin(h, 2);
+            update_kernel<<<(int)h->h_chunks.size(), 256, 0, h->stream>>>(h->d_upd, h->d_chunks, h->d_ts, h->S);
+            prof_end(h);
+            prof_begin(h, 0);
+            fc_tick_kernel<<<h->nctaA, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segA, h->d_ctaA, h->d_ts, h->S, 0,
+                                                                  h->label_ring, dev_losses, t_base);
+            prof_end(h);
+            prof_begin(h, 1);
+            fc_tick_kernel<<<h->nctaB, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segB, h->d_ctaB, h->d_ts, h->S, 1,
+                                                                  h->label_ring, dev_losses, t_base);
+            prof_end(h);
+            h->last_launches += (h->h_tiles[1].empty() ? 7 : 8);
         }
     }
     PB_CUDA(h, cudaGetLastError());
@@ -354,6 +506,10 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     h->nctaA = (int)h->h_ctaA.size() - 1;
     h->nctaB = (int)h->h_ctaB.size() - 1;
 
+    rc = validate_conv(h);
+    if (rc != PB_OK) { delete h; return rc; }
+    plan_conv(h);
+    fill_conv_tables(h);     // sizes only; pointers are filled in after the layout
     size_t zero_from = 0;
     h->arena_bytes = layout(h, nullptr, &zero_from);
     e = cudaMalloc((void**)&h->arena, h->arena_bytes);
@@ -364,6 +520,7 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     layout(h, h->arena, &zero_from);
     h->zero_from = zero_from;
     fill_fc_tables(h);
+    fill_conv_tables(h);
     e = cudaMemsetAsync(h->arena, 0, h->arena_bytes, h->stream);
     auto up = [&](void* d, const void* s, size_t n) { if (e == cudaSuccess && n) e = cudaMemcpyAsync(d, s, n, cudaMemcpyHostToDevice, h->stream); };
     up(h->d_fc, h->h_fc.data(), h->h_fc.size() * sizeof(FcStage));
@@ -371,6 +528,12 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     up(h->d_segB, h->h_segB.data(), h->h_segB.size() * sizeof(FcSeg));
     up(h->d_ctaA, h->h_ctaA.data(), h->h_ctaA.size() * sizeof(int));
     up(h->d_ctaB, h->h_ctaB.data(), h->h_ctaB.size() * sizeof(int));
+    up(h->d_gemms, h->h_gemms.data(), h->h_gemms.size() * sizeof(ConvGemm));
+    for (int q = 0; q < 3; ++q) up(h->d_tiles[q], h->h_tiles[q].data(), h->h_tiles[q].size() * sizeof(GemmTile));
+    up(h->d_cs, h->h_cs.data(), h->h_cs.size() * sizeof(ConvStage));
+    up(h->d_map, h->h_map.data(), h->h_map.size() * sizeof(int2));
+    up(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange));
+    up(h->d_chunks, h->h_chunks.data(), h->h_chunks.size() * sizeof(UpdChunk));
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
     if (e != cudaSuccess) {
         std::string m = std::string("pb_create: upload failed: ") + cudaGetErrorString(e);
@@ -387,6 +550,8 @@ int pb_set_weights(pb_handle* h, const float* host_w, size_t n) {
     PB_CUDA(h, cudaMemsetAsync(h->d_ts, 0, sizeof(TickState), h->stream));
     for (const StageHost& x : h->stages)
         PB_CUDA(h, cudaMemcpyAsync(h->d_w + x.dev_off, host_w + x.user_off, x.n_params * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+    // zero velocity: the predicted weights start equal to the weights
+    if (h->d_wh) PB_CUDA(h, cudaMemcpyAsync(h->d_wh, h->d_w, h->dev_params * sizeof(float), cudaMemcpyDeviceToDevice, h->stream));
     PB_CUDA(h, cudaStreamSynchronize(h->stream));
     h->tick = 0;
     return PB_OK;

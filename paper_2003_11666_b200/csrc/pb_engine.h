@@ -5,6 +5,7 @@
 
 #include "../../include/pb.h"
 #include "pb_internal.h"
+#include "conv_types.h"
 
 namespace pb {
 
@@ -32,6 +33,11 @@ struct StageHost {
     float* dx = nullptr; int dx_slots = 0, dx_nparts = 1;          // gradient w.r.t. main input
     float* dskip = nullptr; int dskip_slots = 0;                   // gradient w.r.t. skip input
     std::vector<int> consumers_main, consumers_skip;               // stages reading this output
+    // convolution stages only
+    float *z_ring = nullptr, *stat_ring = nullptr, *zpart = nullptr, *dz = nullptr, *gpart = nullptr;
+    unsigned char *code_ring = nullptr, *arg_ring = nullptr;
+    int split_f = 1, split_d = 1, split_w = 1;                     // K-slices of fprop / dgrad / wgrad
+    int kps_f = 0, kps_d = 0, kps_w = 0;                           // K per slice
 };
 
 struct ProfileClass { double ms = 0; long long launches = 0; };
@@ -65,6 +71,14 @@ struct pb_handle {
     std::vector<pb::FcStage> h_fc;
     std::vector<pb::FcSeg> h_segA, h_segB;
     std::vector<int> h_ctaA, h_ctaB;
+    // convolution tables
+    float *d_wh = nullptr, *d_g = nullptr;
+    std::vector<pb::ConvGemm> h_gemms; pb::ConvGemm* d_gemms = nullptr;
+    std::vector<pb::GemmTile> h_tiles[3]; pb::GemmTile* d_tiles[3] = {nullptr, nullptr, nullptr};
+    std::vector<pb::ConvStage> h_cs; pb::ConvStage* d_cs = nullptr;
+    std::vector<int2> h_map; int2* d_map = nullptr;
+    std::vector<pb::UpdRange> h_upd; pb::UpdRange* d_upd = nullptr;
+    std::vector<pb::UpdChunk> h_chunks; pb::UpdChunk* d_chunks = nullptr;
 
     long long tick = 0, last_launches = 0;
     bool profile = false;

@@ -157,3 +157,40 @@ def test_fc_backward_fd():
     np.testing.assert_allclose(dx, _fd(f, x), rtol=1e-7, atol=1e-9)
     np.testing.assert_allclose(gW, _fd(f, W), rtol=1e-7, atol=1e-9)
     np.testing.assert_allclose(gb, _fd(f, b), rtol=1e-7, atol=1e-9)
+
+
+def test_round_bf16_matches_torch_and_ties_to_even():
+    rng = np.random.default_rng(9)
+    x = np.concatenate([rng.standard_normal(5000) * 10.0 ** rng.integers(-6, 6, 5000),
+                        [0.0, -0.0, 1.0, 1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, 1.0 + 2 ** -7, -1.0 - 2 ** -8]])
+    got = L.round_bf16(x)
+    ref = torch.tensor(x, dtype=torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(got, ref)
+    # 1 + 2^-8 lies half-way between 1 and 1 + 2^-7: the even mantissa (1.0) wins;
+    # 1 + 3*2^-8 lies half-way between 1 + 2^-7 and 1 + 2^-6: the even one is 1 + 2^-6
+    assert L.round_bf16(np.array([1.0 + 2 ** -8]))[0] == 1.0
+    assert L.round_bf16(np.array([1.0 + 3 * 2 ** -8]))[0] == 1.0 + 2 ** -6
+    assert got.dtype == x.dtype
+
+
+def test_conv_with_rounded_operands_is_conv_of_rounded_operands():
+    rng = np.random.default_rng(10)
+    x, W = rng.standard_normal((3, 6, 6)), rng.standard_normal((4, 3, 3, 3))
+    dz = rng.standard_normal((4, 3, 3))
+    z = L.conv2d_forward(W, x, 2, 1, L.round_bf16)
+    zt = F.conv2d(torch.tensor(L.round_bf16(x))[None], torch.tensor(L.round_bf16(W)), stride=2, padding=1)[0]
+    np.testing.assert_allclose(z, zt.numpy(), rtol=1e-12, atol=1e-12)
+    dx, gW = L.conv2d_backward(W, x, dz, 2, 1, L.round_bf16)
+    dx0, gW0 = L.conv2d_backward(L.round_bf16(W), L.round_bf16(x), L.round_bf16(dz), 2, 1)
+    np.testing.assert_array_equal(dx, dx0)
+    np.testing.assert_array_equal(gW, gW0)
+    assert np.abs(z - L.conv2d_forward(W, x, 2, 1)).max() > 1e-4
+
+
+def test_maxpool_gap_reports_the_closest_call():
+    x = np.array([[[1.0, 0.5, 3.0, 2.75], [0.25, 0.0, 1.0, 0.0]]])
+    y, arg, gap = L.maxpool_forward(x, 2, 2, 0, want_gap=True)
+    np.testing.assert_array_equal(y[0, 0], [1.0, 3.0])
+    assert gap == 0.25
+    _, _, gap0 = L.maxpool_forward(np.zeros((1, 2, 2)), 2, 2, 0, want_gap=True)
+    assert gap0 == float("inf")          # no positive maximum: nothing can flip a gradient
