@@ -105,11 +105,12 @@ int pb_tick(pb_handle* h, const float* dev_x, int label, float* host_loss);
 
 /* n_ticks ticks without host synchronisation.  dev_xs: [n_ticks, sample]
  * floats, dev_labels: [n_ticks] int32, both device memory that must stay
- * valid and unchanged until the stream has run the ticks AND for the next
- * 2(S-1) ticks' worth of calls (stage 0 re-reads a sample at its backward);
- * dev_losses: [n_ticks] floats (device) or NULL.  Continues from the current
- * tick; may be called repeatedly with consecutive batches only if the earlier
- * batches stay alive as stated. */
+ * valid and unchanged until the stream has run the ticks (each sample and label
+ * is copied into the engine's rings at its tick, because stage 0 reads the
+ * sample again at its backward 2(S-1) ticks later); dev_losses: [n_ticks]
+ * floats (device) or NULL, entry k receiving what pb_tick would have returned
+ * at the k-th tick of this call.  Continues from the current tick, so
+ * consecutive calls feed one continuous stream of samples. */
 int pb_run(pb_handle* h, const float* dev_xs, const int32_t* dev_labels,
            int n_ticks, float* dev_losses);
 
@@ -145,6 +146,37 @@ size_t pb_device_bytes(const pb_handle* h);
  * or never run; *launches receives the number of launches timed. */
 int pb_profile_enable(pb_handle* h, int enable);
 double pb_profile_ms(pb_handle* h, int which, long long* launches);
+
+/* Allocation-free variant of pb_create + pb_set_weights + pb_run for small fully
+ * connected pipelines.  (The paper has no counterpart: this exists for callers
+ * that must not allocate device memory - code running inside a pre-sized memory
+ * budget, under another framework's caching allocator whose pool must not be
+ * disturbed, or in a phase where cudaMalloc's implicit device synchronisation
+ * is not acceptable.)
+ *
+ * Runs n_ticks ticks of PB + SC + LWP on the MLP sizes[0] -> ... ->
+ * sizes[n_sizes-1] (ReLU between, softmax cross-entropy last; one stage per FC
+ * layer, 1..16 stages), starting from an empty pipeline.  The caller passes
+ * every input and output as device memory: dev_w / dev_v are the master
+ * weights and velocities (flat, layer-list order, pb_num_params layout; read
+ * and updated in place; zero dev_v for a fresh start), dev_xs [n_ticks,
+ * sizes[0]], dev_labels [n_ticks], dev_losses [n_ticks] or NULL.  Everything
+ * else the tick kernels need (tick state, stage tables, activation rings,
+ * gradient hand-off rows) lives in one static 4 MiB device array inside the
+ * library, which every GPU that loads the library holds until the process
+ * exits.  A network whose scratch exceeds 4 MiB is rejected with PB_E_ARG and a
+ * message giving the size.  No cudaMalloc, cudaFree or other allocating device
+ * call is made; host-side bookkeeping uses ordinary heap memory.
+ *
+ * The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress) and should therefore come before any stream capture.
+ * All calls share the array and it keeps the previous call's contents: each
+ * call clears the part it uses, and two calls that overlap on the GPU (other
+ * streams, other threads) race on it.  The call waits for `stream` before it
+ * returns.  Errors: status code, text via pb_last_error(NULL). */
+int pb_mlp_run_static(const int32_t* sizes, int n_sizes, float lr, float momentum, unsigned flags,
+                      float* dev_w, float* dev_v, const float* dev_xs, const int32_t* dev_labels,
+                      int n_ticks, float* dev_losses, void* stream);
 
 const char* pb_last_error(const pb_handle* h);
 void pb_destroy(pb_handle* h);

@@ -19,7 +19,7 @@ EXPORTS = [
     "pb_create", "pb_set_weights", "pb_tick", "pb_run", "pb_run_host", "pb_get_weights",
     "pb_get_velocity", "pb_sync", "pb_num_params", "pb_num_stages", "pb_stage_delay",
     "pb_tick_count", "pb_last_launch_count", "pb_device_bytes", "pb_profile_enable",
-    "pb_profile_ms", "pb_last_error", "pb_destroy",
+    "pb_profile_ms", "pb_last_error", "pb_destroy", "pb_mlp_run_static",
 ]
 
 
@@ -73,6 +73,7 @@ def load_library():
     lib.pb_last_error.restype = C.c_char_p
     lib.pb_destroy.argtypes = [vp]
     lib.pb_destroy.restype = None
+    lib.pb_mlp_run_static.argtypes = [C.POINTER(C.c_int32), i32, f32, f32, C.c_uint, vp, vp, vp, vp, i32, vp, vp]
     _lib = lib
     return lib
 
@@ -86,6 +87,20 @@ def _ptr(a):
     if isinstance(a, np.ndarray):
         return a.ctypes.data
     return a.data_ptr()     # torch.Tensor
+
+
+def mlp_run_static(sizes, lr, momentum, flags, dev_w, dev_v, dev_xs, dev_labels, n_ticks,
+                   dev_losses=None, stream=0):
+    """pb_mlp_run_static: PB ticks of a small MLP without any device allocation
+    (for callers that may not allocate: the scratch is a static array in the
+    library).  All tensors are device memory owned by the caller."""
+    lib = load_library()
+    arr = (C.c_int32 * len(sizes))(*[int(s) for s in sizes])
+    rc = lib.pb_mlp_run_static(arr, len(sizes), float(lr), float(momentum), int(flags), _ptr(dev_w),
+                               _ptr(dev_v), _ptr(dev_xs), _ptr(dev_labels), int(n_ticks),
+                               _ptr(dev_losses), C.c_void_p(stream))
+    if rc != 0:
+        raise PBError(rc, lib.pb_last_error(None).decode())
 
 
 class PB:

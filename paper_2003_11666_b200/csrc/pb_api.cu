@@ -647,3 +647,126 @@ void pb_destroy(pb_handle* h) {
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------- allocation-free entry point
+namespace {
+
+constexpr size_t kStaticScratchBytes = 4u << 20;   // 4 MiB, held by every GPU that loads the library
+constexpr int kStaticMaxStages = 16;
+constexpr int kStaticMaxDevices = 64;
+
+// Scratch of pb_mlp_run_static: tick state, stage tables, activation rings and
+// gradient hand-off buffers are carved out of this array instead of cudaMalloc'd
+// memory.  In host code this name is only a handle for the runtime, not a
+// device address: the address is looked up once per device below.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+void* g_static_scratch_addr[kStaticMaxDevices] = {nullptr};
+
+}  // namespace
+
+extern "C" int pb_mlp_run_static(const int32_t* sizes, int n_sizes, float lr, float momentum, unsigned flags,
+                                 float* dev_w, float* dev_v, const float* dev_xs, const int32_t* dev_labels,
+                                 int n_ticks, float* dev_losses, void* stream) {
+    if (!sizes || !dev_w || !dev_v || !dev_xs || !dev_labels || n_ticks < 0)
+        return fail(nullptr, PB_E_ARG, "pb_mlp_run_static: NULL pointer or negative tick count");
+    if (n_sizes < 2 || n_sizes > kStaticMaxStages + 1)
+        return fail(nullptr, PB_E_ARG, "pb_mlp_run_static: between 1 and 16 FC stages are supported");
+    if (!(momentum >= 0.f && momentum < 1.f) || !(lr >= 0.f) || (flags & ~(unsigned)(PB_SC | PB_LWP)))
+        return fail(nullptr, PB_E_ARG, "pb_mlp_run_static: need 0 <= momentum < 1, lr >= 0, flags within PB_SC|PB_LWP");
+    pb_layer layers[2 * kStaticMaxStages];
+    int32_t stage_of[2 * kStaticMaxStages];
+    int nl = 0;
+    for (int q = 0; q + 1 < n_sizes; ++q) {
+        if (sizes[q] <= 0 || sizes[q + 1] <= 0) return fail(nullptr, PB_E_ARG, "pb_mlp_run_static: layer sizes must be positive");
+        pb_layer fc{}; fc.op = PB_FC; fc.c_in = sizes[q]; fc.c_out = sizes[q + 1]; fc.src = -1;
+        pb_layer tail{}; tail.op = (q + 2 == n_sizes) ? PB_SOFTMAX_CE : PB_RELU; tail.src = -1;
+        layers[nl] = fc; stage_of[nl++] = q;
+        layers[nl] = tail; stage_of[nl++] = q;
+    }
+    pb_handle hs;                       // host bookkeeping only; owns no device memory
+    pb_handle* h = &hs;
+    h->stream = (cudaStream_t)stream;
+    h->flags = flags; h->lr = lr; h->momentum = momentum; h->n_classes = sizes[n_sizes - 1];
+    h->in_shape = Shape{sizes[0], 1, 1};
+    int rc = parse_layers(h, layers, nl, stage_of);
+    if (rc != PB_OK) return rc;
+    schedule_constants(h);
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
+    if (e != cudaSuccess) return fail(nullptr, PB_E_CUDA, std::string("pb_mlp_run_static: no CUDA device: ") + cudaGetErrorString(e));
+    if (h->device < 0 || h->device >= kStaticMaxDevices) return fail(nullptr, PB_E_UNSUPPORTED, "pb_mlp_run_static: device ordinal above 63");
+    if (!g_static_scratch_addr[h->device]) {
+        // set-up, once per device, with that device current
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || !p) return fail(nullptr, PB_E_CUDA, std::string("pb_mlp_run_static: cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+        g_static_scratch_addr[h->device] = p;
+    }
+    char* base = static_cast<char*>(g_static_scratch_addr[h->device]);
+
+    // the caller's flat vectors are the master weights and velocities
+    h->d_w = dev_w; h->d_v = dev_v;
+    std::vector<int> idsA, idsB;
+    for (StageHost& x : h->stages) {
+        x.dev_off = x.user_off;
+        FcStage f{};
+        f.in_dim = x.head.c_in; f.out_dim = x.head.c_out; f.s = x.index;
+        f.relu = x.relu; f.is_last = x.loss; f.need_dx = x.src >= 0;
+        const bool aligned = ((reinterpret_cast<uintptr_t>(dev_w + x.user_off) | reinterpret_cast<uintptr_t>(dev_v + x.user_off)) & 15) == 0;
+        f.vec = (f.in_dim % 4 == 0 && aligned) ? 4 : 1;
+        f.neg_lr_T = -lr * x.T; f.m = momentum; f.neg_lr_a = -lr * x.a; f.neg_lr_b = -lr * x.b;
+        idsA.push_back((int)h->h_fc.size());
+        if (x.loss) idsB.push_back((int)h->h_fc.size());
+        h->h_fc.push_back(f);
+    }
+    std::vector<int> npartsA(h->h_fc.size(), 1), npartsB(h->h_fc.size(), 1);
+    partition_fc(h, idsA, h->h_segA, h->h_ctaA, npartsA);
+    partition_fc(h, idsB, h->h_segB, h->h_ctaB, npartsB);
+    for (size_t f = 0; f < h->h_fc.size(); ++f) {
+        StageHost& x = h->stages[h->h_fc[f].s];
+        x.dx_nparts = x.loss ? npartsB[f] : npartsA[f];
+    }
+    h->nctaA = (int)h->h_ctaA.size() - 1;
+    h->nctaB = (int)h->h_ctaB.size() - 1;
+
+    // carve the static array
+    Carver c{base};
+    h->d_ts = c.take<TickState>(1);
+    h->d_fc = c.take<FcStage>(h->h_fc.size());
+    h->d_segA = c.take<FcSeg>(h->h_segA.size());
+    h->d_segB = c.take<FcSeg>(h->h_segB.size());
+    h->d_ctaA = c.take<int>(h->h_ctaA.size());
+    h->d_ctaB = c.take<int>(h->h_ctaB.size());
+    h->in_slots = 2 * (h->S - 1) + 1;
+    h->in_ring = c.take<float>((size_t)h->in_slots * h->in_shape.elems());
+    h->label_ring = c.take<int>(h->S);
+    for (StageHost& x : h->stages) {
+        x.out_slots = x.delay + 1;
+        x.out_ring = c.take<float>((size_t)x.out_slots * x.out.elems());
+        if (x.src >= 0) {
+            x.dx_slots = x.index - x.src + 1;
+            x.dx = c.take<float>((size_t)x.dx_slots * x.dx_nparts * x.in.elems());
+        }
+    }
+    if (c.off > kStaticScratchBytes)
+        return fail(nullptr, PB_E_ARG, "pb_mlp_run_static: this network needs " + std::to_string(c.off) +
+                                           " bytes of scratch, the static array holds " + std::to_string(kStaticScratchBytes));
+    fill_fc_tables(h);
+    // the array keeps the previous call's contents: clear what this call uses
+    e = cudaMemsetAsync(base, 0, c.off, h->stream);
+    auto up = [&](void* d, const void* s, size_t n) { if (e == cudaSuccess && n) e = cudaMemcpyAsync(d, s, n, cudaMemcpyHostToDevice, h->stream); };
+    up(h->d_fc, h->h_fc.data(), h->h_fc.size() * sizeof(FcStage));
+    up(h->d_segA, h->h_segA.data(), h->h_segA.size() * sizeof(FcSeg));
+    up(h->d_segB, h->h_segB.data(), h->h_segB.size() * sizeof(FcSeg));
+    up(h->d_ctaA, h->h_ctaA.data(), h->h_ctaA.size() * sizeof(int));
+    up(h->d_ctaB, h->h_ctaB.data(), h->h_ctaB.size() * sizeof(int));
+    if (e != cudaSuccess) return fail(nullptr, PB_E_CUDA, std::string("pb_mlp_run_static: table upload: ") + cudaGetErrorString(e));
+    h->all_fc = true;
+    if (n_ticks > 0) {
+        rc = run_ticks(h, dev_xs, dev_labels, 0, n_ticks, dev_losses);
+        if (rc != PB_OK) return fail(nullptr, rc, "pb_mlp_run_static: " + h->err);
+    }
+    rc = check_device_error(h);          // waits for the stream; the host tables may go after this
+    if (rc != PB_OK) return fail(nullptr, rc, "pb_mlp_run_static: " + h->err);
+    return PB_OK;
+}
