@@ -133,6 +133,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=64)
     ap.add_argument("--impl", default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default=WORKLOAD,
+                    help="mlp4 | mlp16x2048 (default, the headline) | vgg11 | resnet20 | resnet50")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -153,7 +155,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
         dist.barrier()
-    wl = workload(WORKLOAD)
+    wl = workload(args.workload)
     K, W = args.steps, max(args.warmup, 3)
     S = wl.n_stages
     seed = wl.seed + 1000 * rank            # replicas see different sample streams
@@ -200,16 +202,26 @@ def main():
     kp = min(K, 512)
     eng.run(xd[W:W + kp], yd[W:W + kp], kp, losses[W:W + kp])
     eng.sync()
-    k_ms, k_n = eng.profile_ms(0)
+    classes = {name: eng.profile_ms(c) for c, name in enumerate(("fc_phase0", "fc_phase1", "update", "conv_simt", "conv_tc_fprop",
+                                                               "conv_post_fwd", "conv_post_bwd", "conv_tc_wgrad", "conv_tc_dgrad"))}
     eng.profile_enable(False)
     P = eng.num_params
     p_last = wl.layers[-2].c_in * wl.layers[-2].c_out + wl.layers[-2].c_out
-    alg_bytes = 16.0 * (P - p_last)          # one read and one write of (w, v) per updated parameter
     peak, peak_kind = measured_peaks()
+    all_fc = all(int(L.op) in (0, 3, 7) for L in wl.layers)
+    if all_fc:
+        # one read and one write of (w, v) per parameter updated by the launch
+        k_ms, k_n = classes["fc_phase0"]
+        alg_bytes, kernel = 16.0 * (P - p_last), "fc_tick_kernel(phase 0)"
+    else:
+        # conv parameters: read w, v, g; write w, v, predicted w
+        k_ms, k_n = classes["update"]
+        alg_bytes, kernel = 28.0 * (P - p_last), "update_kernel"
     achieved = alg_bytes / (k_ms / k_n * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "fc_tick_kernel(phase 0)", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_source": peak_kind,
-                "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": k_ms / k_n, "launches_timed": k_n}
+                "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": k_ms / k_n, "launches_timed": k_n,
+                "us_per_tick_by_class": {n: (1e3 * m / kp if c else 0.0) for n, (m, c) in classes.items()}}
 
     # ---- end to end through the host-buffer entry point (pinned memory, copies timed)
     eng.set_weights(he_normal_weights(wl.seed, wl))
@@ -233,12 +245,13 @@ def main():
             cpu, _ = time_oracle(wl, budget_s=15.0, max_ticks=8)
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
                 "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                "dtype": "f32", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "stages": S, "params": P, "batch": 1,
+                "dtype": "bf16" if wl.flags & 8 else "f32", "data": "synthetic",
+                "config": {"workload": args.workload, "stages": S, "params": P, "batch": 1,
                            "parallelism": "replicas x%d" % world if world > 1 else "1 gpu",
                            "l2": "weights+velocity %.0f MB stream from HBM every tick (> 126 MB L2), no flush needed" % (8e-6 * P),
-                           "note": "literal lr 0.005 diverges (losses finite on %d of %d timed ticks); "
-                                   "kernel work does not depend on the values" % (finite_ticks, K)},
+                           "note": "literal hyper-parameters; losses finite on %d of %d timed ticks "
+                                   "(the deep MLP and ResNet-50 runs diverge); kernel work does not depend "
+                                   "on the values" % (finite_ticks, K)},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
                 "roofline": roofline, "cpu_baseline": cpu}
         print(json.dumps(line))

@@ -140,7 +140,9 @@ size_t pb_device_bytes(const pb_handle* h);
 
 /* Timing hooks for benchmarks: device time in milliseconds that the kernel
  * class `which` (0 = FC tick kernel, 1 = last-stage loss/backward kernel,
- * 2 = update kernel, 3 = conv kernels) took over the last pb_run, measured
+ * 2 = update kernel, 3 = float32 conv GEMMs, 4 = tensor-core fprop, 5 = conv
+ * normalise/activate/pool forward, 6 = its backward, 7 = tensor-core wgrad,
+ * 8 = tensor-core dgrad) took over the last pb_run, measured
  * with CUDA events on the engine's stream when enabled (enable != 0 costs a
  * pair of event records per launch).  Returns a negative value when disabled
  * or never run; *launches receives the number of launches timed. */

@@ -14,6 +14,7 @@ constexpr float kGnEps = 1e-5f;
 
 struct GroupShared {
     float red[kGroupThreads / 32];
+    float wp1[kGroupThreads / 32], wp2[kGroupThreads / 32];
     float s1[kMaxGroupChannels], s2[kMaxGroupChannels];
     float bc[4];
 };
@@ -78,6 +79,7 @@ conv_post_fwd_kernel(const ConvStage* __restrict__ stages, const int2* __restric
     const bool pooled = st.pool_k > 0 || st.avgpool;
     const size_t oelems = (size_t)st.co * st.out_h * st.out_w;
     float* __restrict__ out = st.out_ring + (size_t)slot * oelems;
+    __nv_bfloat16* __restrict__ out16 = st.out16 ? st.out16 + (size_t)slot * oelems : nullptr;
     auto act = [&](int e) -> float {
         const int c = c0 + e / hw, p = e % hw;
         float v = fmaf(gam[c] * rstd, z[e] - mean, bet[c]);
@@ -88,7 +90,11 @@ conv_post_fwd_kernel(const ConvStage* __restrict__ stages, const int2* __restric
         const float v = act(e);
         const bool pass = st.relu ? v > 0.f : true;
         code[e] = pass ? 1 : 0;
-        if (!pooled) out[(size_t)c0 * hw + e] = pass ? v : 0.f;
+        if (!pooled) {
+            const float a = pass ? v : 0.f;
+            out[(size_t)c0 * hw + e] = a;
+            if (out16) out16[(size_t)(e % hw) * st.co + c0 + e / hw] = __float2bfloat16_rn(a);
+        }
     }
     if (st.pool_k > 0) {
         // 4a. max-pool: first maximum in row-major window order; padding never wins
@@ -107,6 +113,7 @@ conv_post_fwd_kernel(const ConvStage* __restrict__ stages, const int2* __restric
                     if (v > best) { best = v; bpos = r * k + s; }
                 }
             out[(size_t)c0 * ohw + o] = best;
+            if (out16) out16[(size_t)op * st.co + c0 + cl] = __float2bfloat16_rn(best);
             arg[o] = (unsigned char)bpos;
         }
     } else if (st.avgpool) {
@@ -158,47 +165,62 @@ conv_post_bwd_kernel(const ConvStage* __restrict__ stages, const int2* __restric
     const int ohw = st.out_h * st.out_w;
     const unsigned char* __restrict__ arg = st.pool_k > 0 ? st.arg_ring + (size_t)slot * oelems + (size_t)c0 * ohw : nullptr;
 
-    // 1. gradient w.r.t. the normalised activation, per-channel sums (one warp per channel)
-    for (int cl = warp; cl < cpg; cl += kGroupThreads / 32) {
-        const int c = c0 + cl;
+    // 1. gradient w.r.t. the normalised activation and per-channel sums.  All warps
+    //    stay busy: a channel is shared by `wpc` warps when there are fewer channels
+    //    than warps; their partial sums are combined in a fixed order.
+    constexpr int kWarps = kGroupThreads / 32;
+    const int wpc = cpg < kWarps ? kWarps / cpg : 1;
+    const int cpp = kWarps / wpc;                        // channels per pass
+    for (int base = 0; base < cpg; base += cpp) {
+        const int cl = base + warp / wpc, sub = warp % wpc;
         float a1 = 0.f, a2 = 0.f;
-        const float davg = st.avgpool ? gather_out_delta(st, oelems, c, j) / (float)hw : 0.f;
-        for (int p = lane; p < hw; p += 32) {
-            const int e = cl * hw + p;
-            float d;
-            if (st.avgpool) {
-                d = davg;
-            } else if (st.pool_k > 0) {
-                // every pooling window that contains this element and chose it
-                const int y = p / st.ow, x = p % st.ow, k = st.pool_k, ps = st.pool_stride, pp = st.pool_pad;
-                d = 0.f;
-                for (int r = 0; r < k; ++r) {
-                    const int ty = y + pp - r;
-                    if (ty < 0 || ty % ps) continue;
-                    const int py = ty / ps;
-                    if (py >= st.out_h) continue;
-                    for (int s = 0; s < k; ++s) {
-                        const int tx = x + pp - s;
-                        if (tx < 0 || tx % ps) continue;
-                        const int px = tx / ps;
-                        if (px >= st.out_w) continue;
-                        const int o = cl * ohw + py * st.out_w + px;
-                        if (arg[o] == r * k + s) d += gather_out_delta(st, oelems, (size_t)c0 * ohw + o, j);
+        if (cl < cpg && warp < cpp * wpc) {
+            const int c = c0 + cl;
+            const float davg = st.avgpool ? gather_out_delta(st, oelems, c, j) / (float)hw : 0.f;
+            for (int p = sub * 32 + lane; p < hw; p += 32 * wpc) {
+                const int e = cl * hw + p;
+                float d;
+                if (st.avgpool) {
+                    d = davg;
+                } else if (st.pool_k > 0) {
+                    // every pooling window that contains this element and chose it
+                    const int y = p / st.ow, x = p % st.ow, k = st.pool_k, ps = st.pool_stride, pp = st.pool_pad;
+                    d = 0.f;
+                    for (int r = 0; r < k; ++r) {
+                        const int ty = y + pp - r;
+                        if (ty < 0 || ty % ps) continue;
+                        const int py = ty / ps;
+                        if (py >= st.out_h) continue;
+                        for (int s = 0; s < k; ++s) {
+                            const int tx = x + pp - s;
+                            if (tx < 0 || tx % ps) continue;
+                            const int px = tx / ps;
+                            if (px >= st.out_w) continue;
+                            const int o = cl * ohw + py * st.out_w + px;
+                            if (arg[o] == r * k + s) d += gather_out_delta(st, oelems, (size_t)c0 * ohw + o, j);
+                        }
                     }
+                } else {
+                    d = gather_out_delta(st, oelems, (size_t)c0 * hw + e, j);
                 }
-            } else {
-                d = gather_out_delta(st, oelems, (size_t)c0 * hw + e, j);
+                d = code[e] ? d : 0.f;
+                dz[e] = d;
+                a1 += d;
+                a2 = fmaf(d, (z[e] - mean) * rstd, a2);
             }
-            d = code[e] ? d : 0.f;
-            dz[e] = d;
-            a1 += d;
-            a2 = fmaf(d, (z[e] - mean) * rstd, a2);
         }
         a1 = warp_sum(a1);
         a2 = warp_sum(a2);
-        if (lane == 0) { sh.s1[cl] = a1; sh.s2[cl] = a2; }
+        if (lane == 0) { sh.wp1[warp] = a1; sh.wp2[warp] = a2; }
+        __syncthreads();
+        if (tid < cpp && base + tid < cpg) {
+            float t1 = 0.f, t2 = 0.f;
+            for (int q = 0; q < wpc; ++q) { t1 += sh.wp1[tid * wpc + q]; t2 += sh.wp2[tid * wpc + q]; }
+            sh.s1[base + tid] = t1;
+            sh.s2[base + tid] = t2;
+        }
+        __syncthreads();
     }
-    __syncthreads();
     // 2. gradients of scale and shift; group means with the CURRENT scale
     const float* __restrict__ gam = st.w + st.nw;
     if (tid < cpg) {
@@ -234,7 +256,9 @@ conv_post_bwd_kernel(const ConvStage* __restrict__ stages, const int2* __restric
     for (int e = tid; e < n; e += kGroupThreads) {
         const int c = c0 + e / hw;
         const float zh = (z[e] - mean) * rstd;
-        dz[e] = rstd * (fmaf(dz[e], gam[c], -m1) - zh * m2);
+        const float d = rstd * (fmaf(dz[e], gam[c], -m1) - zh * m2);
+        dz[e] = d;
+        if (st.dz16) st.dz16[(size_t)(e % hw) * st.co + c] = __float2bfloat16_rn(d);
     }
 }
 
@@ -256,9 +280,25 @@ update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ 
         const float w = R.w[e], v = R.v[e];
         const float vn = fmaf(R.m, v, g);
         const float wn = fmaf(R.neg_lr_a, vn, fmaf(R.neg_lr_b, g, w));
+        const float wh = fmaf(R.neg_lr_T, vn, wn);
         R.v[e] = vn;
         R.w[e] = wn;
-        R.wh[e] = fmaf(R.neg_lr_T, vn, wn);
+        R.wh[e] = wh;
+        if (R.w16) { R.w16[e] = __float2bfloat16_rn(wn); R.wh16[e] = __float2bfloat16_rn(wh); }
+    }
+}
+
+// bfloat16 copies of freshly loaded weights (w_hat = w while the velocity is zero)
+__global__ void __launch_bounds__(256)
+cast_weights_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ chunks) {
+    const UpdChunk ch = chunks[blockIdx.x];
+    const UpdRange& R = ranges[ch.range];
+    if (!R.w16) return;
+    const int end = min(R.n, ch.start + kUpdChunk);
+    for (int e = ch.start + threadIdx.x; e < end; e += 256) {
+        const __nv_bfloat16 b = __float2bfloat16_rn(R.w[e]);
+        R.w16[e] = b;
+        R.wh16[e] = b;
     }
 }
 

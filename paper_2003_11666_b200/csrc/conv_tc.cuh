@@ -1,0 +1,287 @@
+// Tensor-core (tcgen05) implicit GEMM for the bfloat16 convolution path.
+//
+// The three GEMMs of a convolution stage run on the 5th-generation tensor
+// cores: 128 x BN tiles of D accumulate in tensor memory (fp32), operands are
+// bfloat16 and are gathered straight from the NHWC activation ring / gradient
+// scratch / KRSC weight copies into 128-byte-swizzled shared-memory tiles by
+// the block's threads (implicit im2col: no staging buffer in global memory).
+//   fprop  D[c_out, pixel]      A = predicted weights (K-major)   B = im2col(x)      (K-major)
+//   dgrad  D[c_in, in pixel]    A = weights, read transposed (MN-major)  B = scattered dz (K-major)
+//   wgrad  D[c_out, (r,s,c_in)] A = dz (MN-major)                 B = im2col(x)      (MN-major)
+// with K ordered (r, s, channel) so that 8 consecutive K (one 16-byte unit)
+// are 8 consecutive channels of one pixel.  Two shared-memory stages: while
+// the tensor core works on one K-chunk of 64 the threads gather the next.
+// Every mbarrier wait is bounded; on expiry the block records an error, skips
+// its stores, frees its tensor memory and returns.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "conv_types.h"
+
+namespace pb {
+
+constexpr int kTcThreads = 128;
+constexpr int kTcBM = 128;
+constexpr int kTcChunk = 64;                  // K elements per shared-memory stage
+constexpr int kTcStageBytes = 16384 * 2;      // A tile + B tile
+constexpr int kTcSmemBytes = 2 * kTcStageBytes + 1024;
+constexpr int kTcWaitLimit = 1 << 22;
+
+struct ConvGemmTC {
+    int mode, M, N, K;
+    int ci, co, k, stride, pad, ih, iw, oh, ow;
+    int s, bn;                    // stage index; N-tile width (64 or 128)
+    int nsplit, k_per_split;      // k_per_split is a multiple of kTcChunk
+    const __nv_bfloat16* a;       // fprop: predicted weights; dgrad: weights; wgrad: dz (NHWC)
+    const __nv_bfloat16* b;       // fprop/wgrad: NHWC activation ring; dgrad: dz (NHWC)
+    int b_slots, b_elems;
+    float* c;                     // [c_slots][nsplit][M*N]
+    int c_slots;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Shared-memory matrix descriptor: start address, leading/stride byte offsets
+// (all >> 4), descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t tc_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 x bf16, operand
+// majorness, N >> 3 and M >> 4.
+__device__ __forceinline__ uint32_t tc_idesc(int M, int N, int a_mn, int b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t kmajor_off(int row, int unit) {
+    return (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((unit ^ (row & 7)) << 4));
+}
+__device__ __forceinline__ uint32_t mnmajor_off(int k, int mu) {
+    return (uint32_t)((mu >> 3) * 8192 + (k >> 3) * 1024 + (k & 7) * 128 + (((mu & 7) ^ (k & 7)) << 4));
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done = 0;
+    for (int it = 0; it < kTcWaitLimit && !done; ++it) {
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    }
+    return done != 0;
+}
+
+__device__ __forceinline__ uint4 ldg16(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+
+__global__ void __launch_bounds__(kTcThreads)
+conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, TickState* ts, int S) {
+    extern __shared__ unsigned char tc_smem_raw[];
+    __shared__ uint64_t mbar[2];
+    __shared__ uint32_t tmem_base_sh;
+    const GemmTile tl = tiles[blockIdx.x];
+    const ConvGemmTC& G = gemms[tl.gemm];
+    const long long t = ts->tick;
+    const long long smp = (G.mode == kFprop) ? t - G.s : t - 2LL * (S - 1) + G.s;
+    if (smp < 0) return;                                   // uniform: before any allocation
+    unsigned char* smem = (unsigned char*)(((uintptr_t)tc_smem_raw + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int M = G.M, N = G.N, BN = G.bn;
+    const int kb = tl.split * G.k_per_split, ke = min(G.K, kb + G.k_per_split);
+    const int nchunks = (ke - kb + kTcChunk - 1) / kTcChunk;
+    const __nv_bfloat16* __restrict__ A = G.a;
+    const __nv_bfloat16* __restrict__ B = G.b + (size_t)(smp % G.b_slots) * G.b_elems;
+    float* __restrict__ Cp = G.c + ((size_t)(smp % G.c_slots) * G.nsplit + tl.split) * ((size_t)M * N);
+    const int CI = G.ci, CO = G.co, ksz = G.k, st = G.stride, pad = G.pad, ih = G.ih, iw = G.iw, oh = G.oh, ow = G.ow;
+
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(128) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&mbar[0])) : "memory");
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&mbar[1])) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_base_sh;
+    const int a_mn = G.mode != kFprop, b_mn = G.mode == kWgrad;
+    const uint32_t idesc = tc_idesc(kTcBM, BN, a_mn, b_mn);
+
+    // ---- per-thread invariants of the gathers
+    // K-major tiles: this thread fills unit (tid & 7) of rows (tid >> 3) + 16 i, i = 0..7
+    // MN-major tiles of width 128: unit (tid & 15) of k-rows (tid >> 4) + 8 i; width 64: unit (tid & 7) of (tid >> 3) + 16 i (k < 64 -> i < 4)
+    const int ku = tid & 7, krow0 = tid >> 3;
+    int bp[8], bq[8];             // K-major B rows: pixel coordinates (fprop: output pixel; dgrad: input pixel)
+    bool bok[8];
+    if (G.mode != kWgrad) {
+        const int wdt = (G.mode == kFprop) ? ow : iw;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int n = tl.n0 + krow0 + 16 * i;
+            bok[i] = (krow0 + 16 * i) < BN && n < N;
+            bp[i] = n / wdt; bq[i] = n - bp[i] * wdt;
+        }
+    }
+    // wgrad B: this thread's 8 consecutive n = (r, s, ci..ci+7)
+    const int b_units_per_k = BN >> 3;                      // 16 or 8
+    const int bmu = tid % b_units_per_k, bk0 = tid / b_units_per_k, bkstep = kTcThreads / b_units_per_k;
+    int wr = 0, wsx = 0, wci = 0;
+    bool wok = false;
+    if (G.mode == kWgrad) {
+        const int n = tl.n0 + bmu * 8;
+        wok = n < N;
+        const int rs = n / CI; wci = n - rs * CI; wr = rs / ksz; wsx = rs - wr * ksz;
+    }
+    const int amu = tid & 15, ak0 = tid >> 4;               // MN-major A (width 128)
+    const bool a_m_ok = (tl.m0 + amu * 8) < M;
+
+    bool failed = false;
+    for (int c = 0; c < nchunks; ++c) {
+        const int stg = c & 1;
+        unsigned char* sA = smem + stg * kTcStageBytes;
+        unsigned char* sB = sA + 16384;
+        if (c >= 2) {
+            // the MMAs of chunk c-2 read this stage: wait until they are done
+            if (!mbar_wait(smem_u32(&mbar[stg]), (uint32_t)(((c >> 1) - 1) & 1))) failed = true;
+        }
+        const int k0 = kb + c * kTcChunk;
+        // ---------------- A tile
+        if (G.mode == kFprop) {
+            const int k = k0 + ku * 8;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int row = krow0 + 16 * i, m = tl.m0 + row;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (m < M && k < ke) v = ldg16(A + (size_t)m * G.K + k);
+                *reinterpret_cast<uint4*>(sA + kmajor_off(row, ku)) = v;
+            }
+        } else if (G.mode == kDgrad) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int kl = ak0 + 8 * i, k = k0 + kl;          // k = rs * CO + co
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (a_m_ok && k < ke) {
+                    const int rs = k / CO, co = k - rs * CO;
+                    v = ldg16(A + ((size_t)co * (ksz * ksz) + rs) * CI + tl.m0 + amu * 8);
+                }
+                *reinterpret_cast<uint4*>(sA + mnmajor_off(kl, amu)) = v;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int kl = ak0 + 8 * i, k = k0 + kl;          // k = output pixel
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (a_m_ok && k < ke) v = ldg16(A + (size_t)k * CO + tl.m0 + amu * 8);
+                *reinterpret_cast<uint4*>(sA + mnmajor_off(kl, amu)) = v;
+            }
+        }
+        // ---------------- B tile
+        if (G.mode == kFprop) {
+            const int k = k0 + ku * 8;
+            const int rs = k / CI, ci = k - rs * CI, r = rs / ksz, s = rs - r * ksz;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int row = krow0 + 16 * i;
+                if (row >= BN) break;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                const int y = bp[i] * st + r - pad, x = bq[i] * st + s - pad;
+                if (bok[i] && k < ke && y >= 0 && y < ih && x >= 0 && x < iw) v = ldg16(B + ((size_t)y * iw + x) * CI + ci);
+                *reinterpret_cast<uint4*>(sB + kmajor_off(row, ku)) = v;
+            }
+        } else if (G.mode == kDgrad) {
+            const int k = k0 + ku * 8;
+            const int rs = k / CO, co = k - rs * CO, r = rs / ksz, s = rs - r * ksz;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int row = krow0 + 16 * i;
+                if (row >= BN) break;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                const int ty = bp[i] + pad - r, tx = bq[i] + pad - s;
+                if (bok[i] && k < ke && ty >= 0 && tx >= 0) {
+                    const int p = ty / st, q = tx / st;
+                    if (p * st == ty && q * st == tx && p < oh && q < ow) v = ldg16(B + ((size_t)p * ow + q) * CO + co);
+                }
+                *reinterpret_cast<uint4*>(sB + kmajor_off(row, ku)) = v;
+            }
+        } else {
+            for (int kl = bk0; kl < kTcChunk; kl += bkstep) {
+                const int k = k0 + kl;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (wok && k < ke) {
+                    const int p = k / ow, q = k - p * ow;
+                    const int y = p * st + wr - pad, x = q * st + wsx - pad;
+                    if (y >= 0 && y < ih && x >= 0 && x < iw) v = ldg16(B + ((size_t)y * iw + x) * CI + wci);
+                }
+                *reinterpret_cast<uint4*>(sB + mnmajor_off(kl, bmu)) = v;
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (__syncthreads_or(failed)) { failed = true; break; }
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+            for (int j = 0; j < kTcChunk / 16; ++j) {
+                const uint64_t da = a_mn ? tc_desc(smem_u32(sA) + j * 2048, 8192, 1024) : tc_desc(smem_u32(sA) + j * 32, 16, 1024);
+                const uint64_t db = b_mn ? tc_desc(smem_u32(sB) + j * 2048, 8192, 1024) : tc_desc(smem_u32(sB) + j * 32, 16, 1024);
+                const uint32_t acc = (c > 0 || j > 0) ? 1u : 0u;
+                asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+                             "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                             ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+            }
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&mbar[stg])) : "memory");
+        }
+    }
+    // the last commit covers every MMA issued before it
+    if (!failed && nchunks > 0) {
+        const int last = nchunks - 1;
+        if (!mbar_wait(smem_u32(&mbar[last & 1]), (uint32_t)((last >> 1) & 1))) failed = true;
+    }
+    failed = __syncthreads_or(failed);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (!failed) {
+        // epilogue: warp w reads lanes 32w..32w+31 (rows of D), 32 columns per load
+        const int m = tl.m0 + warp * 32 + lane;
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+            if (tl.n0 + c0 >= N) break;                         // uniform
+            uint32_t r[32];
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                         "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+                           "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+                           "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+                           "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                         : "r"(taddr) : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (m < M) {
+                float* dst = Cp + (size_t)m * N + tl.n0 + c0;
+                const int nleft = N - (tl.n0 + c0);
+                if (nleft >= 32 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        reinterpret_cast<float4*>(dst)[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                                                        __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 32; ++q)
+                        if (q < nleft) dst[q] = __uint_as_float(r[q]);
+                }
+            }
+        }
+    } else if (tid == 0) {
+        ts->error = kErrWait;
+        ts->error_info = tl.gemm;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(128) : "memory");
+}
+
+}  // namespace pb

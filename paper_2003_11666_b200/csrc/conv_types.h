@@ -1,12 +1,14 @@
 // Device-side descriptors of convolution stages.
 #pragma once
+#include <cuda_bf16.h>
+
 #include "pb_internal.h"
 
 namespace pb {
 
 constexpr int kGemmThreads = 256;
 constexpr int kBM = 64, kBN = 64, kBK = 16;
-constexpr int kGroupThreads = 256;
+constexpr int kGroupThreads = 1024;
 constexpr int kMaxGroupChannels = 64;      // channels per normalisation group
 
 enum GemmMode { kFprop = 0, kDgrad = 1, kWgrad = 2 };
@@ -47,6 +49,7 @@ struct ConvStage {
     unsigned char* code_ring;    // [slots][co*oh*ow] bit0: ReLU passed
     unsigned char* arg_ring;     // [slots][co*out_h*out_w] max-pool winner position in its window
     float* out_ring;             // [slots][co*out_h*out_w]
+    __nv_bfloat16* out16;        // [slots][out_h*out_w][co] bfloat16 NHWC copy for the tensor-core path (or nullptr)
     int slots;                   // D_s + 1 (all the rings above)
     const float* wh;             // predicted parameters: weights, then gamma, then beta
     const float* w;              // current parameters
@@ -58,12 +61,14 @@ struct ConvStage {
     // backward
     int n_dsrc; DeltaSrc dsrc[kMaxDeltaSrc];
     float* dz;                   // scratch [co*oh*ow]
+    __nv_bfloat16* dz16;         // scratch [oh*ow][co] bfloat16 NHWC copy (or nullptr)
 };
 
 // A range of parameters updated together: v <- m v + g, w <- w - lr (a v + b g),
 // w_hat <- w - lr T v, with g the sum of nparts partial gradients.
 struct UpdRange {
     float *w, *v, *wh;
+    __nv_bfloat16 *w16, *wh16;   // bfloat16 copies of w and w_hat in the same order (or nullptr)
     const float* g; int nparts; long long part_stride;
     int n;
     int s;

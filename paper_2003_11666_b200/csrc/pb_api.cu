@@ -173,10 +173,32 @@ void choose_split(int M, int N, int K, int num_sms, int& nsplit, int& kps) {
     nsplit = ceil_div(K, kps);
 }
 
+void choose_split_tc(int M, int N, int bn, int K, int num_sms, int& nsplit, int& kps) {
+    const int tiles = ceil_div(M, kTcBM) * ceil_div(N, bn);
+    int want = ceil_div(2 * num_sms, tiles);
+    int by_k = K / (2 * kTcChunk);
+    if (by_k < 1) by_k = 1;
+    nsplit = std::max(1, std::min(std::min(want, by_k), 16));
+    kps = ceil_div(ceil_div(K, nsplit), kTcChunk) * kTcChunk;
+    nsplit = ceil_div(K, kps);
+}
+
+int tc_bn(int N) { return N <= 64 ? 64 : 128; }
+
 void plan_conv(pb_handle* h) {
     for (StageHost& x : h->stages) {
         if (x.head_op != PB_CONV2D) continue;
         const int k2 = x.head.k * x.head.k;
+        x.tc = (h->flags & PB_CONV_BF16) && x.src >= 0 && x.head.c_in % 8 == 0 && x.head.c_out % 8 == 0 &&
+               h->stages[x.src].head_op == PB_CONV2D;
+        if (x.tc) {
+            const int opix = x.z.h * x.z.w, ipix = x.in.h * x.in.w;
+            choose_split_tc(x.head.c_out, opix, tc_bn(opix), x.head.c_in * k2, h->num_sms, x.split_f, x.kps_f);
+            choose_split_tc(x.head.c_in, ipix, tc_bn(ipix), x.head.c_out * k2, h->num_sms, x.split_d, x.kps_d);
+            choose_split_tc(x.head.c_out, x.head.c_in * k2, tc_bn(x.head.c_in * k2), opix, h->num_sms, x.split_w, x.kps_w);
+            x.dx_nparts = x.split_d;
+            continue;
+        }
         choose_split(x.head.c_out, x.z.h * x.z.w, x.head.c_in * k2, h->num_sms, x.split_f, x.kps_f);
         choose_split(x.head.c_in, x.in.h * x.in.w, x.head.c_out * k2, h->num_sms, x.split_d, x.kps_d);
         choose_split(x.head.c_out, x.head.c_in * k2, x.z.h * x.z.w, h->num_sms, x.split_w, x.kps_w);
@@ -184,15 +206,16 @@ void plan_conv(pb_handle* h) {
     }
 }
 
-void add_tiles(std::vector<GemmTile>& tiles, int gemm, int M, int N, int nsplit) {
+void add_tiles(std::vector<GemmTile>& tiles, int gemm, int M, int N, int nsplit, int bm = kBM, int bn = kBN) {
     for (int q = 0; q < nsplit; ++q)
-        for (int m0 = 0; m0 < M; m0 += kBM)
-            for (int n0 = 0; n0 < N; n0 += kBN) tiles.push_back(GemmTile{gemm, m0, n0, q});
+        for (int m0 = 0; m0 < M; m0 += bm)
+            for (int n0 = 0; n0 < N; n0 += bn) tiles.push_back(GemmTile{gemm, m0, n0, q});
 }
 
 void fill_conv_tables(pb_handle* h) {
-    h->h_gemms.clear(); h->h_cs.clear(); h->h_map.clear(); h->h_upd.clear(); h->h_chunks.clear();
+    h->h_gemms.clear(); h->h_cs.clear(); h->h_map.clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear();
     for (auto& t : h->h_tiles) t.clear();
+    for (auto& t : h->h_tctiles) t.clear();
     const int bf = (h->flags & PB_CONV_BF16) ? 1 : 0;
     for (const StageHost& x : h->stages) {
         if (x.head_op != PB_CONV2D) continue;
@@ -200,6 +223,33 @@ void fill_conv_tables(pb_handle* h) {
         const int k2 = L.k * L.k, opix = x.z.h * x.z.w, ipix = x.in.h * x.in.w, nw = L.c_out * L.c_in * k2;
         const float* xin = x.src < 0 ? h->in_ring : h->stages[x.src].out_ring;
         const int xin_slots = x.src < 0 ? h->in_slots : h->stages[x.src].out_slots;
+        if (x.tc) {
+            const StageHost& y = h->stages[x.src];
+            ConvGemmTC t{};
+            t.ci = L.c_in; t.co = L.c_out; t.k = L.k; t.stride = L.stride; t.pad = L.pad;
+            t.ih = x.in.h; t.iw = x.in.w; t.oh = x.z.h; t.ow = x.z.w; t.s = x.index;
+            // fprop: D[c_out, out pixel]
+            t.mode = kFprop; t.M = L.c_out; t.N = opix; t.K = L.c_in * k2; t.bn = tc_bn(t.N);
+            t.nsplit = x.split_f; t.k_per_split = x.kps_f;
+            t.a = h->d_wh16 + x.dev_off; t.b = y.out16; t.b_slots = y.out_slots; t.b_elems = x.in.elems();
+            t.c = x.zpart; t.c_slots = 1;
+            add_tiles(h->h_tctiles[0], (int)h->h_tc.size(), t.M, t.N, t.nsplit, kTcBM, t.bn);
+            h->h_tc.push_back(t);
+            // dgrad: D[c_in, in pixel]
+            t.mode = kDgrad; t.M = L.c_in; t.N = ipix; t.K = L.c_out * k2; t.bn = tc_bn(t.N);
+            t.nsplit = x.split_d; t.k_per_split = x.kps_d;
+            t.a = h->d_w16 + x.dev_off; t.b = x.dz16; t.b_slots = 1; t.b_elems = x.z.elems();
+            t.c = x.dx; t.c_slots = x.dx_slots;
+            add_tiles(h->h_tctiles[1], (int)h->h_tc.size(), t.M, t.N, t.nsplit, kTcBM, t.bn);
+            h->h_tc.push_back(t);
+            // wgrad: D[c_out, (r, s, c_in)]
+            t.mode = kWgrad; t.M = L.c_out; t.N = L.c_in * k2; t.K = opix; t.bn = tc_bn(t.N);
+            t.nsplit = x.split_w; t.k_per_split = x.kps_w;
+            t.a = x.dz16; t.b = y.out16; t.b_slots = y.out_slots; t.b_elems = x.in.elems();
+            t.c = x.gpart; t.c_slots = 1;
+            add_tiles(h->h_tctiles[2], (int)h->h_tc.size(), t.M, t.N, t.nsplit, kTcBM, t.bn);
+            h->h_tc.push_back(t);
+        }
         ConvGemm g{};
         g.ci = L.c_in; g.co = L.c_out; g.k = L.k; g.stride = L.stride; g.pad = L.pad;
         g.ih = x.in.h; g.iw = x.in.w; g.oh = x.z.h; g.ow = x.z.w; g.s = x.index; g.bf16 = bf;
@@ -207,21 +257,21 @@ void fill_conv_tables(pb_handle* h) {
         g.mode = kFprop; g.M = L.c_out; g.N = opix; g.K = L.c_in * k2; g.nsplit = x.split_f; g.k_per_split = x.kps_f;
         g.a = h->d_wh + x.dev_off; g.b = xin; g.b_slots = xin_slots; g.b_elems = x.in.elems();
         g.c = x.zpart; g.c_slots = 1;
-        add_tiles(h->h_tiles[0], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
+        if (!x.tc) add_tiles(h->h_tiles[0], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
         h->h_gemms.push_back(g);
         // dgrad (not for the first stage: nobody needs the gradient of the input)
         if (x.src >= 0) {
             g.mode = kDgrad; g.M = L.c_in; g.N = ipix; g.K = L.c_out * k2; g.nsplit = x.split_d; g.k_per_split = x.kps_d;
             g.a = h->d_w + x.dev_off; g.b = x.dz; g.b_slots = 1; g.b_elems = x.z.elems();
             g.c = x.dx; g.c_slots = x.dx_slots;
-            add_tiles(h->h_tiles[1], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
+            if (!x.tc) add_tiles(h->h_tiles[1], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
             h->h_gemms.push_back(g);
         }
         // wgrad
         g.mode = kWgrad; g.M = L.c_out; g.N = L.c_in * k2; g.K = opix; g.nsplit = x.split_w; g.k_per_split = x.kps_w;
         g.a = x.dz; g.b = xin; g.b_slots = xin_slots; g.b_elems = x.in.elems();
         g.c = x.gpart; g.c_slots = 1;
-        add_tiles(h->h_tiles[2], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
+        if (!x.tc) add_tiles(h->h_tiles[2], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
         h->h_gemms.push_back(g);
 
         ConvStage c{};
@@ -233,6 +283,7 @@ void fill_conv_tables(pb_handle* h) {
         c.zpart = x.zpart; c.z_nsplit = x.split_f;
         c.z_ring = x.z_ring; c.stat_ring = x.stat_ring; c.code_ring = x.code_ring; c.arg_ring = x.arg_ring;
         c.out_ring = x.out_ring; c.slots = x.out_slots;
+        c.out16 = x.out16; c.dz16 = x.dz16;
         c.wh = h->d_wh + x.dev_off; c.w = h->d_w + x.dev_off; c.g = h->d_g + x.dev_off; c.nw = nw;
         if (x.has_skip) {
             const StageHost& y = h->stages[x.skip_src];
@@ -251,9 +302,10 @@ void fill_conv_tables(pb_handle* h) {
         r.s = x.index; r.neg_lr_T = -h->lr * x.T; r.m = h->momentum; r.neg_lr_a = -h->lr * x.a; r.neg_lr_b = -h->lr * x.b;
         r.w = h->d_w + x.dev_off; r.v = h->d_v + x.dev_off; r.wh = h->d_wh + x.dev_off;
         r.g = x.gpart; r.nparts = x.split_w; r.part_stride = nw; r.n = nw;
+        if (x.tc) { r.w16 = h->d_w16 + x.dev_off; r.wh16 = h->d_wh16 + x.dev_off; }
         for (int st = 0; st < r.n; st += kUpdChunk) h->h_chunks.push_back(UpdChunk{(int)h->h_upd.size(), st});
         h->h_upd.push_back(r);
-        r.w += nw; r.v += nw; r.wh += nw;
+        r.w += nw; r.v += nw; r.wh += nw; r.w16 = nullptr; r.wh16 = nullptr;
         r.g = h->d_g + x.dev_off + nw; r.nparts = 1; r.part_stride = 0; r.n = 2 * L.c_out;
         for (int st = 0; st < r.n; st += kUpdChunk) h->h_chunks.push_back(UpdChunk{(int)h->h_upd.size(), st});
         h->h_upd.push_back(r);
@@ -310,11 +362,17 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     h->d_map = c.take<int2>(h->h_map.size() + 1);
     h->d_upd = c.take<UpdRange>(h->h_upd.size() + 1);
     h->d_chunks = c.take<UpdChunk>(h->h_chunks.size() + 1);
+    h->d_tc = c.take<ConvGemmTC>(h->h_tc.size() + 1);
+    for (int q = 0; q < 3; ++q) h->d_tctiles[q] = c.take<GemmTile>(h->h_tctiles[q].size() + 1);
     h->d_w = c.take<float>(h->dev_params);
     if (!h->all_fc) h->d_wh = c.take<float>(h->dev_params);
     *zero_from = c.off;
     h->d_v = c.take<float>(h->dev_params);
     if (!h->all_fc) h->d_g = c.take<float>(h->dev_params);
+    if (h->flags & PB_CONV_BF16) {
+        h->d_w16 = c.take<__nv_bfloat16>(h->dev_params);
+        h->d_wh16 = c.take<__nv_bfloat16>(h->dev_params);
+    }
     h->in_slots = 2 * (h->S - 1) + 1;
     h->in_ring = c.take<float>((size_t)h->in_slots * h->in_shape.elems());
     h->label_ring = c.take<int>(h->S);
@@ -339,6 +397,10 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
             x.zpart = c.take<float>((size_t)x.split_f * ze);
             x.dz = c.take<float>(ze);
             x.gpart = c.take<float>((size_t)x.split_w * nw);
+            if (h->flags & PB_CONV_BF16) {
+                x.out16 = c.take<__nv_bfloat16>((size_t)x.out_slots * x.out.elems());
+                x.dz16 = c.take<__nv_bfloat16>(ze);
+            }
         }
     }
     return c.off;
@@ -417,15 +479,35 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             h->last_launches += 2;
         } else {
             // forward chain: convolutions -> normalise/activate/pool; FC forward
-            prof_begin(h, 3);
-            conv_gemm_kernel<<<(int)h->h_tiles[0].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[0], h->d_ts, h->S);
+            if (!h->h_tiles[0].empty()) {
+                prof_begin(h, 3);
+                conv_gemm_kernel<<<(int)h->h_tiles[0].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[0], h->d_ts, h->S);
+                prof_end(h);
+            }
+            if (!h->h_tctiles[0].empty()) {
+                prof_begin(h, 4);
+                conv_tc_kernel<<<(int)h->h_tctiles[0].size(), kTcThreads, kTcSmemBytes, h->stream>>>(h->d_tc, h->d_tctiles[0], h->d_ts, h->S);
+                prof_end(h);
+            }
+            prof_begin(h, 5);
             conv_post_fwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts);
-            // backward chain: through pool/ReLU/GroupNorm -> data and weight gradients
-            conv_post_bwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts, h->S);
-            if (!h->h_tiles[1].empty())
-                conv_gemm_kernel<<<(int)h->h_tiles[1].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[1], h->d_ts, h->S);
-            conv_gemm_kernel<<<(int)h->h_tiles[2].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[2], h->d_ts, h->S);
             prof_end(h);
+            // backward chain: through pool/ReLU/GroupNorm -> data and weight gradients
+            prof_begin(h, 6);
+            conv_post_bwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts, h->S);
+            prof_end(h);
+            for (int q = 1; q < 3; ++q) {
+                if (!h->h_tiles[q].empty()) {
+                    prof_begin(h, 3);
+                    conv_gemm_kernel<<<(int)h->h_tiles[q].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[q], h->d_ts, h->S);
+                    prof_end(h);
+                }
+                if (!h->h_tctiles[q].empty()) {
+                    prof_begin(h, q == 1 ? 8 : 7);
+                    conv_tc_kernel<<<(int)h->h_tctiles[q].size(), kTcThreads, kTcSmemBytes, h->stream>>>(h->d_tc, h->d_tctiles[q], h->d_ts, h->S);
+                    prof_end(h);
+                }
+            }
             prof_begin(h, 2);
             update_kernel<<<(int)h->h_chunks.size(), 256, 0, h->stream>>>(h->d_upd, h->d_chunks, h->d_ts, h->S);
             prof_end(h);
@@ -437,7 +519,8 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             fc_tick_kernel<<<h->nctaB, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segB, h->d_ctaB, h->d_ts, h->S, 1,
                                                                   h->label_ring, dev_losses, t_base);
             prof_end(h);
-            h->last_launches += (h->h_tiles[1].empty() ? 7 : 8);
+            h->last_launches += 5;      // post_fwd, post_bwd, update, two FC phases
+            for (int q = 0; q < 3; ++q) h->last_launches += (h->h_tiles[q].empty() ? 0 : 1) + (h->h_tctiles[q].empty() ? 0 : 1);
         }
     }
     PB_CUDA(h, cudaGetLastError());
@@ -534,6 +617,10 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     up(h->d_map, h->h_map.data(), h->h_map.size() * sizeof(int2));
     up(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange));
     up(h->d_chunks, h->h_chunks.data(), h->h_chunks.size() * sizeof(UpdChunk));
+    up(h->d_tc, h->h_tc.data(), h->h_tc.size() * sizeof(ConvGemmTC));
+    for (int q = 0; q < 3; ++q) up(h->d_tctiles[q], h->h_tctiles[q].data(), h->h_tctiles[q].size() * sizeof(GemmTile));
+    if (e == cudaSuccess && !h->h_tc.empty())
+        e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
     if (e != cudaSuccess) {
         std::string m = std::string("pb_create: upload failed: ") + cudaGetErrorString(e);
@@ -548,10 +635,25 @@ int pb_set_weights(pb_handle* h, const float* host_w, size_t n) {
     if (!host_w || n != h->n_params) return fail(h, PB_E_ARG, "pb_set_weights: need pb_num_params() floats");
     PB_CUDA(h, cudaMemsetAsync(h->arena + h->zero_from, 0, h->arena_bytes - h->zero_from, h->stream));
     PB_CUDA(h, cudaMemsetAsync(h->d_ts, 0, sizeof(TickState), h->stream));
-    for (const StageHost& x : h->stages)
-        PB_CUDA(h, cudaMemcpyAsync(h->d_w + x.dev_off, host_w + x.user_off, x.n_params * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+    std::vector<float> tmp;
+    for (const StageHost& x : h->stages) {
+        const float* src = host_w + x.user_off;
+        if (x.tc) {
+            // tensor-core stages keep conv weights as [c_out][r][s][c_in]
+            tmp.assign(src, src + x.n_params);
+            const int CI = x.head.c_in, k2 = x.head.k * x.head.k;
+            for (int co = 0; co < x.head.c_out; ++co)
+                for (int ci = 0; ci < CI; ++ci)
+                    for (int rs = 0; rs < k2; ++rs) tmp[((size_t)co * k2 + rs) * CI + ci] = src[((size_t)co * CI + ci) * k2 + rs];
+            src = tmp.data();
+        }
+        PB_CUDA(h, cudaMemcpyAsync(h->d_w + x.dev_off, src, x.n_params * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+        if (x.tc) PB_CUDA(h, cudaStreamSynchronize(h->stream));     // tmp is reused
+    }
     // zero velocity: the predicted weights start equal to the weights
     if (h->d_wh) PB_CUDA(h, cudaMemcpyAsync(h->d_wh, h->d_w, h->dev_params * sizeof(float), cudaMemcpyDeviceToDevice, h->stream));
+    if (h->d_w16 && !h->h_chunks.empty())
+        cast_weights_kernel<<<(int)h->h_chunks.size(), 256, 0, h->stream>>>(h->d_upd, h->d_chunks);
     PB_CUDA(h, cudaStreamSynchronize(h->stream));
     h->tick = 0;
     return PB_OK;
@@ -609,7 +711,21 @@ static int get_params(pb_handle* h, const float* dev, float* host, size_t n, con
     if (!host || n != h->n_params) return fail(h, PB_E_ARG, std::string(who) + ": need pb_num_params() floats");
     for (const StageHost& x : h->stages)
         PB_CUDA(h, cudaMemcpyAsync(host + x.user_off, dev + x.dev_off, x.n_params * sizeof(float), cudaMemcpyDeviceToHost, h->stream));
-    return check_device_error(h);
+    int rc = check_device_error(h);
+    if (rc != PB_OK) return rc;
+    std::vector<float> tmp;
+    for (const StageHost& x : h->stages) {
+        if (!x.tc) continue;
+        // back from [c_out][r][s][c_in] to the caller's [c_out][c_in][r][s]
+        float* dst = host + x.user_off;
+        const int CI = x.head.c_in, k2 = x.head.k * x.head.k;
+        const size_t nw = (size_t)x.head.c_out * CI * k2;
+        tmp.assign(dst, dst + nw);
+        for (int co = 0; co < x.head.c_out; ++co)
+            for (int ci = 0; ci < CI; ++ci)
+                for (int rs = 0; rs < k2; ++rs) dst[((size_t)co * CI + ci) * k2 + rs] = tmp[((size_t)co * k2 + rs) * CI + ci];
+    }
+    return PB_OK;
 }
 
 int pb_get_weights(pb_handle* h, float* host_w, size_t n) { return get_params(h, h ? h->d_w : nullptr, host_w, n, "pb_get_weights"); }
@@ -630,7 +746,7 @@ int pb_profile_enable(pb_handle* h, int enable) {
 }
 
 double pb_profile_ms(pb_handle* h, int which, long long* launches) {
-    if (!h || which < 0 || which >= 4 || h->prof[which].launches == 0) { if (launches) *launches = 0; return -1.0; }
+    if (!h || which < 0 || which >= 9 || h->prof[which].launches == 0) { if (launches) *launches = 0; return -1.0; }
     if (launches) *launches = h->prof[which].launches;
     return h->prof[which].ms;
 }

@@ -6,6 +6,7 @@
 #include "../../include/pb.h"
 #include "pb_internal.h"
 #include "conv_types.h"
+#include "conv_tc.cuh"
 
 namespace pb {
 
@@ -38,6 +39,8 @@ struct StageHost {
     unsigned char *code_ring = nullptr, *arg_ring = nullptr;
     int split_f = 1, split_d = 1, split_w = 1;                     // K-slices of fprop / dgrad / wgrad
     int kps_f = 0, kps_d = 0, kps_w = 0;                           // K per slice
+    bool tc = false;                                               // tensor-core path, weights kept as [co][r][s][ci]
+    __nv_bfloat16 *out16 = nullptr, *dz16 = nullptr;
 };
 
 struct ProfileClass { double ms = 0; long long launches = 0; };
@@ -73,6 +76,9 @@ struct pb_handle {
     std::vector<int> h_ctaA, h_ctaB;
     // convolution tables
     float *d_wh = nullptr, *d_g = nullptr;
+    __nv_bfloat16 *d_w16 = nullptr, *d_wh16 = nullptr;
+    std::vector<pb::ConvGemmTC> h_tc; pb::ConvGemmTC* d_tc = nullptr;
+    std::vector<pb::GemmTile> h_tctiles[3]; pb::GemmTile* d_tctiles[3] = {nullptr, nullptr, nullptr};
     std::vector<pb::ConvGemm> h_gemms; pb::ConvGemm* d_gemms = nullptr;
     std::vector<pb::GemmTile> h_tiles[3]; pb::GemmTile* d_tiles[3] = {nullptr, nullptr, nullptr};
     std::vector<pb::ConvStage> h_cs; pb::ConvStage* d_cs = nullptr;
@@ -82,7 +88,7 @@ struct pb_handle {
 
     long long tick = 0, last_launches = 0;
     bool profile = false;
-    pb::ProfileClass prof[4];
+    pb::ProfileClass prof[9];
     std::vector<cudaEvent_t> ev_pool; size_t ev_used = 0;
     std::vector<int> ev_class;
     std::string err;

@@ -61,7 +61,7 @@ struct TickState {
     int error_info;
 };
 
-enum ErrorCode { kErrNone = 0, kErrSegRows = 1, kErrLabel = 2, kErrSlot = 3 };
+enum ErrorCode { kErrNone = 0, kErrSegRows = 1, kErrLabel = 2, kErrSlot = 3, kErrWait = 4 };
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
