@@ -153,12 +153,12 @@ __device__ void gemm_tile(const ConvGemm& G, const GemmTile& tl, long long smp,
 
 __global__ void __launch_bounds__(kGemmThreads)
 conv_gemm_kernel(const ConvGemm* __restrict__ gemms, const GemmTile* __restrict__ tiles,
-                 const TickState* __restrict__ ts, int S) {
+                 const TickState* __restrict__ ts, int S, int par) {
     __shared__ __align__(16) float As[kBK][kBM + 4];
     __shared__ __align__(16) float Bs[kBK][kBN + 4];
     const GemmTile tl = tiles[blockIdx.x];
     const ConvGemm& G = gemms[tl.gemm];
-    const long long t = ts->tick;
+    const long long t = ts->cnt[par];
     const long long smp = (G.mode == kFprop) ? t - G.s : t - 2LL * (S - 1) + G.s;
     if (smp < 0) return;
     switch (G.k) {

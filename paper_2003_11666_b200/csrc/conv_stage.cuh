@@ -39,11 +39,11 @@ __device__ __forceinline__ float skip_value(const ConvStage& st, const float* __
 // grid: one block per (stage, group); `map` gives (stage, group) per block.
 __global__ void __launch_bounds__(kGroupThreads)
 conv_post_fwd_kernel(const ConvStage* __restrict__ stages, const int2* __restrict__ map,
-                     const TickState* __restrict__ ts) {
+                     const TickState* __restrict__ ts, int par) {
     __shared__ GroupShared sh;
     const ConvStage& st = stages[map[blockIdx.x].x];
     const int grp = map[blockIdx.x].y;
-    const long long i = ts->tick - st.s;
+    const long long i = ts->cnt[par] - st.s;
     if (i < 0) return;
     const int slot = ring_slot(i, st.slots);
     const int hw = st.oh * st.ow, cpg = st.cpg, n = cpg * hw, c0 = grp * cpg;
@@ -146,11 +146,11 @@ __device__ __forceinline__ float gather_out_delta(const ConvStage& st, size_t oe
 
 __global__ void __launch_bounds__(kGroupThreads)
 conv_post_bwd_kernel(const ConvStage* __restrict__ stages, const int2* __restrict__ map,
-                     const TickState* __restrict__ ts, int S) {
+                     const TickState* __restrict__ ts, int S, int par) {
     __shared__ GroupShared sh;
     const ConvStage& st = stages[map[blockIdx.x].x];
     const int grp = map[blockIdx.x].y;
-    const long long j = ts->tick - 2LL * (S - 1) + st.s;
+    const long long j = ts->cnt[par] - 2LL * (S - 1) + st.s;
     if (j < 0) return;
     const int slot = ring_slot(j, st.slots);
     const int hw = st.oh * st.ow, cpg = st.cpg, n = cpg * hw, c0 = grp * cpg;
@@ -268,10 +268,10 @@ conv_post_bwd_kernel(const ConvStage* __restrict__ stages, const int2* __restric
 // weights the next forward will use.
 __global__ void __launch_bounds__(256)
 update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ chunks,
-              const TickState* __restrict__ ts, int S) {
+              const TickState* __restrict__ ts, int S, int par) {
     const UpdChunk ch = chunks[blockIdx.x];
     const UpdRange& R = ranges[ch.range];
-    const long long j = ts->tick - 2LL * (S - 1) + R.s;
+    const long long j = ts->cnt[par] - 2LL * (S - 1) + R.s;
     if (j < 0) return;
     const int end = min(R.n, ch.start + kUpdChunk);
     for (int e = ch.start + threadIdx.x; e < end; e += 256) {

@@ -79,13 +79,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ uint4 ldg16(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
 
 __global__ void __launch_bounds__(kTcThreads)
-conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, TickState* ts, int S) {
+conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, TickState* ts, int S, int par) {
     extern __shared__ unsigned char tc_smem_raw[];
     __shared__ uint64_t mbar[2];
     __shared__ uint32_t tmem_base_sh;
     const GemmTile tl = tiles[blockIdx.x];
     const ConvGemmTC& G = gemms[tl.gemm];
-    const long long t = ts->tick;
+    const long long t = ts->cnt[par];
     const long long smp = (G.mode == kFprop) ? t - G.s : t - 2LL * (S - 1) + G.s;
     if (smp < 0) return;                                   // uniform: before any allocation
     unsigned char* smem = (unsigned char*)(((uintptr_t)tc_smem_raw + 1023) & ~(uintptr_t)1023);

@@ -105,7 +105,7 @@ __device__ __forceinline__ float gather_delta(const FcStage& st, int r, long lon
 template <int VEC>
 __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int S, int phase,
                            const int* __restrict__ label_ring, float* __restrict__ loss_out,
-                           FcShared& sh, TickState* ts) {
+                           FcShared& sh, TickState* ts, const float* __restrict__ x_now, int label_now) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long i = t - st.s;                        // forward sample
     const long long j = t - 2LL * (S - 1) + st.s;        // backward sample
@@ -121,6 +121,12 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
     const int in = st.in_dim, out = st.out_dim;
     const float* __restrict__ xf = st.xin + (size_t)ring_slot(i < 0 ? 0 : i, st.xin_slots) * in;
     const float* __restrict__ xb = st.xin + (size_t)ring_slot(j < 0 ? 0 : j, st.xin_slots) * in;
+    // when this launch also ingests the sample, the input ring slot of tick t is being
+    // written by other blocks: read the caller's copy of the current sample instead
+    if (x_now && st.s == 0) {
+        xf = x_now;
+        if (j == t) xb = x_now;
+    }
 
     // ---- gradient w.r.t. this band's pre-activations
     __syncthreads();   // shared memory may still be in use by the previous segment
@@ -156,7 +162,7 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
             rest = 0.f;
             for (int k = 0; k < kFcWarps; ++k) rest += sh.red[k];
             const float sum = 1.f + rest;
-            int label = label_ring[ring_slot(j, S)];
+            int label = (x_now && j == t) ? label_now : label_ring[ring_slot(j, S)];
             if (label < 0 || label >= out) {
                 if (tid == 0) { ts->error = kErrLabel; ts->error_info = label; }
                 label = 0;
@@ -303,23 +309,41 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
     }
 }
 
+// One launch per tick for fully connected pipelines: phase 0 of every stage, the
+// fused last stage, and (ingest != 0) the copy of the new sample and label into
+// their rings.  When the last stage is too large for one block it gets its own
+// phase-1 launch; `publish` marks the launch that ends the tick.
 __global__ void __launch_bounds__(kFcThreads, 2)
 fc_tick_kernel(const FcStage* __restrict__ stages, const FcSeg* __restrict__ segs,
-               const int* __restrict__ cta_seg_begin, TickState* ts, int S, int phase,
-               const int* __restrict__ label_ring, float* __restrict__ losses, long long t_base) {
+               const int* __restrict__ cta_seg_begin, TickState* ts, int S, int phase, int par, int publish,
+               int* __restrict__ label_ring, float* __restrict__ losses, long long t_base,
+               const float* __restrict__ xs, const int* __restrict__ labels, int label_value,
+               float* __restrict__ in_ring, int in_slots, int elems) {
     __shared__ FcShared sh;
-    const long long t = ts->tick;
+    const long long t = ts->cnt[par];
     float* loss_out = losses ? losses + (t - t_base) : nullptr;
+    const float* x_now = nullptr;
+    int label_now = 0;
+    if (xs) {
+        // ingest: every block copies a slice of the sample; block 0 files the label
+        x_now = xs + (size_t)(t - t_base) * elems;
+        label_now = labels ? labels[t - t_base] : label_value;
+        float* dst = in_ring + (size_t)(t % in_slots) * elems;
+        for (int k = blockIdx.x * kFcThreads + threadIdx.x; k < elems; k += gridDim.x * kFcThreads) dst[k] = x_now[k];
+        if (blockIdx.x == 0 && threadIdx.x == 0) label_ring[t % S] = label_now;
+    }
     for (int q = cta_seg_begin[blockIdx.x]; q < cta_seg_begin[blockIdx.x + 1]; ++q) {
         const FcSeg seg = segs[q];
         const FcStage& st = stages[seg.stage];
-        if (st.vec == 4) fc_segment<4>(st, seg, t, S, phase, label_ring, loss_out, sh, ts);
-        else fc_segment<1>(st, seg, t, S, phase, label_ring, loss_out, sh, ts);
+        const int nph = seg.fused ? 2 : 1;
+        for (int ph = 0; ph < nph; ++ph) {
+            const int phs = seg.fused ? ph : phase;
+            if (st.vec == 4) fc_segment<4>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+            else fc_segment<1>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+            __syncthreads();      // the logits written by phase 0 are read by phase 1
+        }
     }
-    // the last kernel of a tick publishes the next tick number
-    if (phase == 1 && blockIdx.x == 0 && threadIdx.x == 0) {
-        ts->next = t + 1;
-    }
+    if (publish && blockIdx.x == 0 && threadIdx.x == 0) ts->cnt[par ^ 1] = t + 1;
 }
 
 }  // namespace pb

@@ -134,7 +134,7 @@ void schedule_constants(pb_handle* h) {
 
 // Split FC stages into row bands, one or more per thread block, of about equal bytes.
 void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSeg>& segs,
-                  std::vector<int>& cta_begin, std::vector<int>& nparts) {
+                  std::vector<int>& cta_begin, std::vector<int>& nparts, bool fuse_last) {
     double total = 0;
     for (int f : fc_ids) total += (double)h->h_fc[f].out_dim * h->h_fc[f].in_dim * 8.0;
     const double target = 2.0 * h->num_sms;
@@ -143,8 +143,18 @@ void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSe
     segs.clear(); cta_begin.clear();
     cta_begin.push_back(0);
     double rem = budget;
+    // a small last stage runs whole in one block (forward, loss, backward, update),
+    // placed first so that it overlaps the long bands of the other stages
     for (int f : fc_ids) {
         const FcStage& st = h->h_fc[f];
+        if (!fuse_last || !st.is_last) continue;
+        segs.push_back(FcSeg{f, 0, st.out_dim, 0, 1});
+        cta_begin.push_back((int)segs.size());
+        nparts[f] = 1;
+    }
+    for (int f : fc_ids) {
+        const FcStage& st = h->h_fc[f];
+        if (fuse_last && st.is_last) continue;
         const double row_bytes = st.in_dim * 8.0;
         int r = 0, part = 0;
         while (r < st.out_dim) {
@@ -152,7 +162,7 @@ void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSe
             if (n < 1) n = 1;
             if (n > kFcMaxSegRows) n = kFcMaxSegRows;
             if (n > st.out_dim - r) n = st.out_dim - r;
-            segs.push_back(FcSeg{f, r, r + n, part++});
+            segs.push_back(FcSeg{f, r, r + n, part++, 0});
             r += n;
             rem -= n * row_bytes;
             if (rem < row_bytes * 0.5) { cta_begin.push_back((int)segs.size()); rem = budget; }
@@ -325,16 +335,15 @@ int validate_conv(pb_handle* h) {
     return PB_OK;
 }
 
-__global__ void ingest_kernel(TickState* ts, const float* __restrict__ xs, const int* __restrict__ labels,
-                              int label_value, float* __restrict__ in_ring, int in_slots, int elems,
-                              int* __restrict__ label_ring, int S, long long t_base) {
-    const long long t = ts->next;
+__global__ void ingest_kernel(const TickState* __restrict__ ts, int par, const float* __restrict__ xs,
+                              const int* __restrict__ labels, int label_value, float* __restrict__ in_ring,
+                              int in_slots, int elems, int* __restrict__ label_ring, int S, long long t_base) {
+    const long long t = ts->cnt[par];
     const float* src = xs + (size_t)(t - t_base) * elems;
     float* dst = in_ring + (size_t)(t % in_slots) * elems;
     for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < elems; k += gridDim.x * blockDim.x) dst[k] = src[k];
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         label_ring[t % S] = labels ? labels[t - t_base] : label_value;
-        ts->tick = t;
     }
 }
 
@@ -463,63 +472,74 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
     const long long t_base = h->tick;
     h->last_launches = 0;
     if (h->profile) for (auto& p : h->prof) p = ProfileClass{};
+    const bool fused_last = h->nctaB == 0;      // the last stage rides in the phase-0 launch
     for (int k = 0; k < n_ticks; ++k) {
-        ingest_kernel<<<ingest_blocks, 256, 0, h->stream>>>(h->d_ts, dev_xs, dev_labels, label_value, h->in_ring,
-                                                            h->in_slots, elems, h->label_ring, h->S, t_base);
-        h->last_launches += 1;
+        const int par = (int)((t_base + k) & 1);
         if (h->all_fc) {
+            // one launch: ingest + every stage (two when the last stage needs its own)
             prof_begin(h, 0);
-            fc_tick_kernel<<<h->nctaA, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segA, h->d_ctaA, h->d_ts, h->S, 0,
-                                                                  h->label_ring, dev_losses, t_base);
+            fc_tick_kernel<<<h->nctaA, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segA, h->d_ctaA, h->d_ts, h->S, 0, par,
+                                                                  fused_last ? 1 : 0, h->label_ring, dev_losses, t_base,
+                                                                  dev_xs, dev_labels, label_value, h->in_ring, h->in_slots, elems);
             prof_end(h);
-            prof_begin(h, 1);
-            fc_tick_kernel<<<h->nctaB, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segB, h->d_ctaB, h->d_ts, h->S, 1,
-                                                                  h->label_ring, dev_losses, t_base);
-            prof_end(h);
-            h->last_launches += 2;
+            h->last_launches += 1;
+            if (!fused_last) {
+                prof_begin(h, 1);
+                fc_tick_kernel<<<h->nctaB, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segB, h->d_ctaB, h->d_ts, h->S, 1, par, 1,
+                                                                      h->label_ring, dev_losses, t_base,
+                                                                      nullptr, nullptr, 0, nullptr, 0, 0);
+                prof_end(h);
+                h->last_launches += 1;
+            }
         } else {
+            ingest_kernel<<<ingest_blocks, 256, 0, h->stream>>>(h->d_ts, par, dev_xs, dev_labels, label_value, h->in_ring,
+                                                                h->in_slots, elems, h->label_ring, h->S, t_base);
             // forward chain: convolutions -> normalise/activate/pool; FC forward
             if (!h->h_tiles[0].empty()) {
                 prof_begin(h, 3);
-                conv_gemm_kernel<<<(int)h->h_tiles[0].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[0], h->d_ts, h->S);
+                conv_gemm_kernel<<<(int)h->h_tiles[0].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[0], h->d_ts, h->S, par);
                 prof_end(h);
             }
             if (!h->h_tctiles[0].empty()) {
                 prof_begin(h, 4);
-                conv_tc_kernel<<<(int)h->h_tctiles[0].size(), kTcThreads, kTcSmemBytes, h->stream>>>(h->d_tc, h->d_tctiles[0], h->d_ts, h->S);
+                conv_tc_kernel<<<(int)h->h_tctiles[0].size(), kTcThreads, kTcSmemBytes, h->stream>>>(h->d_tc, h->d_tctiles[0], h->d_ts, h->S, par);
                 prof_end(h);
             }
             prof_begin(h, 5);
-            conv_post_fwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts);
+            conv_post_fwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts, par);
             prof_end(h);
             // backward chain: through pool/ReLU/GroupNorm -> data and weight gradients
             prof_begin(h, 6);
-            conv_post_bwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts, h->S);
+            conv_post_bwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts, h->S, par);
             prof_end(h);
             for (int q = 1; q < 3; ++q) {
                 if (!h->h_tiles[q].empty()) {
                     prof_begin(h, 3);
-                    conv_gemm_kernel<<<(int)h->h_tiles[q].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[q], h->d_ts, h->S);
+                    conv_gemm_kernel<<<(int)h->h_tiles[q].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[q], h->d_ts, h->S, par);
                     prof_end(h);
                 }
                 if (!h->h_tctiles[q].empty()) {
                     prof_begin(h, q == 1 ? 8 : 7);
-                    conv_tc_kernel<<<(int)h->h_tctiles[q].size(), kTcThreads, kTcSmemBytes, h->stream>>>(h->d_tc, h->d_tctiles[q], h->d_ts, h->S);
+                    conv_tc_kernel<<<(int)h->h_tctiles[q].size(), kTcThreads, kTcSmemBytes, h->stream>>>(h->d_tc, h->d_tctiles[q], h->d_ts, h->S, par);
                     prof_end(h);
                 }
             }
             prof_begin(h, 2);
-            update_kernel<<<(int)h->h_chunks.size(), 256, 0, h->stream>>>(h->d_upd, h->d_chunks, h->d_ts, h->S);
+            update_kernel<<<(int)h->h_chunks.size(), 256, 0, h->stream>>>(h->d_upd, h->d_chunks, h->d_ts, h->S, par);
             prof_end(h);
             prof_begin(h, 0);
-            fc_tick_kernel<<<h->nctaA, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segA, h->d_ctaA, h->d_ts, h->S, 0,
-                                                                  h->label_ring, dev_losses, t_base);
+            fc_tick_kernel<<<h->nctaA, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segA, h->d_ctaA, h->d_ts, h->S, 0, par,
+                                                                  fused_last ? 1 : 0, h->label_ring, dev_losses, t_base,
+                                                                  nullptr, nullptr, 0, nullptr, 0, 0);
             prof_end(h);
-            prof_begin(h, 1);
-            fc_tick_kernel<<<h->nctaB, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segB, h->d_ctaB, h->d_ts, h->S, 1,
-                                                                  h->label_ring, dev_losses, t_base);
-            prof_end(h);
-            h->last_launches += 5;      // post_fwd, post_bwd, update, two FC phases
+            if (!fused_last) {
+                prof_begin(h, 1);
+                fc_tick_kernel<<<h->nctaB, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segB, h->d_ctaB, h->d_ts, h->S, 1, par, 1,
+                                                                      h->label_ring, dev_losses, t_base,
+                                                                      nullptr, nullptr, 0, nullptr, 0, 0);
+                prof_end(h);
+            }
+            h->last_launches += 5 + (fused_last ? 0 : 1);      // ingest, post_fwd, post_bwd, update, FC
             for (int q = 0; q < 3; ++q) h->last_launches += (h->h_tiles[q].empty() ? 0 : 1) + (h->h_tctiles[q].empty() ? 0 : 1);
         }
     }
@@ -580,11 +600,15 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
         h->h_fc.push_back(f);
     }
     std::vector<int> npartsA(h->h_fc.size(), 1), npartsB(h->h_fc.size(), 1);
-    partition_fc(h, idsA, h->h_segA, h->h_ctaA, npartsA);
-    partition_fc(h, idsB, h->h_segB, h->h_ctaB, npartsB);
+    // a last stage of at most 256 rows and 64 K weights is fused into the phase-0 launch
+    bool fuse_last = false;
+    for (int f : idsB) fuse_last = h->h_fc[f].out_dim <= kFcMaxSegRows && (long long)h->h_fc[f].out_dim * h->h_fc[f].in_dim <= 65536;
+    partition_fc(h, idsA, h->h_segA, h->h_ctaA, npartsA, fuse_last);
+    if (fuse_last) { h->h_segB.clear(); h->h_ctaB.assign(1, 0); }
+    else partition_fc(h, idsB, h->h_segB, h->h_ctaB, npartsB, false);
     for (size_t f = 0; f < h->h_fc.size(); ++f) {
         StageHost& x = h->stages[h->h_fc[f].s];
-        x.dx_nparts = x.loss ? npartsB[f] : npartsA[f];
+        x.dx_nparts = (x.loss && !fuse_last) ? npartsB[f] : npartsA[f];
     }
     h->nctaA = (int)h->h_ctaA.size() - 1;
     h->nctaB = (int)h->h_ctaB.size() - 1;
@@ -836,11 +860,15 @@ extern "C" int pb_mlp_run_static(const int32_t* sizes, int n_sizes, float lr, fl
         h->h_fc.push_back(f);
     }
     std::vector<int> npartsA(h->h_fc.size(), 1), npartsB(h->h_fc.size(), 1);
-    partition_fc(h, idsA, h->h_segA, h->h_ctaA, npartsA);
-    partition_fc(h, idsB, h->h_segB, h->h_ctaB, npartsB);
+    // a last stage of at most 256 rows and 64 K weights is fused into the phase-0 launch
+    bool fuse_last = false;
+    for (int f : idsB) fuse_last = h->h_fc[f].out_dim <= kFcMaxSegRows && (long long)h->h_fc[f].out_dim * h->h_fc[f].in_dim <= 65536;
+    partition_fc(h, idsA, h->h_segA, h->h_ctaA, npartsA, fuse_last);
+    if (fuse_last) { h->h_segB.clear(); h->h_ctaB.assign(1, 0); }
+    else partition_fc(h, idsB, h->h_segB, h->h_ctaB, npartsB, false);
     for (size_t f = 0; f < h->h_fc.size(); ++f) {
         StageHost& x = h->stages[h->h_fc[f].s];
-        x.dx_nparts = x.loss ? npartsB[f] : npartsA[f];
+        x.dx_nparts = (x.loss && !fuse_last) ? npartsB[f] : npartsA[f];
     }
     h->nctaA = (int)h->h_ctaA.size() - 1;
     h->nctaB = (int)h->h_ctaB.size() - 1;

@@ -48,15 +48,16 @@ struct FcSeg {
     int stage;             // index into the FcStage table
     int row0, row1;
     int part;              // which partial row of the stage's dx buffer it writes
+    int fused;             // last stage, whole in this block: loss, backward and update follow its forward here
 };
 
 // Tick state that lives on the device so that launches need no per-tick
-// arguments.  The first kernel of a tick copies `next` to `tick`, the
-// last one writes `next = tick + 1`; no kernel reads a field that another block
-// of the same launch writes.
+// arguments besides a parity bit.  Every kernel of tick t is launched with
+// par = t & 1 and reads cnt[par]; the last kernel of the tick writes
+// cnt[par ^ 1] = t + 1.  No kernel reads a field that another block of the
+// same launch writes.
 struct TickState {
-    long long tick;        // tick being run; written by the first kernel of a tick
-    long long next;        // tick to run next; written by the last kernel of a tick
+    long long cnt[2];
     int error;             // first failed index check (0 = none)
     int error_info;
 };

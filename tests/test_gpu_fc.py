@@ -71,7 +71,7 @@ def test_run_matches_tick_by_tick_and_loss_is_delayed():
     assert np.isnan(got[:S - 1]).all() and np.isfinite(got[S - 1:]).all()
     np.testing.assert_array_equal(got[S - 1:], np.array(one[S - 1:], dtype=np.float32))
     np.testing.assert_array_equal(a.get_weights(), b.get_weights())
-    assert a.tick_count == n and a.last_launch_count == 3 * n
+    assert a.tick_count == n and a.last_launch_count == n      # one launch per tick
     # host-buffer entry point gives the same numbers
     c = make_engine(wl)
     hl = np.zeros(n, dtype=np.float32)
