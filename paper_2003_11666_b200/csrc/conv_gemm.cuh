@@ -156,8 +156,14 @@ conv_gemm_kernel(const ConvGemm* __restrict__ gemms, const GemmTile* __restrict_
                  const TickState* __restrict__ ts, int S, int par) {
     __shared__ __align__(16) float As[kBK][kBM + 4];
     __shared__ __align__(16) float Bs[kBK][kBN + 4];
+    __shared__ ConvGemm G;                                 // descriptor copy (no re-reads through global memory)
     const GemmTile tl = tiles[blockIdx.x];
-    const ConvGemm& G = gemms[tl.gemm];
+    {
+        const int* s_ = reinterpret_cast<const int*>(&gemms[tl.gemm]);
+        int* d_ = reinterpret_cast<int*>(&G);
+        for (int k = threadIdx.x; k < (int)(sizeof(ConvGemm) / 4); k += kGemmThreads) d_[k] = s_[k];
+    }
+    __syncthreads();
     const long long t = ts->cnt[par];
     const long long smp = (G.mode == kFprop) ? t - G.s : t - 2LL * (S - 1) + G.s;
     if (smp < 0) return;

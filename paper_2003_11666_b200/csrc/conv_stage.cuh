@@ -1,9 +1,18 @@
 // Per-stage normalisation / activation / pooling kernels and the fused update.
 //
 // A convolution stage is  conv -> GroupNorm -> (+skip) -> ReLU -> (max-pool |
-// global average pool).  One thread block owns one normalisation group of one
-// stage, so every reduction (group statistics, per-channel gradient sums)
-// stays inside the block and has a fixed order.
+// global average pool).  The elements of a normalisation group are cut into
+// chunks of at most kPostChunk elements (whole channels when the image is
+// small, pieces of one channel when it is large) and ONE WARP owns a chunk:
+// no block-wide barrier is needed, every lane holds kPostPer elements in
+// registers, and a resident block keeps eight independent chunks in flight,
+// which is what hides the (serial) load latencies of such small pieces of work.
+// Whatever needs the whole group goes through small partial tables that every
+// warp of the group combines in the same fixed order:
+//   forward : conv_stats_kernel     (sum the K-slices, keep z, chunk mean / M2)
+//             conv_apply_fwd_kernel (merge statistics, normalise, skip, ReLU, pool)
+//   backward: conv_bwd_dn_kernel    (gradient at the normalised activation, channel sums)
+//             conv_bwd_dz_kernel    (scale/shift gradients, gradient at the conv output)
 #pragma once
 #include "conv_types.h"
 #include "fc_kernels.cuh"   // ring_slot, warp_sum
@@ -11,256 +20,381 @@
 namespace pb {
 
 constexpr float kGnEps = 1e-5f;
-
-struct GroupShared {
-    float red[kGroupThreads / 32];
-    float wp1[kGroupThreads / 32], wp2[kGroupThreads / 32];
-    float s1[kMaxGroupChannels], s2[kMaxGroupChannels];
-    float bc[4];
-};
-
-__device__ __forceinline__ float block_sum(float x, GroupShared& sh) {
-    x = warp_sum(x);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = x;
-    __syncthreads();
-    float tot = 0.f;
-#pragma unroll
-    for (int k = 0; k < kGroupThreads / 32; ++k) tot += sh.red[k];
-    return tot;
-}
+constexpr int kPostPer = kPostChunk / 32;       // elements per lane
 
 __device__ __forceinline__ float skip_value(const ConvStage& st, const float* __restrict__ sk, int c, int y, int x) {
     if (st.skip_mode == 0) return sk[((size_t)c * st.skip_h + y) * st.skip_w + x];
     return c < st.skip_c ? sk[((size_t)c * st.skip_h + 2 * y) * st.skip_w + 2 * x] : 0.f;
 }
 
-// ---------------------------------------------------------------- forward
-// grid: one block per (stage, group); `map` gives (stage, group) per block.
-__global__ void __launch_bounds__(kGroupThreads)
-conv_post_fwd_kernel(const ConvStage* __restrict__ stages, const int2* __restrict__ map,
-                     const TickState* __restrict__ ts, int par) {
-    __shared__ GroupShared sh;
-    const ConvStage& st = stages[map[blockIdx.x].x];
-    const int grp = map[blockIdx.x].y;
-    const long long i = ts->cnt[par] - st.s;
-    if (i < 0) return;
-    const int slot = ring_slot(i, st.slots);
-    const int hw = st.oh * st.ow, cpg = st.cpg, n = cpg * hw, c0 = grp * cpg;
-    const size_t zelems = (size_t)st.co * hw;
-    float* __restrict__ z = st.z_ring + (size_t)slot * zelems + (size_t)c0 * hw;
-    const float* __restrict__ zp = st.zpart + (size_t)c0 * hw;
-    const int tid = threadIdx.x;
+// Elements lane, lane+32, ... of a chunk as (channel, pixel) without divisions: the
+// walker starts at element `lane` and advances by 32 elements per step (np >= 1).
+struct ChunkWalk {
+    int cl, p, e;
+    __device__ __forceinline__ ChunkWalk(const PostChunk& ch, int lane) {
+        e = lane; cl = lane / ch.np; p = lane - cl * ch.np;
+    }
+    __device__ __forceinline__ void get(const PostChunk& ch, int c0, int n, int& c, int& pix, bool& ok) const {
+        ok = e < n;
+        c = c0 + ch.cl0 + (ok ? cl : ch.ncl - 1);
+        pix = ch.p0 + (ok ? p : ch.np - 1);
+    }
+    __device__ __forceinline__ void next(const PostChunk& ch) {
+        e += 32; p += 32;
+        while (p >= ch.np && e < ch.ncl * ch.np) { p -= ch.np; ++cl; }
+    }
+};
 
-    // 1. add the K-slices of the convolution, keep z, group mean
+__device__ __forceinline__ int slot_of(long long sample, int slots) { return (int)((unsigned)sample % (unsigned)slots); }
+
+// ---------------------------------------------------------------- forward, step 1
+__device__ void conv_stats_chunk(const ConvStage& st, const PostChunk& ch, long long t, int lane) {
+    const long long i = t - st.s;
+    if (i < 0) return;
+    const int slot = slot_of(i, st.slots);
+    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np;
+    const size_t zelems = (size_t)st.co * hw;
+    float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
+    const float* __restrict__ zp = st.zpart;
+    float vals[kPostPer];
+    unsigned idx[kPostPer];
+    bool ok[kPostPer];
+    {
+        ChunkWalk w(ch, lane);
+#pragma unroll
+        for (int k = 0; k < kPostPer; ++k) {
+            int c, p;
+            w.get(ch, c0, n, c, p, ok[k]);
+            w.next(ch);
+            idx[k] = (unsigned)(c * hw + p);
+            vals[k] = 0.f;
+        }
+    }
+    // the K-slice loop is outside so that each step issues kPostPer independent loads
+    for (int q = 0; q < st.z_nsplit; ++q) {
+        const float* __restrict__ zq = zp + (size_t)q * zelems;
+#pragma unroll
+        for (int k = 0; k < kPostPer; ++k) vals[k] += zq[idx[k]];
+    }
     float sum = 0.f;
-    for (int e = tid; e < n; e += kGroupThreads) {
-        float v = 0.f;
-        for (int q = 0; q < st.z_nsplit; ++q) v += zp[(size_t)q * zelems + e];
-        z[e] = v;
-        sum += v;
-    }
-    const float mean = block_sum(sum, sh) / (float)n;
-    // 2. biased variance about the mean
+#pragma unroll
+    for (int k = 0; k < kPostPer; ++k)
+        if (ok[k]) { z[idx[k]] = vals[k]; sum += vals[k]; }
+    const float mean = warp_sum(sum) / (float)n;
     float sq = 0.f;
-    for (int e = tid; e < n; e += kGroupThreads) { const float d = z[e] - mean; sq = fmaf(d, d, sq); }
-    const float var = block_sum(sq, sh) / (float)n;
-    const float rstd = rsqrtf(var + kGnEps);
-    if (tid == 0) {
-        st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0] = mean;
-        st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 1] = rstd;
+#pragma unroll
+    for (int k = 0; k < kPostPer; ++k)
+        if (ok[k]) { const float d = vals[k] - mean; sq = fmaf(d, d, sq); }
+    const float m2 = warp_sum(sq);
+    if (lane == 0) {
+        float* f = st.fstat + ((size_t)ch.grp * st.fstat_stride + ch.idx) * 3;
+        f[0] = (float)n; f[1] = mean; f[2] = m2;
     }
-    // 3. normalise with the predicted scale/shift, add the skip input, activate
+}
+
+// ---------------------------------------------------------------- forward, step 2
+__device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, long long t, int lane) {
+    const long long i = t - st.s;
+    if (i < 0) return;
+    const int slot = slot_of(i, st.slots);
+    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np;
+    const size_t zelems = (size_t)st.co * hw;
+    const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
+    // group statistics from the chunk partials (the same arithmetic in every warp of the group)
+    const float* __restrict__ f = st.fstat + (size_t)ch.grp * st.fstat_stride * 3;
+    float tot = 0.f, wsum = 0.f;
+    for (int k = lane; k < ch.nidx; k += 32) { tot += f[3 * k]; wsum = fmaf(f[3 * k], f[3 * k + 1], wsum); }
+    tot = warp_sum(tot);
+    const float mean = warp_sum(wsum) / tot;
+    float m2 = 0.f;
+    for (int k = lane; k < ch.nidx; k += 32) { const float d = f[3 * k + 1] - mean; m2 += f[3 * k + 2] + f[3 * k] * d * d; }
+    const float rstd = rsqrtf(warp_sum(m2) / tot + kGnEps);
+    if (ch.idx == 0 && lane == 0) {
+        st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0] = mean;
+        st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1] = rstd;
+    }
     const float* __restrict__ gam = st.wh + st.nw;
     const float* __restrict__ bet = gam + st.co;
     const float* __restrict__ sk = st.skip_ring
-        ? st.skip_ring + (size_t)ring_slot(i, st.skip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
-    unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems + (size_t)c0 * hw;
+        ? st.skip_ring + (size_t)slot_of(i, st.skip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
+    unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems;
     const bool pooled = st.pool_k > 0 || st.avgpool;
     const size_t oelems = (size_t)st.co * st.out_h * st.out_w;
     float* __restrict__ out = st.out_ring + (size_t)slot * oelems;
     __nv_bfloat16* __restrict__ out16 = st.out16 ? st.out16 + (size_t)slot * oelems : nullptr;
-    auto act = [&](int e) -> float {
-        const int c = c0 + e / hw, p = e % hw;
-        float v = fmaf(gam[c] * rstd, z[e] - mean, bet[c]);
+    auto act = [&](int c, int p) -> float {
+        float v = fmaf(gam[c] * rstd, z[(size_t)c * hw + p] - mean, bet[c]);
         if (sk) v += skip_value(st, sk, c, p / st.ow, p % st.ow);
         return v;
     };
-    for (int e = tid; e < n; e += kGroupThreads) {
-        const float v = act(e);
-        const bool pass = st.relu ? v > 0.f : true;
-        code[e] = pass ? 1 : 0;
-        if (!pooled) {
-            const float a = pass ? v : 0.f;
-            out[(size_t)c0 * hw + e] = a;
-            if (out16) out16[(size_t)(e % hw) * st.co + c0 + e / hw] = __float2bfloat16_rn(a);
+    {
+        int cc[kPostPer], pp[kPostPer];
+        bool ok[kPostPer];
+        float zv[kPostPer], sv[kPostPer];
+        ChunkWalk w(ch, lane);
+#pragma unroll
+        for (int k = 0; k < kPostPer; ++k) {          // all loads of the lane's elements first
+            w.get(ch, c0, n, cc[k], pp[k], ok[k]);
+            w.next(ch);
+            zv[k] = z[(size_t)cc[k] * hw + pp[k]];
+            sv[k] = sk ? skip_value(st, sk, cc[k], pp[k] / st.ow, pp[k] % st.ow) : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < kPostPer; ++k) {
+            if (!ok[k]) continue;
+            const int c = cc[k], p = pp[k];
+            const float v = fmaf(gam[c] * rstd, zv[k] - mean, bet[c]) + sv[k];
+            const bool pass = st.relu ? v > 0.f : true;
+            code[(size_t)c * hw + p] = pass ? 1 : 0;
+            if (!pooled) {
+                const float a = pass ? v : 0.f;
+                out[(size_t)c * hw + p] = a;
+                if (out16) out16[(size_t)p * st.co + c] = __float2bfloat16_rn(a);
+            }
         }
     }
     if (st.pool_k > 0) {
-        // 4a. max-pool: first maximum in row-major window order; padding never wins
+        // max-pool: this chunk owns the pooled pixels [p0*ohw/hw, (p0+np)*ohw/hw) of its channels;
+        // first maximum in row-major window order, padding never wins
         const int ohw = st.out_h * st.out_w, k = st.pool_k;
-        unsigned char* __restrict__ arg = st.arg_ring + (size_t)slot * oelems + (size_t)c0 * ohw;
-        for (int o = tid; o < cpg * ohw; o += kGroupThreads) {
-            const int cl = o / ohw, op = o % ohw, py = op / st.out_w, px = op % st.out_w;
+        const int o0 = (int)((long long)ch.p0 * ohw / hw), o1 = (int)((long long)(ch.p0 + ch.np) * ohw / hw);
+        const int no = o1 - o0;
+        unsigned char* __restrict__ arg = st.arg_ring + (size_t)slot * oelems;
+        for (int e = lane; e < ch.ncl * no; e += 32) {
+            const int c = c0 + ch.cl0 + e / no, op = o0 + e % no, py = op / st.out_w, px = op % st.out_w;
             float best = -INFINITY;
             int bpos = 0;
             for (int r = 0; r < k; ++r)
                 for (int s = 0; s < k; ++s) {
                     const int y = py * st.pool_stride + r - st.pool_pad, x = px * st.pool_stride + s - st.pool_pad;
                     if (y < 0 || y >= st.oh || x < 0 || x >= st.ow) continue;
-                    float v = act(cl * hw + y * st.ow + x);
+                    float v = act(c, y * st.ow + x);
                     if (st.relu) v = fmaxf(v, 0.f);
                     if (v > best) { best = v; bpos = r * k + s; }
                 }
-            out[(size_t)c0 * ohw + o] = best;
-            if (out16) out16[(size_t)op * st.co + c0 + cl] = __float2bfloat16_rn(best);
-            arg[o] = (unsigned char)bpos;
+            out[(size_t)c * ohw + op] = best;
+            if (out16) out16[(size_t)op * st.co + c] = __float2bfloat16_rn(best);
+            arg[(size_t)c * ohw + op] = (unsigned char)bpos;
         }
     } else if (st.avgpool) {
-        // 4b. global average per channel: one warp per channel, fixed order
-        const int lane = tid & 31, warp = tid >> 5;
-        for (int cl = warp; cl < cpg; cl += kGroupThreads / 32) {
+        // global average per channel (chunks of such stages hold whole channels)
+        for (int cl = 0; cl < ch.ncl; ++cl) {
+            const int c = c0 + ch.cl0 + cl;
             float a = 0.f;
             for (int p = lane; p < hw; p += 32) {
-                float v = act(cl * hw + p);
+                float v = act(c, p);
                 if (st.relu) v = fmaxf(v, 0.f);
                 a += v;
             }
             a = warp_sum(a);
-            if (lane == 0) out[c0 + cl] = a / (float)hw;
+            if (lane == 0) out[c] = a / (float)hw;
         }
     }
 }
 
-// ---------------------------------------------------------------- backward
+// ---------------------------------------------------------------- backward, step 1
 // Gradient w.r.t. the stage output element `o` for backward sample j.
 __device__ __forceinline__ float gather_out_delta(const ConvStage& st, size_t oelems, size_t o, long long j) {
     float d = 0.f;
     for (int q = 0; q < st.n_dsrc; ++q) {
         const DeltaSrc& ds = st.dsrc[q];
-        const float* p = ds.ptr + ((size_t)ring_slot(j, ds.slots) * ds.nparts) * oelems + o;
+        const float* p = ds.ptr + ((size_t)slot_of(j, ds.slots) * ds.nparts) * oelems + o;
         for (int k = 0; k < ds.nparts; ++k) d += p[(size_t)k * oelems];
     }
     return d;
 }
 
-__global__ void __launch_bounds__(kGroupThreads)
-conv_post_bwd_kernel(const ConvStage* __restrict__ stages, const int2* __restrict__ map,
-                     const TickState* __restrict__ ts, int S, int par) {
-    __shared__ GroupShared sh;
-    const ConvStage& st = stages[map[blockIdx.x].x];
-    const int grp = map[blockIdx.x].y;
-    const long long j = ts->cnt[par] - 2LL * (S - 1) + st.s;
+__device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long long t, int S, int lane) {
+    const long long j = t - 2LL * (S - 1) + st.s;
     if (j < 0) return;
-    const int slot = ring_slot(j, st.slots);
-    const int hw = st.oh * st.ow, cpg = st.cpg, n = cpg * hw, c0 = grp * cpg;
+    const int slot = slot_of(j, st.slots);
+    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np;
     const size_t zelems = (size_t)st.co * hw;
     const size_t oelems = (size_t)st.co * st.out_h * st.out_w;
-    const float* __restrict__ z = st.z_ring + (size_t)slot * zelems + (size_t)c0 * hw;
-    const unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems + (size_t)c0 * hw;
-    const float mean = st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0];
-    const float rstd = st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 1];
-    float* __restrict__ dz = st.dz + (size_t)c0 * hw;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
+    const unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems;
+    const float mean = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0];
+    const float rstd = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1];
+    float* __restrict__ dz = st.dz;
     const int ohw = st.out_h * st.out_w;
-    const unsigned char* __restrict__ arg = st.pool_k > 0 ? st.arg_ring + (size_t)slot * oelems + (size_t)c0 * ohw : nullptr;
-
-    // 1. gradient w.r.t. the normalised activation and per-channel sums.  All warps
-    //    stay busy: a channel is shared by `wpc` warps when there are fewer channels
-    //    than warps; their partial sums are combined in a fixed order.
-    constexpr int kWarps = kGroupThreads / 32;
-    const int wpc = cpg < kWarps ? kWarps / cpg : 1;
-    const int cpp = kWarps / wpc;                        // channels per pass
-    for (int base = 0; base < cpg; base += cpp) {
-        const int cl = base + warp / wpc, sub = warp % wpc;
-        float a1 = 0.f, a2 = 0.f;
-        if (cl < cpg && warp < cpp * wpc) {
-            const int c = c0 + cl;
-            const float davg = st.avgpool ? gather_out_delta(st, oelems, c, j) / (float)hw : 0.f;
-            for (int p = sub * 32 + lane; p < hw; p += 32 * wpc) {
-                const int e = cl * hw + p;
-                float d;
-                if (st.avgpool) {
-                    d = davg;
-                } else if (st.pool_k > 0) {
-                    // every pooling window that contains this element and chose it
-                    const int y = p / st.ow, x = p % st.ow, k = st.pool_k, ps = st.pool_stride, pp = st.pool_pad;
-                    d = 0.f;
-                    for (int r = 0; r < k; ++r) {
-                        const int ty = y + pp - r;
-                        if (ty < 0 || ty % ps) continue;
-                        const int py = ty / ps;
-                        if (py >= st.out_h) continue;
-                        for (int s = 0; s < k; ++s) {
-                            const int tx = x + pp - s;
-                            if (tx < 0 || tx % ps) continue;
-                            const int px = tx / ps;
-                            if (px >= st.out_w) continue;
-                            const int o = cl * ohw + py * st.out_w + px;
-                            if (arg[o] == r * k + s) d += gather_out_delta(st, oelems, (size_t)c0 * ohw + o, j);
-                        }
-                    }
-                } else {
-                    d = gather_out_delta(st, oelems, (size_t)c0 * hw + e, j);
-                }
-                d = code[e] ? d : 0.f;
-                dz[e] = d;
-                a1 += d;
-                a2 = fmaf(d, (z[e] - mean) * rstd, a2);
+    int cc[kPostPer];
+    unsigned idx[kPostPer];
+    bool ok[kPostPer];
+    float d[kPostPer], zv[kPostPer];
+    unsigned char cd[kPostPer];
+    ChunkWalk wk(ch, lane);
+#pragma unroll
+    for (int k = 0; k < kPostPer; ++k) {
+        int p;
+        wk.get(ch, c0, n, cc[k], p, ok[k]);
+        wk.next(ch);
+        idx[k] = (unsigned)(cc[k] * hw + p);
+        zv[k] = z[idx[k]];
+        cd[k] = code[idx[k]];
+        d[k] = 0.f;
+    }
+    if (!st.avgpool && st.pool_k == 0) {
+        // plain stage: the consumers' partial rows line up with this stage's elements
+        for (int q = 0; q < st.n_dsrc; ++q) {
+            const float* __restrict__ bp = st.dsrc[q].ptr + (size_t)slot_of(j, st.dsrc[q].slots) * st.dsrc[q].nparts * oelems;
+            const int np_ = st.dsrc[q].nparts;
+            for (int kp = 0; kp < np_; ++kp, bp += oelems) {
+#pragma unroll
+                for (int k = 0; k < kPostPer; ++k) d[k] += bp[idx[k]];
             }
         }
+    } else if (st.avgpool) {
+#pragma unroll
+        for (int k = 0; k < kPostPer; ++k) d[k] = gather_out_delta(st, oelems, cc[k], j) / (float)hw;
+    } else {
+        // max-pool: every window that contains the element and chose it
+        const unsigned char* __restrict__ arg = st.arg_ring + (size_t)slot * oelems;
+        const int kk = st.pool_k, ps = st.pool_stride, pp = st.pool_pad;
+#pragma unroll 1
+        for (int k = 0; k < kPostPer; ++k) {
+            if (!ok[k]) continue;
+            const int p = (int)idx[k] - cc[k] * hw;
+            const int y = p / st.ow, x = p % st.ow;
+            float a = 0.f;
+            for (int r = 0; r < kk; ++r) {
+                const int ty = y + pp - r;
+                if (ty < 0 || ty % ps) continue;
+                const int py = ty / ps;
+                if (py >= st.out_h) continue;
+                for (int s = 0; s < kk; ++s) {
+                    const int tx = x + pp - s;
+                    if (tx < 0 || tx % ps) continue;
+                    const int px = tx / ps;
+                    if (px >= st.out_w) continue;
+                    const size_t o = (size_t)cc[k] * ohw + py * st.out_w + px;
+                    if (arg[o] == r * kk + s) a += gather_out_delta(st, oelems, o, j);
+                }
+            }
+            d[k] = a;
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kPostPer; ++k) {
+        d[k] = (ok[k] && cd[k]) ? d[k] : 0.f;
+        if (ok[k]) dz[idx[k]] = d[k];
+        zv[k] = d[k] * ((zv[k] - mean) * rstd);          // d * zhat
+    }
+    // per-channel sums of d and d*zhat over this chunk's pixels
+    const int piece = ch.p0 / kPostChunk;
+    for (int cl = 0; cl < ch.ncl; ++cl) {
+        const int c = c0 + ch.cl0 + cl;
+        float a1 = 0.f, a2 = 0.f;
+#pragma unroll
+        for (int k = 0; k < kPostPer; ++k)
+            if (cc[k] == c) { a1 += d[k]; a2 += zv[k]; }
         a1 = warp_sum(a1);
         a2 = warp_sum(a2);
-        if (lane == 0) { sh.wp1[warp] = a1; sh.wp2[warp] = a2; }
-        __syncthreads();
-        if (tid < cpp && base + tid < cpg) {
-            float t1 = 0.f, t2 = 0.f;
-            for (int q = 0; q < wpc; ++q) { t1 += sh.wp1[tid * wpc + q]; t2 += sh.wp2[tid * wpc + q]; }
-            sh.s1[base + tid] = t1;
-            sh.s2[base + tid] = t2;
+        if (lane == 0) {
+            float* b = st.bsum + ((size_t)c * st.npieces + piece) * 2;
+            b[0] = a1; b[1] = a2;
         }
-        __syncthreads();
-    }
-    // 2. gradients of scale and shift; group means with the CURRENT scale
-    const float* __restrict__ gam = st.w + st.nw;
-    if (tid < cpg) {
-        st.g[st.nw + c0 + tid] = sh.s2[tid];
-        st.g[st.nw + st.co + c0 + tid] = sh.s1[tid];
-    }
-    if (tid == 0) {
-        float m1 = 0.f, m2 = 0.f;
-        for (int cl = 0; cl < cpg; ++cl) { m1 = fmaf(gam[c0 + cl], sh.s1[cl], m1); m2 = fmaf(gam[c0 + cl], sh.s2[cl], m2); }
-        sh.bc[0] = m1 / (float)n;
-        sh.bc[1] = m2 / (float)n;
-    }
-    __syncthreads();
-    const float m1 = sh.bc[0], m2 = sh.bc[1];
-    // 3. skip gradient (taken before normalisation) and gradient w.r.t. the conv output
-    if (st.dskip) {
-        float* __restrict__ dsk = st.dskip + (size_t)ring_slot(j, st.dskip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w);
-        if (st.skip_mode == 0) {
-            for (int e = tid; e < n; e += kGroupThreads) dsk[(size_t)c0 * hw + e] = dz[e];
-        } else {
-            const int shw = st.skip_h * st.skip_w;
-            for (int cl = 0; cl < cpg; ++cl) {
-                const int c = c0 + cl;
-                if (c >= st.skip_c) break;
-                for (int p = tid; p < shw; p += kGroupThreads) {
-                    const int y = p / st.skip_w, x = p % st.skip_w;
-                    dsk[(size_t)c * shw + p] = ((y | x) & 1) ? 0.f : dz[cl * hw + (y >> 1) * st.ow + (x >> 1)];
-                }
-            }
-        }
-        __syncthreads();
-    }
-    for (int e = tid; e < n; e += kGroupThreads) {
-        const int c = c0 + e / hw;
-        const float zh = (z[e] - mean) * rstd;
-        const float d = rstd * (fmaf(dz[e], gam[c], -m1) - zh * m2);
-        dz[e] = d;
-        if (st.dz16) st.dz16[(size_t)(e % hw) * st.co + c] = __float2bfloat16_rn(d);
     }
 }
+
+// ---------------------------------------------------------------- backward, step 2
+__device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long long t, int S, int lane) {
+    const long long j = t - 2LL * (S - 1) + st.s;
+    if (j < 0) return;
+    const int slot = slot_of(j, st.slots);
+    const int hw = st.oh * st.ow, cpg = st.cpg, c0 = ch.grp * cpg, n = ch.ncl * ch.np;
+    const size_t zelems = (size_t)st.co * hw;
+    const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
+    const float mean = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0];
+    const float rstd = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1];
+    float* __restrict__ dz = st.dz;
+    // channel sums of the whole group (pieces added in order), gradients of scale and
+    // shift, group means with the CURRENT scale
+    const float* __restrict__ gam = st.w + st.nw;
+    float m1 = 0.f, m2 = 0.f;
+    for (int cl = lane; cl < cpg; cl += 32) {
+        float t1 = 0.f, t2 = 0.f;
+        const float* __restrict__ b = st.bsum + (size_t)(c0 + cl) * st.npieces * 2;
+        for (int q = 0; q < st.npieces; ++q) { t1 += b[2 * q]; t2 += b[2 * q + 1]; }
+        if (ch.idx == 0) {
+            st.g[st.nw + c0 + cl] = t2;
+            st.g[st.nw + st.co + c0 + cl] = t1;
+        }
+        m1 = fmaf(gam[c0 + cl], t1, m1);
+        m2 = fmaf(gam[c0 + cl], t2, m2);
+    }
+    m1 = warp_sum(m1) / (float)(cpg * hw);
+    m2 = warp_sum(m2) / (float)(cpg * hw);
+    float* __restrict__ dsk = st.dskip
+        ? st.dskip + (size_t)slot_of(j, st.dskip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
+    int cc[kPostPer], pp[kPostPer];
+    bool ok[kPostPer];
+    float dnv[kPostPer], zv[kPostPer];
+    ChunkWalk wk(ch, lane);
+#pragma unroll
+    for (int k = 0; k < kPostPer; ++k) {              // all loads of the lane's elements first
+        wk.get(ch, c0, n, cc[k], pp[k], ok[k]);
+        wk.next(ch);
+        const size_t idx = (size_t)cc[k] * hw + pp[k];
+        dnv[k] = dz[idx];
+        zv[k] = z[idx];
+    }
+#pragma unroll
+    for (int k = 0; k < kPostPer; ++k) {
+        if (!ok[k]) continue;
+        const int c = cc[k], p = pp[k];
+        const size_t idx = (size_t)c * hw + p;
+        const float dn = dnv[k];
+        // the skip input joined after the normalisation: it receives dn itself
+        if (dsk) {
+            if (st.skip_mode == 0) {
+                dsk[idx] = dn;
+            } else if (c < st.skip_c) {
+                const int y = p / st.ow, x = p % st.ow;
+                for (int dy = 0; dy < 2; ++dy)
+                    for (int dx = 0; dx < 2; ++dx) {
+                        const int ys = 2 * y + dy, xs = 2 * x + dx;
+                        if (ys < st.skip_h && xs < st.skip_w)
+                            dsk[((size_t)c * st.skip_h + ys) * st.skip_w + xs] = (dy | dx) ? 0.f : dn;
+                    }
+            }
+        }
+        const float zh = (zv[k] - mean) * rstd;
+        const float dd = rstd * (fmaf(dn, gam[c], -m1) - zh * m2);
+        dz[idx] = dd;
+        if (st.dz16) st.dz16[(size_t)p * st.co + c] = __float2bfloat16_rn(dd);
+    }
+}
+
+// ---------------------------------------------------------------- launch wrappers
+// Persistent blocks: every warp walks the chunk table with a grid stride.  The
+// stage descriptors are kept in shared memory (one copy per stage of the launch
+// would not fit, so each warp re-reads its chunk's descriptor into its own slot).
+#define PB_POST_KERNEL(NAME, CHUNK, ...)                                                          \
+    __global__ void __launch_bounds__(kPostThreads, 2) NAME(const ConvStage* __restrict__ stages,  \
+                                                            const PostChunk* __restrict__ chunks, int nchunks, \
+                                                            const TickState* __restrict__ ts, int S, int par) { \
+        __shared__ ConvStage sst[kPostThreads / 32];                                               \
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;                                \
+        const long long t = ts->cnt[par];                                                          \
+        int loaded = -1;                                                                           \
+        for (int ci = blockIdx.x * (kPostThreads / 32) + warp; ci < nchunks; ci += gridDim.x * (kPostThreads / 32)) { \
+            const PostChunk ch = chunks[ci];                                                       \
+            if (ch.stage != loaded) {                                                              \
+                __syncwarp();                                                                      \
+                const int* s_ = reinterpret_cast<const int*>(&stages[ch.stage]);                   \
+                int* d_ = reinterpret_cast<int*>(&sst[warp]);                                      \
+                for (int k = lane; k < (int)(sizeof(ConvStage) / 4); k += 32) d_[k] = s_[k];       \
+                __syncwarp();                                                                      \
+                loaded = ch.stage;                                                                 \
+            }                                                                                      \
+            CHUNK(sst[warp], ch, t, __VA_ARGS__);                                                  \
+        }                                                                                          \
+    }
+PB_POST_KERNEL(conv_stats_kernel, conv_stats_chunk, lane)
+PB_POST_KERNEL(conv_apply_fwd_kernel, conv_apply_fwd_chunk, lane)
+PB_POST_KERNEL(conv_bwd_dn_kernel, conv_bwd_dn_chunk, S, lane)
+PB_POST_KERNEL(conv_bwd_dz_kernel, conv_bwd_dz_chunk, S, lane)
+#undef PB_POST_KERNEL
 
 // ---------------------------------------------------------------- update
 // Fused SC + LWP step for materialised gradients (convolution stages):

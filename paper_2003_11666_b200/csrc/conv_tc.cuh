@@ -83,8 +83,14 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
     extern __shared__ unsigned char tc_smem_raw[];
     __shared__ uint64_t mbar[2];
     __shared__ uint32_t tmem_base_sh;
+    __shared__ ConvGemmTC G;                               // descriptor copy (no re-reads through global memory)
     const GemmTile tl = tiles[blockIdx.x];
-    const ConvGemmTC& G = gemms[tl.gemm];
+    {
+        const int* s_ = reinterpret_cast<const int*>(&gemms[tl.gemm]);
+        int* d_ = reinterpret_cast<int*>(&G);
+        for (int k = threadIdx.x; k < (int)(sizeof(ConvGemmTC) / 4); k += kTcThreads) d_[k] = s_[k];
+    }
+    __syncthreads();
     const long long t = ts->cnt[par];
     const long long smp = (G.mode == kFprop) ? t - G.s : t - 2LL * (S - 1) + G.s;
     if (smp < 0) return;                                   // uniform: before any allocation

@@ -8,7 +8,8 @@ namespace pb {
 
 constexpr int kGemmThreads = 256;
 constexpr int kBM = 64, kBN = 64, kBK = 16;
-constexpr int kGroupThreads = 1024;
+constexpr int kPostThreads = 256;         // normalisation / activation kernels
+constexpr int kPostChunk = 256;           // elements per warp of those kernels
 constexpr int kMaxGroupChannels = 64;      // channels per normalisation group
 
 enum GemmMode { kFprop = 0, kDgrad = 1, kWgrad = 2 };
@@ -46,6 +47,8 @@ struct ConvStage {
     const float* zpart; int z_nsplit;    // fprop partial sums [nsplit][co*oh*ow]
     float* z_ring;               // [slots][co*oh*ow] conv output, kept for the backward
     float* stat_ring;            // [slots][2*groups] mean, rstd
+    float* fstat; int fstat_stride;      // forward chunk partials [groups][fstat_stride][3]: count, mean, M2
+    float* bsum; int npieces;            // backward channel partials [co][npieces][2]
     unsigned char* code_ring;    // [slots][co*oh*ow] bit0: ReLU passed
     unsigned char* arg_ring;     // [slots][co*out_h*out_w] max-pool winner position in its window
     float* out_ring;             // [slots][co*out_h*out_w]
@@ -75,6 +78,11 @@ struct UpdRange {
     float neg_lr_T, m, neg_lr_a, neg_lr_b;
 };
 struct UpdChunk { int range, start; };
+
+// One warp's share of the normalisation kernels: channels [cl0, cl0+ncl) of group `grp`
+// (relative to the group), pixels [p0, p0+np); chunk `idx` of `nidx` in its group.
+// Either ncl >= 1 whole channels (p0 = 0, np = all pixels) or a piece of one channel.
+struct PostChunk { int stage, grp, cl0, ncl, p0, np, idx, nidx; };
 constexpr int kUpdChunk = 4096;
 
 }  // namespace pb

@@ -47,7 +47,7 @@ template <> __device__ __forceinline__ void vstore<4>(float* p, const float (&r)
 template <> __device__ __forceinline__ void vstore<1>(float* p, const float (&r)[1]) { *p = r[0]; }
 
 __device__ __forceinline__ int ring_slot(long long sample, int slots) {
-    return (int)(sample % slots);
+    return (int)((unsigned)sample % (unsigned)slots);   // samples stay far below 2^32
 }
 
 __device__ __forceinline__ float warp_sum(float x) {
@@ -320,6 +320,7 @@ fc_tick_kernel(const FcStage* __restrict__ stages, const FcSeg* __restrict__ seg
                const float* __restrict__ xs, const int* __restrict__ labels, int label_value,
                float* __restrict__ in_ring, int in_slots, int elems) {
     __shared__ FcShared sh;
+    __shared__ FcStage sst;
     const long long t = ts->cnt[par];
     float* loss_out = losses ? losses + (t - t_base) : nullptr;
     const float* x_now = nullptr;
@@ -334,7 +335,16 @@ fc_tick_kernel(const FcStage* __restrict__ stages, const FcSeg* __restrict__ seg
     }
     for (int q = cta_seg_begin[blockIdx.x]; q < cta_seg_begin[blockIdx.x + 1]; ++q) {
         const FcSeg seg = segs[q];
-        const FcStage& st = stages[seg.stage];
+        // the stage descriptor goes through shared memory: the kernel stores to global
+        // memory in its loops, so fields behind a global reference would be re-read
+        __syncthreads();
+        {
+            const int* s_ = reinterpret_cast<const int*>(&stages[seg.stage]);
+            int* d_ = reinterpret_cast<int*>(&sst);
+            for (int k = threadIdx.x; k < (int)(sizeof(FcStage) / 4); k += kFcThreads) d_[k] = s_[k];
+        }
+        __syncthreads();
+        const FcStage& st = sst;
         const int nph = seg.fused ? 2 : 1;
         for (int ph = 0; ph < nph; ++ph) {
             const int phs = seg.fused ? ph : phase;

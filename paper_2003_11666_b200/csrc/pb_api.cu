@@ -132,40 +132,55 @@ void schedule_constants(pb_handle* h) {
     h->dev_params = dev_off;
 }
 
-// Split FC stages into row bands, one or more per thread block, of about equal bytes.
+// Split FC stages into row bands, one or more per thread block, of equal bytes:
+// block k owns the rows whose cumulative byte offset falls in [k*B, (k+1)*B), so
+// the block count is exact and the launch is one balanced wave.
 void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSeg>& segs,
                   std::vector<int>& cta_begin, std::vector<int>& nparts, bool fuse_last) {
-    double total = 0;
-    for (int f : fc_ids) total += (double)h->h_fc[f].out_dim * h->h_fc[f].in_dim * 8.0;
-    const double target = 2.0 * h->num_sms;
-    double budget = total / target;
-    if (budget < 48.0 * 1024) budget = 48.0 * 1024;
     segs.clear(); cta_begin.clear();
     cta_begin.push_back(0);
-    double rem = budget;
     // a small last stage runs whole in one block (forward, loss, backward, update),
     // placed first so that it overlaps the long bands of the other stages
+    int fused_ctas = 0;
     for (int f : fc_ids) {
         const FcStage& st = h->h_fc[f];
         if (!fuse_last || !st.is_last) continue;
         segs.push_back(FcSeg{f, 0, st.out_dim, 0, 1});
         cta_begin.push_back((int)segs.size());
         nparts[f] = 1;
+        ++fused_ctas;
     }
+    double total = 0;
+    for (int f : fc_ids) {
+        const FcStage& st = h->h_fc[f];
+        if (fuse_last && st.is_last) continue;
+        total += (double)st.out_dim * st.in_dim * 8.0;
+    }
+    if (total <= 0) return;
+    int ncta = 2 * h->num_sms - fused_ctas;       // two resident blocks per SM
+    const int by_size = (int)(total / (48.0 * 1024)) + 1;      // at least 48 KB of weights per block
+    if (ncta > by_size) ncta = by_size;
+    if (ncta < 1) ncta = 1;
+    const double budget = total / ncta;
+    double acc = 0;
+    int cur = 0;                        // block that owns the bytes at offset acc
     for (int f : fc_ids) {
         const FcStage& st = h->h_fc[f];
         if (fuse_last && st.is_last) continue;
         const double row_bytes = st.in_dim * 8.0;
         int r = 0, part = 0;
         while (r < st.out_dim) {
-            int n = (int)(rem / row_bytes);
+            // rows until the next block boundary (at least one), capped by the segment limit
+            const double room = (cur + 1) * budget - acc;
+            int n = (int)(room / row_bytes + 0.5);
             if (n < 1) n = 1;
             if (n > kFcMaxSegRows) n = kFcMaxSegRows;
             if (n > st.out_dim - r) n = st.out_dim - r;
             segs.push_back(FcSeg{f, r, r + n, part++, 0});
             r += n;
-            rem -= n * row_bytes;
-            if (rem < row_bytes * 0.5) { cta_begin.push_back((int)segs.size()); rem = budget; }
+            acc += n * row_bytes;
+            const int owner = std::min(ncta - 1, (int)((acc + 0.5 * row_bytes) / budget));
+            if (owner != cur) { cta_begin.push_back((int)segs.size()); cur = owner; }
         }
         nparts[f] = part;
     }
@@ -199,6 +214,11 @@ void plan_conv(pb_handle* h) {
     for (StageHost& x : h->stages) {
         if (x.head_op != PB_CONV2D) continue;
         const int k2 = x.head.k * x.head.k;
+        {
+            const int hw = x.z.h * x.z.w, cpg = x.head.c_out / x.gn_groups;
+            x.npieces = hw <= kPostChunk ? 1 : ceil_div(hw, kPostChunk);
+            x.fstat_stride = hw <= kPostChunk ? ceil_div(cpg, std::max(1, kPostChunk / hw)) : cpg * x.npieces;
+        }
         x.tc = (h->flags & PB_CONV_BF16) && x.src >= 0 && x.head.c_in % 8 == 0 && x.head.c_out % 8 == 0 &&
                h->stages[x.src].head_op == PB_CONV2D;
         if (x.tc) {
@@ -223,7 +243,7 @@ void add_tiles(std::vector<GemmTile>& tiles, int gemm, int M, int N, int nsplit,
 }
 
 void fill_conv_tables(pb_handle* h) {
-    h->h_gemms.clear(); h->h_cs.clear(); h->h_map.clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear();
+    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear();
     for (auto& t : h->h_tiles) t.clear();
     for (auto& t : h->h_tctiles) t.clear();
     const int bf = (h->flags & PB_CONV_BF16) ? 1 : 0;
@@ -305,7 +325,25 @@ void fill_conv_tables(pb_handle* h) {
         for (int q : x.consumers_main) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dx, y.dx_slots, y.dx_nparts}; }
         for (int q : x.consumers_skip) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dskip, y.dskip_slots, 1}; }
         c.dz = x.dz;
-        for (int gq = 0; gq < x.gn_groups; ++gq) h->h_map.push_back(make_int2((int)h->h_cs.size(), gq));
+        c.fstat = x.fstat; c.fstat_stride = x.fstat_stride; c.bsum = x.bsum; c.npieces = x.npieces;
+        {
+            // chunks of the normalisation kernels: whole channels while they fit, else pieces of one channel
+            const int hw = x.z.h * x.z.w, cpg = c.cpg;
+            for (int gq = 0; gq < x.gn_groups; ++gq) {
+                const size_t first = h->h_pchunks.size();
+                if (hw <= kPostChunk) {
+                    const int per = std::max(1, kPostChunk / hw);
+                    for (int cl = 0; cl < cpg; cl += per)
+                        h->h_pchunks.push_back(PostChunk{(int)h->h_cs.size(), gq, cl, std::min(per, cpg - cl), 0, hw, 0, 0});
+                } else {
+                    for (int cl = 0; cl < cpg; ++cl)
+                        for (int p0 = 0; p0 < hw; p0 += kPostChunk)
+                            h->h_pchunks.push_back(PostChunk{(int)h->h_cs.size(), gq, cl, 1, p0, std::min(kPostChunk, hw - p0), 0, 0});
+                }
+                const int nidx = (int)(h->h_pchunks.size() - first);
+                for (int q = 0; q < nidx; ++q) { h->h_pchunks[first + q].idx = q; h->h_pchunks[first + q].nidx = nidx; }
+            }
+        }
         h->h_cs.push_back(c);
 
         UpdRange r{};
@@ -328,6 +366,7 @@ int validate_conv(pb_handle* h) {
         if (x.gn_groups <= 0) return fail(nullptr, PB_E_UNSUPPORTED, "a CONV2D stage needs a GROUPNORM layer");
         if (x.head.c_out / x.gn_groups > kMaxGroupChannels) return fail(nullptr, PB_E_UNSUPPORTED, "more than 64 channels per normalisation group");
         if (x.has_pool && x.avgpool) return fail(nullptr, PB_E_UNSUPPORTED, "max-pool and average pool in one stage");
+        if (x.avgpool && x.z.h * x.z.w > kPostChunk) return fail(nullptr, PB_E_UNSUPPORTED, "global average pool over more than 256 pixels");
         if ((int)(x.consumers_main.size() + x.consumers_skip.size()) > kMaxDeltaSrc) return fail(nullptr, PB_E_UNSUPPORTED, "too many consumers of one stage");
     }
     for (const StageHost& x : h->stages)
@@ -368,7 +407,7 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     h->d_gemms = c.take<ConvGemm>(h->h_gemms.size() + 1);
     for (int q = 0; q < 3; ++q) h->d_tiles[q] = c.take<GemmTile>(h->h_tiles[q].size() + 1);
     h->d_cs = c.take<ConvStage>(h->h_cs.size() + 1);
-    h->d_map = c.take<int2>(h->h_map.size() + 1);
+    h->d_pchunks = c.take<PostChunk>(h->h_pchunks.size() + 1);
     h->d_upd = c.take<UpdRange>(h->h_upd.size() + 1);
     h->d_chunks = c.take<UpdChunk>(h->h_chunks.size() + 1);
     h->d_tc = c.take<ConvGemmTC>(h->h_tc.size() + 1);
@@ -406,6 +445,8 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
             x.zpart = c.take<float>((size_t)x.split_f * ze);
             x.dz = c.take<float>(ze);
             x.gpart = c.take<float>((size_t)x.split_w * nw);
+            x.fstat = c.take<float>((size_t)x.gn_groups * x.fstat_stride * 3);
+            x.bsum = c.take<float>((size_t)x.head.c_out * x.npieces * 2);
             if (h->flags & PB_CONV_BF16) {
                 x.out16 = c.take<__nv_bfloat16>((size_t)x.out_slots * x.out.elems());
                 x.dz16 = c.take<__nv_bfloat16>(ze);
@@ -473,6 +514,8 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
     h->last_launches = 0;
     if (h->profile) for (auto& p : h->prof) p = ProfileClass{};
     const bool fused_last = h->nctaB == 0;      // the last stage rides in the phase-0 launch
+    const int npc = (int)h->h_pchunks.size();
+    const int post_grid = std::max(1, std::min(ceil_div(npc, kPostThreads / 32), 2 * h->num_sms));
     for (int k = 0; k < n_ticks; ++k) {
         const int par = (int)((t_base + k) & 1);
         if (h->all_fc) {
@@ -506,11 +549,13 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
                 prof_end(h);
             }
             prof_begin(h, 5);
-            conv_post_fwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts, par);
+            conv_stats_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
+            conv_apply_fwd_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
             prof_end(h);
             // backward chain: through pool/ReLU/GroupNorm -> data and weight gradients
             prof_begin(h, 6);
-            conv_post_bwd_kernel<<<(int)h->h_map.size(), kGroupThreads, 0, h->stream>>>(h->d_cs, h->d_map, h->d_ts, h->S, par);
+            conv_bwd_dn_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
+            conv_bwd_dz_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
             prof_end(h);
             for (int q = 1; q < 3; ++q) {
                 if (!h->h_tiles[q].empty()) {
@@ -539,7 +584,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
                                                                       nullptr, nullptr, 0, nullptr, 0, 0);
                 prof_end(h);
             }
-            h->last_launches += 5 + (fused_last ? 0 : 1);      // ingest, post_fwd, post_bwd, update, FC
+            h->last_launches += 7 + (fused_last ? 0 : 1);      // ingest, 2 + 2 normalisation kernels, update, FC
             for (int q = 0; q < 3; ++q) h->last_launches += (h->h_tiles[q].empty() ? 0 : 1) + (h->h_tctiles[q].empty() ? 0 : 1);
         }
     }
@@ -638,7 +683,7 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     up(h->d_gemms, h->h_gemms.data(), h->h_gemms.size() * sizeof(ConvGemm));
     for (int q = 0; q < 3; ++q) up(h->d_tiles[q], h->h_tiles[q].data(), h->h_tiles[q].size() * sizeof(GemmTile));
     up(h->d_cs, h->h_cs.data(), h->h_cs.size() * sizeof(ConvStage));
-    up(h->d_map, h->h_map.data(), h->h_map.size() * sizeof(int2));
+    up(h->d_pchunks, h->h_pchunks.data(), h->h_pchunks.size() * sizeof(PostChunk));
     up(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange));
     up(h->d_chunks, h->h_chunks.data(), h->h_chunks.size() * sizeof(UpdChunk));
     up(h->d_tc, h->h_tc.data(), h->h_tc.size() * sizeof(ConvGemmTC));
