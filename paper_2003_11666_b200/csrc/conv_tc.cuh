@@ -9,8 +9,9 @@
 //   dgrad  D[c_in, in pixel]    A = weights, read transposed (MN-major)  B = scattered dz (K-major)
 //   wgrad  D[c_out, (r,s,c_in)] A = dz (MN-major)                 B = im2col(x)      (MN-major)
 // with K ordered (r, s, channel) so that 8 consecutive K (one 16-byte unit)
-// are 8 consecutive channels of one pixel.  Two shared-memory stages: while
-// the tensor core works on one K-chunk of 64 the threads gather the next.
+// are 8 consecutive channels of one pixel.  The gather uses 16-byte asynchronous
+// copies (cp.async, zero-filled outside the image) into a three-stage ring: two
+// K-chunks of 64 are in flight while the tensor core works on a third.
 // Every mbarrier wait is bounded; on expiry the block records an error, skips
 // its stores, frees its tensor memory and returns.
 #pragma once
@@ -24,7 +25,8 @@ constexpr int kTcThreads = 128;
 constexpr int kTcBM = 128;
 constexpr int kTcChunk = 64;                  // K elements per shared-memory stage
 constexpr int kTcStageBytes = 16384 * 2;      // A tile + B tile
-constexpr int kTcSmemBytes = 2 * kTcStageBytes + 1024;
+constexpr int kTcStages = 3;                  // shared-memory stages of the operand pipeline
+constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + 1024;
 constexpr int kTcWaitLimit = 1 << 22;
 
 struct ConvGemmTC {
@@ -76,12 +78,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     return done != 0;
 }
 
-__device__ __forceinline__ uint4 ldg16(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+// 16-byte asynchronous global -> shared copy; with ok == false the destination is zero-filled
+__device__ __forceinline__ void cp_async16(unsigned char* dst, const __nv_bfloat16* src, bool ok) {
+    const int sz = ok ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(sz) : "memory");
+}
 
 __global__ void __launch_bounds__(kTcThreads)
 conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, TickState* ts, int S, int par) {
     extern __shared__ unsigned char tc_smem_raw[];
-    __shared__ uint64_t mbar[2];
+    __shared__ uint64_t mbar[kTcStages];
     __shared__ uint32_t tmem_base_sh;
     __shared__ ConvGemmTC G;                               // descriptor copy (no re-reads through global memory)
     const GemmTile tl = tiles[blockIdx.x];
@@ -109,8 +115,8 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (tid == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&mbar[0])) : "memory");
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&mbar[1])) : "memory");
+        for (int q = 0; q < kTcStages; ++q)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&mbar[q])) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -148,15 +154,10 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
     const int amu = tid & 15, ak0 = tid >> 4;               // MN-major A (width 128)
     const bool a_m_ok = (tl.m0 + amu * 8) < M;
 
-    bool failed = false;
-    for (int c = 0; c < nchunks; ++c) {
-        const int stg = c & 1;
-        unsigned char* sA = smem + stg * kTcStageBytes;
+    // gather of K-chunk c into its stage (every unit is written: data or zeros)
+    auto gather = [&](int c) {
+        unsigned char* sA = smem + (c % kTcStages) * kTcStageBytes;
         unsigned char* sB = sA + 16384;
-        if (c >= 2) {
-            // the MMAs of chunk c-2 read this stage: wait until they are done
-            if (!mbar_wait(smem_u32(&mbar[stg]), (uint32_t)(((c >> 1) - 1) & 1))) failed = true;
-        }
         const int k0 = kb + c * kTcChunk;
         // ---------------- A tile
         if (G.mode == kFprop) {
@@ -164,28 +165,23 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int row = krow0 + 16 * i, m = tl.m0 + row;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (m < M && k < ke) v = ldg16(A + (size_t)m * G.K + k);
-                *reinterpret_cast<uint4*>(sA + kmajor_off(row, ku)) = v;
+                const bool ok = m < M && k < ke;
+                cp_async16(sA + kmajor_off(row, ku), ok ? A + (size_t)m * G.K + k : A, ok);
             }
         } else if (G.mode == kDgrad) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int kl = ak0 + 8 * i, k = k0 + kl;          // k = rs * CO + co
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (a_m_ok && k < ke) {
-                    const int rs = k / CO, co = k - rs * CO;
-                    v = ldg16(A + ((size_t)co * (ksz * ksz) + rs) * CI + tl.m0 + amu * 8);
-                }
-                *reinterpret_cast<uint4*>(sA + mnmajor_off(kl, amu)) = v;
+                const bool ok = a_m_ok && k < ke;
+                const int rs = k / CO, co = k - rs * CO;
+                cp_async16(sA + mnmajor_off(kl, amu), ok ? A + ((size_t)co * (ksz * ksz) + rs) * CI + tl.m0 + amu * 8 : A, ok);
             }
         } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int kl = ak0 + 8 * i, k = k0 + kl;          // k = output pixel
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (a_m_ok && k < ke) v = ldg16(A + (size_t)k * CO + tl.m0 + amu * 8);
-                *reinterpret_cast<uint4*>(sA + mnmajor_off(kl, amu)) = v;
+                const bool ok = a_m_ok && k < ke;
+                cp_async16(sA + mnmajor_off(kl, amu), ok ? A + (size_t)k * CO + tl.m0 + amu * 8 : A, ok);
             }
         }
         // ---------------- B tile
@@ -196,10 +192,9 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
             for (int i = 0; i < 8; ++i) {
                 const int row = krow0 + 16 * i;
                 if (row >= BN) break;
-                uint4 v = make_uint4(0, 0, 0, 0);
                 const int y = bp[i] * st + r - pad, x = bq[i] * st + s - pad;
-                if (bok[i] && k < ke && y >= 0 && y < ih && x >= 0 && x < iw) v = ldg16(B + ((size_t)y * iw + x) * CI + ci);
-                *reinterpret_cast<uint4*>(sB + kmajor_off(row, ku)) = v;
+                const bool ok = bok[i] && k < ke && y >= 0 && y < ih && x >= 0 && x < iw;
+                cp_async16(sB + kmajor_off(row, ku), ok ? B + ((size_t)y * iw + x) * CI + ci : B, ok);
             }
         } else if (G.mode == kDgrad) {
             const int k = k0 + ku * 8;
@@ -208,26 +203,33 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
             for (int i = 0; i < 8; ++i) {
                 const int row = krow0 + 16 * i;
                 if (row >= BN) break;
-                uint4 v = make_uint4(0, 0, 0, 0);
                 const int ty = bp[i] + pad - r, tx = bq[i] + pad - s;
-                if (bok[i] && k < ke && ty >= 0 && tx >= 0) {
-                    const int p = ty / st, q = tx / st;
-                    if (p * st == ty && q * st == tx && p < oh && q < ow) v = ldg16(B + ((size_t)p * ow + q) * CO + co);
-                }
-                *reinterpret_cast<uint4*>(sB + kmajor_off(row, ku)) = v;
+                const int p = ty / st, q = tx / st;
+                const bool ok = bok[i] && k < ke && ty >= 0 && tx >= 0 && p * st == ty && q * st == tx && p < oh && q < ow;
+                cp_async16(sB + kmajor_off(row, ku), ok ? B + ((size_t)p * ow + q) * CO + co : B, ok);
             }
         } else {
             for (int kl = bk0; kl < kTcChunk; kl += bkstep) {
                 const int k = k0 + kl;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (wok && k < ke) {
-                    const int p = k / ow, q = k - p * ow;
-                    const int y = p * st + wr - pad, x = q * st + wsx - pad;
-                    if (y >= 0 && y < ih && x >= 0 && x < iw) v = ldg16(B + ((size_t)y * iw + x) * CI + wci);
-                }
-                *reinterpret_cast<uint4*>(sB + mnmajor_off(kl, bmu)) = v;
+                const int p = k / ow, q = k - p * ow;
+                const int y = p * st + wr - pad, x = q * st + wsx - pad;
+                const bool ok = wok && k < ke && y >= 0 && y < ih && x >= 0 && x < iw;
+                cp_async16(sB + mnmajor_off(kl, bmu), ok ? B + ((size_t)y * iw + x) * CI + wci : B, ok);
             }
         }
+    };
+
+    bool failed = false;
+    for (int c = 0; c < kTcStages - 1; ++c) {
+        if (c < nchunks) gather(c);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    for (int c = 0; c < nchunks; ++c) {
+        const int stg = c % kTcStages;
+        unsigned char* sA = smem + stg * kTcStageBytes;
+        unsigned char* sB = sA + 16384;
+        // this thread's copies of chunk c have landed; make them visible to the tensor core
+        asm volatile("cp.async.wait_group %0;" ::"n"(kTcStages - 2) : "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         if (__syncthreads_or(failed)) { failed = true; break; }
         if (tid == 0) {
@@ -243,11 +245,19 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
             }
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&mbar[stg])) : "memory");
         }
+        // refill the stage that chunk c-1 used, once its MMAs have read it
+        const int nxt = c + kTcStages - 1;
+        if (nxt < nchunks) {
+            if (c >= 1 && !mbar_wait(smem_u32(&mbar[(c - 1) % kTcStages]), (uint32_t)(((c - 1) / kTcStages) & 1))) failed = true;
+            gather(nxt);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     // the last commit covers every MMA issued before it
     if (!failed && nchunks > 0) {
         const int last = nchunks - 1;
-        if (!mbar_wait(smem_u32(&mbar[last & 1]), (uint32_t)((last >> 1) & 1))) failed = true;
+        if (!mbar_wait(smem_u32(&mbar[last % kTcStages]), (uint32_t)((last / kTcStages) & 1))) failed = true;
     }
     failed = __syncthreads_or(failed);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
