@@ -27,64 +27,93 @@ __device__ __forceinline__ float skip_value(const ConvStage& st, const float* __
     return c < st.skip_c ? sk[((size_t)c * st.skip_h + 2 * y) * st.skip_w + 2 * x] : 0.f;
 }
 
-// Elements lane, lane+32, ... of a chunk as (channel, pixel) without divisions: the
-// walker starts at element `lane` and advances by 32 elements per step (np >= 1).
+// A lane works on units of VEC consecutive pixels of one channel (VEC = 4 when the
+// image size is a multiple of 4: float4 / uchar4 accesses, a quarter of the index
+// arithmetic).  Units lane, lane+32, ... of a chunk are walked without divisions.
+template <int VEC>
 struct ChunkWalk {
-    int cl, p, e;
+    int cl, p, e, npu;          // channel in chunk, pixel offset, unit index, units per channel
     __device__ __forceinline__ ChunkWalk(const PostChunk& ch, int lane) {
-        e = lane; cl = lane / ch.np; p = lane - cl * ch.np;
+        npu = ch.np / VEC;
+        e = lane; cl = lane / npu; p = (lane - cl * npu) * VEC;
     }
-    __device__ __forceinline__ void get(const PostChunk& ch, int c0, int n, int& c, int& pix, bool& ok) const {
-        ok = e < n;
+    __device__ __forceinline__ void get(const PostChunk& ch, int c0, int nunits, int& c, int& pix, bool& ok) const {
+        ok = e < nunits;
         c = c0 + ch.cl0 + (ok ? cl : ch.ncl - 1);
-        pix = ch.p0 + (ok ? p : ch.np - 1);
+        pix = ch.p0 + (ok ? p : ch.np - VEC);
     }
     __device__ __forceinline__ void next(const PostChunk& ch) {
-        e += 32; p += 32;
-        while (p >= ch.np && e < ch.ncl * ch.np) { p -= ch.np; ++cl; }
+        e += 32; p += 32 * VEC;
+        while (p >= ch.np && e < ch.ncl * npu) { p -= ch.np; ++cl; }
     }
 };
 
 __device__ __forceinline__ int slot_of(long long sample, int slots) { return (int)((unsigned)sample % (unsigned)slots); }
 
+template <int VEC> __device__ __forceinline__ void ldb(unsigned char (&r)[VEC], const unsigned char* p);
+template <> __device__ __forceinline__ void ldb<4>(unsigned char (&r)[4], const unsigned char* p) {
+    const uchar4 q = *reinterpret_cast<const uchar4*>(p); r[0] = q.x; r[1] = q.y; r[2] = q.z; r[3] = q.w;
+}
+template <> __device__ __forceinline__ void ldb<1>(unsigned char (&r)[1], const unsigned char* p) { r[0] = *p; }
+template <int VEC> __device__ __forceinline__ void stb(unsigned char* p, const unsigned char (&r)[VEC]);
+template <> __device__ __forceinline__ void stb<4>(unsigned char* p, const unsigned char (&r)[4]) {
+    *reinterpret_cast<uchar4*>(p) = make_uchar4(r[0], r[1], r[2], r[3]);
+}
+template <> __device__ __forceinline__ void stb<1>(unsigned char* p, const unsigned char (&r)[1]) { *p = r[0]; }
+
 // ---------------------------------------------------------------- forward, step 1
+template <int VEC>
 __device__ void conv_stats_chunk(const ConvStage& st, const PostChunk& ch, long long t, int lane) {
+    constexpr int U = kPostPer / VEC;
     const long long i = t - st.s;
     if (i < 0) return;
     const int slot = slot_of(i, st.slots);
-    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np;
+    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np, nunits = n / VEC;
     const size_t zelems = (size_t)st.co * hw;
     float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
     const float* __restrict__ zp = st.zpart;
-    float vals[kPostPer];
-    unsigned idx[kPostPer];
-    bool ok[kPostPer];
+    float vals[U][VEC];
+    unsigned idx[U];
+    bool ok[U];
     {
-        ChunkWalk w(ch, lane);
+        ChunkWalk<VEC> w(ch, lane);
 #pragma unroll
-        for (int k = 0; k < kPostPer; ++k) {
+        for (int u = 0; u < U; ++u) {
             int c, p;
-            w.get(ch, c0, n, c, p, ok[k]);
+            w.get(ch, c0, nunits, c, p, ok[u]);
             w.next(ch);
-            idx[k] = (unsigned)(c * hw + p);
-            vals[k] = 0.f;
+            idx[u] = (unsigned)(c * hw + p);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) vals[u][e] = 0.f;
         }
     }
-    // the K-slice loop is outside so that each step issues kPostPer independent loads
+    // the K-slice loop is outside so that each step issues U independent loads
     for (int q = 0; q < st.z_nsplit; ++q) {
         const float* __restrict__ zq = zp + (size_t)q * zelems;
 #pragma unroll
-        for (int k = 0; k < kPostPer; ++k) vals[k] += zq[idx[k]];
+        for (int u = 0; u < U; ++u) {
+            float r[VEC];
+            vload<VEC>(r, zq + idx[u]);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) vals[u][e] += r[e];
+        }
     }
     float sum = 0.f;
 #pragma unroll
-    for (int k = 0; k < kPostPer; ++k)
-        if (ok[k]) { z[idx[k]] = vals[k]; sum += vals[k]; }
+    for (int u = 0; u < U; ++u)
+        if (ok[u]) {
+            vstore<VEC>(z + idx[u], vals[u]);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) sum += vals[u][e];
+        }
     const float mean = warp_sum(sum) / (float)n;
     float sq = 0.f;
 #pragma unroll
-    for (int k = 0; k < kPostPer; ++k)
-        if (ok[k]) { const float d = vals[k] - mean; sq = fmaf(d, d, sq); }
+    for (int u = 0; u < U; ++u)
+        if (ok[u]) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) { const float d = vals[u][e] - mean; sq = fmaf(d, d, sq); }
+        }
     const float m2 = warp_sum(sq);
     if (lane == 0) {
         float* f = st.fstat + ((size_t)ch.grp * st.fstat_stride + ch.idx) * 3;
@@ -93,11 +122,13 @@ __device__ void conv_stats_chunk(const ConvStage& st, const PostChunk& ch, long 
 }
 
 // ---------------------------------------------------------------- forward, step 2
+template <int VEC>
 __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, long long t, int lane) {
+    constexpr int U = kPostPer / VEC;
     const long long i = t - st.s;
     if (i < 0) return;
     const int slot = slot_of(i, st.slots);
-    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np;
+    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np, nunits = n / VEC;
     const size_t zelems = (size_t)st.co * hw;
     const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
     // group statistics from the chunk partials (the same arithmetic in every warp of the group)
@@ -128,28 +159,47 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
         return v;
     };
     {
-        int cc[kPostPer], pp[kPostPer];
-        bool ok[kPostPer];
-        float zv[kPostPer], sv[kPostPer];
-        ChunkWalk w(ch, lane);
+        int cc[U], pp[U];
+        bool ok[U];
+        float zv[U][VEC], sv[U][VEC];
+        ChunkWalk<VEC> w(ch, lane);
 #pragma unroll
-        for (int k = 0; k < kPostPer; ++k) {          // all loads of the lane's elements first
-            w.get(ch, c0, n, cc[k], pp[k], ok[k]);
+        for (int u = 0; u < U; ++u) {                 // all loads of the lane's units first
+            w.get(ch, c0, nunits, cc[u], pp[u], ok[u]);
             w.next(ch);
-            zv[k] = z[(size_t)cc[k] * hw + pp[k]];
-            sv[k] = sk ? skip_value(st, sk, cc[k], pp[k] / st.ow, pp[k] % st.ow) : 0.f;
+            vload<VEC>(zv[u], z + (size_t)cc[u] * hw + pp[u]);
+            if (!sk) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) sv[u][e] = 0.f;
+            } else if (st.skip_mode == 0) {
+                // identity skips share this stage's indexing
+                vload<VEC>(sv[u], sk + (size_t)cc[u] * hw + pp[u]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) sv[u][e] = skip_value(st, sk, cc[u], (pp[u] + e) / st.ow, (pp[u] + e) % st.ow);
+            }
         }
 #pragma unroll
-        for (int k = 0; k < kPostPer; ++k) {
-            if (!ok[k]) continue;
-            const int c = cc[k], p = pp[k];
-            const float v = fmaf(gam[c] * rstd, zv[k] - mean, bet[c]) + sv[k];
-            const bool pass = st.relu ? v > 0.f : true;
-            code[(size_t)c * hw + p] = pass ? 1 : 0;
+        for (int u = 0; u < U; ++u) {
+            if (!ok[u]) continue;
+            const int c = cc[u], p = pp[u];
+            const float gs = gam[c] * rstd, bb = bet[c];
+            float a[VEC];
+            unsigned char cd[VEC];
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+                const float v = fmaf(gs, zv[u][e] - mean, bb) + sv[u][e];
+                const bool pass = st.relu ? v > 0.f : true;
+                cd[e] = pass ? 1 : 0;
+                a[e] = pass ? v : 0.f;
+            }
+            stb<VEC>(code + (size_t)c * hw + p, cd);
             if (!pooled) {
-                const float a = pass ? v : 0.f;
-                out[(size_t)c * hw + p] = a;
-                if (out16) out16[(size_t)p * st.co + c] = __float2bfloat16_rn(a);
+                vstore<VEC>(out + (size_t)c * hw + p, a);
+                if (out16) {
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) out16[(size_t)(p + e) * st.co + c] = __float2bfloat16_rn(a[e]);
+                }
             }
         }
     }
@@ -204,11 +254,13 @@ __device__ __forceinline__ float gather_out_delta(const ConvStage& st, size_t oe
     return d;
 }
 
+template <int VEC>
 __device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long long t, int S, int lane) {
+    constexpr int U = kPostPer / VEC;
     const long long j = t - 2LL * (S - 1) + st.s;
     if (j < 0) return;
     const int slot = slot_of(j, st.slots);
-    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np;
+    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np, nunits = n / VEC;
     const size_t zelems = (size_t)st.co * hw;
     const size_t oelems = (size_t)st.co * st.out_h * st.out_w;
     const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
@@ -217,67 +269,86 @@ __device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long
     const float rstd = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1];
     float* __restrict__ dz = st.dz;
     const int ohw = st.out_h * st.out_w;
-    int cc[kPostPer];
-    unsigned idx[kPostPer];
-    bool ok[kPostPer];
-    float d[kPostPer], zv[kPostPer];
-    unsigned char cd[kPostPer];
-    ChunkWalk wk(ch, lane);
+    int cc[U];
+    unsigned idx[U];
+    bool ok[U];
+    float d[U][VEC], zv[U][VEC];
+    unsigned char cd[U][VEC];
+    ChunkWalk<VEC> wk(ch, lane);
 #pragma unroll
-    for (int k = 0; k < kPostPer; ++k) {
+    for (int u = 0; u < U; ++u) {
         int p;
-        wk.get(ch, c0, n, cc[k], p, ok[k]);
+        wk.get(ch, c0, nunits, cc[u], p, ok[u]);
         wk.next(ch);
-        idx[k] = (unsigned)(cc[k] * hw + p);
-        zv[k] = z[idx[k]];
-        cd[k] = code[idx[k]];
-        d[k] = 0.f;
+        idx[u] = (unsigned)(cc[u] * hw + p);
+        vload<VEC>(zv[u], z + idx[u]);
+        ldb<VEC>(cd[u], code + idx[u]);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) d[u][e] = 0.f;
     }
     if (!st.avgpool && st.pool_k == 0) {
         // plain stage: the consumers' partial rows line up with this stage's elements
         for (int q = 0; q < st.n_dsrc; ++q) {
-            const float* __restrict__ bp = st.dsrc[q].ptr + (size_t)slot_of(j, st.dsrc[q].slots) * st.dsrc[q].nparts * oelems;
+            const float* bp = st.dsrc[q].ptr + (size_t)slot_of(j, st.dsrc[q].slots) * st.dsrc[q].nparts * oelems;
             const int np_ = st.dsrc[q].nparts;
             for (int kp = 0; kp < np_; ++kp, bp += oelems) {
 #pragma unroll
-                for (int k = 0; k < kPostPer; ++k) d[k] += bp[idx[k]];
+                for (int u = 0; u < U; ++u) {
+                    float r[VEC];
+                    vload<VEC>(r, bp + idx[u]);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) d[u][e] += r[e];
+                }
             }
         }
     } else if (st.avgpool) {
 #pragma unroll
-        for (int k = 0; k < kPostPer; ++k) d[k] = gather_out_delta(st, oelems, cc[k], j) / (float)hw;
+        for (int u = 0; u < U; ++u) {
+            const float a = gather_out_delta(st, oelems, cc[u], j) / (float)hw;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) d[u][e] = a;
+        }
     } else {
         // max-pool: every window that contains the element and chose it
         const unsigned char* __restrict__ arg = st.arg_ring + (size_t)slot * oelems;
         const int kk = st.pool_k, ps = st.pool_stride, pp = st.pool_pad;
 #pragma unroll 1
-        for (int k = 0; k < kPostPer; ++k) {
-            if (!ok[k]) continue;
-            const int p = (int)idx[k] - cc[k] * hw;
-            const int y = p / st.ow, x = p % st.ow;
-            float a = 0.f;
-            for (int r = 0; r < kk; ++r) {
-                const int ty = y + pp - r;
-                if (ty < 0 || ty % ps) continue;
-                const int py = ty / ps;
-                if (py >= st.out_h) continue;
-                for (int s = 0; s < kk; ++s) {
-                    const int tx = x + pp - s;
-                    if (tx < 0 || tx % ps) continue;
-                    const int px = tx / ps;
-                    if (px >= st.out_w) continue;
-                    const size_t o = (size_t)cc[k] * ohw + py * st.out_w + px;
-                    if (arg[o] == r * kk + s) a += gather_out_delta(st, oelems, o, j);
+        for (int u = 0; u < U; ++u) {
+            if (!ok[u]) continue;
+#pragma unroll 1
+            for (int e = 0; e < VEC; ++e) {
+                const int p = (int)idx[u] - cc[u] * hw + e;
+                const int y = p / st.ow, x = p % st.ow;
+                float a = 0.f;
+                for (int r = 0; r < kk; ++r) {
+                    const int ty = y + pp - r;
+                    if (ty < 0 || ty % ps) continue;
+                    const int py = ty / ps;
+                    if (py >= st.out_h) continue;
+                    for (int s = 0; s < kk; ++s) {
+                        const int tx = x + pp - s;
+                        if (tx < 0 || tx % ps) continue;
+                        const int px = tx / ps;
+                        if (px >= st.out_w) continue;
+                        const size_t o = (size_t)cc[u] * ohw + py * st.out_w + px;
+                        if (arg[o] == r * kk + s) a += gather_out_delta(st, oelems, o, j);
+                    }
                 }
+                d[u][e] = a;
             }
-            d[k] = a;
         }
     }
+    float s1[U], s2[U];
 #pragma unroll
-    for (int k = 0; k < kPostPer; ++k) {
-        d[k] = (ok[k] && cd[k]) ? d[k] : 0.f;
-        if (ok[k]) dz[idx[k]] = d[k];
-        zv[k] = d[k] * ((zv[k] - mean) * rstd);          // d * zhat
+    for (int u = 0; u < U; ++u) {
+        s1[u] = 0.f; s2[u] = 0.f;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            d[u][e] = (ok[u] && cd[u][e]) ? d[u][e] : 0.f;
+            s1[u] += d[u][e];
+            s2[u] = fmaf(d[u][e], (zv[u][e] - mean) * rstd, s2[u]);      // d * zhat
+        }
+        if (ok[u]) vstore<VEC>(dz + idx[u], d[u]);
     }
     // per-channel sums of d and d*zhat over this chunk's pixels
     const int piece = ch.p0 / kPostChunk;
@@ -285,8 +356,8 @@ __device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long
         const int c = c0 + ch.cl0 + cl;
         float a1 = 0.f, a2 = 0.f;
 #pragma unroll
-        for (int k = 0; k < kPostPer; ++k)
-            if (cc[k] == c) { a1 += d[k]; a2 += zv[k]; }
+        for (int u = 0; u < U; ++u)
+            if (cc[u] == c) { a1 += s1[u]; a2 += s2[u]; }
         a1 = warp_sum(a1);
         a2 = warp_sum(a2);
         if (lane == 0) {
@@ -297,11 +368,13 @@ __device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long
 }
 
 // ---------------------------------------------------------------- backward, step 2
+template <int VEC>
 __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long long t, int S, int lane) {
+    constexpr int U = kPostPer / VEC;
     const long long j = t - 2LL * (S - 1) + st.s;
     if (j < 0) return;
     const int slot = slot_of(j, st.slots);
-    const int hw = st.oh * st.ow, cpg = st.cpg, c0 = ch.grp * cpg, n = ch.ncl * ch.np;
+    const int hw = st.oh * st.ow, cpg = st.cpg, c0 = ch.grp * cpg, n = ch.ncl * ch.np, nunits = n / VEC;
     const size_t zelems = (size_t)st.co * hw;
     const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
     const float mean = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0];
@@ -326,42 +399,52 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
     m2 = warp_sum(m2) / (float)(cpg * hw);
     float* __restrict__ dsk = st.dskip
         ? st.dskip + (size_t)slot_of(j, st.dskip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
-    int cc[kPostPer], pp[kPostPer];
-    bool ok[kPostPer];
-    float dnv[kPostPer], zv[kPostPer];
-    ChunkWalk wk(ch, lane);
+    int cc[U], pp[U];
+    bool ok[U];
+    float dnv[U][VEC], zv[U][VEC];
+    ChunkWalk<VEC> wk(ch, lane);
 #pragma unroll
-    for (int k = 0; k < kPostPer; ++k) {              // all loads of the lane's elements first
-        wk.get(ch, c0, n, cc[k], pp[k], ok[k]);
+    for (int u = 0; u < U; ++u) {                     // all loads of the lane's units first
+        wk.get(ch, c0, nunits, cc[u], pp[u], ok[u]);
         wk.next(ch);
-        const size_t idx = (size_t)cc[k] * hw + pp[k];
-        dnv[k] = dz[idx];
-        zv[k] = z[idx];
+        const size_t idx = (size_t)cc[u] * hw + pp[u];
+        vload<VEC>(dnv[u], dz + idx);
+        vload<VEC>(zv[u], z + idx);
     }
 #pragma unroll
-    for (int k = 0; k < kPostPer; ++k) {
-        if (!ok[k]) continue;
-        const int c = cc[k], p = pp[k];
+    for (int u = 0; u < U; ++u) {
+        if (!ok[u]) continue;
+        const int c = cc[u], p = pp[u];
         const size_t idx = (size_t)c * hw + p;
-        const float dn = dnv[k];
         // the skip input joined after the normalisation: it receives dn itself
         if (dsk) {
             if (st.skip_mode == 0) {
-                dsk[idx] = dn;
+                vstore<VEC>(dsk + idx, dnv[u]);
             } else if (c < st.skip_c) {
-                const int y = p / st.ow, x = p % st.ow;
-                for (int dy = 0; dy < 2; ++dy)
-                    for (int dx = 0; dx < 2; ++dx) {
-                        const int ys = 2 * y + dy, xs = 2 * x + dx;
-                        if (ys < st.skip_h && xs < st.skip_w)
-                            dsk[((size_t)c * st.skip_h + ys) * st.skip_w + xs] = (dy | dx) ? 0.f : dn;
-                    }
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) {
+                    const int y = (p + e) / st.ow, x = (p + e) % st.ow;
+                    for (int dy = 0; dy < 2; ++dy)
+                        for (int dx = 0; dx < 2; ++dx) {
+                            const int ys = 2 * y + dy, xs = 2 * x + dx;
+                            if (ys < st.skip_h && xs < st.skip_w)
+                                dsk[((size_t)c * st.skip_h + ys) * st.skip_w + xs] = (dy | dx) ? 0.f : dnv[u][e];
+                        }
+                }
             }
         }
-        const float zh = (zv[k] - mean) * rstd;
-        const float dd = rstd * (fmaf(dn, gam[c], -m1) - zh * m2);
-        dz[idx] = dd;
-        if (st.dz16) st.dz16[(size_t)p * st.co + c] = __float2bfloat16_rn(dd);
+        const float g = gam[c];
+        float dd[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            const float zh = (zv[u][e] - mean) * rstd;
+            dd[e] = rstd * (fmaf(dnv[u][e], g, -m1) - zh * m2);
+        }
+        vstore<VEC>(dz + idx, dd);
+        if (st.dz16) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) st.dz16[(size_t)(p + e) * st.co + c] = __float2bfloat16_rn(dd[e]);
+        }
     }
 }
 
@@ -387,7 +470,8 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
                 __syncwarp();                                                                      \
                 loaded = ch.stage;                                                                 \
             }                                                                                      \
-            CHUNK(sst[warp], ch, t, __VA_ARGS__);                                                  \
+            if (sst[warp].vec4) CHUNK<4>(sst[warp], ch, t, __VA_ARGS__);                           \
+            else CHUNK<1>(sst[warp], ch, t, __VA_ARGS__);                                          \
         }                                                                                          \
     }
 PB_POST_KERNEL(conv_stats_kernel, conv_stats_chunk, lane)
@@ -408,6 +492,41 @@ update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ 
     const long long j = ts->cnt[par] - 2LL * (S - 1) + R.s;
     if (j < 0) return;
     const int end = min(R.n, ch.start + kUpdChunk);
+    const bool vec = ((reinterpret_cast<uintptr_t>(R.w) | reinterpret_cast<uintptr_t>(R.v) | reinterpret_cast<uintptr_t>(R.wh) |
+                       reinterpret_cast<uintptr_t>(R.g)) & 15) == 0 && (R.part_stride & 3) == 0 && (R.n & 3) == 0 &&
+                     (!R.w16 || ((reinterpret_cast<uintptr_t>(R.w16) | reinterpret_cast<uintptr_t>(R.wh16)) & 7) == 0);
+    if (vec) {
+        // four parameters per thread and step (kUpdChunk and ch.start are multiples of 4)
+        for (int e = ch.start + 4 * threadIdx.x; e < end; e += 4 * 256) {
+            float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int q = 0; q < R.nparts; ++q) {
+                const float4 p = *reinterpret_cast<const float4*>(R.g + (size_t)q * R.part_stride + e);
+                g.x += p.x; g.y += p.y; g.z += p.z; g.w += p.w;
+            }
+            const float4 w = *reinterpret_cast<const float4*>(R.w + e), v = *reinterpret_cast<const float4*>(R.v + e);
+            float4 vn, wn, wh;
+            vn.x = fmaf(R.m, v.x, g.x); vn.y = fmaf(R.m, v.y, g.y); vn.z = fmaf(R.m, v.z, g.z); vn.w = fmaf(R.m, v.w, g.w);
+            wn.x = fmaf(R.neg_lr_a, vn.x, fmaf(R.neg_lr_b, g.x, w.x)); wn.y = fmaf(R.neg_lr_a, vn.y, fmaf(R.neg_lr_b, g.y, w.y));
+            wn.z = fmaf(R.neg_lr_a, vn.z, fmaf(R.neg_lr_b, g.z, w.z)); wn.w = fmaf(R.neg_lr_a, vn.w, fmaf(R.neg_lr_b, g.w, w.w));
+            wh.x = fmaf(R.neg_lr_T, vn.x, wn.x); wh.y = fmaf(R.neg_lr_T, vn.y, wn.y);
+            wh.z = fmaf(R.neg_lr_T, vn.z, wn.z); wh.w = fmaf(R.neg_lr_T, vn.w, wn.w);
+            *reinterpret_cast<float4*>(R.v + e) = vn;
+            *reinterpret_cast<float4*>(R.w + e) = wn;
+            if (R.w16) {
+                // tensor-core stages read only the bfloat16 copies of the conv weights
+                __nv_bfloat162 a0 = __floats2bfloat162_rn(wn.x, wn.y), a1 = __floats2bfloat162_rn(wn.z, wn.w);
+                __nv_bfloat162 b0 = __floats2bfloat162_rn(wh.x, wh.y), b1 = __floats2bfloat162_rn(wh.z, wh.w);
+                uint2 ua, ub;
+                ua.x = *reinterpret_cast<unsigned*>(&a0); ua.y = *reinterpret_cast<unsigned*>(&a1);
+                ub.x = *reinterpret_cast<unsigned*>(&b0); ub.y = *reinterpret_cast<unsigned*>(&b1);
+                *reinterpret_cast<uint2*>(R.w16 + e) = ua;
+                *reinterpret_cast<uint2*>(R.wh16 + e) = ub;
+            } else {
+                *reinterpret_cast<float4*>(R.wh + e) = wh;
+            }
+        }
+        return;
+    }
     for (int e = ch.start + threadIdx.x; e < end; e += 256) {
         float g = 0.f;
         for (int q = 0; q < R.nparts; ++q) g += R.g[(size_t)q * R.part_stride + e];
@@ -417,8 +536,8 @@ update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ 
         const float wh = fmaf(R.neg_lr_T, vn, wn);
         R.v[e] = vn;
         R.w[e] = wn;
-        R.wh[e] = wh;
         if (R.w16) { R.w16[e] = __float2bfloat16_rn(wn); R.wh16[e] = __float2bfloat16_rn(wh); }
+        else R.wh[e] = wh;
     }
 }
 

@@ -41,6 +41,7 @@ struct ConvStage {
     int co, oh, ow;              // conv output (z) shape
     int groups, cpg;             // GroupNorm groups, channels per group
     int relu, avgpool;
+    int vec4;                    // oh*ow is a multiple of 4: the element kernels use 4-wide accesses
     int pool_k, pool_stride, pool_pad;   // pool_k == 0: no max-pool
     int out_h, out_w;            // stage output spatial shape (after pooling)
     // forward

@@ -308,6 +308,7 @@ void fill_conv_tables(pb_handle* h) {
         c.s = x.index; c.co = L.c_out; c.oh = x.z.h; c.ow = x.z.w;
         c.groups = x.gn_groups; c.cpg = L.c_out / x.gn_groups;
         c.relu = x.relu; c.avgpool = x.avgpool;
+        c.vec4 = ((x.z.h * x.z.w) % 4 == 0) ? 1 : 0;
         c.pool_k = x.has_pool ? x.pool_k : 0; c.pool_stride = x.pool_stride; c.pool_pad = x.pool_pad;
         c.out_h = x.out.h; c.out_w = x.out.w;
         c.zpart = x.zpart; c.z_nsplit = x.split_f;
