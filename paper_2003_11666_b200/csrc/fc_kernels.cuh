@@ -46,6 +46,13 @@ template <> __device__ __forceinline__ void vstore<4>(float* p, const float (&r)
 }
 template <> __device__ __forceinline__ void vstore<1>(float* p, const float (&r)[1]) { *p = r[0]; }
 
+// streaming store: updated weights are not read again before the next tick
+template <int VEC> __device__ __forceinline__ void vstore_stream(float* p, const float (&r)[VEC]);
+template <> __device__ __forceinline__ void vstore_stream<4>(float* p, const float (&r)[4]) {
+    __stcs(reinterpret_cast<float4*>(p), make_float4(r[0], r[1], r[2], r[3]));
+}
+template <> __device__ __forceinline__ void vstore_stream<1>(float* p, const float (&r)[1]) { __stcs(p, r[0]); }
+
 __device__ __forceinline__ int ring_slot(long long sample, int slots) {
     return (int)((unsigned)sample % (unsigned)slots);   // samples stay far below 2^32
 }
@@ -204,11 +211,13 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
                 if (do_bwd) vload<VEC>(xbr[c], xb + col[c]);
             }
         }
-        // rows of this row split, four at a time
-        for (int r0 = rs * 4; r0 < rows; r0 += nrs * 4) {
-            float wv[4][kFcChunksPerSweep][VEC], vv[4][kFcChunksPerSweep][VEC];
+        // Rows of this row split, two at a time, software-pipelined: the loads of the
+        // next pair are issued before the current pair is used, so a warp always has a
+        // full set of loads in flight while it computes and stores.
+        const int step = nrs * 2;
+        auto load_pair = [&](float (&wv)[2][kFcChunksPerSweep][VEC], float (&vv)[2][kFcChunksPerSweep][VEC], int r0) {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < 2; ++u) {
                 const int r = r0 + u;
 #pragma unroll
                 for (int c = 0; c < kFcChunksPerSweep; ++c) {
@@ -221,9 +230,11 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
                     }
                 }
             }
-            float facc[4];
+        };
+        auto use_pair = [&](float (&wv)[2][kFcChunksPerSweep][VEC], float (&vv)[2][kFcChunksPerSweep][VEC], int r0) {
+            float facc[2];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < 2; ++u) {
                 const int r = r0 + u;
                 facc[u] = 0.f;
                 const float d = (do_bwd && r < rows) ? sh.delta[r] : 0.f;
@@ -242,18 +253,38 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
                     }
                     if (do_bwd && r < rows && cok[c]) {
                         const size_t off = (size_t)(seg.row0 + r) * in + col[c];
-                        vstore<VEC>(st.w + off, wn);
-                        vstore<VEC>(st.v + off, vn);
+                        vstore_stream<VEC>(st.w + off, wn);
+                        vstore_stream<VEC>(st.v + off, vn);
                     }
                 }
             }
-            if (do_fwd) {
-                const float tot = warp_sum4(facc[0], facc[1], facc[2], facc[3], lane);
-                const int q = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
-                if ((lane & 7) == 0 && r0 + q < rows) {
+            if (do_fwd && r0 < rows) {
+                // two row sums with 5 shuffles: lanes 0-15 end with row r0, lanes 16-31 with row r0+1
+                const bool hi = lane & 16;
+                float keep = hi ? facc[1] : facc[0];
+                const float send = hi ? facc[0] : facc[1];
+                keep += __shfl_xor_sync(0xffffffffu, send, 16);
+                keep += __shfl_xor_sync(0xffffffffu, keep, 8);
+                keep += __shfl_xor_sync(0xffffffffu, keep, 4);
+                keep += __shfl_xor_sync(0xffffffffu, keep, 2);
+                keep += __shfl_xor_sync(0xffffffffu, keep, 1);
+                const int q = lane >> 4;
+                if ((lane & 15) == 0 && r0 + q < rows) {
                     float* slot = &sh.rowpart[cg][r0 + q];
-                    *slot = (c0 == 0 ? 0.f : *slot) + tot;
+                    *slot = (c0 == 0 ? 0.f : *slot) + keep;
                 }
+            }
+        };
+        {
+            float wa[2][kFcChunksPerSweep][VEC], va[2][kFcChunksPerSweep][VEC];
+            float wb[2][kFcChunksPerSweep][VEC], vb[2][kFcChunksPerSweep][VEC];
+            int r0 = rs * 2;
+            load_pair(wa, va, r0);
+            for (; r0 < rows; r0 += 2 * step) {
+                load_pair(wb, vb, r0 + step);
+                use_pair(wa, va, r0);
+                load_pair(wa, va, r0 + 2 * step);
+                use_pair(wb, vb, r0 + step);
             }
         }
         // column partials: combine the row splits in a fixed order, then store
