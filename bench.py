@@ -217,9 +217,12 @@ def main():
         # conv parameters: read w, v, g; write w, v, predicted w
         k_ms, k_n = classes["update"]
         alg_bytes, kernel = 28.0 * (P - p_last), "update_kernel"
+    # DRAM bytes per launch of that kernel from the ncu capture summarised under profiles/
+    # (dram__bytes_read.sum + dram__bytes_write.sum, steady-state tick); None where not captured
+    traffic = {"mlp16x2048": 506.60e6 + 448.82e6}.get(args.workload) if all_fc else None
     achieved = alg_bytes / (k_ms / k_n * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_source": peak_kind,
+                "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind,
                 "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": k_ms / k_n, "launches_timed": k_n,
                 "us_per_tick_by_class": {n: (1e3 * m / kp if c else 0.0) for n, (m, c) in classes.items()}}
 
