@@ -85,6 +85,27 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(ms, world, device="cuda"):
+    """Slowest rank's time: the job is done when the last replica is."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world, ticks_per_rank, ms):
+    """Whole-job ticks/s: every replica ran `ticks_per_rank` ticks within `ms`."""
+    return world * ticks_per_rank / (ms * 1e-3)
+
+
+def replica_seed(base_seed, rank):
+    """Replicas see different sample streams."""
+    return base_seed + 1000 * rank
+
+
 def time_oracle(wl, budget_s=20.0, max_ticks=None):
     """Times the CPU checker as it stands on steady-state ticks of `wl`."""
     from oracle import PBOracle
@@ -158,7 +179,7 @@ def main():
     wl = workload(args.workload)
     K, W = args.steps, max(args.warmup, 3)
     S = wl.n_stages
-    seed = wl.seed + 1000 * rank            # replicas see different sample streams
+    seed = replica_seed(wl.seed, rank)
     x, y = make_inputs(seed, K + W, wl.sample_elems, wl.n_classes)
     stream = torch.cuda.current_stream()
     eng = pbm.PB(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, wl.lr, wl.momentum,
@@ -171,13 +192,6 @@ def main():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
-
-    def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
 
     # ---- device-resident timing: W warm-up ticks (fills the pipeline), then K ticks
     eng.run(xd[:W], yd[:W], W, losses[:W])
@@ -193,9 +207,9 @@ def main():
     e1.record(stream)
     barrier()
     launches = eng.last_launch_count
-    ms = max_over_ranks(e0.elapsed_time(e1))
+    ms = max_over_ranks(e0.elapsed_time(e1), world)
     clocks = sampler.stop() if rank == 0 else None
-    value = world * K / (ms * 1e-3)
+    value = job_value(world, K, ms)
 
     # ---- per-kernel durations (CUDA events on the engine's stream, separate pass)
     eng.profile_enable(True)
@@ -236,8 +250,8 @@ def main():
     t0 = time.perf_counter()
     eng.run_host(hx[W:], hy[W:], K, hl[W:])
     torch.cuda.synchronize()
-    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
-    e2e = {"value": world * K / (e2e_ms * 1e-3), "unit": UNIT,
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, world)
+    e2e = {"value": job_value(world, K, e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": wl.sample_elems * 4 + 4, "d2h_bytes_per_step": 4}
     finite_ticks = int(np.isfinite(hl[W:].numpy()).sum())
     eng.destroy()

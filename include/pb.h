@@ -110,7 +110,8 @@ int pb_tick(pb_handle* h, const float* dev_x, int label, float* host_loss);
  * sample again at its backward 2(S-1) ticks later); dev_losses: [n_ticks]
  * floats (device) or NULL, entry k receiving what pb_tick would have returned
  * at the k-th tick of this call.  Continues from the current tick, so
- * consecutive calls feed one continuous stream of samples. */
+ * consecutive calls feed one continuous stream of samples.  n_ticks == 0 is a
+ * no-op (the pointers are not examined); a negative count is PB_E_ARG. */
 int pb_run(pb_handle* h, const float* dev_xs, const int32_t* dev_labels,
            int n_ticks, float* dev_losses);
 

@@ -200,7 +200,7 @@ void choose_split(int M, int N, int K, int num_sms, int& nsplit, int& kps) {
 
 void choose_split_tc(int M, int N, int bn, int K, int num_sms, int& nsplit, int& kps) {
     const int tiles = ceil_div(M, kTcBM) * ceil_div(N, bn);
-    int want = ceil_div(2 * num_sms, tiles);
+    int want = ceil_div(num_sms, tiles);
     int by_k = K / (2 * kTcChunk);
     if (by_k < 1) by_k = 1;
     nsplit = std::max(1, std::min(std::min(want, by_k), 16));
@@ -743,15 +743,15 @@ int pb_tick(pb_handle* h, const float* dev_x, int label, float* host_loss) {
 
 int pb_run(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int n_ticks, float* dev_losses) {
     if (!h) return PB_E_ARG;
+    if (n_ticks == 0) return PB_OK;         // nothing to do; the pointers are not looked at
     if (!dev_xs || !dev_labels || n_ticks < 0) return fail(h, PB_E_ARG, "pb_run: NULL pointer or negative count");
-    if (n_ticks == 0) return PB_OK;
     return run_ticks(h, dev_xs, dev_labels, 0, n_ticks, dev_losses);
 }
 
 int pb_run_host(pb_handle* h, const float* host_xs, const int32_t* host_labels, int n_ticks, float* host_losses) {
     if (!h) return PB_E_ARG;
-    if (!host_xs || !host_labels || n_ticks < 0) return fail(h, PB_E_ARG, "pb_run_host: NULL pointer or negative count");
     if (n_ticks == 0) return PB_OK;
+    if (!host_xs || !host_labels || n_ticks < 0) return fail(h, PB_E_ARG, "pb_run_host: NULL pointer or negative count");
     const size_t xb = (size_t)n_ticks * h->in_shape.elems() * sizeof(float);
     const size_t lb = (size_t)n_ticks * sizeof(int32_t), fb = (size_t)n_ticks * sizeof(float);
     const size_t o1 = align_up(xb, 256), o2 = o1 + align_up(lb, 256), need = o2 + align_up(fb, 256);

@@ -113,3 +113,49 @@ def test_bad_arguments_are_reported_not_thrown_across_the_abi():
     with pytest.raises(PBError):
         e.tick(0, 99)
     e.destroy()
+
+
+def test_single_stage_network_on_the_gpu():
+    # S = 1: delay 0, the sample and its label are consumed in the tick that ingests them
+    wl = mlp([40, 6], lr=0.01, seed=8)
+    w = compare_ticks(wl, 20, TOL)
+    assert w["ticks"] == 20
+
+
+def test_last_stage_too_large_to_fuse_uses_its_own_launch():
+    # 300 outputs (> 256 rows): the loss/backward of the last stage is a second launch
+    import torch
+    wl = mlp([96, 64, 300], lr=0.002, seed=9)
+    w = compare_ticks(wl, 2 * (wl.n_stages - 1) + 16, TOL)
+    assert w["ticks"] == 2 * (wl.n_stages - 1) + 16
+    e = make_engine(wl)
+    x, y = make_inputs(wl.seed, 4, wl.sample_elems, wl.n_classes)
+    e.run(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda(), 4)
+    e.sync()
+    assert e.last_launch_count == 8
+    e.destroy()
+
+
+def test_consecutive_runs_and_ticks_form_one_stream_and_zero_ticks_is_a_no_op():
+    import torch
+    wl = mlp([48, 40, 24, 5], lr=0.003, seed=10)
+    n = 30
+    x, y = make_inputs(wl.seed, n, wl.sample_elems, wl.n_classes)
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    a, b = make_engine(wl), make_engine(wl)
+    la = torch.zeros(n, device="cuda")
+    a.run(xd, yd, n, la)
+    lb = torch.zeros(n, device="cuda")
+    b.run(xd[:7], yd[:7], 7, lb[:7])
+    b.run(xd[7:7], yd[7:7], 0, None)                       # nothing happens
+    one = b.tick(xd[7], int(y[7]))                           # odd tick count in between
+    b.run(xd[8:], yd[8:], n - 8, lb[8:])
+    a.sync(); b.sync()
+    S = wl.n_stages
+    got_a, got_b = la.cpu().numpy(), lb.cpu().numpy()
+    got_b[7] = one
+    np.testing.assert_array_equal(got_a[S - 1:], got_b[S - 1:])
+    np.testing.assert_array_equal(a.get_weights(), b.get_weights())
+    np.testing.assert_array_equal(a.get_velocity(), b.get_velocity())
+    assert b.tick_count == n
+    a.destroy(); b.destroy()
