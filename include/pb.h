@@ -74,8 +74,11 @@ typedef struct {
 
 /* Mitigation switches (Section "Methods").  PB_SC: a = m^D, b = (1-m^D)/(1-m),
  * else a = 1, b = 0.  PB_LWP: forward weights w_hat = w - lr*T*v with T = D,
- * else T = 0.  PB_CONV_BF16: convolutions multiply bf16 operands with fp32
- * accumulation; master weights, velocity and everything else stay fp32. */
+ * else T = 0.  PB_LWP_WFORM (with PB_LWP): predict with the weight-difference
+ * form w_hat = w + T (w - w_previous) instead of the velocity form; the two
+ * differ once SC is on (Section "Combined Mitigation").  PB_CONV_BF16:
+ * convolutions multiply bf16 operands with fp32 accumulation; master weights,
+ * velocity and everything else stay fp32. */
 enum { PB_SC = 1, PB_LWP = 2, PB_LWP_WFORM = 4, PB_CONV_BF16 = 8 };
 
 /* Builds the engine.  layers/stage_of_layer: host arrays of n_layers entries,
@@ -93,6 +96,14 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
 /* Copies n = pb_num_params() floats from host memory into the master weights,
  * zeroes the velocity and restarts the pipeline at tick 0. */
 int pb_set_weights(pb_handle* h, const float* host_w, size_t n);
+
+/* Over- or under-compensation (paper: generalized Spike Compensation with
+ * other a, b, e.g. SC_2D; Appendix "Extended Weight Prediction Horizons",
+ * T = alpha D).  Stage s then uses a = m^(sc_delay_scale * D_s),
+ * b = (1 - a)/(1 - m) and T = horizon_scale * D_s; (1, 1) is the default
+ * SC_D + LWP_D.  Takes effect for ticks issued after the call; synchronises
+ * the stream.  Scales must be >= 0. */
+int pb_set_mitigation(pb_handle* h, float sc_delay_scale, float horizon_scale);
 
 /* One tick.  dev_x: the new sample (in_c*in_h*in_w floats, device memory; it
  * is copied into the engine's input ring, so it may be reused after the call

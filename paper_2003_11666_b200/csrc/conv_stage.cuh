@@ -508,8 +508,13 @@ update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ 
             vn.x = fmaf(R.m, v.x, g.x); vn.y = fmaf(R.m, v.y, g.y); vn.z = fmaf(R.m, v.z, g.z); vn.w = fmaf(R.m, v.w, g.w);
             wn.x = fmaf(R.neg_lr_a, vn.x, fmaf(R.neg_lr_b, g.x, w.x)); wn.y = fmaf(R.neg_lr_a, vn.y, fmaf(R.neg_lr_b, g.y, w.y));
             wn.z = fmaf(R.neg_lr_a, vn.z, fmaf(R.neg_lr_b, g.z, w.z)); wn.w = fmaf(R.neg_lr_a, vn.w, fmaf(R.neg_lr_b, g.w, w.w));
-            wh.x = fmaf(R.neg_lr_T, vn.x, wn.x); wh.y = fmaf(R.neg_lr_T, vn.y, wn.y);
-            wh.z = fmaf(R.neg_lr_T, vn.z, wn.z); wh.w = fmaf(R.neg_lr_T, vn.w, wn.w);
+            if (R.wform) {
+                wh.x = fmaf(R.T_w, wn.x - w.x, wn.x); wh.y = fmaf(R.T_w, wn.y - w.y, wn.y);
+                wh.z = fmaf(R.T_w, wn.z - w.z, wn.z); wh.w = fmaf(R.T_w, wn.w - w.w, wn.w);
+            } else {
+                wh.x = fmaf(R.neg_lr_T, vn.x, wn.x); wh.y = fmaf(R.neg_lr_T, vn.y, wn.y);
+                wh.z = fmaf(R.neg_lr_T, vn.z, wn.z); wh.w = fmaf(R.neg_lr_T, vn.w, wn.w);
+            }
             *reinterpret_cast<float4*>(R.v + e) = vn;
             *reinterpret_cast<float4*>(R.w + e) = wn;
             if (R.w16) {
@@ -533,7 +538,7 @@ update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ 
         const float w = R.w[e], v = R.v[e];
         const float vn = fmaf(R.m, v, g);
         const float wn = fmaf(R.neg_lr_a, vn, fmaf(R.neg_lr_b, g, w));
-        const float wh = fmaf(R.neg_lr_T, vn, wn);
+        const float wh = R.wform ? fmaf(R.T_w, wn - w, wn) : fmaf(R.neg_lr_T, vn, wn);
         R.v[e] = vn;
         R.w[e] = wn;
         if (R.w16) { R.w16[e] = __float2bfloat16_rn(wn); R.wh16[e] = __float2bfloat16_rn(wh); }

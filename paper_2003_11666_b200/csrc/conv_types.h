@@ -77,6 +77,7 @@ struct UpdRange {
     int n;
     int s;
     float neg_lr_T, m, neg_lr_a, neg_lr_b;
+    float T_w; int wform;        // weight-difference form: w_hat = w_new + T (w_new - w_old)
 };
 struct UpdChunk { int range, start; };
 

@@ -109,7 +109,7 @@ __device__ __forceinline__ float gather_delta(const FcStage& st, int r, long lon
 // phase 0: every stage's forward, and backward + update of every stage but the
 //          last (whose gradient only exists once its own forward is done);
 // phase 1: the last stage's loss, backward and update.
-template <int VEC>
+template <int VEC, bool WF>
 __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int S, int phase,
                            const int* __restrict__ label_ring, float* __restrict__ loss_out,
                            FcShared& sh, TickState* ts, const float* __restrict__ x_now, int label_now) {
@@ -193,7 +193,7 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
     while (ncg * 2 <= nchunks && ncg * 2 <= kFcWarps) ncg *= 2;
     const int nrs = kFcWarps / ncg;
     const int cg = warp % ncg, rs = warp / ncg;
-    const float nlT = st.neg_lr_T, m = st.m, nla = st.neg_lr_a, nlb = st.neg_lr_b;
+    const float nlT = st.neg_lr_T, m = st.m, nla = st.neg_lr_a, nlb = st.neg_lr_b, Tw = st.T_w;
     const bool want_dx = do_bwd && st.need_dx;
 
     for (int c0 = 0; c0 < nchunks; c0 += ncg * kFcChunksPerSweep) {
@@ -215,23 +215,28 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
         // next pair are issued before the current pair is used, so a warp always has a
         // full set of loads in flight while it computes and stores.
         const int step = nrs * 2;
-        auto load_pair = [&](float (&wv)[2][kFcChunksPerSweep][VEC], float (&vv)[2][kFcChunksPerSweep][VEC], int r0) {
+        // (WF: the weight-difference form keeps its predicted weights in memory; they ride
+        //  in the slot of the velocity operand's twin `hv`)
+        auto load_pair = [&](float (&wv)[2][kFcChunksPerSweep][VEC], float (&vv)[2][kFcChunksPerSweep][VEC],
+                             float (&hv)[2][kFcChunksPerSweep][VEC], int r0) {
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
                 const int r = r0 + u;
 #pragma unroll
                 for (int c = 0; c < kFcChunksPerSweep; ++c) {
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) { wv[u][c][e] = 0.f; vv[u][c][e] = 0.f; }
+                    for (int e = 0; e < VEC; ++e) { wv[u][c][e] = 0.f; vv[u][c][e] = 0.f; if (WF) hv[u][c][e] = 0.f; }
                     if (r < rows && cok[c]) {
                         const size_t off = (size_t)(seg.row0 + r) * in + col[c];
                         vload_stream<VEC>(wv[u][c], st.w + off);
                         if (do_bwd) vload_stream<VEC>(vv[u][c], st.v + off);
+                        if (WF && do_fwd) vload_stream<VEC>(hv[u][c], st.wh + off);
                     }
                 }
             }
         };
-        auto use_pair = [&](float (&wv)[2][kFcChunksPerSweep][VEC], float (&vv)[2][kFcChunksPerSweep][VEC], int r0) {
+        auto use_pair = [&](float (&wv)[2][kFcChunksPerSweep][VEC], float (&vv)[2][kFcChunksPerSweep][VEC],
+                            float (&hv)[2][kFcChunksPerSweep][VEC], int r0) {
             float facc[2];
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
@@ -240,21 +245,23 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
                 const float d = (do_bwd && r < rows) ? sh.delta[r] : 0.f;
 #pragma unroll
                 for (int c = 0; c < kFcChunksPerSweep; ++c) {
-                    float wn[VEC], vn[VEC];
+                    float wn[VEC], vn[VEC], hn[VEC];
 #pragma unroll
                     for (int e = 0; e < VEC; ++e) {
                         const float w = wv[u][c][e], v = vv[u][c][e];
-                        const float what = fmaf(nlT, v, w);          // w_hat = w - lr T v
+                        const float what = WF ? hv[u][c][e] : fmaf(nlT, v, w);   // w_hat = w - lr T v (or the stored prediction)
                         facc[u] = fmaf(what, xfr[c][e], facc[u]);     // forward  (W_hat x)
                         cacc[c][e] = fmaf(w, d, cacc[c][e]);          // backward (W^T delta)
                         const float g = d * xbr[c][e];                // rank-1 gradient
                         vn[e] = fmaf(m, v, g);                        // v <- m v + g
                         wn[e] = fmaf(nla, vn[e], fmaf(nlb, g, w));    // w <- w - lr (a v + b g)
+                        hn[e] = fmaf(Tw, wn[e] - w, wn[e]);           // w_hat = w_new + T (w_new - w_old)
                     }
                     if (do_bwd && r < rows && cok[c]) {
                         const size_t off = (size_t)(seg.row0 + r) * in + col[c];
                         vstore_stream<VEC>(st.w + off, wn);
                         vstore_stream<VEC>(st.v + off, vn);
+                        if (WF) vstore_stream<VEC>(st.wh + off, hn);
                     }
                 }
             }
@@ -276,15 +283,16 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
             }
         };
         {
-            float wa[2][kFcChunksPerSweep][VEC], va[2][kFcChunksPerSweep][VEC];
-            float wb[2][kFcChunksPerSweep][VEC], vb[2][kFcChunksPerSweep][VEC];
+            // (ha / hb are only touched when WF is set; otherwise they cost nothing)
+            float wa[2][kFcChunksPerSweep][VEC], va[2][kFcChunksPerSweep][VEC], ha[2][kFcChunksPerSweep][VEC];
+            float wb[2][kFcChunksPerSweep][VEC], vb[2][kFcChunksPerSweep][VEC], hb[2][kFcChunksPerSweep][VEC];
             int r0 = rs * 2;
-            load_pair(wa, va, r0);
+            load_pair(wa, va, ha, r0);
             for (; r0 < rows; r0 += 2 * step) {
-                load_pair(wb, vb, r0 + step);
-                use_pair(wa, va, r0);
-                load_pair(wa, va, r0 + 2 * step);
-                use_pair(wb, vb, r0 + step);
+                load_pair(wb, vb, hb, r0 + step);
+                use_pair(wa, va, ha, r0);
+                load_pair(wa, va, ha, r0 + 2 * step);
+                use_pair(wb, vb, hb, r0 + step);
             }
         }
         // column partials: combine the row splits in a fixed order, then store
@@ -327,15 +335,17 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
         if (do_fwd) {
             float y = 0.f;
             for (int k = 0; k < ncg; ++k) y += sh.rowpart[k][r];
-            y += fmaf(nlT, vb, b);
+            y += WF ? st.wh[(size_t)out * in + row] : fmaf(nlT, vb, b);
             if (st.relu) y = fmaxf(y, 0.f);
             st.out[(size_t)ring_slot(i, st.out_slots) * out + row] = y;
         }
         if (do_bwd) {
             const float g = sh.delta[r];
             const float vn = fmaf(m, vb, g);
+            const float bn = fmaf(nla, vn, fmaf(nlb, g, b));
             vbias[row] = vn;
-            bias[row] = fmaf(nla, vn, fmaf(nlb, g, b));
+            bias[row] = bn;
+            if (WF) st.wh[(size_t)out * in + row] = fmaf(Tw, bn - b, bn);
         }
     }
 }
@@ -379,8 +389,13 @@ fc_tick_kernel(const FcStage* __restrict__ stages, const FcSeg* __restrict__ seg
         const int nph = seg.fused ? 2 : 1;
         for (int ph = 0; ph < nph; ++ph) {
             const int phs = seg.fused ? ph : phase;
-            if (st.vec == 4) fc_segment<4>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
-            else fc_segment<1>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+            if (st.wh) {
+                if (st.vec == 4) fc_segment<4, true>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+                else fc_segment<1, true>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+            } else {
+                if (st.vec == 4) fc_segment<4, false>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+                else fc_segment<1, false>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+            }
             __syncthreads();      // the logits written by phase 0 are read by phase 1
         }
     }

@@ -108,21 +108,28 @@ int parse_layers(pb_handle* h, const pb_layer* layers, int n_layers, const int32
     return PB_OK;
 }
 
+// SC coefficients for the delay alpha_sc * D and LWP horizon alpha_T * D of one stage
+// (alpha = 1: SC_D and LWP_D; alpha = 2: the over-compensating SC_2D / LWP_2D variants).
+void mitigation_constants(const pb_handle* h, StageHost& x) {
+    const double m = h->momentum;
+    double a = 1.0, b = 0.0;
+    if (h->flags & PB_SC) {
+        const double d = (double)h->sc_delay_scale * x.delay;
+        a = std::pow(m, d);
+        b = (1.0 - a) / (1.0 - m);            // 0 <= m < 1 is checked at pb_create
+    }
+    x.a = (float)a; x.b = (float)b;
+    x.T = (h->flags & PB_LWP) ? h->horizon_scale * (float)x.delay : 0.f;
+}
+
 // Per-stage constants: delay (Eq. F_i), SC_D coefficients, LWP horizon.
 void schedule_constants(pb_handle* h) {
     const int S = h->S;
-    const double m = h->momentum;
     size_t dev_off = 0;
     h->all_fc = true;
     for (StageHost& x : h->stages) {
         x.delay = 2 * (S - 1 - x.index);
-        double a = 1.0, b = 0.0;
-        if (h->flags & PB_SC) {
-            a = std::pow(m, (double)x.delay);
-            b = (m == 1.0) ? (double)x.delay : (1.0 - a) / (1.0 - m);
-        }
-        x.a = (float)a; x.b = (float)b;
-        x.T = (h->flags & PB_LWP) ? (float)x.delay : 0.f;
+        mitigation_constants(h, x);
         x.dev_off = dev_off;
         dev_off += align_up(x.n_params, 64);
         if (x.head_op != PB_FC) h->all_fc = false;
@@ -349,6 +356,7 @@ void fill_conv_tables(pb_handle* h) {
 
         UpdRange r{};
         r.s = x.index; r.neg_lr_T = -h->lr * x.T; r.m = h->momentum; r.neg_lr_a = -h->lr * x.a; r.neg_lr_b = -h->lr * x.b;
+        r.T_w = x.T; r.wform = (h->flags & PB_LWP_WFORM) ? 1 : 0;
         r.w = h->d_w + x.dev_off; r.v = h->d_v + x.dev_off; r.wh = h->d_wh + x.dev_off;
         r.g = x.gpart; r.nparts = x.split_w; r.part_stride = nw; r.n = nw;
         if (x.tc) { r.w16 = h->d_w16 + x.dev_off; r.wh16 = h->d_wh16 + x.dev_off; }
@@ -414,7 +422,7 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     h->d_tc = c.take<ConvGemmTC>(h->h_tc.size() + 1);
     for (int q = 0; q < 3; ++q) h->d_tctiles[q] = c.take<GemmTile>(h->h_tctiles[q].size() + 1);
     h->d_w = c.take<float>(h->dev_params);
-    if (!h->all_fc) h->d_wh = c.take<float>(h->dev_params);
+    if (!h->all_fc || (h->flags & PB_LWP_WFORM)) h->d_wh = c.take<float>(h->dev_params);
     *zero_from = c.off;
     h->d_v = c.take<float>(h->dev_params);
     if (!h->all_fc) h->d_g = c.take<float>(h->dev_params);
@@ -462,6 +470,9 @@ void fill_fc_tables(pb_handle* h) {
         const StageHost& x = h->stages[f.s];
         f.w = h->d_w + x.dev_off;
         f.v = h->d_v + x.dev_off;
+        f.neg_lr_T = -h->lr * x.T; f.m = h->momentum; f.neg_lr_a = -h->lr * x.a; f.neg_lr_b = -h->lr * x.b;
+        f.T_w = x.T;
+        f.wh = ((h->flags & PB_LWP_WFORM) && h->d_wh) ? h->d_wh + x.dev_off : nullptr;
         if (x.src < 0) { f.xin = h->in_ring; f.xin_slots = h->in_slots; }
         else { f.xin = h->stages[x.src].out_ring; f.xin_slots = h->stages[x.src].out_slots; }
         f.out = x.out_ring; f.out_slots = x.out_slots;
@@ -617,7 +628,7 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
         return fail(nullptr, PB_E_ARG, "pb_create: NULL pointer or non-positive size");
     if (!(momentum >= 0.f && momentum < 1.f) || !(lr >= 0.f)) return fail(nullptr, PB_E_ARG, "pb_create: need 0 <= momentum < 1 and lr >= 0");
     if (flags & ~(unsigned)(PB_SC | PB_LWP | PB_LWP_WFORM | PB_CONV_BF16)) return fail(nullptr, PB_E_ARG, "pb_create: unknown flag");
-    if (flags & PB_LWP_WFORM) return fail(nullptr, PB_E_UNSUPPORTED, "pb_create: the weight-difference form of LWP is not built");
+    if ((flags & PB_LWP_WFORM) && !(flags & PB_LWP)) return fail(nullptr, PB_E_ARG, "pb_create: PB_LWP_WFORM needs PB_LWP");
     for (int q = 1; q < n_layers; ++q)
         if (stage_of_layer[q] < stage_of_layer[q - 1]) return fail(nullptr, PB_E_ARG, "pb_create: stage indices must not decrease");
     pb_handle* h = new (std::nothrow) pb_handle();
@@ -726,6 +737,24 @@ int pb_set_weights(pb_handle* h, const float* host_w, size_t n) {
         cast_weights_kernel<<<(int)h->h_chunks.size(), 256, 0, h->stream>>>(h->d_upd, h->d_chunks);
     PB_CUDA(h, cudaStreamSynchronize(h->stream));
     h->tick = 0;
+    return PB_OK;
+}
+
+int pb_set_mitigation(pb_handle* h, float sc_delay_scale, float horizon_scale) {
+    if (!h) return PB_E_ARG;
+    if (!(sc_delay_scale >= 0.f) || !(horizon_scale >= 0.f)) return fail(h, PB_E_ARG, "pb_set_mitigation: scales must be >= 0");
+    h->sc_delay_scale = sc_delay_scale;
+    h->horizon_scale = horizon_scale;
+    for (StageHost& x : h->stages) mitigation_constants(h, x);
+    fill_fc_tables(h);
+    fill_conv_tables(h);
+    // the tables take effect for launches issued after this call (stream order)
+    PB_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (!h->h_fc.empty())
+        PB_CUDA(h, cudaMemcpyAsync(h->d_fc, h->h_fc.data(), h->h_fc.size() * sizeof(FcStage), cudaMemcpyHostToDevice, h->stream));
+    if (!h->h_upd.empty())
+        PB_CUDA(h, cudaMemcpyAsync(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange), cudaMemcpyHostToDevice, h->stream));
+    PB_CUDA(h, cudaStreamSynchronize(h->stream));
     return PB_OK;
 }
 

@@ -38,6 +38,8 @@ struct FcStage {
     int n_dsrc;
     DeltaSrc dsrc[kMaxDeltaSrc];
     float neg_lr_T;        // -lr * T      (LWP horizon)
+    float T_w;             // T itself, for the weight-difference form
+    float* wh;             // stored predicted weights (weight-difference form only), else nullptr
     float m;               // momentum
     float neg_lr_a;        // -lr * a      (spike compensation)
     float neg_lr_b;        // -lr * b

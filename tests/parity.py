@@ -38,7 +38,7 @@ def make_engine(wl):
 
 
 def compare_ticks(wl, n_ticks, tol, check_every=1, finite_limit=1e30, loose_after=None,
-                  fragile_margin=None, fragile_tol=None, spread_factor=None):
+                  fragile_margin=None, fragile_tol=None, spread_factor=None, mitigation=None):
     """Tick both sides one sample at a time; returns the worst errors seen.
 
     The window ends early (returning the tick) once the checker's own state
@@ -59,10 +59,15 @@ def compare_ticks(wl, n_ticks, tol, check_every=1, finite_limit=1e30, loose_afte
     max(tol, spread_factor * distance between its float32 and float64 runs)."""
     import torch
     x, y = make_inputs(wl.seed, n_ticks, wl.sample_elems, wl.n_classes)
-    o = make_oracle(wl, margins=fragile_margin is not None)
+    okw = {}
+    if mitigation is not None:       # (SC delay scale, LWP horizon scale), e.g. (2, 2) for SC_2D + LWP_2D
+        okw = dict(sc_delay_scale=mitigation[0], horizon_scale=mitigation[1])
+    o = make_oracle(wl, margins=fragile_margin is not None, **okw)
     fragile_tick = None
-    o32 = make_oracle(wl, dtype=np.float32) if spread_factor is not None else None
+    o32 = make_oracle(wl, dtype=np.float32, **okw) if spread_factor is not None else None
     eng = make_engine(wl)
+    if mitigation is not None:
+        eng.set_mitigation(*mitigation)
     xd = torch.from_numpy(x).cuda()
     worst = {"loss": 0.0, "w": 0.0, "v": 0.0, "ticks": 0, "fragile_tick": None, "strict_w": 0.0, "strict_v": 0.0}
     for t in range(n_ticks):

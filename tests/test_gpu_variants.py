@@ -1,0 +1,53 @@
+"""Mitigation variants of the paper on the GPU against the CPU checker: the
+weight-difference form of LWP (with and without SC), over-compensation
+(SC_2D, LWP_2D) and horizons T = alpha D."""
+import pytest
+
+from pb_workloads import mlp, tiny_cnn, tiny_resnet
+from tests.parity import compare_ticks
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-4
+
+
+@pytest.mark.parametrize("make", [lambda f: mlp([48, 40, 33, 24, 5], lr=0.003, seed=31, flags=f),
+                                  lambda f: tiny_cnn(flags=f), lambda f: _resnet(f)])
+@pytest.mark.parametrize("flags", [7, 6])
+def test_weight_difference_form(make, flags):
+    wl = make(flags)
+    n = 2 * (wl.n_stages - 1) + 20
+    w = compare_ticks(wl, n, TOL)
+    assert w["ticks"] == n
+
+
+def _resnet(flags):
+    wl = tiny_resnet()
+    wl.flags = flags
+    return wl
+
+
+@pytest.mark.parametrize("make", [lambda: mlp([48, 40, 33, 24, 5], lr=0.003, seed=32), tiny_cnn])
+@pytest.mark.parametrize("scales", [(2.0, 2.0), (2.0, 1.0), (1.0, 2.0), (0.0, 0.5)])
+def test_over_and_under_compensation(make, scales):
+    wl = make()
+    n = 2 * (wl.n_stages - 1) + 20
+    w = compare_ticks(wl, n, TOL, mitigation=scales)
+    assert w["ticks"] == n
+
+
+def test_mitigation_scale_arguments_are_checked():
+    from paper_2003_11666_b200 import PBError
+    from tests.parity import make_engine
+    e = make_engine(mlp([8, 6, 4]))
+    with pytest.raises(PBError):
+        e.set_mitigation(-1.0, 1.0)
+    e.set_mitigation(1.0, 1.0)
+    e.destroy()
+
+
+def test_wform_needs_lwp():
+    from paper_2003_11666_b200 import PB, PBError
+    wl = mlp([8, 6, 4])
+    with pytest.raises(PBError):
+        PB(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, 0.1, 0.9, flags=4)

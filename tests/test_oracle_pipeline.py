@@ -187,3 +187,18 @@ def test_rejects_stage_without_head():
     wl = Workload("bad", [Layer(OP.RELU)], [0], (3, 1, 1), 3, 0.1, 0.9, 1, 0)
     with pytest.raises(Exception):
         PBOracle(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, 0.1, 0.9)
+
+
+def test_compensation_scales_set_the_stage_constants():
+    # SC with alpha*D and horizon alpha*D (SC_2D / LWP_2D are alpha = 2): stage s must use
+    # a = m^(alpha_sc D_s), b = (1 - a)/(1 - m), T = alpha_T D_s
+    wl = mlp([6, 5, 4, 3])
+    o = PBOracle(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, 0.1, 0.9, 3,
+                 sc_delay_scale=2, horizon_scale=0.5)
+    o.set_weights(he_normal_weights(wl.seed, wl))
+    for s, opt in enumerate(o.opt):
+        D = 2 * (o.S - 1 - s)
+        assert opt.a == pytest.approx(0.9 ** (2 * D), rel=1e-12)
+        assert opt.b == pytest.approx((1 - 0.9 ** (2 * D)) / 0.1, rel=1e-12, abs=1e-15)
+        assert opt.T == pytest.approx(0.5 * D)
+        assert opt.a / 0.1 + opt.b == pytest.approx(10.0, rel=1e-12)     # total contribution unchanged
