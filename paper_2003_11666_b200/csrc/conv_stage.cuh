@@ -21,6 +21,7 @@ namespace pb {
 
 constexpr float kGnEps = 1e-5f;
 constexpr int kPostPer = kPostChunk / 32;       // elements per lane
+constexpr int kPostRun = 1;                     // consecutive chunks a warp takes at a time (longer runs measured slower)
 
 __device__ __forceinline__ float skip_value(const ConvStage& st, const float* __restrict__ sk, int c, int y, int x) {
     if (st.skip_mode == 0) return sk[((size_t)c * st.skip_h + y) * st.skip_w + x];
@@ -131,19 +132,6 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
     const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np, nunits = n / VEC;
     const size_t zelems = (size_t)st.co * hw;
     const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
-    // group statistics from the chunk partials (the same arithmetic in every warp of the group)
-    const float* __restrict__ f = st.fstat + (size_t)ch.grp * st.fstat_stride * 3;
-    float tot = 0.f, wsum = 0.f;
-    for (int k = lane; k < ch.nidx; k += 32) { tot += f[3 * k]; wsum = fmaf(f[3 * k], f[3 * k + 1], wsum); }
-    tot = warp_sum(tot);
-    const float mean = warp_sum(wsum) / tot;
-    float m2 = 0.f;
-    for (int k = lane; k < ch.nidx; k += 32) { const float d = f[3 * k + 1] - mean; m2 += f[3 * k + 2] + f[3 * k] * d * d; }
-    const float rstd = rsqrtf(warp_sum(m2) / tot + kGnEps);
-    if (ch.idx == 0 && lane == 0) {
-        st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0] = mean;
-        st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1] = rstd;
-    }
     const float* __restrict__ gam = st.wh + st.nw;
     const float* __restrict__ bet = gam + st.co;
     const float* __restrict__ sk = st.skip_ring
@@ -153,18 +141,14 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
     const size_t oelems = (size_t)st.co * st.out_h * st.out_w;
     float* __restrict__ out = st.out_ring + (size_t)slot * oelems;
     __nv_bfloat16* __restrict__ out16 = st.out16 ? st.out16 + (size_t)slot * oelems : nullptr;
-    auto act = [&](int c, int p) -> float {
-        float v = fmaf(gam[c] * rstd, z[(size_t)c * hw + p] - mean, bet[c]);
-        if (sk) v += skip_value(st, sk, c, p / st.ow, p % st.ow);
-        return v;
-    };
+    // the loads of the lane's units go first: they do not depend on the statistics
+    int cc[U], pp[U];
+    bool ok[U];
+    float zv[U][VEC], sv[U][VEC];
     {
-        int cc[U], pp[U];
-        bool ok[U];
-        float zv[U][VEC], sv[U][VEC];
         ChunkWalk<VEC> w(ch, lane);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {                 // all loads of the lane's units first
+        for (int u = 0; u < U; ++u) {
             w.get(ch, c0, nunits, cc[u], pp[u], ok[u]);
             w.next(ch);
             vload<VEC>(zv[u], z + (size_t)cc[u] * hw + pp[u]);
@@ -179,6 +163,26 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
                 for (int e = 0; e < VEC; ++e) sv[u][e] = skip_value(st, sk, cc[u], (pp[u] + e) / st.ow, (pp[u] + e) % st.ow);
             }
         }
+    }
+    // group statistics from the chunk partials (the same arithmetic in every warp of the group)
+    const float* __restrict__ f = st.fstat + (size_t)ch.grp * st.fstat_stride * 3;
+    float tot = 0.f, wsum = 0.f;
+    for (int k = lane; k < ch.nidx; k += 32) { tot += f[3 * k]; wsum = fmaf(f[3 * k], f[3 * k + 1], wsum); }
+    tot = warp_sum(tot);
+    const float mean = warp_sum(wsum) / tot;
+    float m2 = 0.f;
+    for (int k = lane; k < ch.nidx; k += 32) { const float d = f[3 * k + 1] - mean; m2 += f[3 * k + 2] + f[3 * k] * d * d; }
+    const float rstd = rsqrtf(warp_sum(m2) / tot + kGnEps);
+    if (ch.idx == 0 && lane == 0) {
+        st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0] = mean;
+        st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1] = rstd;
+    }
+    auto act = [&](int c, int p) -> float {
+        float v = fmaf(gam[c] * rstd, z[(size_t)c * hw + p] - mean, bet[c]);
+        if (sk) v += skip_value(st, sk, c, p / st.ow, p % st.ow);
+        return v;
+    };
+    {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             if (!ok[u]) continue;
@@ -380,6 +384,19 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
     const float mean = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0];
     const float rstd = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1];
     float* __restrict__ dz = st.dz;
+    // the loads of the lane's units go first: they do not depend on the group sums
+    int cc[U], pp[U];
+    bool ok[U];
+    float dnv[U][VEC], zv[U][VEC];
+    ChunkWalk<VEC> wk(ch, lane);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {                     // all loads of the lane's units first
+        wk.get(ch, c0, nunits, cc[u], pp[u], ok[u]);
+        wk.next(ch);
+        const size_t idx = (size_t)cc[u] * hw + pp[u];
+        vload<VEC>(dnv[u], dz + idx);
+        vload<VEC>(zv[u], z + idx);
+    }
     // channel sums of the whole group (pieces added in order), gradients of scale and
     // shift, group means with the CURRENT scale
     const float* __restrict__ gam = st.w + st.nw;
@@ -399,18 +416,6 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
     m2 = warp_sum(m2) / (float)(cpg * hw);
     float* __restrict__ dsk = st.dskip
         ? st.dskip + (size_t)slot_of(j, st.dskip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
-    int cc[U], pp[U];
-    bool ok[U];
-    float dnv[U][VEC], zv[U][VEC];
-    ChunkWalk<VEC> wk(ch, lane);
-#pragma unroll
-    for (int u = 0; u < U; ++u) {                     // all loads of the lane's units first
-        wk.get(ch, c0, nunits, cc[u], pp[u], ok[u]);
-        wk.next(ch);
-        const size_t idx = (size_t)cc[u] * hw + pp[u];
-        vload<VEC>(dnv[u], dz + idx);
-        vload<VEC>(zv[u], z + idx);
-    }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         if (!ok[u]) continue;
@@ -449,9 +454,10 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
 }
 
 // ---------------------------------------------------------------- launch wrappers
-// Persistent blocks: every warp walks the chunk table with a grid stride.  The
-// stage descriptors are kept in shared memory (one copy per stage of the launch
-// would not fit, so each warp re-reads its chunk's descriptor into its own slot).
+// Persistent blocks.  The chunk table is dealt to the warps in short runs of
+// consecutive chunks, round-robin (chunks are ordered by stage and differ a lot in
+// cost between stages: long contiguous ranges unbalance the warps, single chunks
+// make every warp reload its stage descriptor, kept in shared memory, each time).
 #define PB_POST_KERNEL(NAME, CHUNK, ...)                                                          \
     __global__ void __launch_bounds__(kPostThreads, 2) NAME(const ConvStage* __restrict__ stages,  \
                                                             const PostChunk* __restrict__ chunks, int nchunks, \
@@ -459,8 +465,12 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
         __shared__ ConvStage sst[kPostThreads / 32];                                               \
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;                                \
         const long long t = ts->cnt[par];                                                          \
+        const int nwarps = gridDim.x * (kPostThreads / 32);                                        \
+        const int gw = blockIdx.x * (kPostThreads / 32) + warp;                                    \
         int loaded = -1;                                                                           \
-        for (int ci = blockIdx.x * (kPostThreads / 32) + warp; ci < nchunks; ci += gridDim.x * (kPostThreads / 32)) { \
+        /* runs of kPostRun consecutive chunks, dealt round-robin to the warps */                  \
+        for (int base = gw * kPostRun; base < nchunks; base += nwarps * kPostRun)                  \
+        for (int ci = base; ci < min(nchunks, base + kPostRun); ++ci) {                            \
             const PostChunk ch = chunks[ci];                                                       \
             if (ch.stage != loaded) {                                                              \
                 __syncwarp();                                                                      \
