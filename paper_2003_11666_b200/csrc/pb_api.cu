@@ -490,17 +490,19 @@ void fill_fc_tables(pb_handle* h) {
 }
 
 // ---------------------------------------------------------------- profiling helpers
-void prof_begin(pb_handle* h, int cls) {
+void prof_begin(pb_handle* h, int cls, cudaStream_t st = nullptr) {
+    if (!st) st = h->stream;
     if (!h->profile) return;
     if (h->ev_used + 2 > h->ev_pool.size()) {
         for (int k = 0; k < 2; ++k) { cudaEvent_t e; cudaEventCreate(&e); h->ev_pool.push_back(e); }
     }
     h->ev_class.push_back(cls);
-    cudaEventRecord(h->ev_pool[h->ev_used], h->stream);
+    cudaEventRecord(h->ev_pool[h->ev_used], st);
 }
-void prof_end(pb_handle* h) {
+void prof_end(pb_handle* h, cudaStream_t st = nullptr) {
+    if (!st) st = h->stream;
     if (!h->profile) return;
-    cudaEventRecord(h->ev_pool[h->ev_used + 1], h->stream);
+    cudaEventRecord(h->ev_pool[h->ev_used + 1], st);
     h->ev_used += 2;
 }
 void prof_collect(pb_handle* h) {
@@ -549,7 +551,24 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
         } else {
             ingest_kernel<<<ingest_blocks, 256, 0, h->stream>>>(h->d_ts, par, dev_xs, dev_labels, label_value, h->in_ring,
                                                                 h->in_slots, elems, h->label_ring, h->S, t_base);
-            // forward chain: convolutions -> normalise/activate/pool; FC forward
+            // The FC stages of this tick depend only on what earlier ticks left in the rings
+            // (and on the label just ingested): they run on a side stream beside the conv chain.
+            cudaStream_t fs = h->side ? h->side : h->stream;
+            cudaEventRecord(h->ev_fork, h->stream);
+            cudaStreamWaitEvent(fs, h->ev_fork, 0);
+            prof_begin(h, 0, fs);
+            fc_tick_kernel<<<h->nctaA, kFcThreads, 0, fs>>>(h->d_fc, h->d_segA, h->d_ctaA, h->d_ts, h->S, 0, par,
+                                                           fused_last ? 1 : 0, h->label_ring, dev_losses, t_base,
+                                                           nullptr, nullptr, 0, nullptr, 0, 0);
+            prof_end(h, fs);
+            if (!fused_last) {
+                prof_begin(h, 1, fs);
+                fc_tick_kernel<<<h->nctaB, kFcThreads, 0, fs>>>(h->d_fc, h->d_segB, h->d_ctaB, h->d_ts, h->S, 1, par, 1,
+                                                               h->label_ring, dev_losses, t_base,
+                                                               nullptr, nullptr, 0, nullptr, 0, 0);
+                prof_end(h, fs);
+            }
+            // forward chain: convolutions -> normalise/activate/pool
             if (!h->h_tiles[0].empty()) {
                 prof_begin(h, 3);
                 conv_gemm_kernel<<<(int)h->h_tiles[0].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[0], h->d_ts, h->S, par);
@@ -584,18 +603,9 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             prof_begin(h, 2);
             update_kernel<<<(int)h->h_chunks.size(), 256, 0, h->stream>>>(h->d_upd, h->d_chunks, h->d_ts, h->S, par);
             prof_end(h);
-            prof_begin(h, 0);
-            fc_tick_kernel<<<h->nctaA, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segA, h->d_ctaA, h->d_ts, h->S, 0, par,
-                                                                  fused_last ? 1 : 0, h->label_ring, dev_losses, t_base,
-                                                                  nullptr, nullptr, 0, nullptr, 0, 0);
-            prof_end(h);
-            if (!fused_last) {
-                prof_begin(h, 1);
-                fc_tick_kernel<<<h->nctaB, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segB, h->d_ctaB, h->d_ts, h->S, 1, par, 1,
-                                                                      h->label_ring, dev_losses, t_base,
-                                                                      nullptr, nullptr, 0, nullptr, 0, 0);
-                prof_end(h);
-            }
+            // the conv chain waits for the FC stages before the tick ends
+            cudaEventRecord(h->ev_join, fs);
+            cudaStreamWaitEvent(h->stream, h->ev_join, 0);
             h->last_launches += 7 + (fused_last ? 0 : 1);      // ingest, 2 + 2 normalisation kernels, update, FC
             for (int q = 0; q < 3; ++q) h->last_launches += (h->h_tiles[q].empty() ? 0 : 1) + (h->h_tctiles[q].empty() ? 0 : 1);
         }
@@ -700,6 +710,11 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     up(h->d_chunks, h->h_chunks.data(), h->h_chunks.size() * sizeof(UpdChunk));
     up(h->d_tc, h->h_tc.data(), h->h_tc.size() * sizeof(ConvGemmTC));
     for (int q = 0; q < 3; ++q) up(h->d_tctiles[q], h->h_tctiles[q].data(), h->h_tctiles[q].size() * sizeof(GemmTile));
+    if (e == cudaSuccess && !h->all_fc) {
+        e = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
+    }
     if (e == cudaSuccess && !h->h_tc.empty())
         e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
@@ -856,6 +871,9 @@ void pb_destroy(pb_handle* h) {
     if (!h) return;
     cudaStreamSynchronize(h->stream);
     for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
+    if (h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); }
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->staging) cudaFree(h->staging);
     cudaFree(h->arena);
     delete h;
