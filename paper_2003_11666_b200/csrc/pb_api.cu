@@ -583,23 +583,30 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             conv_stats_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
             conv_apply_fwd_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
             prof_end(h);
-            // backward chain: through pool/ReLU/GroupNorm -> data and weight gradients
-            prof_begin(h, 6);
-            conv_bwd_dn_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
-            conv_bwd_dz_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
-            prof_end(h);
+            // Backward chain: through pool/ReLU/GroupNorm -> data and weight gradients.  It reads
+            // what earlier ticks stored (other ring slots than the forward chain writes) and the
+            // current weights, so it runs on its own stream beside the forward chain; only the
+            // update, which overwrites the predicted weights the forward reads, waits for both.
+            cudaStream_t bs = h->bwd ? h->bwd : h->stream;
+            cudaStreamWaitEvent(bs, h->ev_fork, 0);
+            prof_begin(h, 6, bs);
+            conv_bwd_dn_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
+            conv_bwd_dz_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
+            prof_end(h, bs);
             for (int q = 1; q < 3; ++q) {
                 if (!h->h_tiles[q].empty()) {
-                    prof_begin(h, 3);
-                    conv_gemm_kernel<<<(int)h->h_tiles[q].size(), kGemmThreads, 0, h->stream>>>(h->d_gemms, h->d_tiles[q], h->d_ts, h->S, par);
-                    prof_end(h);
+                    prof_begin(h, 3, bs);
+                    conv_gemm_kernel<<<(int)h->h_tiles[q].size(), kGemmThreads, 0, bs>>>(h->d_gemms, h->d_tiles[q], h->d_ts, h->S, par);
+                    prof_end(h, bs);
                 }
                 if (!h->h_tctiles[q].empty()) {
-                    prof_begin(h, q == 1 ? 8 : 7);
-                    conv_tc_kernel<<<(int)h->h_tctiles[q].size(), kTcThreads, kTcSmemBytes, h->stream>>>(h->d_tc, h->d_tctiles[q], h->d_ts, h->S, par);
-                    prof_end(h);
+                    prof_begin(h, q == 1 ? 8 : 7, bs);
+                    conv_tc_kernel<<<(int)h->h_tctiles[q].size(), kTcThreads, kTcSmemBytes, bs>>>(h->d_tc, h->d_tctiles[q], h->d_ts, h->S, par);
+                    prof_end(h, bs);
                 }
             }
+            cudaEventRecord(h->ev_bjoin, bs);
+            cudaStreamWaitEvent(h->stream, h->ev_bjoin, 0);
             prof_begin(h, 2);
             update_kernel<<<(int)h->h_chunks.size(), 256, 0, h->stream>>>(h->d_upd, h->d_chunks, h->d_ts, h->S, par);
             prof_end(h);
@@ -714,6 +721,8 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
         e = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->bwd, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_bjoin, cudaEventDisableTiming);
     }
     if (e == cudaSuccess && !h->h_tc.empty())
         e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
@@ -872,6 +881,8 @@ void pb_destroy(pb_handle* h) {
     cudaStreamSynchronize(h->stream);
     for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
     if (h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); }
+    if (h->bwd) { cudaStreamSynchronize(h->bwd); cudaStreamDestroy(h->bwd); }
+    if (h->ev_bjoin) cudaEventDestroy(h->ev_bjoin);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->staging) cudaFree(h->staging);

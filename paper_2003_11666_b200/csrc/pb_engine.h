@@ -51,7 +51,8 @@ struct ProfileClass { double ms = 0; long long launches = 0; };
 struct pb_handle {
     cudaStream_t stream = nullptr;
     cudaStream_t side = nullptr;                // FC stages of conv nets run beside the conv chain of the same tick
-    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaStream_t bwd = nullptr;                 // backward chain of a tick, beside its forward chain
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_bjoin = nullptr;
     int device = 0, num_sms = 0;
     unsigned flags = 0;
     float lr = 0, momentum = 0;
