@@ -64,58 +64,63 @@ __device__ void gemm_tile(const ConvGemm& G, const GemmTile& tl, long long smp,
         }
     }
 
-    for (int k0 = kb; k0 < ke; k0 += kBK) {
-        float ra[4], rb[4];
+    // gather of one K step into registers (ra: this thread's 4 elements of the A tile, rb: of the B tile)
+    auto fetch = [&](int k0, float (&ra)[4], float (&rb)[4]) {
         if (G.mode == kFprop) {
-            // A[m, kk] = w_hat[m*K + kk]: 16 consecutive kk per row
-            const int kk = k0 + lo16;
+        // A[m, kk] = w_hat[m*K + kk]: 16 consecutive kk per row
+        const int kk = k0 + lo16;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int m = tl.m0 + hi16 + 16 * q;
-                ra[q] = (m < M && kk < ke) ? A[(size_t)m * G.K + kk] : 0.f;
-            }
-            // B[kk, n] = x[ci, p*st + r - pad, q*st + s - pad]
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int kq = k0 + hi4 + 4 * q;
-                int c, r, s;
-                KDiv<KS>::split(kq, ksz, c, r, s);
-                const int y = n_p * st + r - pad, x = n_q * st + s - pad;
-                rb[q] = (n_ok && kq < ke && y >= 0 && y < ih && x >= 0 && x < iw) ? B[((size_t)c * ih + y) * iw + x] : 0.f;
-            }
-        } else if (G.mode == kDgrad) {
-            // A[m = ci, kk = (co, r, s)] = w[co, ci, r, s];  B[kk, n = (y, x)] = dz[co, (y+pad-r)/st, (x+pad-s)/st]
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int kq = k0 + hi4 + 4 * q;
-                int c, r, s;
-                KDiv<KS>::split(kq, ksz, c, r, s);
-                const int m = tl.m0 + lo64;
-                ra[q] = (m < M && kq < ke) ? A[(((size_t)c * G.ci + m) * ksz + r) * ksz + s] : 0.f;
-                const int ty_ = n_p + pad - r, tx_ = n_q + pad - s;
-                float v = 0.f;
-                if (n_ok && kq < ke && ty_ >= 0 && tx_ >= 0) {
-                    const int p = ty_ / st, qq = tx_ / st;
-                    if (p * st == ty_ && qq * st == tx_ && p < oh && qq < ow) v = B[((size_t)c * oh + p) * ow + qq];
-                }
-                rb[q] = v;
-            }
-        } else {
-            // A[m = co, kk = pixel] = dz[m*K + kk];  B[kk = (p, q), n = (ci, r, s)] = x[ci, p*st+r-pad, q*st+s-pad]
-            const int kk = k0 + lo16;
-            const int p = kk / ow, qq = kk - p * ow;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int m = tl.m0 + hi16 + 16 * q;
-                ra[q] = (m < M && kk < ke) ? A[(size_t)m * G.K + kk] : 0.f;
-                const int y = p * st + wr[q] - pad, x = qq * st + ws[q] - pad;
-                rb[q] = (w_ok[q] && kk < ke && y >= 0 && y < ih && x >= 0 && x < iw) ? B[((size_t)wc[q] * ih + y) * iw + x] : 0.f;
-            }
+        for (int q = 0; q < 4; ++q) {
+            const int m = tl.m0 + hi16 + 16 * q;
+            ra[q] = (m < M && kk < ke) ? A[(size_t)m * G.K + kk] : 0.f;
         }
-        if (bf) {
+        // B[kk, n] = x[ci, p*st + r - pad, q*st + s - pad]
 #pragma unroll
-            for (int q = 0; q < 4; ++q) { ra[q] = round_bf16(ra[q]); rb[q] = round_bf16(rb[q]); }
+        for (int q = 0; q < 4; ++q) {
+            const int kq = k0 + hi4 + 4 * q;
+            int c, r, s;
+            KDiv<KS>::split(kq, ksz, c, r, s);
+            const int y = n_p * st + r - pad, x = n_q * st + s - pad;
+            rb[q] = (n_ok && kq < ke && y >= 0 && y < ih && x >= 0 && x < iw) ? B[((size_t)c * ih + y) * iw + x] : 0.f;
         }
+    } else if (G.mode == kDgrad) {
+        // A[m = ci, kk = (co, r, s)] = w[co, ci, r, s];  B[kk, n = (y, x)] = dz[co, (y+pad-r)/st, (x+pad-s)/st]
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int kq = k0 + hi4 + 4 * q;
+            int c, r, s;
+            KDiv<KS>::split(kq, ksz, c, r, s);
+            const int m = tl.m0 + lo64;
+            ra[q] = (m < M && kq < ke) ? A[(((size_t)c * G.ci + m) * ksz + r) * ksz + s] : 0.f;
+            const int ty_ = n_p + pad - r, tx_ = n_q + pad - s;
+            float v = 0.f;
+            if (n_ok && kq < ke && ty_ >= 0 && tx_ >= 0) {
+                const int p = ty_ / st, qq = tx_ / st;
+                if (p * st == ty_ && qq * st == tx_ && p < oh && qq < ow) v = B[((size_t)c * oh + p) * ow + qq];
+            }
+            rb[q] = v;
+        }
+    } else {
+        // A[m = co, kk = pixel] = dz[m*K + kk];  B[kk = (p, q), n = (ci, r, s)] = x[ci, p*st+r-pad, q*st+s-pad]
+        const int kk = k0 + lo16;
+        const int p = kk / ow, qq = kk - p * ow;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int m = tl.m0 + hi16 + 16 * q;
+            ra[q] = (m < M && kk < ke) ? A[(size_t)m * G.K + kk] : 0.f;
+            const int y = p * st + wr[q] - pad, x = qq * st + ws[q] - pad;
+            rb[q] = (w_ok[q] && kk < ke && y >= 0 && y < ih && x >= 0 && x < iw) ? B[((size_t)wc[q] * ih + y) * iw + x] : 0.f;
+        }
+    }
+    if (bf) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { ra[q] = round_bf16(ra[q]); rb[q] = round_bf16(rb[q]); }
+    }
+    };
+    // Software pipeline: the gather of step k+1 is in flight while step k is multiplied.
+    float ra[4], rb[4];
+    fetch(kb, ra, rb);
+    for (int k0 = kb; k0 < ke; k0 += kBK) {
         __syncthreads();
         if (G.mode == kDgrad) {
 #pragma unroll
@@ -128,6 +133,7 @@ __device__ void gemm_tile(const ConvGemm& G, const GemmTile& tl, long long smp,
             for (int q = 0; q < 4; ++q) { As[lo16][hi16 + 16 * q] = ra[q]; Bs[lo16][hi16 + 16 * q] = rb[q]; }
         }
         __syncthreads();
+        if (k0 + kBK < ke) fetch(k0 + kBK, ra, rb);
 #pragma unroll
         for (int kk = 0; kk < kBK; ++kk) {
             const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);

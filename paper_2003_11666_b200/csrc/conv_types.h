@@ -8,6 +8,7 @@ namespace pb {
 
 constexpr int kGemmThreads = 256;
 constexpr int kBM = 64, kBN = 64, kBK = 16;
+constexpr int kSimtMaxK = 192;             // longest K loop of one float32 tile before K is sliced
 constexpr int kPostThreads = 256;         // normalisation / activation kernels
 constexpr int kPostChunk = 256;           // elements per warp of those kernels
 constexpr int kMaxGroupChannels = 64;      // channels per normalisation group

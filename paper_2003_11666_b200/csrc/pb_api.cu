@@ -196,21 +196,19 @@ void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSe
 
 // ---------------------------------------------------------------- convolution planning
 void choose_split(int M, int N, int K, int num_sms, int& nsplit, int& kps) {
-    const int tiles = ceil_div(M, kBM) * ceil_div(N, kBN);
-    int want = ceil_div(num_sms, tiles);
-    int by_k = K / 64;
-    if (by_k < 1) by_k = 1;
-    nsplit = std::max(1, std::min(std::min(want, by_k), 32));
+    // as for the tensor-core path: slices only bound the K loop of one tile
+    (void)M; (void)N; (void)num_sms;
+    nsplit = std::max(1, std::min(ceil_div(K, kSimtMaxK), 32));
     kps = ceil_div(ceil_div(K, nsplit), kBK) * kBK;
     nsplit = ceil_div(K, kps);
 }
 
 void choose_split_tc(int M, int N, int bn, int K, int num_sms, int& nsplit, int& kps) {
-    const int tiles = ceil_div(M, kTcBM) * ceil_div(N, bn);
-    int want = ceil_div(num_sms, tiles);
-    int by_k = K / (2 * kTcChunk);
-    if (by_k < 1) by_k = 1;
-    nsplit = std::max(1, std::min(std::min(want, by_k), 16));
+    // The grouped launch already holds thousands of tiles, so K is sliced only to bound the
+    // length of one tile's K loop (every slice costs a partial result that must be written
+    // and read back): at most kTcMaxK elements of K per slice.
+    (void)M; (void)N; (void)bn; (void)num_sms;
+    nsplit = std::max(1, std::min(ceil_div(K, kTcMaxK), 16));
     kps = ceil_div(ceil_div(K, nsplit), kTcChunk) * kTcChunk;
     nsplit = ceil_div(K, kps);
 }
