@@ -76,3 +76,28 @@ def test_resnet50_bf16_first_72_ticks():
     w = compare_ticks(wl, 72, TOL_BF16, check_every=4, spread_factor=3.0)
     assert w["ticks"] == 72
     assert w["loss"] <= TOL_BF16
+
+
+@pytest.mark.parametrize("name,ticks", [("resnet20", 96), ("vgg11", 48)])
+def test_two_runs_give_identical_bits(name, ticks):
+    # Forward chain, backward chain and FC stage of a tick run on three streams and every
+    # reduction has a fixed order: two runs of the same samples must agree bit for bit
+    # (a race between the chains, or an atomics-ordered sum, would show up here).
+    import torch
+    from pb_workloads import make_inputs
+    from tests.parity import make_engine
+    wl = workload(name)
+    x, y = make_inputs(wl.seed, ticks, wl.sample_elems, wl.n_classes)
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    outs = []
+    for _ in range(2):
+        e = make_engine(wl)
+        losses = torch.zeros(ticks, device="cuda")
+        e.run(xd, yd, ticks, losses)
+        e.sync()
+        outs.append((losses.cpu().numpy(), e.get_weights(), e.get_velocity()))
+        e.destroy()
+    S = wl.n_stages
+    np.testing.assert_array_equal(outs[0][0][S - 1:], outs[1][0][S - 1:])
+    np.testing.assert_array_equal(outs[0][1], outs[1][1])
+    np.testing.assert_array_equal(outs[0][2], outs[1][2])
