@@ -591,18 +591,26 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             conv_bwd_dn_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
             conv_bwd_dz_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
             prof_end(h, bs);
+            // data gradients (dgrad) and weight gradients (wgrad) both start from dz and write
+            // different buffers: wgrad goes to a stream of its own
+            cudaStream_t ws = h->aux ? h->aux : bs;
+            cudaEventRecord(h->ev_dz, bs);
+            cudaStreamWaitEvent(ws, h->ev_dz, 0);
             for (int q = 1; q < 3; ++q) {
+                cudaStream_t qs = q == 1 ? bs : ws;
                 if (!h->h_tiles[q].empty()) {
-                    prof_begin(h, 3, bs);
-                    conv_gemm_kernel<<<(int)h->h_tiles[q].size(), kGemmThreads, 0, bs>>>(h->d_gemms, h->d_tiles[q], h->d_ts, h->S, par);
-                    prof_end(h, bs);
+                    prof_begin(h, 3, qs);
+                    conv_gemm_kernel<<<(int)h->h_tiles[q].size(), kGemmThreads, 0, qs>>>(h->d_gemms, h->d_tiles[q], h->d_ts, h->S, par);
+                    prof_end(h, qs);
                 }
                 if (!h->h_tctiles[q].empty()) {
-                    prof_begin(h, q == 1 ? 8 : 7, bs);
-                    conv_tc_kernel<<<(int)h->h_tctiles[q].size(), kTcThreads, kTcSmemBytes, bs>>>(h->d_tc, h->d_tctiles[q], h->d_ts, h->S, par);
-                    prof_end(h, bs);
+                    prof_begin(h, q == 1 ? 8 : 7, qs);
+                    conv_tc_kernel<<<(int)h->h_tctiles[q].size(), kTcThreads, kTcSmemBytes, qs>>>(h->d_tc, h->d_tctiles[q], h->d_ts, h->S, par);
+                    prof_end(h, qs);
                 }
             }
+            cudaEventRecord(h->ev_wjoin, ws);
+            cudaStreamWaitEvent(h->stream, h->ev_wjoin, 0);
             cudaEventRecord(h->ev_bjoin, bs);
             cudaStreamWaitEvent(h->stream, h->ev_bjoin, 0);
             prof_begin(h, 2);
@@ -721,6 +729,9 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->bwd, cudaStreamNonBlocking);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_bjoin, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_dz, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_wjoin, cudaEventDisableTiming);
     }
     if (e == cudaSuccess && !h->h_tc.empty())
         e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
@@ -881,6 +892,9 @@ void pb_destroy(pb_handle* h) {
     if (h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); }
     if (h->bwd) { cudaStreamSynchronize(h->bwd); cudaStreamDestroy(h->bwd); }
     if (h->ev_bjoin) cudaEventDestroy(h->ev_bjoin);
+    if (h->aux) { cudaStreamSynchronize(h->aux); cudaStreamDestroy(h->aux); }
+    if (h->ev_dz) cudaEventDestroy(h->ev_dz);
+    if (h->ev_wjoin) cudaEventDestroy(h->ev_wjoin);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->staging) cudaFree(h->staging);

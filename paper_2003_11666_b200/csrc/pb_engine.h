@@ -52,6 +52,8 @@ struct pb_handle {
     cudaStream_t stream = nullptr;
     cudaStream_t side = nullptr;                // FC stages of conv nets run beside the conv chain of the same tick
     cudaStream_t bwd = nullptr;                 // backward chain of a tick, beside its forward chain
+    cudaStream_t aux = nullptr;                 // weight gradients, beside the data gradients
+    cudaEvent_t ev_dz = nullptr, ev_wjoin = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_bjoin = nullptr;
     int device = 0, num_sms = 0;
     unsigned flags = 0;
