@@ -26,6 +26,7 @@ struct ConvGemm {
     int ci, co, k, stride, pad, ih, iw, oh, ow;
     int s;                       // stage index (for the tick arithmetic)
     int bf16;                    // round both operands to bfloat16 before multiplying
+    int tm, tn;                  // per-thread patch (1 or 4): the tile is (16 tm) x (16 tn)
     int nsplit, k_per_split;
     const float* a;              // fprop: w_hat; dgrad: w; wgrad: dz
     const float* b;              // fprop/wgrad: ring of the input activations; dgrad: dz

@@ -292,21 +292,24 @@ void fill_conv_tables(pb_handle* h) {
         g.mode = kFprop; g.M = L.c_out; g.N = opix; g.K = L.c_in * k2; g.nsplit = x.split_f; g.k_per_split = x.kps_f;
         g.a = h->d_wh + x.dev_off; g.b = xin; g.b_slots = xin_slots; g.b_elems = x.in.elems();
         g.c = x.zpart; g.c_slots = 1;
-        if (!x.tc) add_tiles(h->h_tiles[0], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
+        g.tm = g.M <= 16 ? 1 : 4; g.tn = g.N <= 16 ? 1 : 4;        // small problems take small tiles
+        if (!x.tc) add_tiles(h->h_tiles[0], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
         h->h_gemms.push_back(g);
         // dgrad (not for the first stage: nobody needs the gradient of the input)
         if (x.src >= 0) {
             g.mode = kDgrad; g.M = L.c_in; g.N = ipix; g.K = L.c_out * k2; g.nsplit = x.split_d; g.k_per_split = x.kps_d;
             g.a = h->d_w + x.dev_off; g.b = x.dz; g.b_slots = 1; g.b_elems = x.z.elems();
             g.c = x.dx; g.c_slots = x.dx_slots;
-            if (!x.tc) add_tiles(h->h_tiles[1], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
+            g.tm = g.M <= 16 ? 1 : 4; g.tn = g.N <= 16 ? 1 : 4;
+            if (!x.tc) add_tiles(h->h_tiles[1], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
             h->h_gemms.push_back(g);
         }
         // wgrad
         g.mode = kWgrad; g.M = L.c_out; g.N = L.c_in * k2; g.K = opix; g.nsplit = x.split_w; g.k_per_split = x.kps_w;
         g.a = x.dz; g.b = xin; g.b_slots = xin_slots; g.b_elems = x.in.elems();
         g.c = x.gpart; g.c_slots = 1;
-        if (!x.tc) add_tiles(h->h_tiles[2], (int)h->h_gemms.size(), g.M, g.N, g.nsplit);
+        g.tm = g.M <= 16 ? 1 : 4; g.tn = g.N <= 16 ? 1 : 4;
+        if (!x.tc) add_tiles(h->h_tiles[2], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
         h->h_gemms.push_back(g);
 
         ConvStage c{};
