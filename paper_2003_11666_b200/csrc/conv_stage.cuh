@@ -459,7 +459,7 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
 // cost between stages: long contiguous ranges unbalance the warps, single chunks
 // make every warp reload its stage descriptor, kept in shared memory, each time).
 #define PB_POST_KERNEL(NAME, CHUNK, ...)                                                          \
-    __global__ void __launch_bounds__(kPostThreads, 2) NAME(const ConvStage* __restrict__ stages,  \
+    __global__ void __launch_bounds__(kPostThreads, 4) NAME(const ConvStage* __restrict__ stages,  \
                                                             const PostChunk* __restrict__ chunks, int nchunks, \
                                                             const TickState* __restrict__ ts, int S, int par) { \
         __shared__ ConvStage sst[kPostThreads / 32];                                               \

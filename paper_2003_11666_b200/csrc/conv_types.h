@@ -10,7 +10,7 @@ constexpr int kGemmThreads = 256;
 constexpr int kBM = 64, kBN = 64, kBK = 16;
 constexpr int kSimtMaxK = 192;             // longest K loop of one float32 tile before K is sliced
 constexpr int kPostThreads = 256;         // normalisation / activation kernels
-constexpr int kPostChunk = 256;           // elements per warp of those kernels
+constexpr int kPostChunk = 128;           // elements per warp of those kernels
 constexpr int kMaxGroupChannels = 64;      // channels per normalisation group
 
 enum GemmMode { kFprop = 0, kDgrad = 1, kWgrad = 2 };

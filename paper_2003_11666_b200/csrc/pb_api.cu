@@ -376,7 +376,7 @@ int validate_conv(pb_handle* h) {
         if (x.gn_groups <= 0) return fail(nullptr, PB_E_UNSUPPORTED, "a CONV2D stage needs a GROUPNORM layer");
         if (x.head.c_out / x.gn_groups > kMaxGroupChannels) return fail(nullptr, PB_E_UNSUPPORTED, "more than 64 channels per normalisation group");
         if (x.has_pool && x.avgpool) return fail(nullptr, PB_E_UNSUPPORTED, "max-pool and average pool in one stage");
-        if (x.avgpool && x.z.h * x.z.w > kPostChunk) return fail(nullptr, PB_E_UNSUPPORTED, "global average pool over more than 256 pixels");
+        if (x.avgpool && x.z.h * x.z.w > kPostChunk) return fail(nullptr, PB_E_UNSUPPORTED, "global average pool over more than 128 pixels");
         if ((int)(x.consumers_main.size() + x.consumers_skip.size()) > kMaxDeltaSrc) return fail(nullptr, PB_E_UNSUPPORTED, "too many consumers of one stage");
     }
     for (const StageHost& x : h->stages)
@@ -530,7 +530,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
     if (h->profile) for (auto& p : h->prof) p = ProfileClass{};
     const bool fused_last = h->nctaB == 0;      // the last stage rides in the phase-0 launch
     const int npc = (int)h->h_pchunks.size();
-    const int post_grid = std::max(1, std::min(ceil_div(npc, kPostThreads / 32), 2 * h->num_sms));
+    const int post_grid = std::max(1, std::min(ceil_div(npc, kPostThreads / 32), 4 * h->num_sms));
     for (int k = 0; k < n_ticks; ++k) {
         const int par = (int)((t_base + k) & 1);
         if (h->all_fc) {
