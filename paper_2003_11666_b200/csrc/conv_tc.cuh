@@ -21,9 +21,13 @@
 
 namespace pb {
 
-constexpr int kTcThreads = 128;
-constexpr int kTcBM = 128;
 constexpr int kTcChunk = 64;                  // K elements per shared-memory stage
+constexpr int kTcThreads = 256;                // 8 warps gather; warps 0-3 / 4-7 split the columns in the epilogue
+constexpr int kTcRowsPerPass = kTcThreads / 8; // K-major tiles: rows filled per pass (8 units of 16 bytes per row)
+constexpr int kTcPasses = 128 / kTcRowsPerPass;
+constexpr int kTcKPerPass = kTcThreads / 16;   // MN-major tiles of width 128: k rows filled per pass
+constexpr int kTcKPasses = kTcChunk / kTcKPerPass;
+constexpr int kTcBM = 128;
 constexpr int kTcStageBytes = 16384 * 2;      // A tile + B tile
 constexpr int kTcStages = 3;                  // shared-memory stages of the operand pipeline
 constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + 1024;
@@ -128,17 +132,17 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
     const uint32_t idesc = tc_idesc(kTcBM, BN, a_mn, b_mn);
 
     // ---- per-thread invariants of the gathers
-    // K-major tiles: this thread fills unit (tid & 7) of rows (tid >> 3) + 16 i, i = 0..7
-    // MN-major tiles of width 128: unit (tid & 15) of k-rows (tid >> 4) + 8 i; width 64: unit (tid & 7) of (tid >> 3) + 16 i (k < 64 -> i < 4)
+    // K-major tiles: this thread fills unit (tid & 7) of rows (tid >> 3) + kTcRowsPerPass i
+    // MN-major tiles of width 128: unit (tid & 15) of k-rows (tid >> 4) + kTcKPerPass i
     const int ku = tid & 7, krow0 = tid >> 3;
-    int bp[8], bq[8];             // K-major B rows: pixel coordinates (fprop: output pixel; dgrad: input pixel)
-    bool bok[8];
+    int bp[kTcPasses], bq[kTcPasses];   // K-major B rows: pixel coordinates (fprop: output pixel; dgrad: input pixel)
+    bool bok[kTcPasses];
     if (G.mode != kWgrad) {
         const int wdt = (G.mode == kFprop) ? ow : iw;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int n = tl.n0 + krow0 + 16 * i;
-            bok[i] = (krow0 + 16 * i) < BN && n < N;
+        for (int i = 0; i < kTcPasses; ++i) {
+            const int n = tl.n0 + krow0 + kTcRowsPerPass * i;
+            bok[i] = (krow0 + kTcRowsPerPass * i) < BN && n < N;
             bp[i] = n / wdt; bq[i] = n - bp[i] * wdt;
         }
     }
@@ -164,23 +168,23 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
         if (G.mode == kFprop) {
             const int k = k0 + ku * 8;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int row = krow0 + 16 * i, m = tl.m0 + row;
+            for (int i = 0; i < kTcPasses; ++i) {
+                const int row = krow0 + kTcRowsPerPass * i, m = tl.m0 + row;
                 const bool ok = m < M && k < ke;
                 cp_async16(sA + kmajor_off(row, ku), ok ? A + (size_t)m * G.K + k : A, ok);
             }
         } else if (G.mode == kDgrad) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int kl = ak0 + 8 * i, k = k0 + kl;          // k = rs * CO + co
+            for (int i = 0; i < kTcKPasses; ++i) {
+                const int kl = ak0 + kTcKPerPass * i, k = k0 + kl;          // k = rs * CO + co
                 const bool ok = a_m_ok && k < ke;
                 const int rs = k / CO, co = k - rs * CO;
                 cp_async16(sA + mnmajor_off(kl, amu), ok ? A + ((size_t)co * (ksz * ksz) + rs) * CI + tl.m0 + amu * 8 : A, ok);
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int kl = ak0 + 8 * i, k = k0 + kl;          // k = output pixel
+            for (int i = 0; i < kTcKPasses; ++i) {
+                const int kl = ak0 + kTcKPerPass * i, k = k0 + kl;          // k = output pixel
                 const bool ok = a_m_ok && k < ke;
                 cp_async16(sA + mnmajor_off(kl, amu), ok ? A + (size_t)k * CO + tl.m0 + amu * 8 : A, ok);
             }
@@ -190,8 +194,8 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
             const int k = k0 + ku * 8;
             const int rs = k / CI, ci = k - rs * CI, r = rs / ksz, s = rs - r * ksz;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int row = krow0 + 16 * i;
+            for (int i = 0; i < kTcPasses; ++i) {
+                const int row = krow0 + kTcRowsPerPass * i;
                 if (row >= BN) break;
                 const int y = bp[i] * st + r - pad, x = bq[i] * st + s - pad;
                 const bool ok = bok[i] && k < ke && y >= 0 && y < ih && x >= 0 && x < iw;
@@ -201,8 +205,8 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
             const int k = k0 + ku * 8;
             const int rs = k / CO, co = k - rs * CO, r = rs / ksz, s = rs - r * ksz;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int row = krow0 + 16 * i;
+            for (int i = 0; i < kTcPasses; ++i) {
+                const int row = krow0 + kTcRowsPerPass * i;
                 if (row >= BN) break;
                 const int ty = bp[i] + pad - r, tx = bq[i] + pad - s;
                 const int p = ty / st, q = tx / st;
@@ -264,11 +268,14 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (!failed) {
         // epilogue: warp w reads lanes 32w..32w+31 (rows of D), 32 columns per load
-        const int m = tl.m0 + warp * 32 + lane;
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        // (a warp may only touch the TMEM lanes of its quarter, warp % 4; the two warps of a
+        //  quarter take one half of the columns each)
+        const int quarter = warp & 3, half = warp >> 2;
+        const int m = tl.m0 + quarter * 32 + lane;
+        for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
             if (tl.n0 + c0 >= N) break;                         // uniform
             uint32_t r[32];
-            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
+            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0;
             asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                          "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
                          : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
