@@ -233,7 +233,7 @@ def main():
         alg_bytes, kernel = 28.0 * (P - p_last), "update_kernel"
     # DRAM bytes per launch of that kernel from the ncu capture summarised under profiles/
     # (dram__bytes_read.sum + dram__bytes_write.sum, steady-state tick); None where not captured
-    traffic = {"mlp16x2048": 506.60e6 + 448.82e6}.get(args.workload) if all_fc else None
+    traffic = {"mlp16x2048": 506.77e6 + 448.64e6}.get(args.workload) if all_fc else None
     achieved = alg_bytes / (k_ms / k_n * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind,
