@@ -233,7 +233,7 @@ def main():
         alg_bytes, kernel = 28.0 * (P - p_last), "update_kernel"
     # DRAM bytes per launch of that kernel from the ncu capture summarised under profiles/
     # (dram__bytes_read.sum + dram__bytes_write.sum, steady-state tick); None where not captured
-    traffic = {"mlp16x2048": 506.77e6 + 448.64e6}.get(args.workload) if all_fc else None
+    traffic = None   # the counters on file predate the two-wave partition
     achieved = alg_bytes / (k_ms / k_n * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind,

@@ -141,7 +141,8 @@ void schedule_constants(pb_handle* h) {
 
 // Split FC stages into row bands, one or more per thread block, of equal bytes:
 // block k owns the rows whose cumulative byte offset falls in [k*B, (k+1)*B), so
-// the block count is exact and the launch is one balanced wave.
+// the first wave is exact and balanced.  Networks whose weights are far larger than
+// the cache also get a second wave of short blocks (see below).
 void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSeg>& segs,
                   std::vector<int>& cta_begin, std::vector<int>& nparts, bool fuse_last) {
     segs.clear(); cta_begin.clear();
@@ -157,11 +158,26 @@ void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSe
         nparts[f] = 1;
         ++fused_ctas;
     }
-    double total = 0;
+    // The first wave (two resident blocks per SM) takes all but a small share of every
+    // stage's rows; the rest goes to short blocks of kFcTailRows rows that the hardware
+    // hands to whichever SM finishes its band first, which evens out the SMs' speeds.
+    const double tail_frac = kFcTailFraction;
+    const int tail_rows = kFcTailRows;
+    std::vector<int> main_rows(h->h_fc.size(), 0);
+    double total = 0, all_bytes = 0;
     for (int f : fc_ids) {
         const FcStage& st = h->h_fc[f];
         if (fuse_last && st.is_last) continue;
-        total += (double)st.out_dim * st.in_dim * 8.0;
+        all_bytes += (double)st.out_dim * st.in_dim * 8.0;
+    }
+    const bool with_tail = tail_frac > 0 && all_bytes >= 2.0 * h->num_sms * 1024.0 * 1024.0;
+    for (int f : fc_ids) {
+        const FcStage& st = h->h_fc[f];
+        if (fuse_last && st.is_last) continue;
+        int tail = with_tail ? (int)(st.out_dim * tail_frac / tail_rows + 0.5) * tail_rows : 0;
+        if (tail > st.out_dim - 1) tail = 0;
+        main_rows[f] = st.out_dim - tail;
+        total += (double)main_rows[f] * st.in_dim * 8.0;
     }
     if (total <= 0) return;
     int ncta = 2 * h->num_sms - fused_ctas;       // two resident blocks per SM
@@ -176,13 +192,13 @@ void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSe
         if (fuse_last && st.is_last) continue;
         const double row_bytes = st.in_dim * 8.0;
         int r = 0, part = 0;
-        while (r < st.out_dim) {
+        while (r < main_rows[f]) {
             // rows until the next block boundary (at least one), capped by the segment limit
             const double room = (cur + 1) * budget - acc;
             int n = (int)(room / row_bytes + 0.5);
             if (n < 1) n = 1;
             if (n > kFcMaxSegRows) n = kFcMaxSegRows;
-            if (n > st.out_dim - r) n = st.out_dim - r;
+            if (n > main_rows[f] - r) n = main_rows[f] - r;
             segs.push_back(FcSeg{f, r, r + n, part++, 0});
             r += n;
             acc += n * row_bytes;
@@ -192,6 +208,14 @@ void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSe
         nparts[f] = part;
     }
     if (cta_begin.back() != (int)segs.size()) cta_begin.push_back((int)segs.size());
+    for (int f : fc_ids) {
+        const FcStage& st = h->h_fc[f];
+        if (fuse_last && st.is_last) continue;
+        for (int r = main_rows[f]; r < st.out_dim; r += kFcTailRows) {
+            segs.push_back(FcSeg{f, r, std::min(st.out_dim, r + kFcTailRows), nparts[f]++, 0});
+            cta_begin.push_back((int)segs.size());
+        }
+    }
 }
 
 // ---------------------------------------------------------------- convolution planning

@@ -10,6 +10,8 @@ constexpr int kFcThreads = 256;
 constexpr int kFcWarps = kFcThreads / 32;
 constexpr int kFcMaxSegRows = 256;  // rows of one FC segment (bounds shared memory)
 constexpr int kFcChunksPerSweep = 2;
+constexpr double kFcTailFraction = 0.10;  // share of a large stage's rows left to short second-wave blocks
+constexpr int kFcTailRows = 16;           // rows of one such block
 
 // Where a stage finds the gradient w.r.t. its output: a consumer's hand-off
 // buffer laid out [slots][nparts][elems]; the reader sums the nparts rows.
