@@ -7,12 +7,15 @@
 // no block-wide barrier is needed, every lane holds kPostPer elements in
 // registers, and a resident block keeps eight independent chunks in flight,
 // which is what hides the (serial) load latencies of such small pieces of work.
-// Whatever needs the whole group goes through small partial tables that every
-// warp of the group combines in the same fixed order:
+// Whatever needs the whole group goes through small partial tables that one warp
+// per group combines in a fixed order:
 //   forward : conv_stats_kernel     (sum the K-slices, keep z, chunk mean / M2)
-//             conv_apply_fwd_kernel (merge statistics, normalise, skip, ReLU, pool)
-//   backward: conv_bwd_dn_kernel    (gradient at the normalised activation, channel sums)
-//             conv_bwd_dz_kernel    (scale/shift gradients, gradient at the conv output)
+//             conv_group_merge_kernel, mode 0 (group mean and 1/std from the chunk partials)
+//             conv_apply_fwd_kernel (normalise, skip, ReLU, pool)
+//   backward: conv_bwd_dn_kernel    (gradient at the normalised activation, channel sums per chunk)
+//             conv_group_merge_kernel, mode 1 (scale/shift gradients, group means)
+//             conv_bwd_dz_kernel    (gradient at the conv output)
+// The merges run once per group (one warp each) instead of once per chunk.
 #pragma once
 #include "conv_types.h"
 #include "fc_kernels.cuh"   // ring_slot, warp_sum
@@ -164,19 +167,8 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
             }
         }
     }
-    // group statistics from the chunk partials (the same arithmetic in every warp of the group)
-    const float* __restrict__ f = st.fstat + (size_t)ch.grp * st.fstat_stride * 3;
-    float tot = 0.f, wsum = 0.f;
-    for (int k = lane; k < ch.nidx; k += 32) { tot += f[3 * k]; wsum = fmaf(f[3 * k], f[3 * k + 1], wsum); }
-    tot = warp_sum(tot);
-    const float mean = warp_sum(wsum) / tot;
-    float m2 = 0.f;
-    for (int k = lane; k < ch.nidx; k += 32) { const float d = f[3 * k + 1] - mean; m2 += f[3 * k + 2] + f[3 * k] * d * d; }
-    const float rstd = rsqrtf(warp_sum(m2) / tot + kGnEps);
-    if (ch.idx == 0 && lane == 0) {
-        st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0] = mean;
-        st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1] = rstd;
-    }
+    const float mean = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0];
+    const float rstd = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1];
     auto act = [&](int c, int p) -> float {
         float v = fmaf(gam[c] * rstd, z[(size_t)c * hw + p] - mean, bet[c]);
         if (sk) v += skip_value(st, sk, c, p / st.ow, p % st.ow);
@@ -397,23 +389,8 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
         vload<VEC>(dnv[u], dz + idx);
         vload<VEC>(zv[u], z + idx);
     }
-    // channel sums of the whole group (pieces added in order), gradients of scale and
-    // shift, group means with the CURRENT scale
-    const float* __restrict__ gam = st.w + st.nw;
-    float m1 = 0.f, m2 = 0.f;
-    for (int cl = lane; cl < cpg; cl += 32) {
-        float t1 = 0.f, t2 = 0.f;
-        const float* __restrict__ b = st.bsum + (size_t)(c0 + cl) * st.npieces * 2;
-        for (int q = 0; q < st.npieces; ++q) { t1 += b[2 * q]; t2 += b[2 * q + 1]; }
-        if (ch.idx == 0) {
-            st.g[st.nw + c0 + cl] = t2;
-            st.g[st.nw + st.co + c0 + cl] = t1;
-        }
-        m1 = fmaf(gam[c0 + cl], t1, m1);
-        m2 = fmaf(gam[c0 + cl], t2, m2);
-    }
-    m1 = warp_sum(m1) / (float)(cpg * hw);
-    m2 = warp_sum(m2) / (float)(cpg * hw);
+    const float* __restrict__ gam = st.w + st.nw;      // the CURRENT scale
+    const float m1 = st.gsum[2 * ch.grp], m2 = st.gsum[2 * ch.grp + 1];
     float* __restrict__ dsk = st.dskip
         ? st.dskip + (size_t)slot_of(j, st.dskip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
 #pragma unroll
@@ -489,6 +466,75 @@ PB_POST_KERNEL(conv_apply_fwd_kernel, conv_apply_fwd_chunk, lane)
 PB_POST_KERNEL(conv_bwd_dn_kernel, conv_bwd_dn_chunk, S, lane)
 PB_POST_KERNEL(conv_bwd_dz_kernel, conv_bwd_dz_chunk, S, lane)
 #undef PB_POST_KERNEL
+
+// ---------------------------------------------------------------- group merges
+// mode 0 (forward): chunk statistics (count, mean, M2) -> group mean and 1/std, kept for the backward.
+// mode 1 (backward): per-chunk channel sums -> gradients of scale and shift, and the two
+// group means the gradient at the conv output needs (with the CURRENT scale).
+__global__ void __launch_bounds__(256)
+conv_group_merge_kernel(const ConvStage* __restrict__ stages, const GroupRef* __restrict__ groups, int ngroups,
+                        const TickState* __restrict__ ts, int S, int par, int mode) {
+    const int lane = threadIdx.x & 31;
+    const int gi = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (gi >= ngroups) return;
+    const GroupRef gr = groups[gi];
+    const ConvStage& st = stages[gr.stage];
+    const long long t = ts->cnt[par];
+    const int hw = st.oh * st.ow, cpg = st.cpg, c0 = gr.grp * cpg;
+    if (mode == 0) {
+        const long long i = t - st.s;
+        if (i < 0) return;
+        const int slot = slot_of(i, st.slots), nidx = st.fstat_stride;
+        const float* __restrict__ f = st.fstat + (size_t)gr.grp * st.fstat_stride * 3;
+        float tot = 0.f, wsum = 0.f;
+        for (int k = lane; k < nidx; k += 32) { tot += f[3 * k]; wsum = fmaf(f[3 * k], f[3 * k + 1], wsum); }
+        tot = warp_sum(tot);
+        const float mean = warp_sum(wsum) / tot;
+        float m2 = 0.f;
+        for (int k = lane; k < nidx; k += 32) { const float d = f[3 * k + 1] - mean; m2 += f[3 * k + 2] + f[3 * k] * d * d; }
+        const float rstd = rsqrtf(warp_sum(m2) / tot + kGnEps);
+        if (lane == 0) {
+            st.stat_ring[((size_t)slot * st.groups + gr.grp) * 2 + 0] = mean;
+            st.stat_ring[((size_t)slot * st.groups + gr.grp) * 2 + 1] = rstd;
+        }
+        return;
+    }
+    const long long j = t - 2LL * (S - 1) + st.s;
+    if (j < 0) return;
+    const float* __restrict__ gam = st.w + st.nw;
+    const int np = st.npieces;
+    float m1 = 0.f, m2 = 0.f;
+    if (np >= 8) {
+        // few channels, many pieces: lanes over the pieces of one channel at a time
+        for (int cl = 0; cl < cpg; ++cl) {
+            const float* __restrict__ b = st.bsum + (size_t)(c0 + cl) * np * 2;
+            float t1 = 0.f, t2 = 0.f;
+            for (int q = lane; q < np; q += 32) { t1 += b[2 * q]; t2 += b[2 * q + 1]; }
+            t1 = warp_sum(t1); t2 = warp_sum(t2);
+            if (lane == 0) {
+                st.g[st.nw + c0 + cl] = t2;
+                st.g[st.nw + st.co + c0 + cl] = t1;
+            }
+            m1 = fmaf(gam[c0 + cl], t1, m1);
+            m2 = fmaf(gam[c0 + cl], t2, m2);
+        }
+    } else {
+        for (int cl = lane; cl < cpg; cl += 32) {
+            const float* __restrict__ b = st.bsum + (size_t)(c0 + cl) * np * 2;
+            float t1 = 0.f, t2 = 0.f;
+            for (int q = 0; q < np; ++q) { t1 += b[2 * q]; t2 += b[2 * q + 1]; }
+            st.g[st.nw + c0 + cl] = t2;
+            st.g[st.nw + st.co + c0 + cl] = t1;
+            m1 = fmaf(gam[c0 + cl], t1, m1);
+            m2 = fmaf(gam[c0 + cl], t2, m2);
+        }
+        m1 = warp_sum(m1); m2 = warp_sum(m2);
+    }
+    if (lane == 0) {
+        st.gsum[2 * gr.grp] = m1 / (float)(cpg * hw);
+        st.gsum[2 * gr.grp + 1] = m2 / (float)(cpg * hw);
+    }
+}
 
 // ---------------------------------------------------------------- update
 // Fused SC + LWP step for materialised gradients (convolution stages):

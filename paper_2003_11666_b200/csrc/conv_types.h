@@ -52,6 +52,7 @@ struct ConvStage {
     float* stat_ring;            // [slots][2*groups] mean, rstd
     float* fstat; int fstat_stride;      // forward chunk partials [groups][fstat_stride][3]: count, mean, M2
     float* bsum; int npieces;            // backward channel partials [co][npieces][2]
+    float* gsum;                 // backward group means [groups][2] (of d*gamma and d*gamma*zhat)
     unsigned char* code_ring;    // [slots][co*oh*ow] bit0: ReLU passed
     unsigned char* arg_ring;     // [slots][co*out_h*out_w] max-pool winner position in its window
     float* out_ring;             // [slots][co*out_h*out_w]
@@ -87,6 +88,8 @@ struct UpdChunk { int range, start; };
 // (relative to the group), pixels [p0, p0+np); chunk `idx` of `nidx` in its group.
 // Either ncl >= 1 whole channels (p0 = 0, np = all pixels) or a piece of one channel.
 struct PostChunk { int stage, grp, cl0, ncl, p0, np, idx, nidx; };
+// One normalisation group of one stage (a warp of the merge kernel).
+struct GroupRef { int stage, grp; };
 constexpr int kUpdChunk = 4096;
 
 }  // namespace pb

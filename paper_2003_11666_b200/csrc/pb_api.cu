@@ -272,7 +272,7 @@ void add_tiles(std::vector<GemmTile>& tiles, int gemm, int M, int N, int nsplit,
 }
 
 void fill_conv_tables(pb_handle* h) {
-    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear();
+    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_groups.clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear();
     for (auto& t : h->h_tiles) t.clear();
     for (auto& t : h->h_tctiles) t.clear();
     const int bf = (h->flags & PB_CONV_BF16) ? 1 : 0;
@@ -358,11 +358,12 @@ void fill_conv_tables(pb_handle* h) {
         for (int q : x.consumers_main) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dx, y.dx_slots, y.dx_nparts}; }
         for (int q : x.consumers_skip) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dskip, y.dskip_slots, 1}; }
         c.dz = x.dz;
-        c.fstat = x.fstat; c.fstat_stride = x.fstat_stride; c.bsum = x.bsum; c.npieces = x.npieces;
+        c.fstat = x.fstat; c.fstat_stride = x.fstat_stride; c.bsum = x.bsum; c.npieces = x.npieces; c.gsum = x.gsum;
         {
             // chunks of the normalisation kernels: whole channels while they fit, else pieces of one channel
             const int hw = x.z.h * x.z.w, cpg = c.cpg;
             for (int gq = 0; gq < x.gn_groups; ++gq) {
+                h->h_groups.push_back(GroupRef{(int)h->h_cs.size(), gq});
                 const size_t first = h->h_pchunks.size();
                 if (hw <= kPostChunk) {
                     const int per = std::max(1, kPostChunk / hw);
@@ -442,6 +443,7 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     for (int q = 0; q < 3; ++q) h->d_tiles[q] = c.take<GemmTile>(h->h_tiles[q].size() + 1);
     h->d_cs = c.take<ConvStage>(h->h_cs.size() + 1);
     h->d_pchunks = c.take<PostChunk>(h->h_pchunks.size() + 1);
+    h->d_groups = c.take<GroupRef>(h->h_groups.size() + 1);
     h->d_upd = c.take<UpdRange>(h->h_upd.size() + 1);
     h->d_chunks = c.take<UpdChunk>(h->h_chunks.size() + 1);
     h->d_tc = c.take<ConvGemmTC>(h->h_tc.size() + 1);
@@ -481,6 +483,7 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
             x.gpart = c.take<float>((size_t)x.split_w * nw);
             x.fstat = c.take<float>((size_t)x.gn_groups * x.fstat_stride * 3);
             x.bsum = c.take<float>((size_t)x.head.c_out * x.npieces * 2);
+            x.gsum = c.take<float>((size_t)x.gn_groups * 2);
             if (h->flags & PB_CONV_BF16) {
                 x.out16 = c.take<__nv_bfloat16>((size_t)x.out_slots * x.out.elems());
                 x.dz16 = c.take<__nv_bfloat16>(ze);
@@ -555,6 +558,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
     const bool fused_last = h->nctaB == 0;      // the last stage rides in the phase-0 launch
     const int npc = (int)h->h_pchunks.size();
     const int post_grid = std::max(1, std::min(ceil_div(npc, kPostThreads / 32), 4 * h->num_sms));
+    const int ngr = (int)h->h_groups.size(), merge_grid = std::max(1, ceil_div(ngr, 8));
     for (int k = 0; k < n_ticks; ++k) {
         const int par = (int)((t_base + k) & 1);
         if (h->all_fc) {
@@ -606,6 +610,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             }
             prof_begin(h, 5);
             conv_stats_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
+            conv_group_merge_kernel<<<merge_grid, 256, 0, h->stream>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 0);
             conv_apply_fwd_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
             prof_end(h);
             // Backward chain: through pool/ReLU/GroupNorm -> data and weight gradients.  It reads
@@ -616,6 +621,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             cudaStreamWaitEvent(bs, h->ev_fork, 0);
             prof_begin(h, 6, bs);
             conv_bwd_dn_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
+            conv_group_merge_kernel<<<merge_grid, 256, 0, bs>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 1);
             conv_bwd_dz_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
             prof_end(h, bs);
             // data gradients (dgrad) and weight gradients (wgrad) both start from dz and write
@@ -646,7 +652,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             // the conv chain waits for the FC stages before the tick ends
             cudaEventRecord(h->ev_join, fs);
             cudaStreamWaitEvent(h->stream, h->ev_join, 0);
-            h->last_launches += 7 + (fused_last ? 0 : 1);      // ingest, 2 + 2 normalisation kernels, update, FC
+            h->last_launches += 9 + (fused_last ? 0 : 1);      // ingest, 3 + 3 normalisation kernels, update, FC
             for (int q = 0; q < 3; ++q) h->last_launches += (h->h_tiles[q].empty() ? 0 : 1) + (h->h_tctiles[q].empty() ? 0 : 1);
         }
     }
@@ -746,6 +752,7 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     for (int q = 0; q < 3; ++q) up(h->d_tiles[q], h->h_tiles[q].data(), h->h_tiles[q].size() * sizeof(GemmTile));
     up(h->d_cs, h->h_cs.data(), h->h_cs.size() * sizeof(ConvStage));
     up(h->d_pchunks, h->h_pchunks.data(), h->h_pchunks.size() * sizeof(PostChunk));
+    up(h->d_groups, h->h_groups.data(), h->h_groups.size() * sizeof(GroupRef));
     up(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange));
     up(h->d_chunks, h->h_chunks.data(), h->h_chunks.size() * sizeof(UpdChunk));
     up(h->d_tc, h->h_tc.data(), h->h_tc.size() * sizeof(ConvGemmTC));

@@ -37,7 +37,7 @@ struct StageHost {
     // convolution stages only
     float *z_ring = nullptr, *stat_ring = nullptr, *zpart = nullptr, *dz = nullptr, *gpart = nullptr;
     unsigned char *code_ring = nullptr, *arg_ring = nullptr;
-    float *fstat = nullptr, *bsum = nullptr; int fstat_stride = 1, npieces = 1;
+    float *fstat = nullptr, *bsum = nullptr, *gsum = nullptr; int fstat_stride = 1, npieces = 1;
     int split_f = 1, split_d = 1, split_w = 1;                     // K-slices of fprop / dgrad / wgrad
     int kps_f = 0, kps_d = 0, kps_w = 0;                           // K per slice
     bool tc = false;                                               // tensor-core path, weights kept as [co][r][s][ci]
@@ -90,6 +90,7 @@ struct pb_handle {
     std::vector<pb::GemmTile> h_tiles[3]; pb::GemmTile* d_tiles[3] = {nullptr, nullptr, nullptr};
     std::vector<pb::ConvStage> h_cs; pb::ConvStage* d_cs = nullptr;
     std::vector<pb::PostChunk> h_pchunks; pb::PostChunk* d_pchunks = nullptr;
+    std::vector<pb::GroupRef> h_groups; pb::GroupRef* d_groups = nullptr;
     std::vector<pb::UpdRange> h_upd; pb::UpdRange* d_upd = nullptr;
     std::vector<pb::UpdChunk> h_chunks; pb::UpdChunk* d_chunks = nullptr;
 
