@@ -2,20 +2,18 @@
 //
 // A convolution stage is  conv -> GroupNorm -> (+skip) -> ReLU -> (max-pool |
 // global average pool).  The elements of a normalisation group are cut into
-// chunks of at most kPostChunk elements (whole channels when the image is
-// small, pieces of one channel when it is large) and ONE WARP owns a chunk:
-// no block-wide barrier is needed, every lane holds kPostPer elements in
-// registers, and a resident block keeps eight independent chunks in flight,
-// which is what hides the (serial) load latencies of such small pieces of work.
-// Whatever needs the whole group goes through small partial tables that one warp
-// per group combines in a fixed order:
+// chunks of at most kPostChunk elements that are contiguous in memory (whole
+// channels when the image is small, a piece of one channel when it is large)
+// and ONE BLOCK owns a chunk: every thread holds kPostPer elements, all its
+// loads are issued before anything is used, and a resident SM keeps six to eight
+// such blocks in flight.  Whatever needs the whole group goes through small
+// partial tables that one warp per group combines in a fixed order:
 //   forward : conv_stats_kernel     (sum the K-slices, keep z, chunk mean / M2)
 //             conv_group_merge_kernel, mode 0 (group mean and 1/std from the chunk partials)
 //             conv_apply_fwd_kernel (normalise, skip, ReLU, pool)
 //   backward: conv_bwd_dn_kernel    (gradient at the normalised activation, channel sums per chunk)
 //             conv_group_merge_kernel, mode 1 (scale/shift gradients, group means)
 //             conv_bwd_dz_kernel    (gradient at the conv output)
-// The merges run once per group (one warp each) instead of once per chunk.
 #pragma once
 #include "conv_types.h"
 #include "fc_kernels.cuh"   // ring_slot, warp_sum
@@ -23,34 +21,13 @@
 namespace pb {
 
 constexpr float kGnEps = 1e-5f;
-constexpr int kPostPer = kPostChunk / 32;       // elements per lane
-constexpr int kPostRun = 1;                     // consecutive chunks a warp takes at a time (longer runs measured slower)
+constexpr int kPostPer = kPostChunk / kPostThreads;       // elements per thread
+constexpr int kPostWarps = kPostThreads / 32;
 
 __device__ __forceinline__ float skip_value(const ConvStage& st, const float* __restrict__ sk, int c, int y, int x) {
     if (st.skip_mode == 0) return sk[((size_t)c * st.skip_h + y) * st.skip_w + x];
     return c < st.skip_c ? sk[((size_t)c * st.skip_h + 2 * y) * st.skip_w + 2 * x] : 0.f;
 }
-
-// A lane works on units of VEC consecutive pixels of one channel (VEC = 4 when the
-// image size is a multiple of 4: float4 / uchar4 accesses, a quarter of the index
-// arithmetic).  Units lane, lane+32, ... of a chunk are walked without divisions.
-template <int VEC>
-struct ChunkWalk {
-    int cl, p, e, npu;          // channel in chunk, pixel offset, unit index, units per channel
-    __device__ __forceinline__ ChunkWalk(const PostChunk& ch, int lane) {
-        npu = ch.np / VEC;
-        e = lane; cl = lane / npu; p = (lane - cl * npu) * VEC;
-    }
-    __device__ __forceinline__ void get(const PostChunk& ch, int c0, int nunits, int& c, int& pix, bool& ok) const {
-        ok = e < nunits;
-        c = c0 + ch.cl0 + (ok ? cl : ch.ncl - 1);
-        pix = ch.p0 + (ok ? p : ch.np - VEC);
-    }
-    __device__ __forceinline__ void next(const PostChunk& ch) {
-        e += 32; p += 32 * VEC;
-        while (p >= ch.np && e < ch.ncl * npu) { p -= ch.np; ++cl; }
-    }
-};
 
 __device__ __forceinline__ int slot_of(long long sample, int slots) { return (int)((unsigned)sample % (unsigned)slots); }
 
@@ -65,78 +42,120 @@ template <> __device__ __forceinline__ void stb<4>(unsigned char* p, const unsig
 }
 template <> __device__ __forceinline__ void stb<1>(unsigned char* p, const unsigned char (&r)[1]) { *p = r[0]; }
 
+// Sum over the block, returned to every thread (two barriers; `red` holds kPostWarps floats).
+__device__ __forceinline__ float block_sum(float x, float* red) {
+    x = warp_sum(x);
+    __syncthreads();                       // `red` may still be read from the previous call
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
+    __syncthreads();
+    float a = 0.f;
+#pragma unroll
+    for (int k = 0; k < kPostWarps; ++k) a += red[k];
+    return a;
+}
+
+// A chunk is the contiguous range [base, base + n) of the stage's [channel][pixel] tensor:
+// unit q (VEC consecutive pixels of one channel) of thread `tid` is unit u*kPostThreads + tid.
+struct ChunkGeom {
+    int hw, n, nunits, base, c_first;
+    __device__ __forceinline__ ChunkGeom(const ConvStage& st, const PostChunk& ch, int vec) {
+        hw = st.oh * st.ow;
+        n = ch.ncl * ch.np;
+        nunits = n / vec;
+        c_first = ch.grp * st.cpg + ch.cl0;
+        base = c_first * hw + ch.p0;
+    }
+};
+
 // ---------------------------------------------------------------- forward, step 1
 template <int VEC>
-__device__ void conv_stats_chunk(const ConvStage& st, const PostChunk& ch, long long t, int lane) {
+__device__ void conv_stats_chunk(const ConvStage& st, const PostChunk& ch, long long t, float* red) {
     constexpr int U = kPostPer / VEC;
     const long long i = t - st.s;
     if (i < 0) return;
+    const int tid = threadIdx.x;
     const int slot = slot_of(i, st.slots);
-    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np, nunits = n / VEC;
-    const size_t zelems = (size_t)st.co * hw;
-    float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
-    const float* __restrict__ zp = st.zpart;
+    const ChunkGeom cg(st, ch, VEC);
+    const size_t zelems = (size_t)st.co * cg.hw;
+    float* __restrict__ z = st.z_ring + (size_t)slot * zelems + cg.base;
+    const float* __restrict__ zp = st.zpart + cg.base;
     float vals[U][VEC];
-    unsigned idx[U];
-    bool ok[U];
-    {
-        ChunkWalk<VEC> w(ch, lane);
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            int c, p;
-            w.get(ch, c0, nunits, c, p, ok[u]);
-            w.next(ch);
-            idx[u] = (unsigned)(c * hw + p);
+    for (int u = 0; u < U; ++u)
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) vals[u][e] = 0.f;
-        }
-    }
+        for (int e = 0; e < VEC; ++e) vals[u][e] = 0.f;
     // the K-slice loop is outside so that each step issues U independent loads
     for (int q = 0; q < st.z_nsplit; ++q) {
         const float* __restrict__ zq = zp + (size_t)q * zelems;
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            float r[VEC];
-            vload<VEC>(r, zq + idx[u]);
+            const int unit = u * kPostThreads + tid;
+            if (unit < cg.nunits) {
+                float r[VEC];
+                vload<VEC>(r, zq + unit * VEC);
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) vals[u][e] += r[e];
+                for (int e = 0; e < VEC; ++e) vals[u][e] += r[e];
+            }
         }
     }
     float sum = 0.f;
 #pragma unroll
-    for (int u = 0; u < U; ++u)
-        if (ok[u]) {
-            vstore<VEC>(z + idx[u], vals[u]);
+    for (int u = 0; u < U; ++u) {
+        const int unit = u * kPostThreads + tid;
+        if (unit < cg.nunits) {
+            vstore<VEC>(z + unit * VEC, vals[u]);
 #pragma unroll
             for (int e = 0; e < VEC; ++e) sum += vals[u][e];
         }
-    const float mean = warp_sum(sum) / (float)n;
+    }
+    const float mean = block_sum(sum, red) / (float)cg.n;
     float sq = 0.f;
 #pragma unroll
     for (int u = 0; u < U; ++u)
-        if (ok[u]) {
+        if (u * kPostThreads + tid < cg.nunits) {
 #pragma unroll
             for (int e = 0; e < VEC; ++e) { const float d = vals[u][e] - mean; sq = fmaf(d, d, sq); }
         }
-    const float m2 = warp_sum(sq);
-    if (lane == 0) {
+    const float m2 = block_sum(sq, red);
+    if (tid == 0) {
         float* f = st.fstat + ((size_t)ch.grp * st.fstat_stride + ch.idx) * 3;
-        f[0] = (float)n; f[1] = mean; f[2] = m2;
+        f[0] = (float)cg.n; f[1] = mean; f[2] = m2;
     }
 }
 
 // ---------------------------------------------------------------- forward, step 2
+// Elementwise over a TILE: channels [cl0, cl0+ncl) (absolute) x pixels [p0, p0+np).  Plain
+// stages are tiled as (a multiple of 8 channels) x (up to 128 pixels), so that the bfloat16
+// [pixel][channel] copy can be written as whole 16-byte runs of 8 channels after a transpose
+// through shared memory; stages that pool keep their group chunks as tiles.
+__device__ __forceinline__ void store_nhwc_tile(const __nv_bfloat16* t16, int rs, const PostChunk& ch, int co,
+                                                __nv_bfloat16* __restrict__ dst) {
+    const int ng = ch.ncl >> 3;
+    for (int idx = threadIdx.x; idx < ch.np * ng; idx += kPostThreads) {
+        const int pix = idx / ng, cgp = idx - pix * ng;
+        const unsigned short* src = reinterpret_cast<const unsigned short*>(t16) + (size_t)(cgp * 8) * rs + pix;
+        uint4 v;
+        v.x = src[0] | ((unsigned)src[rs] << 16);
+        v.y = src[2 * rs] | ((unsigned)src[3 * rs] << 16);
+        v.z = src[4 * rs] | ((unsigned)src[5 * rs] << 16);
+        v.w = src[6 * rs] | ((unsigned)src[7 * rs] << 16);
+        *reinterpret_cast<uint4*>(dst + (size_t)(ch.p0 + pix) * co + ch.cl0 + cgp * 8) = v;
+    }
+}
+
 template <int VEC>
-__device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, long long t, int lane) {
+__device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, long long t, __nv_bfloat16* t16) {
     constexpr int U = kPostPer / VEC;
     const long long i = t - st.s;
     if (i < 0) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int slot = slot_of(i, st.slots);
-    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np, nunits = n / VEC;
+    const int hw = st.oh * st.ow, npu = ch.np / VEC, nunits = ch.ncl * npu, rs = ch.np + 2;
     const size_t zelems = (size_t)st.co * hw;
     const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
     const float* __restrict__ gam = st.wh + st.nw;
     const float* __restrict__ bet = gam + st.co;
+    const float* __restrict__ stat = st.stat_ring + (size_t)slot * st.groups * 2;
     const float* __restrict__ sk = st.skip_ring
         ? st.skip_ring + (size_t)slot_of(i, st.skip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
     unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems;
@@ -144,70 +163,79 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
     const size_t oelems = (size_t)st.co * st.out_h * st.out_w;
     float* __restrict__ out = st.out_ring + (size_t)slot * oelems;
     __nv_bfloat16* __restrict__ out16 = st.out16 ? st.out16 + (size_t)slot * oelems : nullptr;
-    // the loads of the lane's units go first: they do not depend on the statistics
+    const bool transposed = out16 && !pooled && (ch.ncl & 7) == 0 && ch.ncl <= kPostTileChannels && (ch.cl0 & 7) == 0 && (st.co & 7) == 0;
+    // all loads of the thread's units first
     int cc[U], pp[U];
     bool ok[U];
-    float zv[U][VEC], sv[U][VEC];
-    {
-        ChunkWalk<VEC> w(ch, lane);
+    float zv[U][VEC], sv[U][VEC], gs[U], bb[U], mean[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            w.get(ch, c0, nunits, cc[u], pp[u], ok[u]);
-            w.next(ch);
-            vload<VEC>(zv[u], z + (size_t)cc[u] * hw + pp[u]);
-            if (!sk) {
+    for (int u = 0; u < U; ++u) {
+        const int unit = u * kPostThreads + tid;
+        ok[u] = unit < nunits;
+        const int uu = ok[u] ? unit : 0;
+        const int cl = uu / npu;
+        cc[u] = ch.cl0 + cl;
+        pp[u] = ch.p0 + (uu - cl * npu) * VEC;
+        const size_t idx = (size_t)cc[u] * hw + pp[u];
+        const int grp = cc[u] / st.cpg;
+        vload<VEC>(zv[u], z + idx);
+        mean[u] = stat[2 * grp];
+        gs[u] = gam[cc[u]] * stat[2 * grp + 1];
+        bb[u] = bet[cc[u]];
+        if (!sk) {
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) sv[u][e] = 0.f;
-            } else if (st.skip_mode == 0) {
-                // identity skips share this stage's indexing
-                vload<VEC>(sv[u], sk + (size_t)cc[u] * hw + pp[u]);
-            } else {
+            for (int e = 0; e < VEC; ++e) sv[u][e] = 0.f;
+        } else if (st.skip_mode == 0) {
+            vload<VEC>(sv[u], sk + idx);            // identity skips share this stage's indexing
+        } else {
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) sv[u][e] = skip_value(st, sk, cc[u], (pp[u] + e) / st.ow, (pp[u] + e) % st.ow);
-            }
+            for (int e = 0; e < VEC; ++e) sv[u][e] = skip_value(st, sk, cc[u], (pp[u] + e) / st.ow, (pp[u] + e) % st.ow);
         }
     }
-    const float mean = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0];
-    const float rstd = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1];
     auto act = [&](int c, int p) -> float {
-        float v = fmaf(gam[c] * rstd, z[(size_t)c * hw + p] - mean, bet[c]);
+        const int grp = c / st.cpg;
+        float v = fmaf(gam[c] * stat[2 * grp + 1], z[(size_t)c * hw + p] - stat[2 * grp], bet[c]);
         if (sk) v += skip_value(st, sk, c, p / st.ow, p % st.ow);
         return v;
     };
-    {
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (!ok[u]) continue;
-            const int c = cc[u], p = pp[u];
-            const float gs = gam[c] * rstd, bb = bet[c];
-            float a[VEC];
-            unsigned char cd[VEC];
+    for (int u = 0; u < U; ++u) {
+        if (!ok[u]) continue;
+        const int c = cc[u], p = pp[u];
+        float a[VEC];
+        unsigned char cd[VEC];
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-                const float v = fmaf(gs, zv[u][e] - mean, bb) + sv[u][e];
-                const bool pass = st.relu ? v > 0.f : true;
-                cd[e] = pass ? 1 : 0;
-                a[e] = pass ? v : 0.f;
-            }
-            stb<VEC>(code + (size_t)c * hw + p, cd);
-            if (!pooled) {
-                vstore<VEC>(out + (size_t)c * hw + p, a);
-                if (out16) {
+        for (int e = 0; e < VEC; ++e) {
+            const float v = fmaf(gs[u], zv[u][e] - mean[u], bb[u]) + sv[u][e];
+            const bool pass = st.relu ? v > 0.f : true;
+            cd[e] = pass ? 1 : 0;
+            a[e] = pass ? v : 0.f;
+        }
+        stb<VEC>(code + (size_t)c * hw + p, cd);
+        if (!pooled) {
+            vstore<VEC>(out + (size_t)c * hw + p, a);
+            if (transposed) {
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) out16[(size_t)(p + e) * st.co + c] = __float2bfloat16_rn(a[e]);
-                }
+                for (int e = 0; e < VEC; ++e) t16[(c - ch.cl0) * rs + (p - ch.p0) + e] = __float2bfloat16_rn(a[e]);
+            } else if (out16) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) out16[(size_t)(p + e) * st.co + c] = __float2bfloat16_rn(a[e]);
             }
         }
     }
+    if (transposed) {
+        __syncthreads();
+        store_nhwc_tile(t16, rs, ch, st.co, out16);
+    }
     if (st.pool_k > 0) {
-        // max-pool: this chunk owns the pooled pixels [p0*ohw/hw, (p0+np)*ohw/hw) of its channels;
+        // max-pool: this tile owns the pooled pixels [p0*ohw/hw, (p0+np)*ohw/hw) of its channels;
         // first maximum in row-major window order, padding never wins
         const int ohw = st.out_h * st.out_w, k = st.pool_k;
         const int o0 = (int)((long long)ch.p0 * ohw / hw), o1 = (int)((long long)(ch.p0 + ch.np) * ohw / hw);
         const int no = o1 - o0;
         unsigned char* __restrict__ arg = st.arg_ring + (size_t)slot * oelems;
-        for (int e = lane; e < ch.ncl * no; e += 32) {
-            const int c = c0 + ch.cl0 + e / no, op = o0 + e % no, py = op / st.out_w, px = op % st.out_w;
+        for (int e = tid; e < ch.ncl * no; e += kPostThreads) {
+            const int c = ch.cl0 + e / no, op = o0 + e % no, py = op / st.out_w, px = op % st.out_w;
             float best = -INFINITY;
             int bpos = 0;
             for (int r = 0; r < k; ++r)
@@ -223,9 +251,9 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
             arg[(size_t)c * ohw + op] = (unsigned char)bpos;
         }
     } else if (st.avgpool) {
-        // global average per channel (chunks of such stages hold whole channels)
-        for (int cl = 0; cl < ch.ncl; ++cl) {
-            const int c = c0 + ch.cl0 + cl;
+        // global average per channel (tiles of such stages hold whole channels): a warp per channel
+        for (int cl = warp; cl < ch.ncl; cl += kPostWarps) {
+            const int c = ch.cl0 + cl;
             float a = 0.f;
             for (int p = lane; p < hw; p += 32) {
                 float v = act(c, p);
@@ -251,56 +279,71 @@ __device__ __forceinline__ float gather_out_delta(const ConvStage& st, size_t oe
 }
 
 template <int VEC>
-__device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long long t, int S, int lane) {
+__device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long long t, int S, float* red, float* usum) {
     constexpr int U = kPostPer / VEC;
     const long long j = t - 2LL * (S - 1) + st.s;
     if (j < 0) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int slot = slot_of(j, st.slots);
-    const int hw = st.oh * st.ow, c0 = ch.grp * st.cpg, n = ch.ncl * ch.np, nunits = n / VEC;
+    const ChunkGeom cg(st, ch, VEC);
+    const int hw = cg.hw, npu = ch.np / VEC;
     const size_t zelems = (size_t)st.co * hw;
     const size_t oelems = (size_t)st.co * st.out_h * st.out_w;
-    const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
-    const unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems;
+    const float* __restrict__ z = st.z_ring + (size_t)slot * zelems + cg.base;
+    const unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems + cg.base;
     const float mean = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0];
     const float rstd = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1];
-    float* __restrict__ dz = st.dz;
+    float* __restrict__ dz = st.dz + cg.base;
     const int ohw = st.out_h * st.out_w;
-    int cc[U];
-    unsigned idx[U];
     bool ok[U];
     float d[U][VEC], zv[U][VEC];
     unsigned char cd[U][VEC];
-    ChunkWalk<VEC> wk(ch, lane);
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-        int p;
-        wk.get(ch, c0, nunits, cc[u], p, ok[u]);
-        wk.next(ch);
-        idx[u] = (unsigned)(cc[u] * hw + p);
-        vload<VEC>(zv[u], z + idx[u]);
-        ldb<VEC>(cd[u], code + idx[u]);
+        const int unit = u * kPostThreads + tid;
+        ok[u] = unit < cg.nunits;
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) d[u][e] = 0.f;
+        for (int e = 0; e < VEC; ++e) { d[u][e] = 0.f; zv[u][e] = 0.f; cd[u][e] = 0; }
+        if (ok[u]) {
+            vload<VEC>(zv[u], z + unit * VEC);
+            ldb<VEC>(cd[u], code + unit * VEC);
+        }
     }
     if (!st.avgpool && st.pool_k == 0) {
         // plain stage: the consumers' partial rows line up with this stage's elements
         for (int q = 0; q < st.n_dsrc; ++q) {
-            const float* bp = st.dsrc[q].ptr + (size_t)slot_of(j, st.dsrc[q].slots) * st.dsrc[q].nparts * oelems;
+            const float* bp = st.dsrc[q].ptr + (size_t)slot_of(j, st.dsrc[q].slots) * st.dsrc[q].nparts * oelems + cg.base;
             const int np_ = st.dsrc[q].nparts;
             for (int kp = 0; kp < np_; ++kp, bp += oelems) {
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
+                    if (!ok[u]) continue;
                     float r[VEC];
-                    vload<VEC>(r, bp + idx[u]);
+                    vload<VEC>(r, bp + (u * kPostThreads + tid) * VEC);
 #pragma unroll
                     for (int e = 0; e < VEC; ++e) d[u][e] += r[e];
                 }
             }
         }
     } else if (st.avgpool) {
+        // every pixel of a channel receives the same value: a warp gathers it once per
+        // channel (lanes over the consumers' partial rows) and hands it on through shared memory
+        __syncthreads();
+        for (int cl = warp; cl < ch.ncl; cl += kPostWarps) {
+            float a = 0.f;
+            for (int q = 0; q < st.n_dsrc; ++q) {
+                const DeltaSrc& ds = st.dsrc[q];
+                const float* p = ds.ptr + ((size_t)slot_of(j, ds.slots) * ds.nparts) * oelems + cg.c_first + cl;
+                for (int k = lane; k < ds.nparts; k += 32) a += p[(size_t)k * oelems];
+            }
+            a = warp_sum(a);
+            if (lane == 0) usum[cl] = a / (float)hw;
+        }
+        __syncthreads();
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const float a = gather_out_delta(st, oelems, cc[u], j) / (float)hw;
+            if (!ok[u]) continue;
+            const float a = usum[(u * kPostThreads + tid) / npu];
 #pragma unroll
             for (int e = 0; e < VEC; ++e) d[u][e] = a;
         }
@@ -311,9 +354,11 @@ __device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long
 #pragma unroll 1
         for (int u = 0; u < U; ++u) {
             if (!ok[u]) continue;
+            const int unit = u * kPostThreads + tid, cl = unit / npu;
+            const int c = cg.c_first + cl, p0 = ch.p0 + (unit - cl * npu) * VEC;
 #pragma unroll 1
             for (int e = 0; e < VEC; ++e) {
-                const int p = (int)idx[u] - cc[u] * hw + e;
+                const int p = p0 + e;
                 const int y = p / st.ow, x = p % st.ow;
                 float a = 0.f;
                 for (int r = 0; r < kk; ++r) {
@@ -326,7 +371,7 @@ __device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long
                         if (tx < 0 || tx % ps) continue;
                         const int px = tx / ps;
                         if (px >= st.out_w) continue;
-                        const size_t o = (size_t)cc[u] * ohw + py * st.out_w + px;
+                        const size_t o = (size_t)c * ohw + py * st.out_w + px;
                         if (arg[o] == r * kk + s) a += gather_out_delta(st, oelems, o, j);
                     }
                 }
@@ -344,53 +389,77 @@ __device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long
             s1[u] += d[u][e];
             s2[u] = fmaf(d[u][e], (zv[u][e] - mean) * rstd, s2[u]);      // d * zhat
         }
-        if (ok[u]) vstore<VEC>(dz + idx[u], d[u]);
+        if (ok[u]) vstore<VEC>(dz + (u * kPostThreads + tid) * VEC, d[u]);
     }
     // per-channel sums of d and d*zhat over this chunk's pixels
     const int piece = ch.p0 / kPostChunk;
-    for (int cl = 0; cl < ch.ncl; ++cl) {
-        const int c = c0 + ch.cl0 + cl;
+    if (ch.ncl == 1) {
         float a1 = 0.f, a2 = 0.f;
 #pragma unroll
-        for (int u = 0; u < U; ++u)
-            if (cc[u] == c) { a1 += s1[u]; a2 += s2[u]; }
-        a1 = warp_sum(a1);
-        a2 = warp_sum(a2);
-        if (lane == 0) {
-            float* b = st.bsum + ((size_t)c * st.npieces + piece) * 2;
+        for (int u = 0; u < U; ++u) { a1 += s1[u]; a2 += s2[u]; }
+        a1 = block_sum(a1, red);
+        a2 = block_sum(a2, red);
+        if (tid == 0) {
+            float* b = st.bsum + ((size_t)cg.c_first * st.npieces + piece) * 2;
             b[0] = a1; b[1] = a2;
+        }
+    } else {
+        // several whole channels: unit sums go through shared memory, then a warp per channel
+        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int unit = u * kPostThreads + tid;
+            if (unit < cg.nunits) { usum[2 * unit] = s1[u]; usum[2 * unit + 1] = s2[u]; }
+        }
+        __syncthreads();
+        for (int cl = warp; cl < ch.ncl; cl += kPostWarps) {
+            float a1 = 0.f, a2 = 0.f;
+            for (int q = lane; q < npu; q += 32) { a1 += usum[2 * (cl * npu + q)]; a2 += usum[2 * (cl * npu + q) + 1]; }
+            a1 = warp_sum(a1);
+            a2 = warp_sum(a2);
+            if (lane == 0) {
+                float* b = st.bsum + ((size_t)(cg.c_first + cl) * st.npieces + piece) * 2;
+                b[0] = a1; b[1] = a2;
+            }
         }
     }
 }
 
 // ---------------------------------------------------------------- backward, step 2
+// Elementwise over a tile (see the forward step 2).
 template <int VEC>
-__device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long long t, int S, int lane) {
+__device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long long t, int S, __nv_bfloat16* t16) {
     constexpr int U = kPostPer / VEC;
     const long long j = t - 2LL * (S - 1) + st.s;
     if (j < 0) return;
+    const int tid = threadIdx.x;
     const int slot = slot_of(j, st.slots);
-    const int hw = st.oh * st.ow, cpg = st.cpg, c0 = ch.grp * cpg, n = ch.ncl * ch.np, nunits = n / VEC;
+    const int hw = st.oh * st.ow, npu = ch.np / VEC, nunits = ch.ncl * npu, rs = ch.np + 2;
     const size_t zelems = (size_t)st.co * hw;
     const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
-    const float mean = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 0];
-    const float rstd = st.stat_ring[((size_t)slot * st.groups + ch.grp) * 2 + 1];
+    const float* __restrict__ stat = st.stat_ring + (size_t)slot * st.groups * 2;
+    const float* __restrict__ gam = st.w + st.nw;      // the CURRENT scale
     float* __restrict__ dz = st.dz;
-    // the loads of the lane's units go first: they do not depend on the group sums
+    const bool transposed = st.dz16 && (ch.ncl & 7) == 0 && ch.ncl <= kPostTileChannels && (ch.cl0 & 7) == 0 && (st.co & 7) == 0;
     int cc[U], pp[U];
     bool ok[U];
-    float dnv[U][VEC], zv[U][VEC];
-    ChunkWalk<VEC> wk(ch, lane);
+    float dnv[U][VEC], zv[U][VEC], gv[U], mean[U], rstd[U], m1[U], m2[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {                     // all loads of the lane's units first
-        wk.get(ch, c0, nunits, cc[u], pp[u], ok[u]);
-        wk.next(ch);
+    for (int u = 0; u < U; ++u) {                     // all loads of the thread's units first
+        const int unit = u * kPostThreads + tid;
+        ok[u] = unit < nunits;
+        const int uu = ok[u] ? unit : 0;
+        const int cl = uu / npu;
+        cc[u] = ch.cl0 + cl;
+        pp[u] = ch.p0 + (uu - cl * npu) * VEC;
         const size_t idx = (size_t)cc[u] * hw + pp[u];
+        const int grp = cc[u] / st.cpg;
         vload<VEC>(dnv[u], dz + idx);
         vload<VEC>(zv[u], z + idx);
+        gv[u] = gam[cc[u]];
+        mean[u] = stat[2 * grp]; rstd[u] = stat[2 * grp + 1];
+        m1[u] = st.gsum[2 * grp]; m2[u] = st.gsum[2 * grp + 1];
     }
-    const float* __restrict__ gam = st.w + st.nw;      // the CURRENT scale
-    const float m1 = st.gsum[2 * ch.grp], m2 = st.gsum[2 * ch.grp + 1];
     float* __restrict__ dsk = st.dskip
         ? st.dskip + (size_t)slot_of(j, st.dskip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
 #pragma unroll
@@ -415,56 +484,48 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
                 }
             }
         }
-        const float g = gam[c];
         float dd[VEC];
 #pragma unroll
         for (int e = 0; e < VEC; ++e) {
-            const float zh = (zv[u][e] - mean) * rstd;
-            dd[e] = rstd * (fmaf(dnv[u][e], g, -m1) - zh * m2);
+            const float zh = (zv[u][e] - mean[u]) * rstd[u];
+            dd[e] = rstd[u] * (fmaf(dnv[u][e], gv[u], -m1[u]) - zh * m2[u]);
         }
         vstore<VEC>(dz + idx, dd);
-        if (st.dz16) {
+        if (transposed) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) t16[(c - ch.cl0) * rs + (p - ch.p0) + e] = __float2bfloat16_rn(dd[e]);
+        } else if (st.dz16) {
 #pragma unroll
             for (int e = 0; e < VEC; ++e) st.dz16[(size_t)(p + e) * st.co + c] = __float2bfloat16_rn(dd[e]);
         }
     }
+    if (transposed) {
+        __syncthreads();
+        store_nhwc_tile(t16, rs, ch, st.co, st.dz16);
+    }
 }
 
 // ---------------------------------------------------------------- launch wrappers
-// Persistent blocks.  The chunk table is dealt to the warps in short runs of
-// consecutive chunks, round-robin (chunks are ordered by stage and differ a lot in
-// cost between stages: long contiguous ranges unbalance the warps, single chunks
-// make every warp reload its stage descriptor, kept in shared memory, each time).
+// One block per chunk (statistics, channel sums) or tile (elementwise kernels).
 #define PB_POST_KERNEL(NAME, CHUNK, ...)                                                          \
     __global__ void __launch_bounds__(kPostThreads, 4) NAME(const ConvStage* __restrict__ stages,  \
                                                             const PostChunk* __restrict__ chunks, int nchunks, \
                                                             const TickState* __restrict__ ts, int S, int par) { \
-        __shared__ ConvStage sst[kPostThreads / 32];                                               \
-        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;                                \
+        __shared__ float red[kPostWarps];                                                          \
+        __shared__ float usum[2 * kPostChunk];                                                     \
+        __shared__ __align__(16) __nv_bfloat16 t16[kPostChunk + 2 * kPostTileChannels];            \
+        (void)red; (void)usum; (void)t16; (void)S;                                                 \
+        if ((int)blockIdx.x >= nchunks) return;                                                    \
+        const PostChunk ch = chunks[blockIdx.x];                                                   \
         const long long t = ts->cnt[par];                                                          \
-        const int nwarps = gridDim.x * (kPostThreads / 32);                                        \
-        const int gw = blockIdx.x * (kPostThreads / 32) + warp;                                    \
-        int loaded = -1;                                                                           \
-        /* runs of kPostRun consecutive chunks, dealt round-robin to the warps */                  \
-        for (int base = gw * kPostRun; base < nchunks; base += nwarps * kPostRun)                  \
-        for (int ci = base; ci < min(nchunks, base + kPostRun); ++ci) {                            \
-            const PostChunk ch = chunks[ci];                                                       \
-            if (ch.stage != loaded) {                                                              \
-                __syncwarp();                                                                      \
-                const int* s_ = reinterpret_cast<const int*>(&stages[ch.stage]);                   \
-                int* d_ = reinterpret_cast<int*>(&sst[warp]);                                      \
-                for (int k = lane; k < (int)(sizeof(ConvStage) / 4); k += 32) d_[k] = s_[k];       \
-                __syncwarp();                                                                      \
-                loaded = ch.stage;                                                                 \
-            }                                                                                      \
-            if (sst[warp].vec4) CHUNK<4>(sst[warp], ch, t, __VA_ARGS__);                           \
-            else CHUNK<1>(sst[warp], ch, t, __VA_ARGS__);                                          \
-        }                                                                                          \
+        const ConvStage& st = stages[ch.stage];                                                    \
+        if (st.vec4) CHUNK<4>(st, ch, t, __VA_ARGS__);                                             \
+        else CHUNK<1>(st, ch, t, __VA_ARGS__);                                                     \
     }
-PB_POST_KERNEL(conv_stats_kernel, conv_stats_chunk, lane)
-PB_POST_KERNEL(conv_apply_fwd_kernel, conv_apply_fwd_chunk, lane)
-PB_POST_KERNEL(conv_bwd_dn_kernel, conv_bwd_dn_chunk, S, lane)
-PB_POST_KERNEL(conv_bwd_dz_kernel, conv_bwd_dz_chunk, S, lane)
+PB_POST_KERNEL(conv_stats_kernel, conv_stats_chunk, red)
+PB_POST_KERNEL(conv_apply_fwd_kernel, conv_apply_fwd_chunk, t16)
+PB_POST_KERNEL(conv_bwd_dn_kernel, conv_bwd_dn_chunk, S, red, usum)
+PB_POST_KERNEL(conv_bwd_dz_kernel, conv_bwd_dz_chunk, S, t16)
 #undef PB_POST_KERNEL
 
 // ---------------------------------------------------------------- group merges

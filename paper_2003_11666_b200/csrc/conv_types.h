@@ -10,7 +10,9 @@ constexpr int kGemmThreads = 256;
 constexpr int kBM = 64, kBN = 64, kBK = 16;
 constexpr int kSimtMaxK = 192;             // longest K loop of one float32 tile before K is sliced
 constexpr int kPostThreads = 256;         // normalisation / activation kernels
-constexpr int kPostChunk = 128;           // elements per warp of those kernels
+constexpr int kPostChunk = 2048;          // elements per block of those kernels
+constexpr int kPostTilePixels = 128;       // pixels of a tile of the elementwise kernels
+constexpr int kPostTileChannels = 64;      // most channels of such a tile
 constexpr int kMaxGroupChannels = 64;      // channels per normalisation group
 
 enum GemmMode { kFprop = 0, kDgrad = 1, kWgrad = 2 };
@@ -84,8 +86,10 @@ struct UpdRange {
 };
 struct UpdChunk { int range, start; };
 
-// One warp's share of the normalisation kernels: channels [cl0, cl0+ncl) of group `grp`
+// One block's share of the normalisation kernels: channels [cl0, cl0+ncl) of group `grp`
 // (relative to the group), pixels [p0, p0+np); chunk `idx` of `nidx` in its group.
+// The same record describes a tile of the elementwise kernels: there cl0 is an absolute
+// channel and grp is not used.
 // Either ncl >= 1 whole channels (p0 = 0, np = all pixels) or a piece of one channel.
 struct PostChunk { int stage, grp, cl0, ncl, p0, np, idx, nidx; };
 // One normalisation group of one stage (a warp of the merge kernel).

@@ -272,7 +272,7 @@ void add_tiles(std::vector<GemmTile>& tiles, int gemm, int M, int N, int nsplit,
 }
 
 void fill_conv_tables(pb_handle* h) {
-    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_groups.clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear();
+    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_groups.clear(); h->h_ptiles[0].clear(); h->h_ptiles[1].clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear();
     for (auto& t : h->h_tiles) t.clear();
     for (auto& t : h->h_tctiles) t.clear();
     const int bf = (h->flags & PB_CONV_BF16) ? 1 : 0;
@@ -376,7 +376,23 @@ void fill_conv_tables(pb_handle* h) {
                 }
                 const int nidx = (int)(h->h_pchunks.size() - first);
                 for (int q = 0; q < nidx; ++q) { h->h_pchunks[first + q].idx = q; h->h_pchunks[first + q].nidx = nidx; }
+                if (x.has_pool || x.avgpool)      // the forward of a pooling stage works on the group chunks
+                    for (int q = 0; q < nidx; ++q) {
+                        PostChunk tch = h->h_pchunks[first + q];
+                        tch.cl0 += gq * cpg; tch.grp = -1;
+                        h->h_ptiles[0].push_back(tch);
+                    }
             }
+            // tiles of the elementwise kernels: (a multiple of 8 channels) x (up to kPostTilePixels pixels)
+            const int PT = std::min(hw, kPostTilePixels);
+            int CT = std::min(kPostTileChannels, std::max(8, (kPostChunk / PT) / 8 * 8));
+            CT = std::min(CT, (int)L.c_out);
+            for (int c0 = 0; c0 < L.c_out; c0 += CT)
+                for (int p0 = 0; p0 < hw; p0 += PT) {
+                    const PostChunk tch{(int)h->h_cs.size(), -1, c0, std::min(CT, (int)L.c_out - c0), p0, std::min(PT, hw - p0), 0, 0};
+                    if (!(x.has_pool || x.avgpool)) h->h_ptiles[0].push_back(tch);
+                    h->h_ptiles[1].push_back(tch);
+                }
         }
         h->h_cs.push_back(c);
 
@@ -401,7 +417,7 @@ int validate_conv(pb_handle* h) {
         if (x.gn_groups <= 0) return fail(nullptr, PB_E_UNSUPPORTED, "a CONV2D stage needs a GROUPNORM layer");
         if (x.head.c_out / x.gn_groups > kMaxGroupChannels) return fail(nullptr, PB_E_UNSUPPORTED, "more than 64 channels per normalisation group");
         if (x.has_pool && x.avgpool) return fail(nullptr, PB_E_UNSUPPORTED, "max-pool and average pool in one stage");
-        if (x.avgpool && x.z.h * x.z.w > kPostChunk) return fail(nullptr, PB_E_UNSUPPORTED, "global average pool over more than 128 pixels");
+        if (x.avgpool && x.z.h * x.z.w > kPostChunk) return fail(nullptr, PB_E_UNSUPPORTED, "global average pool over more than 2048 pixels");
         if ((int)(x.consumers_main.size() + x.consumers_skip.size()) > kMaxDeltaSrc) return fail(nullptr, PB_E_UNSUPPORTED, "too many consumers of one stage");
     }
     for (const StageHost& x : h->stages)
@@ -444,6 +460,7 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     h->d_cs = c.take<ConvStage>(h->h_cs.size() + 1);
     h->d_pchunks = c.take<PostChunk>(h->h_pchunks.size() + 1);
     h->d_groups = c.take<GroupRef>(h->h_groups.size() + 1);
+    for (int q = 0; q < 2; ++q) h->d_ptiles[q] = c.take<PostChunk>(h->h_ptiles[q].size() + 1);
     h->d_upd = c.take<UpdRange>(h->h_upd.size() + 1);
     h->d_chunks = c.take<UpdChunk>(h->h_chunks.size() + 1);
     h->d_tc = c.take<ConvGemmTC>(h->h_tc.size() + 1);
@@ -557,7 +574,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
     if (h->profile) for (auto& p : h->prof) p = ProfileClass{};
     const bool fused_last = h->nctaB == 0;      // the last stage rides in the phase-0 launch
     const int npc = (int)h->h_pchunks.size();
-    const int post_grid = std::max(1, std::min(ceil_div(npc, kPostThreads / 32), 4 * h->num_sms));
+    const int post_grid = std::max(1, npc);              // one block per chunk
     const int ngr = (int)h->h_groups.size(), merge_grid = std::max(1, ceil_div(ngr, 8));
     for (int k = 0; k < n_ticks; ++k) {
         const int par = (int)((t_base + k) & 1);
@@ -611,7 +628,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             prof_begin(h, 5);
             conv_stats_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
             conv_group_merge_kernel<<<merge_grid, 256, 0, h->stream>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 0);
-            conv_apply_fwd_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
+            conv_apply_fwd_kernel<<<std::max(1, (int)h->h_ptiles[0].size()), kPostThreads, 0, h->stream>>>(h->d_cs, h->d_ptiles[0], (int)h->h_ptiles[0].size(), h->d_ts, h->S, par);
             prof_end(h);
             // Backward chain: through pool/ReLU/GroupNorm -> data and weight gradients.  It reads
             // what earlier ticks stored (other ring slots than the forward chain writes) and the
@@ -622,7 +639,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             prof_begin(h, 6, bs);
             conv_bwd_dn_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
             conv_group_merge_kernel<<<merge_grid, 256, 0, bs>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 1);
-            conv_bwd_dz_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
+            conv_bwd_dz_kernel<<<std::max(1, (int)h->h_ptiles[1].size()), kPostThreads, 0, bs>>>(h->d_cs, h->d_ptiles[1], (int)h->h_ptiles[1].size(), h->d_ts, h->S, par);
             prof_end(h, bs);
             // data gradients (dgrad) and weight gradients (wgrad) both start from dz and write
             // different buffers: wgrad goes to a stream of its own
@@ -753,6 +770,7 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     up(h->d_cs, h->h_cs.data(), h->h_cs.size() * sizeof(ConvStage));
     up(h->d_pchunks, h->h_pchunks.data(), h->h_pchunks.size() * sizeof(PostChunk));
     up(h->d_groups, h->h_groups.data(), h->h_groups.size() * sizeof(GroupRef));
+    for (int q = 0; q < 2; ++q) up(h->d_ptiles[q], h->h_ptiles[q].data(), h->h_ptiles[q].size() * sizeof(PostChunk));
     up(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange));
     up(h->d_chunks, h->h_chunks.data(), h->h_chunks.size() * sizeof(UpdChunk));
     up(h->d_tc, h->h_tc.data(), h->h_tc.size() * sizeof(ConvGemmTC));

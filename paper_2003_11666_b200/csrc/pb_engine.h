@@ -91,6 +91,7 @@ struct pb_handle {
     std::vector<pb::ConvStage> h_cs; pb::ConvStage* d_cs = nullptr;
     std::vector<pb::PostChunk> h_pchunks; pb::PostChunk* d_pchunks = nullptr;
     std::vector<pb::GroupRef> h_groups; pb::GroupRef* d_groups = nullptr;
+    std::vector<pb::PostChunk> h_ptiles[2]; pb::PostChunk* d_ptiles[2] = {nullptr, nullptr};   // tiles of the elementwise kernels: forward, backward
     std::vector<pb::UpdRange> h_upd; pb::UpdRange* d_upd = nullptr;
     std::vector<pb::UpdChunk> h_chunks; pb::UpdChunk* d_chunks = nullptr;
 
