@@ -14,6 +14,14 @@ stage is updated separately with its own delay (Section "Methods").
 The program is written per sample: everything a stage produces is stored
 under the key (stage, sample id), so a stage can only ever read what an
 earlier tick wrote for that sample.
+
+Fill-and-drain mode (`update_size` = N > 0; Section 1 and Appendix
+"Pipelined Backpropagation": mini-batch SGD on a pipeline).  N samples enter on
+N consecutive ticks, the pipeline then drains for 2(S-1) ticks in which nothing
+enters, and only when it is empty are all stages updated, with the mean of the
+N gradients and plain SGD with momentum; one update takes N + 2S - 2 ticks.
+Every sample then sees the same weights forward and backward, so the result
+is ordinary mini-batch SGD with momentum.
 """
 import numpy as np
 
@@ -181,7 +189,7 @@ class PBOracle:
     def __init__(self, layer_list, stage_of_layer, in_shape, n_classes, lr,
                  momentum, flags=FLAG_SC | FLAG_LWP, dtype=np.float64,
                  sc_delay_scale=1, horizon_scale=1, record=False, conv_operands=None,
-                 margins=False):
+                 margins=False, update_size=0):
         """conv_operands: None, or "bf16" to round both operands of every
         convolution product (forward, data gradient, weight gradient) to
         bfloat16 while accumulating in `dtype`.  margins: log in
@@ -197,6 +205,11 @@ class PBOracle:
         if not self.stages[-1].loss:
             raise ValueError("the last stage must end in SOFTMAX_CE")
         self.in_shape = tuple(in_shape)
+        self.update_size = int(update_size)
+        if self.update_size > 0:
+            flags = 0           # no delay between a sample's forward and backward weights: nothing to compensate
+        self.cycle = self.update_size + 2 * (self.S - 1)     # ticks per update when filling and draining
+        self.gsum = None
         self.lr, self.m, self.flags = lr, momentum, flags
         self.sc_delay_scale, self.horizon_scale = sc_delay_scale, horizon_scale
         self.n_params = sum(st.n_params for st in self.stages)
@@ -234,12 +247,22 @@ class PBOracle:
     def get_velocity(self):
         return np.concatenate([o.v for o in self.opt])
 
+    def live(self, i):
+        """Did a sample enter at tick i?  Always (i >= 0) in PB; when filling
+        and draining only during the first N ticks of a cycle."""
+        if i < 0:
+            return False
+        return self.update_size == 0 or i % self.cycle < self.update_size
+
     def tick(self, x, label):
         """One time step with new sample (x, label).  Returns the loss the
-        last stage computed this tick (sample t-(S-1)), NaN while filling."""
+        last stage computed this tick (sample t-(S-1)), NaN while filling.
+        Samples are named by the tick at which they entered; in fill-and-drain
+        mode the (x, label) of a draining tick is ignored."""
         S, t = self.S, self.t
-        self.out[(-1, t)] = np.asarray(x, dtype=self.dtype).reshape(self.in_shape)
-        self.labels[t] = int(label)
+        if self.live(t):
+            self.out[(-1, t)] = np.asarray(x, dtype=self.dtype).reshape(self.in_shape)
+            self.labels[t] = int(label)
 
         # 1. predicted weights from the state left by the previous tick
         theta_hat = [o.predicted() for o in self.opt]
@@ -247,7 +270,7 @@ class PBOracle:
         # 2. forward of sample t-s at stage s
         for st in self.stages:
             s, i = st.index, t - st.index
-            if i < 0:
+            if not self.live(i):
                 continue
             skip_in = self.out[(st.skip[0], i)] if st.skip is not None else None
             y, stash = st.forward(theta_hat[s], self.out[(st.src, i)], skip_in)
@@ -260,7 +283,7 @@ class PBOracle:
         # 3. loss and its gradient at the last stage (same tick: delay 0)
         loss = float("nan")
         i = t - (S - 1)
-        if i >= 0:
+        if self.live(i):
             self.last_logits = self.out[(S - 1, i)].ravel().copy()
             loss, delta = L.softmax_ce(self.out[(S - 1, i)].ravel(), self.labels.pop(i))
             self.dsum[(S - 1, i)] = delta.reshape(-1, 1, 1)
@@ -269,7 +292,7 @@ class PBOracle:
         grads = {}
         for st in self.stages:
             s, j = st.index, t - 2 * (S - 1) + st.index
-            if j < 0:
+            if not self.live(j):
                 continue
             dy = self.dsum.pop((s, j))
             skip_shape = self.stages[st.skip[0]].out_shape if st.skip is not None else None
@@ -288,6 +311,19 @@ class PBOracle:
                 self.grads[(s, j)] = g.copy()
 
         # 5. update every stage that received a gradient
+        if self.update_size > 0:
+            # fill and drain: gradients wait until the pipeline is empty, then every
+            # stage takes one SGDM step with their mean
+            if self.gsum is None:
+                self.gsum = [np.zeros_like(o.w) for o in self.opt]
+            for s, g in grads.items():
+                self.gsum[s] = self.gsum[s] + g
+            if t % self.cycle == self.cycle - 1:
+                for s in range(S):
+                    self.opt[s].update(self.gsum[s] / self.dtype(self.update_size))
+                self.gsum = None
+            self.t += 1
+            return loss
         for s, g in grads.items():
             self.opt[s].update(g)
             if self.record:

@@ -226,6 +226,10 @@ def workload(name):
         return _resnet20()
     if name == "resnet50":
         return _resnet50()
+    if name == "resnet50_112":
+        # the same 54 stages on 112x112 images: a quarter of the activation
+        # memory, for profiler captures that replay kernels many times
+        return _resnet50(hw=112, name="resnet50_112")
     raise KeyError(name)
 
 

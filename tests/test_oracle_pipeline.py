@@ -202,3 +202,64 @@ def test_compensation_scales_set_the_stage_constants():
         assert opt.b == pytest.approx((1 - 0.9 ** (2 * D)) / 0.1, rel=1e-12, abs=1e-15)
         assert opt.T == pytest.approx(0.5 * D)
         assert opt.a / 0.1 + opt.b == pytest.approx(10.0, rel=1e-12)     # total contribution unchanged
+
+
+@pytest.mark.parametrize("make,N", [(lambda: mlp([10, 8, 6, 4], lr=0.05), 3), (tiny_cnn, 4),
+                                    (tiny_resnet, 2), (lambda: tiny_resnet(bottleneck=True), 5),
+                                    (lambda: mlp([9, 5], lr=0.05), 1)])
+def test_fill_and_drain_is_minibatch_sgdm(make, N):
+    # Filling and draining the pipeline for every update is ordinary mini-batch SGD with
+    # momentum (Section 1; Appendix "Pipelined Backpropagation"): torch's SGD on the mean
+    # loss of the N samples of a cycle must give the same weights, velocities and losses,
+    # and one update must take N + 2S - 2 ticks.
+    wl = make()
+    S = wl.n_stages
+    cycle = N + 2 * S - 2
+    o = PBOracle(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, wl.lr, wl.momentum,
+                 wl.flags, update_size=N)
+    w0 = he_normal_weights(wl.seed, wl).astype(np.float64)
+    o.set_weights(w0)
+    stages = torch_ref.build(wl)
+    params = [torch.nn.Parameter(p) for p in _thetas(stages, w0)]
+    ref = torch.optim.SGD(params, lr=wl.lr, momentum=wl.momentum)
+    n_cycles = 3
+    x, y = make_inputs(wl.seed, n_cycles * cycle, wl.sample_elems, wl.n_classes)
+    for c in range(n_cycles):
+        base = c * cycle
+        w_before = o.get_weights().copy()
+        got = [o.tick(x[base + p], y[base + p]) for p in range(cycle)]
+        # nothing moved before the pipeline was empty is checked by the cycle's losses:
+        # every sample of the cycle saw the weights of the cycle's start
+        ref.zero_grad()
+        losses = [torch_ref.network_loss(stages, params, torch.tensor(x[base + p], dtype=torch.float64).view(wl.in_shape),
+                                         y[base + p]) for p in range(N)]
+        (sum(losses) / N).backward()
+        for p in range(cycle):
+            q = p - (S - 1)              # the sample whose loss appears at tick base + p
+            if 0 <= q < N:
+                assert got[p] == pytest.approx(losses[q].item(), rel=1e-10, abs=1e-12)
+            else:
+                assert np.isnan(got[p])
+        ref.step()
+        want = np.concatenate([p.detach().numpy().ravel() for p in params])
+        np.testing.assert_allclose(o.get_weights(), want, rtol=1e-9, atol=1e-12)
+        vel = np.concatenate([ref.state[p]["momentum_buffer"].numpy().ravel() for p in params])
+        np.testing.assert_allclose(o.get_velocity(), vel, rtol=1e-9, atol=1e-12)
+        assert not np.array_equal(o.get_weights(), w_before)
+
+
+def test_fill_and_drain_holds_the_weights_until_the_pipeline_is_empty():
+    wl = mlp([10, 8, 6, 4], lr=0.05)
+    N, S = 3, wl.n_stages
+    cycle = N + 2 * S - 2
+    o = PBOracle(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, wl.lr, wl.momentum,
+                 wl.flags, update_size=N)
+    w0 = he_normal_weights(wl.seed, wl).astype(np.float64)
+    o.set_weights(w0)
+    x, y = make_inputs(wl.seed, cycle, wl.sample_elems, wl.n_classes)
+    for p in range(cycle - 1):
+        o.tick(x[p], y[p])
+        np.testing.assert_array_equal(o.get_weights(), w0)
+    o.tick(x[cycle - 1], y[cycle - 1])
+    assert not np.array_equal(o.get_weights(), w0)
+    assert all(op.version == 1 for op in o.opt)
