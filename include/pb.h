@@ -105,6 +105,23 @@ int pb_set_weights(pb_handle* h, const float* host_w, size_t n);
  * the stream.  Scales must be >= 0. */
 int pb_set_mitigation(pb_handle* h, float sc_delay_scale, float horizon_scale);
 
+/* Fill-and-drain training (Section 1; Appendix "Pipelined Backpropagation":
+ * mini-batch SGD on a pipeline).  With n_samples = N > 0 the engine stops
+ * being asynchronous: time is cut into cycles of N + 2 (S - 1) ticks; a
+ * sample enters at each of the first N ticks of a cycle, nothing enters while
+ * the pipeline drains (the dev_x / dev_xs entry and label of such a tick must
+ * still be valid memory, but their values are not used, and the tick's loss is
+ * NaN when no sample reaches the last stage), and each stage takes ONE plain
+ * SGD-with-momentum step per cycle with the mean of the N gradients,
+ * v <- m v + mean g, w <- w - lr v, once its last backward of the cycle is
+ * done.  Forward and backward of every sample then use the same weights, so
+ * SC and LWP have nothing to compensate and are off in this mode whatever the
+ * flags say; weights and velocities are those of ordinary mini-batch SGD at
+ * every cycle boundary.  N = 0 returns to pipelined backpropagation.  Call it
+ * while the tick count is zero (after pb_create or pb_set_weights), else
+ * PB_E_ARG.  Synchronises the stream. */
+int pb_set_update_size(pb_handle* h, int n_samples);
+
 /* One tick.  dev_x: the new sample (in_c*in_h*in_w floats, device memory; it
  * is copied into the engine's input ring, so it may be reused after the call
  * returns in stream order).  label in [0, n_classes).  If host_loss is not

@@ -20,6 +20,7 @@ EXPORTS = [
     "pb_get_velocity", "pb_sync", "pb_num_params", "pb_num_stages", "pb_stage_delay",
     "pb_tick_count", "pb_last_launch_count", "pb_device_bytes", "pb_profile_enable",
     "pb_profile_ms", "pb_last_error", "pb_destroy", "pb_mlp_run_static", "pb_set_mitigation",
+    "pb_set_update_size",
 ]
 
 
@@ -51,6 +52,7 @@ def load_library():
                               f32, f32, C.c_uint, vp, C.POINTER(vp)]
     lib.pb_set_weights.argtypes = [vp, vp, C.c_size_t]
     lib.pb_set_mitigation.argtypes = [vp, f32, f32]
+    lib.pb_set_update_size.argtypes = [vp, i32]
     lib.pb_tick.argtypes = [vp, vp, i32, C.POINTER(f32)]
     lib.pb_run.argtypes = [vp, vp, vp, i32, vp]
     lib.pb_run_host.argtypes = [vp, vp, vp, i32, vp]
@@ -132,6 +134,9 @@ class PB:
 
     def set_mitigation(self, sc_delay_scale, horizon_scale):
         self._check(self._lib.pb_set_mitigation(self._h, float(sc_delay_scale), float(horizon_scale)))
+
+    def set_update_size(self, n_samples):
+        self._check(self._lib.pb_set_update_size(self._h, int(n_samples)))
 
     def tick(self, dev_x, label, want_loss=True):
         loss = C.c_float(float("nan"))

@@ -207,7 +207,7 @@ conv_gemm_kernel(const ConvGemm* __restrict__ gemms, const GemmTile* __restrict_
     __syncthreads();
     const long long t = ts->cnt[par];
     const long long smp = (G.mode == kFprop) ? t - G.s : t - 2LL * (S - 1) + G.s;
-    if (smp < 0) return;
+    if (!sample_live(ts, smp)) return;
     if (G.tm == 4) {
         if (G.tn == 4) gemm_dispatch_k<4, 4>(G, tl, smp, smem);
         else gemm_dispatch_k<4, 1>(G, tl, smp, smem);

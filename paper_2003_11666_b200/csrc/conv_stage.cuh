@@ -69,10 +69,10 @@ struct ChunkGeom {
 
 // ---------------------------------------------------------------- forward, step 1
 template <int VEC>
-__device__ void conv_stats_chunk(const ConvStage& st, const PostChunk& ch, long long t, float* red) {
+__device__ void conv_stats_chunk(const ConvStage& st, const PostChunk& ch, long long t, const TickState* ts, float* red) {
     constexpr int U = kPostPer / VEC;
     const long long i = t - st.s;
-    if (i < 0) return;
+    if (!sample_live(ts, i)) return;
     const int tid = threadIdx.x;
     const int slot = slot_of(i, st.slots);
     const ChunkGeom cg(st, ch, VEC);
@@ -144,10 +144,10 @@ __device__ __forceinline__ void store_nhwc_tile(const __nv_bfloat16* t16, int rs
 }
 
 template <int VEC>
-__device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, long long t, __nv_bfloat16* t16) {
+__device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, long long t, const TickState* ts, __nv_bfloat16* t16) {
     constexpr int U = kPostPer / VEC;
     const long long i = t - st.s;
-    if (i < 0) return;
+    if (!sample_live(ts, i)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int slot = slot_of(i, st.slots);
     const int hw = st.oh * st.ow, npu = ch.np / VEC, nunits = ch.ncl * npu, rs = ch.np + 2;
@@ -279,10 +279,10 @@ __device__ __forceinline__ float gather_out_delta(const ConvStage& st, size_t oe
 }
 
 template <int VEC>
-__device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long long t, int S, float* red, float* usum) {
+__device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long long t, const TickState* ts, int S, float* red, float* usum) {
     constexpr int U = kPostPer / VEC;
     const long long j = t - 2LL * (S - 1) + st.s;
-    if (j < 0) return;
+    if (!sample_live(ts, j)) return;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int slot = slot_of(j, st.slots);
     const ChunkGeom cg(st, ch, VEC);
@@ -428,10 +428,10 @@ __device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long
 // ---------------------------------------------------------------- backward, step 2
 // Elementwise over a tile (see the forward step 2).
 template <int VEC>
-__device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long long t, int S, __nv_bfloat16* t16) {
+__device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long long t, const TickState* ts, int S, __nv_bfloat16* t16) {
     constexpr int U = kPostPer / VEC;
     const long long j = t - 2LL * (S - 1) + st.s;
-    if (j < 0) return;
+    if (!sample_live(ts, j)) return;
     const int tid = threadIdx.x;
     const int slot = slot_of(j, st.slots);
     const int hw = st.oh * st.ow, npu = ch.np / VEC, nunits = ch.ncl * npu, rs = ch.np + 2;
@@ -519,8 +519,8 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
         const PostChunk ch = chunks[blockIdx.x];                                                   \
         const long long t = ts->cnt[par];                                                          \
         const ConvStage& st = stages[ch.stage];                                                    \
-        if (st.vec4) CHUNK<4>(st, ch, t, __VA_ARGS__);                                             \
-        else CHUNK<1>(st, ch, t, __VA_ARGS__);                                                     \
+        if (st.vec4) CHUNK<4>(st, ch, t, ts, __VA_ARGS__);                                         \
+        else CHUNK<1>(st, ch, t, ts, __VA_ARGS__);                                                 \
     }
 PB_POST_KERNEL(conv_stats_kernel, conv_stats_chunk, red)
 PB_POST_KERNEL(conv_apply_fwd_kernel, conv_apply_fwd_chunk, t16)
@@ -544,7 +544,7 @@ conv_group_merge_kernel(const ConvStage* __restrict__ stages, const GroupRef* __
     const int hw = st.oh * st.ow, cpg = st.cpg, c0 = gr.grp * cpg;
     if (mode == 0) {
         const long long i = t - st.s;
-        if (i < 0) return;
+        if (!sample_live(ts, i)) return;
         const int slot = slot_of(i, st.slots), nidx = st.fstat_stride;
         const float* __restrict__ f = st.fstat + (size_t)gr.grp * st.fstat_stride * 3;
         float tot = 0.f, wsum = 0.f;
@@ -561,7 +561,7 @@ conv_group_merge_kernel(const ConvStage* __restrict__ stages, const GroupRef* __
         return;
     }
     const long long j = t - 2LL * (S - 1) + st.s;
-    if (j < 0) return;
+    if (!sample_live(ts, j)) return;
     const float* __restrict__ gam = st.w + st.nw;
     const int np = st.npieces;
     float m1 = 0.f, m2 = 0.f;
@@ -607,7 +607,9 @@ update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ 
     const UpdChunk ch = chunks[blockIdx.x];
     const UpdRange& R = ranges[ch.range];
     const long long j = ts->cnt[par] - 2LL * (S - 1) + R.s;
-    if (j < 0) return;
+    if (!sample_live(ts, j)) return;
+    float m_eff, nla, gsc;
+    step_coefficients(ts, j, R.m, R.neg_lr_a, m_eff, nla, gsc);
     const int end = min(R.n, ch.start + kUpdChunk);
     const bool vec = ((reinterpret_cast<uintptr_t>(R.w) | reinterpret_cast<uintptr_t>(R.v) | reinterpret_cast<uintptr_t>(R.wh) |
                        reinterpret_cast<uintptr_t>(R.g)) & 15) == 0 && (R.part_stride & 3) == 0 && (R.n & 3) == 0 &&
@@ -620,11 +622,12 @@ update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ 
                 const float4 p = *reinterpret_cast<const float4*>(R.g + (size_t)q * R.part_stride + e);
                 g.x += p.x; g.y += p.y; g.z += p.z; g.w += p.w;
             }
+            g.x *= gsc; g.y *= gsc; g.z *= gsc; g.w *= gsc;
             const float4 w = *reinterpret_cast<const float4*>(R.w + e), v = *reinterpret_cast<const float4*>(R.v + e);
             float4 vn, wn, wh;
-            vn.x = fmaf(R.m, v.x, g.x); vn.y = fmaf(R.m, v.y, g.y); vn.z = fmaf(R.m, v.z, g.z); vn.w = fmaf(R.m, v.w, g.w);
-            wn.x = fmaf(R.neg_lr_a, vn.x, fmaf(R.neg_lr_b, g.x, w.x)); wn.y = fmaf(R.neg_lr_a, vn.y, fmaf(R.neg_lr_b, g.y, w.y));
-            wn.z = fmaf(R.neg_lr_a, vn.z, fmaf(R.neg_lr_b, g.z, w.z)); wn.w = fmaf(R.neg_lr_a, vn.w, fmaf(R.neg_lr_b, g.w, w.w));
+            vn.x = fmaf(m_eff, v.x, g.x); vn.y = fmaf(m_eff, v.y, g.y); vn.z = fmaf(m_eff, v.z, g.z); vn.w = fmaf(m_eff, v.w, g.w);
+            wn.x = fmaf(nla, vn.x, fmaf(R.neg_lr_b, g.x, w.x)); wn.y = fmaf(nla, vn.y, fmaf(R.neg_lr_b, g.y, w.y));
+            wn.z = fmaf(nla, vn.z, fmaf(R.neg_lr_b, g.z, w.z)); wn.w = fmaf(nla, vn.w, fmaf(R.neg_lr_b, g.w, w.w));
             if (R.wform) {
                 wh.x = fmaf(R.T_w, wn.x - w.x, wn.x); wh.y = fmaf(R.T_w, wn.y - w.y, wn.y);
                 wh.z = fmaf(R.T_w, wn.z - w.z, wn.z); wh.w = fmaf(R.T_w, wn.w - w.w, wn.w);
@@ -652,9 +655,10 @@ update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ 
     for (int e = ch.start + threadIdx.x; e < end; e += 256) {
         float g = 0.f;
         for (int q = 0; q < R.nparts; ++q) g += R.g[(size_t)q * R.part_stride + e];
+        g *= gsc;
         const float w = R.w[e], v = R.v[e];
-        const float vn = fmaf(R.m, v, g);
-        const float wn = fmaf(R.neg_lr_a, vn, fmaf(R.neg_lr_b, g, w));
+        const float vn = fmaf(m_eff, v, g);
+        const float wn = fmaf(nla, vn, fmaf(R.neg_lr_b, g, w));
         const float wh = R.wform ? fmaf(R.T_w, wn - w, wn) : fmaf(R.neg_lr_T, vn, wn);
         R.v[e] = vn;
         R.w[e] = wn;

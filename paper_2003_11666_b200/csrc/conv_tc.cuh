@@ -104,7 +104,7 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
     __syncthreads();
     const long long t = ts->cnt[par];
     const long long smp = (G.mode == kFprop) ? t - G.s : t - 2LL * (S - 1) + G.s;
-    if (smp < 0) return;                                   // uniform: before any allocation
+    if (!sample_live(ts, smp)) return;                                   // uniform: before any allocation
     unsigned char* smem = (unsigned char*)(((uintptr_t)tc_smem_raw + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int M = G.M, N = G.N, BN = G.bn;

@@ -116,9 +116,10 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long i = t - st.s;                        // forward sample
     const long long j = t - 2LL * (S - 1) + st.s;        // backward sample
-    const bool do_fwd = phase == 0 && i >= 0;
-    const bool do_bwd = j >= 0 && (st.is_last ? phase == 1 : phase == 0);
-    if (phase == 1 && seg.row0 == 0 && tid == 0 && j < 0 && loss_out) *loss_out = __int_as_float(0x7fc00000);
+    const bool live_j = sample_live(ts, j);
+    const bool do_fwd = phase == 0 && sample_live(ts, i);
+    const bool do_bwd = live_j && (st.is_last ? phase == 1 : phase == 0);
+    if (phase == 1 && seg.row0 == 0 && tid == 0 && !live_j && loss_out) *loss_out = __int_as_float(0x7fc00000);
     if (!do_fwd && !do_bwd) return;
     const int rows = seg.row1 - seg.row0;
     if (rows > kFcMaxSegRows || rows <= 0) {
@@ -193,7 +194,9 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
     while (ncg * 2 <= nchunks && ncg * 2 <= kFcWarps) ncg *= 2;
     const int nrs = kFcWarps / ncg;
     const int cg = warp % ncg, rs = warp / ncg;
-    const float nlT = st.neg_lr_T, m = st.m, nla = st.neg_lr_a, nlb = st.neg_lr_b, Tw = st.T_w;
+    const float nlT = st.neg_lr_T, nlb = st.neg_lr_b, Tw = st.T_w;
+    float m, nla, gsc;
+    step_coefficients(ts, j, st.m, st.neg_lr_a, m, nla, gsc);
     const bool want_dx = do_bwd && st.need_dx;
 
     for (int c0 = 0; c0 < nchunks; c0 += ncg * kFcChunksPerSweep) {
@@ -208,7 +211,11 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
             for (int e = 0; e < VEC; ++e) { xfr[c][e] = 0.f; xbr[c][e] = 0.f; cacc[c][e] = 0.f; }
             if (cok[c]) {
                 if (do_fwd) vload<VEC>(xfr[c], xf + col[c]);
-                if (do_bwd) vload<VEC>(xbr[c], xb + col[c]);
+                if (do_bwd) {
+                    vload<VEC>(xbr[c], xb + col[c]);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) xbr[c][e] *= gsc;
+                }
             }
         }
         // Rows of this row split, two at a time, software-pipelined: the loads of the
@@ -252,7 +259,7 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
                         const float what = WF ? hv[u][c][e] : fmaf(nlT, v, w);   // w_hat = w - lr T v (or the stored prediction)
                         facc[u] = fmaf(what, xfr[c][e], facc[u]);     // forward  (W_hat x)
                         cacc[c][e] = fmaf(w, d, cacc[c][e]);          // backward (W^T delta)
-                        const float g = d * xbr[c][e];                // rank-1 gradient
+                        const float g = d * xbr[c][e];                // rank-1 gradient (xbr carries the 1/N of a mini-batch mean)
                         vn[e] = fmaf(m, v, g);                        // v <- m v + g
                         wn[e] = fmaf(nla, vn[e], fmaf(nlb, g, w));    // w <- w - lr (a v + b g)
                         hn[e] = fmaf(Tw, wn[e] - w, wn[e]);           // w_hat = w_new + T (w_new - w_old)
@@ -340,7 +347,7 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
             st.out[(size_t)ring_slot(i, st.out_slots) * out + row] = y;
         }
         if (do_bwd) {
-            const float g = sh.delta[r];
+            const float g = sh.delta[r] * gsc;
             const float vn = fmaf(m, vb, g);
             const float bn = fmaf(nla, vn, fmaf(nlb, g, b));
             vbias[row] = vn;

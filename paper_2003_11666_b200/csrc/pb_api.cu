@@ -120,6 +120,20 @@ void mitigation_constants(const pb_handle* h, StageHost& x) {
     }
     x.a = (float)a; x.b = (float)b;
     x.T = (h->flags & PB_LWP) ? h->horizon_scale * (float)x.delay : 0.f;
+    if (h->update_size > 0) {
+        // fill and drain: forward and backward of a sample see the same weights; plain SGDM
+        x.a = 1.f; x.b = 0.f; x.T = 0.f;
+    }
+}
+
+// Resets the device-side tick state (tick 0, no error) and files the training mode.
+int reset_tick_state(pb_handle* h) {
+    TickState ts{};
+    ts.fd_n = h->update_size;
+    ts.fd_cycle = h->update_size > 0 ? h->update_size + 2 * (h->S - 1) : 0;
+    cudaError_t e = cudaMemcpyAsync(h->d_ts, &ts, sizeof(ts), cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);      // ts is a stack variable
+    return e == cudaSuccess ? PB_OK : PB_E_CUDA;
 }
 
 // Per-stage constants: delay (Eq. F_i), SC_D coefficients, LWP horizon.
@@ -800,7 +814,7 @@ int pb_set_weights(pb_handle* h, const float* host_w, size_t n) {
     if (!h) return PB_E_ARG;
     if (!host_w || n != h->n_params) return fail(h, PB_E_ARG, "pb_set_weights: need pb_num_params() floats");
     PB_CUDA(h, cudaMemsetAsync(h->arena + h->zero_from, 0, h->arena_bytes - h->zero_from, h->stream));
-    PB_CUDA(h, cudaMemsetAsync(h->d_ts, 0, sizeof(TickState), h->stream));
+    if (reset_tick_state(h) != PB_OK) return fail(h, PB_E_CUDA, "pb_set_weights: could not reset the tick state");
     std::vector<float> tmp;
     for (const StageHost& x : h->stages) {
         const float* src = host_w + x.user_off;
@@ -840,6 +854,23 @@ int pb_set_mitigation(pb_handle* h, float sc_delay_scale, float horizon_scale) {
     if (!h->h_upd.empty())
         PB_CUDA(h, cudaMemcpyAsync(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange), cudaMemcpyHostToDevice, h->stream));
     PB_CUDA(h, cudaStreamSynchronize(h->stream));
+    return PB_OK;
+}
+
+int pb_set_update_size(pb_handle* h, int n_samples) {
+    if (!h) return PB_E_ARG;
+    if (n_samples < 0) return fail(h, PB_E_ARG, "pb_set_update_size: negative update size");
+    if (h->tick != 0) return fail(h, PB_E_ARG, "pb_set_update_size: call it before the first tick (after pb_set_weights)");
+    h->update_size = n_samples;
+    for (StageHost& x : h->stages) mitigation_constants(h, x);
+    fill_fc_tables(h);
+    fill_conv_tables(h);
+    PB_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (!h->h_fc.empty())
+        PB_CUDA(h, cudaMemcpyAsync(h->d_fc, h->h_fc.data(), h->h_fc.size() * sizeof(FcStage), cudaMemcpyHostToDevice, h->stream));
+    if (!h->h_upd.empty())
+        PB_CUDA(h, cudaMemcpyAsync(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange), cudaMemcpyHostToDevice, h->stream));
+    if (reset_tick_state(h) != PB_OK) return fail(h, PB_E_CUDA, "pb_set_update_size: could not write the tick state");
     return PB_OK;
 }
 

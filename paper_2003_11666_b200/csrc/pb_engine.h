@@ -59,6 +59,7 @@ struct pb_handle {
     unsigned flags = 0;
     float lr = 0, momentum = 0;
     float sc_delay_scale = 1.f, horizon_scale = 1.f;     // SC with alpha*D, LWP horizon alpha*D
+    int update_size = 0;                        // > 0: fill-and-drain mini-batch SGD with that many samples per update
     int S = 0, n_classes = 0;
     pb::Shape in_shape;
     size_t n_params = 0, dev_params = 0;

@@ -64,10 +64,41 @@ struct TickState {
     long long cnt[2];
     int error;             // first failed index check (0 = none)
     int error_info;
+    int fd_n;              // fill-and-drain mode: samples per update (0 = pipelined backpropagation)
+    int fd_cycle;          // ... and ticks per update, fd_n + 2 (S - 1)
 };
 
 enum ErrorCode { kErrNone = 0, kErrSegRows = 1, kErrLabel = 2, kErrSlot = 3, kErrWait = 4 };
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+#ifdef __CUDACC__
+// Samples are named by the tick at which they entered.  In pipelined backpropagation
+// one enters at every tick; when the pipeline is filled and drained for every update
+// (mini-batch SGD, Section 1), only at the first fd_n ticks of a cycle.
+__device__ __forceinline__ bool sample_live(const TickState* ts, long long i) {
+    if (i < 0) return false;
+    const int n = ts->fd_n;
+    return n == 0 || (int)(i % ts->fd_cycle) < n;
+}
+
+// Coefficients of the update that backward sample j triggers:
+//   v <- m_eff v + gscale g ;  w <- w + nla_eff v + neg_lr_b (gscale g).
+// Pipelined backpropagation: the stage's own constants.  Fill and drain: the velocity
+// collects the mean gradient of the cycle (decayed once, at the cycle's first sample)
+// and the weights move once, at its last sample, so that every sample of the cycle
+// sees the same weights; the stage tables then hold a = 1, b = 0, T = 0.
+__device__ __forceinline__ void step_coefficients(const TickState* ts, long long j, float m, float neg_lr_a,
+                                                  float& m_eff, float& nla_eff, float& gscale) {
+    const int n = ts->fd_n;
+    m_eff = m; nla_eff = neg_lr_a; gscale = 1.f;
+    if (n > 0 && j >= 0) {
+        const int pos = (int)(j % ts->fd_cycle);
+        m_eff = pos == 0 ? m : 1.f;
+        nla_eff = pos == n - 1 ? neg_lr_a : 0.f;
+        gscale = 1.f / (float)n;
+    }
+}
+#endif
 
 }  // namespace pb
