@@ -601,7 +601,7 @@ conv_group_merge_kernel(const ConvStage* __restrict__ stages, const GroupRef* __
 // Fused SC + LWP step for materialised gradients (convolution stages):
 // reads w, v and the gradient slices once, writes w, v and the predicted
 // weights the next forward will use.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 6)
 update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ chunks,
               const TickState* __restrict__ ts, int S, int par) {
     const UpdChunk ch = chunks[blockIdx.x];

@@ -89,6 +89,12 @@ __device__ __forceinline__ void cp_async16(unsigned char* dst, const __nv_bfloat
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(sz) : "memory");
 }
 
+// Quotient a / b for 0 <= a < 2^21 and b <= 2^13 from the float reciprocal of b: the
+// product (a + 0.5) / b is at least 0.5 / b away from every integer, far more than its
+// rounding error (about 2e-7 a / b), so rounding down gives the exact quotient.  A
+// negative a gives a negative result (only ever used to reject the element).
+__device__ __forceinline__ int quot(int a, float inv_b) { return __float2int_rd(((float)a + 0.5f) * inv_b); }
+
 __global__ void __launch_bounds__(kTcThreads)
 conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, TickState* ts, int S, int par) {
     extern __shared__ unsigned char tc_smem_raw[];
@@ -114,6 +120,9 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
     const __nv_bfloat16* __restrict__ B = G.b + (size_t)(smp % G.b_slots) * G.b_elems;
     float* __restrict__ Cp = G.c + ((size_t)(smp % G.c_slots) * G.nsplit + tl.split) * ((size_t)M * N);
     const int CI = G.ci, CO = G.co, ksz = G.k, st = G.stride, pad = G.pad, ih = G.ih, iw = G.iw, oh = G.oh, ow = G.ow;
+    // the gathers divide by these for every 16-byte unit: reciprocals once per block
+    const float inv_ci = 1.f / (float)CI, inv_co = 1.f / (float)CO, inv_ksz = 1.f / (float)ksz,
+                inv_st = 1.f / (float)st, inv_ow = 1.f / (float)ow;
 
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(128) : "memory");
@@ -139,22 +148,24 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
     bool bok[kTcPasses];
     if (G.mode != kWgrad) {
         const int wdt = (G.mode == kFprop) ? ow : iw;
+        const float inv_wdt = 1.f / (float)wdt;
 #pragma unroll
         for (int i = 0; i < kTcPasses; ++i) {
             const int n = tl.n0 + krow0 + kTcRowsPerPass * i;
             bok[i] = (krow0 + kTcRowsPerPass * i) < BN && n < N;
-            bp[i] = n / wdt; bq[i] = n - bp[i] * wdt;
+            bp[i] = quot(n, inv_wdt); bq[i] = n - bp[i] * wdt;
         }
     }
     // wgrad B: this thread's 8 consecutive n = (r, s, ci..ci+7)
     const int b_units_per_k = BN >> 3;                      // 16 or 8
-    const int bmu = tid % b_units_per_k, bk0 = tid / b_units_per_k, bkstep = kTcThreads / b_units_per_k;
+    const int bshift = BN == 128 ? 4 : 3;                   // log2 of b_units_per_k
+    const int bmu = tid & (b_units_per_k - 1), bk0 = tid >> bshift, bkstep = kTcThreads >> bshift;
     int wr = 0, wsx = 0, wci = 0;
     bool wok = false;
     if (G.mode == kWgrad) {
         const int n = tl.n0 + bmu * 8;
         wok = n < N;
-        const int rs = n / CI; wci = n - rs * CI; wr = rs / ksz; wsx = rs - wr * ksz;
+        const int rs = quot(n, inv_ci); wci = n - rs * CI; wr = quot(rs, inv_ksz); wsx = rs - wr * ksz;
     }
     const int amu = tid & 15, ak0 = tid >> 4;               // MN-major A (width 128)
     const bool a_m_ok = (tl.m0 + amu * 8) < M;
@@ -178,7 +189,7 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
             for (int i = 0; i < kTcKPasses; ++i) {
                 const int kl = ak0 + kTcKPerPass * i, k = k0 + kl;          // k = rs * CO + co
                 const bool ok = a_m_ok && k < ke;
-                const int rs = k / CO, co = k - rs * CO;
+                const int rs = quot(k, inv_co), co = k - rs * CO;
                 cp_async16(sA + mnmajor_off(kl, amu), ok ? A + ((size_t)co * (ksz * ksz) + rs) * CI + tl.m0 + amu * 8 : A, ok);
             }
         } else {
@@ -192,7 +203,7 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
         // ---------------- B tile
         if (G.mode == kFprop) {
             const int k = k0 + ku * 8;
-            const int rs = k / CI, ci = k - rs * CI, r = rs / ksz, s = rs - r * ksz;
+            const int rs = quot(k, inv_ci), ci = k - rs * CI, r = quot(rs, inv_ksz), s = rs - r * ksz;
 #pragma unroll
             for (int i = 0; i < kTcPasses; ++i) {
                 const int row = krow0 + kTcRowsPerPass * i;
@@ -203,20 +214,20 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict_
             }
         } else if (G.mode == kDgrad) {
             const int k = k0 + ku * 8;
-            const int rs = k / CO, co = k - rs * CO, r = rs / ksz, s = rs - r * ksz;
+            const int rs = quot(k, inv_co), co = k - rs * CO, r = quot(rs, inv_ksz), s = rs - r * ksz;
 #pragma unroll
             for (int i = 0; i < kTcPasses; ++i) {
                 const int row = krow0 + kTcRowsPerPass * i;
                 if (row >= BN) break;
                 const int ty = bp[i] + pad - r, tx = bq[i] + pad - s;
-                const int p = ty / st, q = tx / st;
+                const int p = quot(ty, inv_st), q = quot(tx, inv_st);
                 const bool ok = bok[i] && k < ke && ty >= 0 && tx >= 0 && p * st == ty && q * st == tx && p < oh && q < ow;
                 cp_async16(sB + kmajor_off(row, ku), ok ? B + ((size_t)p * ow + q) * CO + co : B, ok);
             }
         } else {
             for (int kl = bk0; kl < kTcChunk; kl += bkstep) {
                 const int k = k0 + kl;
-                const int p = k / ow, q = k - p * ow;
+                const int p = quot(k, inv_ow), q = k - p * ow;
                 const int y = p * st + wr - pad, x = q * st + wsx - pad;
                 const bool ok = wok && k < ke && y >= 0 && y < ih && x >= 0 && x < iw;
                 cp_async16(sB + mnmajor_off(kl, bmu), ok ? B + ((size_t)y * iw + x) * CI + wci : B, ok);

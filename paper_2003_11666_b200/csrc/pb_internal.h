@@ -79,7 +79,7 @@ __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; 
 __device__ __forceinline__ bool sample_live(const TickState* ts, long long i) {
     if (i < 0) return false;
     const int n = ts->fd_n;
-    return n == 0 || (int)(i % ts->fd_cycle) < n;
+    return n == 0 || (int)((unsigned)i % (unsigned)ts->fd_cycle) < n;      // ticks stay far below 2^32
 }
 
 // Coefficients of the update that backward sample j triggers:
@@ -93,7 +93,7 @@ __device__ __forceinline__ void step_coefficients(const TickState* ts, long long
     const int n = ts->fd_n;
     m_eff = m; nla_eff = neg_lr_a; gscale = 1.f;
     if (n > 0 && j >= 0) {
-        const int pos = (int)(j % ts->fd_cycle);
+        const int pos = (int)((unsigned)j % (unsigned)ts->fd_cycle);
         m_eff = pos == 0 ? m : 1.f;
         nla_eff = pos == n - 1 ? neg_lr_a : 0.f;
         gscale = 1.f / (float)n;
