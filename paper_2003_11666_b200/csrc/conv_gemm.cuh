@@ -41,6 +41,7 @@ __device__ void gemm_tile(const ConvGemm& G, const GemmTile& tl, long long smp, 
     float* __restrict__ Cp = G.c + ((size_t)(smp % G.c_slots) * G.nsplit + tl.split) * ((size_t)M * N);
     const int ksz = G.k, st = G.stride, pad = G.pad, ih = G.ih, iw = G.iw, oh = G.oh, ow = G.ow;
     const bool bf = G.bf16 != 0;
+    const float inv_st = 1.f / (float)st, inv_ow = 1.f / (float)ow;     // see quot()
 
     float acc[TM][TN];
 #pragma unroll
@@ -110,7 +111,7 @@ __device__ void gemm_tile(const ConvGemm& G, const GemmTile& tl, long long smp, 
                 const int ty_ = n_p + pad - r, tx_ = n_q + pad - s;
                 float v = 0.f;
                 if (n_ok && kq < ke && ty_ >= 0 && tx_ >= 0) {
-                    const int p = ty_ / st, qq = tx_ / st;
+                    const int p = quot(ty_, inv_st), qq = quot(tx_, inv_st);
                     if (p * st == ty_ && qq * st == tx_ && p < oh && qq < ow) v = B[((size_t)c * oh + p) * ow + qq];
                 }
                 rb[q] = v;
@@ -118,7 +119,7 @@ __device__ void gemm_tile(const ConvGemm& G, const GemmTile& tl, long long smp, 
         } else {
             // A[m = co, kk = pixel] = dz[m*K + kk];  B[kk = (p, q), n = (ci, r, s)] = x[ci, p*st+r-pad, q*st+s-pad]
             const int kk = k0 + lo16;
-            const int p = kk / ow, qq = kk - p * ow;
+            const int p = quot(kk, inv_ow), qq = kk - p * ow;
 #pragma unroll
             for (int q = 0; q < TM; ++q) {
                 const int m = tl.m0 + hi16 + 16 * q;

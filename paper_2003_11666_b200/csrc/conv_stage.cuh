@@ -7,13 +7,19 @@
 // and ONE BLOCK owns a chunk: every thread holds kPostPer elements, all its
 // loads are issued before anything is used, and a resident SM keeps six to eight
 // such blocks in flight.  Whatever needs the whole group goes through small
-// partial tables that one warp per group combines in a fixed order:
-//   forward : conv_stats_kernel     (sum the K-slices, keep z, chunk mean / M2)
-//             conv_group_merge_kernel, mode 0 (group mean and 1/std from the chunk partials)
-//             conv_apply_fwd_kernel (normalise, skip, ReLU, pool)
-//   backward: conv_bwd_dn_kernel    (gradient at the normalised activation, channel sums per chunk)
-//             conv_group_merge_kernel, mode 1 (scale/shift gradients, group means)
-//             conv_bwd_dz_kernel    (gradient at the conv output)
+// partial tables that are combined in a fixed order.  Both directions are ONE launch:
+// the groups of a stage are bundled (whole groups, at least 8 channels where bfloat16
+// copies are written); every block does the first step for its chunk, then counts
+// itself in at the bundle's counter, and the block that arrives last - by then all
+// partials of the bundle are in memory - merges them and does the second step for the
+// bundle's tiles.  Nobody waits for anybody, and the merge order is the table's, not
+// the arrival order, so results do not depend on scheduling.
+//   forward  (conv_fwd_post_kernel): conv_stats_chunk (sum the K-slices, keep z, chunk
+//             mean / M2) -> group_merge_fwd (group mean and 1/std) -> conv_apply_fwd_chunk
+//             (normalise, skip, ReLU, pool)
+//   backward (conv_bwd_post_kernel): conv_bwd_dn_chunk (gradient at the normalised
+//             activation, channel sums per chunk) -> group_merge_bwd (scale/shift
+//             gradients, group means) -> conv_bwd_dz_chunk (gradient at the conv output)
 #pragma once
 #include "conv_types.h"
 #include "fc_kernels.cuh"   // ring_slot, warp_sum
@@ -30,6 +36,15 @@ __device__ __forceinline__ float skip_value(const ConvStage& st, const float* __
 }
 
 __device__ __forceinline__ int slot_of(long long sample, int slots) { return (int)((unsigned)sample % (unsigned)slots); }
+
+// Loads of data that OTHER blocks of the same launch have written (read by the block
+// that closes a bundle): served by the L2 cache, never by a non-coherent path.
+template <int VEC> __device__ __forceinline__ void vload_cg(float (&r)[VEC], const float* p);
+template <> __device__ __forceinline__ void vload_cg<4>(float (&r)[4], const float* p) {
+    const float4 q = __ldcg(reinterpret_cast<const float4*>(p));
+    r[0] = q.x; r[1] = q.y; r[2] = q.z; r[3] = q.w;
+}
+template <> __device__ __forceinline__ void vload_cg<1>(float (&r)[1], const float* p) { r[0] = __ldcg(p); }
 
 template <int VEC> __device__ __forceinline__ void ldb(unsigned char (&r)[VEC], const unsigned char* p);
 template <> __device__ __forceinline__ void ldb<4>(unsigned char (&r)[4], const unsigned char* p) {
@@ -143,7 +158,9 @@ __device__ __forceinline__ void store_nhwc_tile(const __nv_bfloat16* t16, int rs
     }
 }
 
-template <int VEC>
+// CG: the tile's inputs were written by other blocks of the SAME launch (the caller is the
+// block that closes a bundle): they are then loaded through the L2 cache.
+template <int VEC, bool CG>
 __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, long long t, const TickState* ts, __nv_bfloat16* t16) {
     constexpr int U = kPostPer / VEC;
     const long long i = t - st.s;
@@ -152,10 +169,10 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
     const int slot = slot_of(i, st.slots);
     const int hw = st.oh * st.ow, npu = ch.np / VEC, nunits = ch.ncl * npu, rs = ch.np + 2;
     const size_t zelems = (size_t)st.co * hw;
-    const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
+    const float* z = st.z_ring + (size_t)slot * zelems;
     const float* __restrict__ gam = st.wh + st.nw;
     const float* __restrict__ bet = gam + st.co;
-    const float* __restrict__ stat = st.stat_ring + (size_t)slot * st.groups * 2;
+    const float* stat = st.stat_ring + (size_t)slot * st.groups * 2;     // may have been written by this very block
     const float* __restrict__ sk = st.skip_ring
         ? st.skip_ring + (size_t)slot_of(i, st.skip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
     unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems;
@@ -178,7 +195,7 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
         pp[u] = ch.p0 + (uu - cl * npu) * VEC;
         const size_t idx = (size_t)cc[u] * hw + pp[u];
         const int grp = cc[u] / st.cpg;
-        vload<VEC>(zv[u], z + idx);
+        if (CG) vload_cg<VEC>(zv[u], z + idx); else vload<VEC>(zv[u], z + idx);
         mean[u] = stat[2 * grp];
         gs[u] = gam[cc[u]] * stat[2 * grp + 1];
         bb[u] = bet[cc[u]];
@@ -194,7 +211,8 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
     }
     auto act = [&](int c, int p) -> float {
         const int grp = c / st.cpg;
-        float v = fmaf(gam[c] * stat[2 * grp + 1], z[(size_t)c * hw + p] - stat[2 * grp], bet[c]);
+        const float zc = CG ? __ldcg(z + (size_t)c * hw + p) : z[(size_t)c * hw + p];
+        float v = fmaf(gam[c] * stat[2 * grp + 1], zc - stat[2 * grp], bet[c]);
         if (sk) v += skip_value(st, sk, c, p / st.ow, p % st.ow);
         return v;
     };
@@ -427,7 +445,7 @@ __device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long
 
 // ---------------------------------------------------------------- backward, step 2
 // Elementwise over a tile (see the forward step 2).
-template <int VEC>
+template <int VEC, bool CG>
 __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long long t, const TickState* ts, int S, __nv_bfloat16* t16) {
     constexpr int U = kPostPer / VEC;
     const long long j = t - 2LL * (S - 1) + st.s;
@@ -454,7 +472,7 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
         pp[u] = ch.p0 + (uu - cl * npu) * VEC;
         const size_t idx = (size_t)cc[u] * hw + pp[u];
         const int grp = cc[u] / st.cpg;
-        vload<VEC>(dnv[u], dz + idx);
+        if (CG) vload_cg<VEC>(dnv[u], dz + idx); else vload<VEC>(dnv[u], dz + idx);
         vload<VEC>(zv[u], z + idx);
         gv[u] = gam[cc[u]];
         mean[u] = stat[2 * grp]; rstd[u] = stat[2 * grp + 1];
@@ -505,72 +523,37 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
     }
 }
 
-// ---------------------------------------------------------------- launch wrappers
-// One block per chunk (statistics, channel sums) or tile (elementwise kernels).
-#define PB_POST_KERNEL(NAME, CHUNK, ...)                                                          \
-    __global__ void __launch_bounds__(kPostThreads, 4) NAME(const ConvStage* __restrict__ stages,  \
-                                                            const PostChunk* __restrict__ chunks, int nchunks, \
-                                                            const TickState* __restrict__ ts, int S, int par) { \
-        __shared__ float red[kPostWarps];                                                          \
-        __shared__ float usum[2 * kPostChunk];                                                     \
-        __shared__ __align__(16) __nv_bfloat16 t16[kPostChunk + 2 * kPostTileChannels];            \
-        (void)red; (void)usum; (void)t16; (void)S;                                                 \
-        if ((int)blockIdx.x >= nchunks) return;                                                    \
-        const PostChunk ch = chunks[blockIdx.x];                                                   \
-        const long long t = ts->cnt[par];                                                          \
-        const ConvStage& st = stages[ch.stage];                                                    \
-        if (st.vec4) CHUNK<4>(st, ch, t, ts, __VA_ARGS__);                                         \
-        else CHUNK<1>(st, ch, t, ts, __VA_ARGS__);                                                 \
-    }
-PB_POST_KERNEL(conv_stats_kernel, conv_stats_chunk, red)
-PB_POST_KERNEL(conv_apply_fwd_kernel, conv_apply_fwd_chunk, t16)
-PB_POST_KERNEL(conv_bwd_dn_kernel, conv_bwd_dn_chunk, S, red, usum)
-PB_POST_KERNEL(conv_bwd_dz_kernel, conv_bwd_dz_chunk, S, t16)
-#undef PB_POST_KERNEL
-
 // ---------------------------------------------------------------- group merges
-// mode 0 (forward): chunk statistics (count, mean, M2) -> group mean and 1/std, kept for the backward.
-// mode 1 (backward): per-chunk channel sums -> gradients of scale and shift, and the two
-// group means the gradient at the conv output needs (with the CURRENT scale).
-__global__ void __launch_bounds__(256)
-conv_group_merge_kernel(const ConvStage* __restrict__ stages, const GroupRef* __restrict__ groups, int ngroups,
-                        const TickState* __restrict__ ts, int S, int par, int mode) {
-    const int lane = threadIdx.x & 31;
-    const int gi = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (gi >= ngroups) return;
-    const GroupRef gr = groups[gi];
-    const ConvStage& st = stages[gr.stage];
-    const long long t = ts->cnt[par];
-    const int hw = st.oh * st.ow, cpg = st.cpg, c0 = gr.grp * cpg;
-    if (mode == 0) {
-        const long long i = t - st.s;
-        if (!sample_live(ts, i)) return;
-        const int slot = slot_of(i, st.slots), nidx = st.fstat_stride;
-        const float* __restrict__ f = st.fstat + (size_t)gr.grp * st.fstat_stride * 3;
-        float tot = 0.f, wsum = 0.f;
-        for (int k = lane; k < nidx; k += 32) { tot += f[3 * k]; wsum = fmaf(f[3 * k], f[3 * k + 1], wsum); }
-        tot = warp_sum(tot);
-        const float mean = warp_sum(wsum) / tot;
-        float m2 = 0.f;
-        for (int k = lane; k < nidx; k += 32) { const float d = f[3 * k + 1] - mean; m2 += f[3 * k + 2] + f[3 * k] * d * d; }
-        const float rstd = rsqrtf(warp_sum(m2) / tot + kGnEps);
-        if (lane == 0) {
-            st.stat_ring[((size_t)slot * st.groups + gr.grp) * 2 + 0] = mean;
-            st.stat_ring[((size_t)slot * st.groups + gr.grp) * 2 + 1] = rstd;
-        }
-        return;
+// forward: chunk statistics (count, mean, M2) -> group mean and 1/std, kept for the backward.
+__device__ __forceinline__ void group_merge_fwd(const ConvStage& st, int grp, long long t, int lane) {
+    const int slot = slot_of(t - st.s, st.slots), nidx = st.fstat_stride;
+    const float* f = st.fstat + (size_t)grp * st.fstat_stride * 3;
+    float tot = 0.f, wsum = 0.f;
+    for (int k = lane; k < nidx; k += 32) { const float n = __ldcg(f + 3 * k); tot += n; wsum = fmaf(n, __ldcg(f + 3 * k + 1), wsum); }
+    tot = warp_sum(tot);
+    const float mean = warp_sum(wsum) / tot;
+    float m2 = 0.f;
+    for (int k = lane; k < nidx; k += 32) { const float d = __ldcg(f + 3 * k + 1) - mean; m2 += __ldcg(f + 3 * k + 2) + __ldcg(f + 3 * k) * d * d; }
+    const float rstd = rsqrtf(warp_sum(m2) / tot + kGnEps);
+    if (lane == 0) {
+        st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0] = mean;
+        st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 1] = rstd;
     }
-    const long long j = t - 2LL * (S - 1) + st.s;
-    if (!sample_live(ts, j)) return;
+}
+
+// backward: per-chunk channel sums -> gradients of scale and shift, and the two group
+// means the gradient at the conv output needs (with the CURRENT scale).
+__device__ __forceinline__ void group_merge_bwd(const ConvStage& st, int grp, int lane) {
+    const int hw = st.oh * st.ow, cpg = st.cpg, c0 = grp * cpg;
     const float* __restrict__ gam = st.w + st.nw;
     const int np = st.npieces;
     float m1 = 0.f, m2 = 0.f;
     if (np >= 8) {
         // few channels, many pieces: lanes over the pieces of one channel at a time
         for (int cl = 0; cl < cpg; ++cl) {
-            const float* __restrict__ b = st.bsum + (size_t)(c0 + cl) * np * 2;
+            const float* b = st.bsum + (size_t)(c0 + cl) * np * 2;
             float t1 = 0.f, t2 = 0.f;
-            for (int q = lane; q < np; q += 32) { t1 += b[2 * q]; t2 += b[2 * q + 1]; }
+            for (int q = lane; q < np; q += 32) { t1 += __ldcg(b + 2 * q); t2 += __ldcg(b + 2 * q + 1); }
             t1 = warp_sum(t1); t2 = warp_sum(t2);
             if (lane == 0) {
                 st.g[st.nw + c0 + cl] = t2;
@@ -581,9 +564,9 @@ conv_group_merge_kernel(const ConvStage* __restrict__ stages, const GroupRef* __
         }
     } else {
         for (int cl = lane; cl < cpg; cl += 32) {
-            const float* __restrict__ b = st.bsum + (size_t)(c0 + cl) * np * 2;
+            const float* b = st.bsum + (size_t)(c0 + cl) * np * 2;
             float t1 = 0.f, t2 = 0.f;
-            for (int q = 0; q < np; ++q) { t1 += b[2 * q]; t2 += b[2 * q + 1]; }
+            for (int q = 0; q < np; ++q) { t1 += __ldcg(b + 2 * q); t2 += __ldcg(b + 2 * q + 1); }
             st.g[st.nw + c0 + cl] = t2;
             st.g[st.nw + st.co + c0 + cl] = t1;
             m1 = fmaf(gam[c0 + cl], t1, m1);
@@ -592,9 +575,126 @@ conv_group_merge_kernel(const ConvStage* __restrict__ stages, const GroupRef* __
         m1 = warp_sum(m1); m2 = warp_sum(m2);
     }
     if (lane == 0) {
-        st.gsum[2 * gr.grp] = m1 / (float)(cpg * hw);
-        st.gsum[2 * gr.grp + 1] = m2 / (float)(cpg * hw);
+        st.gsum[2 * grp] = m1 / (float)(cpg * hw);
+        st.gsum[2 * grp + 1] = m2 / (float)(cpg * hw);
     }
+}
+
+// ---------------------------------------------------------------- the two launches
+// Counts this block in at its bundle; true (for every thread) in the block that arrives
+// last, which also clears the counter for the next launch.  Every thread's stores of
+// the first step are fenced before the count, so the last block sees all of them.
+__device__ __forceinline__ bool bundle_closed_by_me(int* counter, int nchunks, int* flag) {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int old = atomicAdd(counter, 1);
+        const int last = old == nchunks - 1;
+        if (last) *counter = 0;
+        *flag = last;
+        __threadfence();
+    }
+    __syncthreads();
+    return *flag != 0;
+}
+
+__global__ void __launch_bounds__(kPostThreads, 4)
+conv_fwd_post_kernel(const ConvStage* __restrict__ stages, const PostChunk* __restrict__ chunks, int nchunks,
+                     const PostBundle* __restrict__ bundles, const PostChunk* __restrict__ tiles, int* __restrict__ counters,
+                     const TickState* __restrict__ ts, int S, int par) {
+    __shared__ float red[kPostWarps];
+    __shared__ __align__(16) __nv_bfloat16 t16[kPostChunk + 2 * kPostTileChannels];
+    __shared__ int last_flag;
+    (void)S;
+    if ((int)blockIdx.x >= nchunks) return;
+    const PostChunk ch = chunks[blockIdx.x];
+    const long long t = ts->cnt[par];
+    const ConvStage& st = stages[ch.stage];
+    if (!sample_live(ts, t - st.s)) return;                 // uniform over the bundle: nobody counts in
+    if (st.vec4) conv_stats_chunk<4>(st, ch, t, ts, red);
+    else conv_stats_chunk<1>(st, ch, t, ts, red);
+    if (ch.bundle < 0) return;                              // merged and finished by the launches that follow
+    const PostBundle bd = bundles[ch.bundle];
+    if (!bundle_closed_by_me(counters + ch.bundle, bd.nchunks, &last_flag)) return;
+    for (int g = threadIdx.x >> 5; g < bd.ngrp; g += kPostWarps) group_merge_fwd(st, bd.grp0 + g, t, threadIdx.x & 31);
+    __syncthreads();
+    for (int q = 0; q < bd.nftiles; ++q) {
+        const PostChunk tl = tiles[bd.ftile0 + q];
+        if (st.vec4) conv_apply_fwd_chunk<4, true>(st, tl, t, ts, t16);
+        else conv_apply_fwd_chunk<1, true>(st, tl, t, ts, t16);
+        __syncthreads();                                     // t16 is reused by the next tile
+    }
+}
+
+__global__ void __launch_bounds__(kPostThreads, 4)
+conv_bwd_post_kernel(const ConvStage* __restrict__ stages, const PostChunk* __restrict__ chunks, int nchunks,
+                     const PostBundle* __restrict__ bundles, const PostChunk* __restrict__ tiles, int* __restrict__ counters,
+                     const TickState* __restrict__ ts, int S, int par) {
+    __shared__ float red[kPostWarps];
+    __shared__ __align__(16) float usum[2 * kPostChunk];
+    __shared__ int last_flag;
+    if ((int)blockIdx.x >= nchunks) return;
+    const PostChunk ch = chunks[blockIdx.x];
+    const long long t = ts->cnt[par];
+    const ConvStage& st = stages[ch.stage];
+    if (!sample_live(ts, t - 2LL * (S - 1) + st.s)) return;
+    if (st.vec4) conv_bwd_dn_chunk<4>(st, ch, t, ts, S, red, usum);
+    else conv_bwd_dn_chunk<1>(st, ch, t, ts, S, red, usum);
+    if (ch.bundle < 0) return;
+    const PostBundle bd = bundles[ch.bundle];
+    if (!bundle_closed_by_me(counters + ch.bundle, bd.nchunks, &last_flag)) return;
+    for (int g = threadIdx.x >> 5; g < bd.ngrp; g += kPostWarps) group_merge_bwd(st, bd.grp0 + g, threadIdx.x & 31);
+    __syncthreads();
+    // the transposing tile of the second step lives in the space of the first step's sums
+    __nv_bfloat16* t16 = reinterpret_cast<__nv_bfloat16*>(usum);
+    for (int q = 0; q < bd.nbtiles; ++q) {
+        const PostChunk tl = tiles[bd.btile0 + q];
+        if (st.vec4) conv_bwd_dz_chunk<4, true>(st, tl, t, ts, S, t16);
+        else conv_bwd_dz_chunk<1, true>(st, tl, t, ts, S, t16);
+        __syncthreads();
+    }
+}
+
+// Stages that are not fused: one warp per group merges the partials ...
+__global__ void __launch_bounds__(256)
+conv_group_merge_kernel(const ConvStage* __restrict__ stages, const GroupRef* __restrict__ groups, int ngroups,
+                        const TickState* __restrict__ ts, int S, int par, int mode) {
+    const int gi = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (gi >= ngroups) return;
+    const GroupRef gr = groups[gi];
+    const ConvStage& st = stages[gr.stage];
+    const long long t = ts->cnt[par];
+    if (mode == 0) {
+        if (sample_live(ts, t - st.s)) group_merge_fwd(st, gr.grp, t, threadIdx.x & 31);
+    } else {
+        if (sample_live(ts, t - 2LL * (S - 1) + st.s)) group_merge_bwd(st, gr.grp, threadIdx.x & 31);
+    }
+}
+
+// ... and the second step runs one block per tile.
+__global__ void __launch_bounds__(kPostThreads, 4)
+conv_apply_fwd_kernel(const ConvStage* __restrict__ stages, const PostChunk* __restrict__ tiles, int ntiles,
+                      const TickState* __restrict__ ts, int S, int par) {
+    __shared__ __align__(16) __nv_bfloat16 t16[kPostChunk + 2 * kPostTileChannels];
+    (void)S;
+    if ((int)blockIdx.x >= ntiles) return;
+    const PostChunk tl = tiles[blockIdx.x];
+    const long long t = ts->cnt[par];
+    const ConvStage& st = stages[tl.stage];
+    if (st.vec4) conv_apply_fwd_chunk<4, false>(st, tl, t, ts, t16);
+    else conv_apply_fwd_chunk<1, false>(st, tl, t, ts, t16);
+}
+
+__global__ void __launch_bounds__(kPostThreads, 4)
+conv_bwd_dz_kernel(const ConvStage* __restrict__ stages, const PostChunk* __restrict__ tiles, int ntiles,
+                   const TickState* __restrict__ ts, int S, int par) {
+    __shared__ __align__(16) __nv_bfloat16 t16[kPostChunk + 2 * kPostTileChannels];
+    if ((int)blockIdx.x >= ntiles) return;
+    const PostChunk tl = tiles[blockIdx.x];
+    const long long t = ts->cnt[par];
+    const ConvStage& st = stages[tl.stage];
+    if (st.vec4) conv_bwd_dz_chunk<4, false>(st, tl, t, ts, S, t16);
+    else conv_bwd_dz_chunk<1, false>(st, tl, t, ts, S, t16);
 }
 
 // ---------------------------------------------------------------- update

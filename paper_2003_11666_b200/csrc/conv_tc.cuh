@@ -89,12 +89,6 @@ __device__ __forceinline__ void cp_async16(unsigned char* dst, const __nv_bfloat
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(sz) : "memory");
 }
 
-// Quotient a / b for 0 <= a < 2^21 and b <= 2^13 from the float reciprocal of b: the
-// product (a + 0.5) / b is at least 0.5 / b away from every integer, far more than its
-// rounding error (about 2e-7 a / b), so rounding down gives the exact quotient.  A
-// negative a gives a negative result (only ever used to reject the element).
-__device__ __forceinline__ int quot(int a, float inv_b) { return __float2int_rd(((float)a + 0.5f) * inv_b); }
-
 __global__ void __launch_bounds__(kTcThreads)
 conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, TickState* ts, int S, int par) {
     extern __shared__ unsigned char tc_smem_raw[];

@@ -13,6 +13,7 @@ constexpr int kPostThreads = 256;         // normalisation / activation kernels
 constexpr int kPostChunk = 2048;          // elements per block of those kernels
 constexpr int kPostTilePixels = 128;       // pixels of a tile of the elementwise kernels
 constexpr int kPostTileChannels = 64;      // most channels of such a tile
+constexpr int kPostFuseTiles = 4;           // a bundle with at most this many second-step tiles is finished by its closing block
 constexpr int kMaxGroupChannels = 64;      // channels per normalisation group
 
 enum GemmMode { kFprop = 0, kDgrad = 1, kWgrad = 2 };
@@ -91,9 +92,20 @@ struct UpdChunk { int range, start; };
 // The same record describes a tile of the elementwise kernels: there cl0 is an absolute
 // channel and grp is not used.
 // Either ncl >= 1 whole channels (p0 = 0, np = all pixels) or a piece of one channel.
-struct PostChunk { int stage, grp, cl0, ncl, p0, np, idx, nidx; };
-// One normalisation group of one stage (a warp of the merge kernel).
+struct PostChunk { int stage, grp, cl0, ncl, p0, np, idx, nidx, bundle; };   // bundle < 0: the stage is not fused
+// A bundle: groups [grp0, grp0 + ngrp) of one stage, whose nchunks chunks are closed by
+// one block that then works through the bundle's tiles of the second step.
+// One normalisation group of a stage that is not fused (a warp of the merge kernel).
 struct GroupRef { int stage, grp; };
+struct PostBundle { int stage, grp0, ngrp, nchunks, ftile0, nftiles, btile0, nbtiles; };
 constexpr int kUpdChunk = 4096;
+
+#ifdef __CUDACC__
+// Quotient a / b for 0 <= a < 2^21 and b <= 2^13 from the float reciprocal of b: the
+// product (a + 0.5) / b is at least 0.5 / b away from every integer, far more than its
+// rounding error (about 2e-7 a / b), so rounding down gives the exact quotient.  A
+// negative a gives a negative result (only ever used to reject the element).
+__device__ __forceinline__ int quot(int a, float inv_b) { return __float2int_rd(((float)a + 0.5f) * inv_b); }
+#endif
 
 }  // namespace pb

@@ -286,7 +286,17 @@ void add_tiles(std::vector<GemmTile>& tiles, int gemm, int M, int N, int nsplit,
 }
 
 void fill_conv_tables(pb_handle* h) {
-    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_groups.clear(); h->h_ptiles[0].clear(); h->h_ptiles[1].clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear();
+    {
+        // first-step blocks of the normalisation launches over the whole network
+        long long chunks = 0;
+        for (const StageHost& x : h->stages) {
+            if (x.head_op != PB_CONV2D) continue;
+            const int hw = x.z.h * x.z.w, cpg = x.head.c_out / x.gn_groups;
+            chunks += (long long)x.gn_groups * (hw <= kPostChunk ? ceil_div(cpg, std::max(1, kPostChunk / hw)) : cpg * ceil_div(hw, kPostChunk));
+        }
+        h->post_fuse = chunks <= 8LL * h->num_sms;       // under two waves of four blocks per SM
+    }
+    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_bundles.clear(); h->h_groups.clear(); h->h_ptiles[0].clear(); h->h_ptiles[1].clear(); h->h_dtiles[0].clear(); h->h_dtiles[1].clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear();
     for (auto& t : h->h_tiles) t.clear();
     for (auto& t : h->h_tctiles) t.clear();
     const int bf = (h->flags & PB_CONV_BF16) ? 1 : 0;
@@ -360,7 +370,7 @@ void fill_conv_tables(pb_handle* h) {
         c.zpart = x.zpart; c.z_nsplit = x.split_f;
         c.z_ring = x.z_ring; c.stat_ring = x.stat_ring; c.code_ring = x.code_ring; c.arg_ring = x.arg_ring;
         c.out_ring = x.out_ring; c.slots = x.out_slots;
-        c.out16 = x.out16; c.dz16 = x.dz16;
+        c.out16 = x.out16; c.dz16 = x.tc ? x.dz16 : nullptr;     // only tensor-core stages read the bfloat16 gradient
         c.wh = h->d_wh + x.dev_off; c.w = h->d_w + x.dev_off; c.g = h->d_g + x.dev_off; c.nw = nw;
         if (x.has_skip) {
             const StageHost& y = h->stages[x.skip_src];
@@ -374,39 +384,91 @@ void fill_conv_tables(pb_handle* h) {
         c.dz = x.dz;
         c.fstat = x.fstat; c.fstat_stride = x.fstat_stride; c.bsum = x.bsum; c.npieces = x.npieces; c.gsum = x.gsum;
         {
-            // chunks of the normalisation kernels: whole channels while they fit, else pieces of one channel
-            const int hw = x.z.h * x.z.w, cpg = c.cpg;
-            for (int gq = 0; gq < x.gn_groups; ++gq) {
-                h->h_groups.push_back(GroupRef{(int)h->h_cs.size(), gq});
-                const size_t first = h->h_pchunks.size();
-                if (hw <= kPostChunk) {
-                    const int per = std::max(1, kPostChunk / hw);
-                    for (int cl = 0; cl < cpg; cl += per)
-                        h->h_pchunks.push_back(PostChunk{(int)h->h_cs.size(), gq, cl, std::min(per, cpg - cl), 0, hw, 0, 0});
-                } else {
-                    for (int cl = 0; cl < cpg; ++cl)
-                        for (int p0 = 0; p0 < hw; p0 += kPostChunk)
-                            h->h_pchunks.push_back(PostChunk{(int)h->h_cs.size(), gq, cl, 1, p0, std::min(kPostChunk, hw - p0), 0, 0});
+            // Chunks of the first step: whole channels while they fit, else pieces of one channel.
+            // Tiles of the second step: (a multiple of 8 channels) x pixels, up to kPostChunk
+            // elements; the forward of a pooling stage works on the group chunks instead.
+            // In small networks (the first step is under two waves of blocks, so launch latency
+            // dominates) stages are FUSED: their groups are bundled (whole groups, at least 8
+            // channels where bfloat16 copies are written, whose 16-byte runs hold 8 channels of a
+            // pixel), tiles stay inside a bundle and the block that closes a bundle finishes it.
+            // Elsewhere, and for a stage with a bundle of more than kPostFuseTiles tiles, the
+            // three-launch form stays (closing blocks working through several tiles each would
+            // be the tail of a launch that is already many waves long).
+            const int hw = x.z.h * x.z.w, cpg = c.cpg, stage_idx = (int)h->h_cs.size();
+            const bool need16 = x.tc && L.c_out % 8 == 0 && 8 % cpg == 0;
+            const int gpb = need16 && cpg < 8 ? 8 / cpg : 1;           // groups per bundle
+            const bool pooled = x.has_pool || x.avgpool;
+            auto tile_shape = [&](int channels, int& CT, int& PT) {
+                CT = std::min(kPostTileChannels, std::max(8, (kPostChunk / std::min(hw, kPostTilePixels)) / 8 * 8));
+                CT = std::min(CT, channels);
+                PT = CT * hw <= kPostChunk ? hw : std::min(hw, std::max(4, (kPostChunk / CT) / 4 * 4));
+            };
+            auto chunks_of_group = [&](int gq) {
+                int n = 0;
+                if (hw <= kPostChunk) n = ceil_div(cpg, std::max(1, kPostChunk / hw));
+                else n = cpg * ceil_div(hw, kPostChunk);
+                return n;
+            };
+            bool fuse = h->post_fuse;
+            if (fuse) {
+                int CT, PT;
+                tile_shape(gpb * cpg, CT, PT);
+                const int btiles = ceil_div(gpb * cpg, CT) * ceil_div(hw, PT);
+                const int ftiles = pooled ? gpb * chunks_of_group(0) : btiles;
+                fuse = btiles <= kPostFuseTiles && ftiles <= kPostFuseTiles;
+            }
+            for (int g0 = 0; g0 < x.gn_groups; g0 += gpb) {
+                PostBundle bd{};
+                bd.stage = stage_idx; bd.grp0 = g0; bd.ngrp = std::min(gpb, x.gn_groups - g0);
+                const int bundle_idx = fuse ? (int)h->h_bundles.size() : -1;
+                bd.ftile0 = (int)h->h_ptiles[0].size(); bd.btile0 = (int)h->h_ptiles[1].size();
+                for (int gq = g0; gq < g0 + bd.ngrp; ++gq) {
+                    if (!fuse) h->h_groups.push_back(GroupRef{stage_idx, gq});
+                    const size_t first = h->h_pchunks.size();
+                    if (hw <= kPostChunk) {
+                        const int per = std::max(1, kPostChunk / hw);
+                        for (int cl = 0; cl < cpg; cl += per)
+                            h->h_pchunks.push_back(PostChunk{stage_idx, gq, cl, std::min(per, cpg - cl), 0, hw, 0, 0, bundle_idx});
+                    } else {
+                        for (int cl = 0; cl < cpg; ++cl)
+                            for (int p0 = 0; p0 < hw; p0 += kPostChunk)
+                                h->h_pchunks.push_back(PostChunk{stage_idx, gq, cl, 1, p0, std::min(kPostChunk, hw - p0), 0, 0, bundle_idx});
+                    }
+                    const int nidx = (int)(h->h_pchunks.size() - first);
+                    for (int q = 0; q < nidx; ++q) { h->h_pchunks[first + q].idx = q; h->h_pchunks[first + q].nidx = nidx; }
+                    bd.nchunks += nidx;
+                    if (pooled)
+                        for (int q = 0; q < nidx; ++q) {
+                            PostChunk tch = h->h_pchunks[first + q];
+                            tch.cl0 += gq * cpg; tch.grp = -1;
+                            (fuse ? h->h_ptiles[0] : h->h_dtiles[0]).push_back(tch);
+                        }
                 }
-                const int nidx = (int)(h->h_pchunks.size() - first);
-                for (int q = 0; q < nidx; ++q) { h->h_pchunks[first + q].idx = q; h->h_pchunks[first + q].nidx = nidx; }
-                if (x.has_pool || x.avgpool)      // the forward of a pooling stage works on the group chunks
-                    for (int q = 0; q < nidx; ++q) {
-                        PostChunk tch = h->h_pchunks[first + q];
-                        tch.cl0 += gq * cpg; tch.grp = -1;
-                        h->h_ptiles[0].push_back(tch);
+                if (!fuse) continue;
+                const int c_lo = g0 * cpg, c_hi = (g0 + bd.ngrp) * cpg;
+                int CT, PT;
+                tile_shape(c_hi - c_lo, CT, PT);
+                for (int c0 = c_lo; c0 < c_hi; c0 += CT)
+                    for (int p0 = 0; p0 < hw; p0 += PT) {
+                        const PostChunk tch{stage_idx, -1, c0, std::min(CT, c_hi - c0), p0, std::min(PT, hw - p0), 0, 0, bundle_idx};
+                        if (!pooled) h->h_ptiles[0].push_back(tch);
+                        h->h_ptiles[1].push_back(tch);
+                    }
+                bd.nftiles = (int)h->h_ptiles[0].size() - bd.ftile0;
+                bd.nbtiles = (int)h->h_ptiles[1].size() - bd.btile0;
+                h->h_bundles.push_back(bd);
+            }
+            if (!fuse) {
+                // stage-wide tiles for the launches of their own
+                int CT, PT;
+                tile_shape(L.c_out, CT, PT);
+                for (int c0 = 0; c0 < L.c_out; c0 += CT)
+                    for (int p0 = 0; p0 < hw; p0 += PT) {
+                        const PostChunk tch{stage_idx, -1, c0, std::min(CT, (int)L.c_out - c0), p0, std::min(PT, hw - p0), 0, 0, -1};
+                        if (!pooled) h->h_dtiles[0].push_back(tch);
+                        h->h_dtiles[1].push_back(tch);
                     }
             }
-            // tiles of the elementwise kernels: (a multiple of 8 channels) x (up to kPostTilePixels pixels)
-            const int PT = std::min(hw, kPostTilePixels);
-            int CT = std::min(kPostTileChannels, std::max(8, (kPostChunk / PT) / 8 * 8));
-            CT = std::min(CT, (int)L.c_out);
-            for (int c0 = 0; c0 < L.c_out; c0 += CT)
-                for (int p0 = 0; p0 < hw; p0 += PT) {
-                    const PostChunk tch{(int)h->h_cs.size(), -1, c0, std::min(CT, (int)L.c_out - c0), p0, std::min(PT, hw - p0), 0, 0};
-                    if (!(x.has_pool || x.avgpool)) h->h_ptiles[0].push_back(tch);
-                    h->h_ptiles[1].push_back(tch);
-                }
         }
         h->h_cs.push_back(c);
 
@@ -473,8 +535,10 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     for (int q = 0; q < 3; ++q) h->d_tiles[q] = c.take<GemmTile>(h->h_tiles[q].size() + 1);
     h->d_cs = c.take<ConvStage>(h->h_cs.size() + 1);
     h->d_pchunks = c.take<PostChunk>(h->h_pchunks.size() + 1);
+    h->d_bundles = c.take<PostBundle>(h->h_bundles.size() + 1);
     h->d_groups = c.take<GroupRef>(h->h_groups.size() + 1);
     for (int q = 0; q < 2; ++q) h->d_ptiles[q] = c.take<PostChunk>(h->h_ptiles[q].size() + 1);
+    for (int q = 0; q < 2; ++q) h->d_dtiles[q] = c.take<PostChunk>(h->h_dtiles[q].size() + 1);
     h->d_upd = c.take<UpdRange>(h->h_upd.size() + 1);
     h->d_chunks = c.take<UpdChunk>(h->h_chunks.size() + 1);
     h->d_tc = c.take<ConvGemmTC>(h->h_tc.size() + 1);
@@ -483,6 +547,7 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     if (!h->all_fc || (h->flags & PB_LWP_WFORM)) h->d_wh = c.take<float>(h->dev_params);
     *zero_from = c.off;
     h->d_v = c.take<float>(h->dev_params);
+    for (int q = 0; q < 2; ++q) h->d_bcnt[q] = c.take<int>(h->h_bundles.size() + 1);   // bundle counters (zero between launches)
     if (!h->all_fc) h->d_g = c.take<float>(h->dev_params);
     if (h->flags & PB_CONV_BF16) {
         h->d_w16 = c.take<__nv_bfloat16>(h->dev_params);
@@ -589,7 +654,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
     const bool fused_last = h->nctaB == 0;      // the last stage rides in the phase-0 launch
     const int npc = (int)h->h_pchunks.size();
     const int post_grid = std::max(1, npc);              // one block per chunk
-    const int ngr = (int)h->h_groups.size(), merge_grid = std::max(1, ceil_div(ngr, 8));
+    const int ngr = (int)h->h_groups.size();             // groups of the stages that keep the three-launch form
     for (int k = 0; k < n_ticks; ++k) {
         const int par = (int)((t_base + k) & 1);
         if (h->all_fc) {
@@ -640,9 +705,11 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
                 prof_end(h);
             }
             prof_begin(h, 5);
-            conv_stats_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
-            conv_group_merge_kernel<<<merge_grid, 256, 0, h->stream>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 0);
-            conv_apply_fwd_kernel<<<std::max(1, (int)h->h_ptiles[0].size()), kPostThreads, 0, h->stream>>>(h->d_cs, h->d_ptiles[0], (int)h->h_ptiles[0].size(), h->d_ts, h->S, par);
+            conv_fwd_post_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_bundles, h->d_ptiles[0], h->d_bcnt[0], h->d_ts, h->S, par);
+            if (ngr > 0)
+                conv_group_merge_kernel<<<ceil_div(ngr, 8), 256, 0, h->stream>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 0);
+            if (!h->h_dtiles[0].empty())
+                conv_apply_fwd_kernel<<<(int)h->h_dtiles[0].size(), kPostThreads, 0, h->stream>>>(h->d_cs, h->d_dtiles[0], (int)h->h_dtiles[0].size(), h->d_ts, h->S, par);
             prof_end(h);
             // Backward chain: through pool/ReLU/GroupNorm -> data and weight gradients.  It reads
             // what earlier ticks stored (other ring slots than the forward chain writes) and the
@@ -651,9 +718,11 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             cudaStream_t bs = h->bwd ? h->bwd : h->stream;
             cudaStreamWaitEvent(bs, h->ev_fork, 0);
             prof_begin(h, 6, bs);
-            conv_bwd_dn_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_ts, h->S, par);
-            conv_group_merge_kernel<<<merge_grid, 256, 0, bs>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 1);
-            conv_bwd_dz_kernel<<<std::max(1, (int)h->h_ptiles[1].size()), kPostThreads, 0, bs>>>(h->d_cs, h->d_ptiles[1], (int)h->h_ptiles[1].size(), h->d_ts, h->S, par);
+            conv_bwd_post_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_bundles, h->d_ptiles[1], h->d_bcnt[1], h->d_ts, h->S, par);
+            if (ngr > 0)
+                conv_group_merge_kernel<<<ceil_div(ngr, 8), 256, 0, bs>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 1);
+            if (!h->h_dtiles[1].empty())
+                conv_bwd_dz_kernel<<<(int)h->h_dtiles[1].size(), kPostThreads, 0, bs>>>(h->d_cs, h->d_dtiles[1], (int)h->h_dtiles[1].size(), h->d_ts, h->S, par);
             prof_end(h, bs);
             // data gradients (dgrad) and weight gradients (wgrad) both start from dz and write
             // different buffers: wgrad goes to a stream of its own
@@ -683,7 +752,8 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             // the conv chain waits for the FC stages before the tick ends
             cudaEventRecord(h->ev_join, fs);
             cudaStreamWaitEvent(h->stream, h->ev_join, 0);
-            h->last_launches += 9 + (fused_last ? 0 : 1);      // ingest, 3 + 3 normalisation kernels, update, FC
+            h->last_launches += 5 + (fused_last ? 0 : 1);      // ingest, the two normalisation kernels, update, FC
+            h->last_launches += (h->h_dtiles[0].empty() ? 0 : 1) + (h->h_dtiles[1].empty() ? 0 : 1) + (ngr > 0 ? 2 : 0);
             for (int q = 0; q < 3; ++q) h->last_launches += (h->h_tiles[q].empty() ? 0 : 1) + (h->h_tctiles[q].empty() ? 0 : 1);
         }
     }
@@ -783,8 +853,10 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     for (int q = 0; q < 3; ++q) up(h->d_tiles[q], h->h_tiles[q].data(), h->h_tiles[q].size() * sizeof(GemmTile));
     up(h->d_cs, h->h_cs.data(), h->h_cs.size() * sizeof(ConvStage));
     up(h->d_pchunks, h->h_pchunks.data(), h->h_pchunks.size() * sizeof(PostChunk));
+    up(h->d_bundles, h->h_bundles.data(), h->h_bundles.size() * sizeof(PostBundle));
     up(h->d_groups, h->h_groups.data(), h->h_groups.size() * sizeof(GroupRef));
     for (int q = 0; q < 2; ++q) up(h->d_ptiles[q], h->h_ptiles[q].data(), h->h_ptiles[q].size() * sizeof(PostChunk));
+    for (int q = 0; q < 2; ++q) up(h->d_dtiles[q], h->h_dtiles[q].data(), h->h_dtiles[q].size() * sizeof(PostChunk));
     up(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange));
     up(h->d_chunks, h->h_chunks.data(), h->h_chunks.size() * sizeof(UpdChunk));
     up(h->d_tc, h->h_tc.data(), h->h_tc.size() * sizeof(ConvGemmTC));

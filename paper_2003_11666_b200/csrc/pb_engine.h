@@ -91,7 +91,11 @@ struct pb_handle {
     std::vector<pb::GemmTile> h_tiles[3]; pb::GemmTile* d_tiles[3] = {nullptr, nullptr, nullptr};
     std::vector<pb::ConvStage> h_cs; pb::ConvStage* d_cs = nullptr;
     std::vector<pb::PostChunk> h_pchunks; pb::PostChunk* d_pchunks = nullptr;
-    std::vector<pb::GroupRef> h_groups; pb::GroupRef* d_groups = nullptr;
+    std::vector<pb::PostChunk> h_dtiles[2]; pb::PostChunk* d_dtiles[2] = {nullptr, nullptr};   // tiles of large bundles: launches of their own
+    std::vector<pb::GroupRef> h_groups; pb::GroupRef* d_groups = nullptr;      // groups merged by the merge kernel
+    bool post_fuse = false;                     // normalisation steps of a stage fused into one launch
+    std::vector<pb::PostBundle> h_bundles; pb::PostBundle* d_bundles = nullptr;
+    int* d_bcnt[2] = {nullptr, nullptr};        // bundle counters of the forward / backward launch
     std::vector<pb::PostChunk> h_ptiles[2]; pb::PostChunk* d_ptiles[2] = {nullptr, nullptr};   // tiles of the elementwise kernels: forward, backward
     std::vector<pb::UpdRange> h_upd; pb::UpdRange* d_upd = nullptr;
     std::vector<pb::UpdChunk> h_chunks; pb::UpdChunk* d_chunks = nullptr;
