@@ -245,7 +245,9 @@ def main():
     hx = torch.from_numpy(x).pin_memory()
     hy = torch.from_numpy(y).pin_memory()
     hl = torch.zeros(K + W).pin_memory()
-    eng.run_host(hx[:W], hy[:W], W, hl[:W])
+    # warm-up of the same size as the timed call: it fills the pipeline and sizes the
+    # library's staging buffer, so that the timed call allocates nothing
+    eng.run_host(hx[W:], hy[W:], K, hl[W:])
     barrier()
     t0 = time.perf_counter()
     eng.run_host(hx[W:], hy[W:], K, hl[W:])

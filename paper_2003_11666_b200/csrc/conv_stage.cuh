@@ -598,6 +598,37 @@ __device__ __forceinline__ bool bundle_closed_by_me(int* counter, int nchunks, i
     return *flag != 0;
 }
 
+// What the closing block does: merge the bundle's groups, then its tiles of the second
+// step.  Kept out of line so that its registers do not weigh on the first step, which
+// every block runs.
+__device__ __noinline__ void close_bundle_fwd(const ConvStage* __restrict__ stages, const PostBundle* __restrict__ bundles, int bundle,
+                                              const PostChunk* __restrict__ tiles, long long t, const TickState* ts, __nv_bfloat16* t16) {
+    const PostBundle bd = bundles[bundle];
+    const ConvStage& st = stages[bd.stage];
+    for (int g = threadIdx.x >> 5; g < bd.ngrp; g += kPostWarps) group_merge_fwd(st, bd.grp0 + g, t, threadIdx.x & 31);
+    __syncthreads();
+    for (int q = 0; q < bd.nftiles; ++q) {
+        const PostChunk tl = tiles[bd.ftile0 + q];
+        if (st.vec4) conv_apply_fwd_chunk<4, true>(st, tl, t, ts, t16);
+        else conv_apply_fwd_chunk<1, true>(st, tl, t, ts, t16);
+        __syncthreads();                                     // t16 is reused by the next tile
+    }
+}
+
+__device__ __noinline__ void close_bundle_bwd(const ConvStage* __restrict__ stages, const PostBundle* __restrict__ bundles, int bundle,
+                                              const PostChunk* __restrict__ tiles, long long t, const TickState* ts, int S, __nv_bfloat16* t16) {
+    const PostBundle bd = bundles[bundle];
+    const ConvStage& st = stages[bd.stage];
+    for (int g = threadIdx.x >> 5; g < bd.ngrp; g += kPostWarps) group_merge_bwd(st, bd.grp0 + g, threadIdx.x & 31);
+    __syncthreads();
+    for (int q = 0; q < bd.nbtiles; ++q) {
+        const PostChunk tl = tiles[bd.btile0 + q];
+        if (st.vec4) conv_bwd_dz_chunk<4, true>(st, tl, t, ts, S, t16);
+        else conv_bwd_dz_chunk<1, true>(st, tl, t, ts, S, t16);
+        __syncthreads();
+    }
+}
+
 __global__ void __launch_bounds__(kPostThreads, 4)
 conv_fwd_post_kernel(const ConvStage* __restrict__ stages, const PostChunk* __restrict__ chunks, int nchunks,
                      const PostBundle* __restrict__ bundles, const PostChunk* __restrict__ tiles, int* __restrict__ counters,
@@ -613,17 +644,10 @@ conv_fwd_post_kernel(const ConvStage* __restrict__ stages, const PostChunk* __re
     if (!sample_live(ts, t - st.s)) return;                 // uniform over the bundle: nobody counts in
     if (st.vec4) conv_stats_chunk<4>(st, ch, t, ts, red);
     else conv_stats_chunk<1>(st, ch, t, ts, red);
-    if (ch.bundle < 0) return;                              // merged and finished by the launches that follow
-    const PostBundle bd = bundles[ch.bundle];
-    if (!bundle_closed_by_me(counters + ch.bundle, bd.nchunks, &last_flag)) return;
-    for (int g = threadIdx.x >> 5; g < bd.ngrp; g += kPostWarps) group_merge_fwd(st, bd.grp0 + g, t, threadIdx.x & 31);
-    __syncthreads();
-    for (int q = 0; q < bd.nftiles; ++q) {
-        const PostChunk tl = tiles[bd.ftile0 + q];
-        if (st.vec4) conv_apply_fwd_chunk<4, true>(st, tl, t, ts, t16);
-        else conv_apply_fwd_chunk<1, true>(st, tl, t, ts, t16);
-        __syncthreads();                                     // t16 is reused by the next tile
-    }
+    const int bundle = chunks[blockIdx.x].bundle;
+    if (bundle < 0) return;                                 // merged and finished by the launches that follow
+    if (!bundle_closed_by_me(counters + bundle, bundles[bundle].nchunks, &last_flag)) return;
+    close_bundle_fwd(stages, bundles, bundle, tiles, ts->cnt[par], ts, t16);
 }
 
 __global__ void __launch_bounds__(kPostThreads, 4)
@@ -640,19 +664,11 @@ conv_bwd_post_kernel(const ConvStage* __restrict__ stages, const PostChunk* __re
     if (!sample_live(ts, t - 2LL * (S - 1) + st.s)) return;
     if (st.vec4) conv_bwd_dn_chunk<4>(st, ch, t, ts, S, red, usum);
     else conv_bwd_dn_chunk<1>(st, ch, t, ts, S, red, usum);
-    if (ch.bundle < 0) return;
-    const PostBundle bd = bundles[ch.bundle];
-    if (!bundle_closed_by_me(counters + ch.bundle, bd.nchunks, &last_flag)) return;
-    for (int g = threadIdx.x >> 5; g < bd.ngrp; g += kPostWarps) group_merge_bwd(st, bd.grp0 + g, threadIdx.x & 31);
-    __syncthreads();
+    const int bundle = chunks[blockIdx.x].bundle;
+    if (bundle < 0) return;
+    if (!bundle_closed_by_me(counters + bundle, bundles[bundle].nchunks, &last_flag)) return;
     // the transposing tile of the second step lives in the space of the first step's sums
-    __nv_bfloat16* t16 = reinterpret_cast<__nv_bfloat16*>(usum);
-    for (int q = 0; q < bd.nbtiles; ++q) {
-        const PostChunk tl = tiles[bd.btile0 + q];
-        if (st.vec4) conv_bwd_dz_chunk<4, true>(st, tl, t, ts, S, t16);
-        else conv_bwd_dz_chunk<1, true>(st, tl, t, ts, S, t16);
-        __syncthreads();
-    }
+    close_bundle_bwd(stages, bundles, bundle, tiles, ts->cnt[par], ts, S, reinterpret_cast<__nv_bfloat16*>(usum));
 }
 
 // Stages that are not fused: one warp per group merges the partials ...

@@ -361,7 +361,7 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
 // fused last stage, and (ingest != 0) the copy of the new sample and label into
 // their rings.  When the last stage is too large for one block it gets its own
 // phase-1 launch; `publish` marks the launch that ends the tick.
-__global__ void __launch_bounds__(kFcThreads, 2)
+__global__ void __launch_bounds__(kFcThreads, kFcBlocksPerSM)
 fc_tick_kernel(const FcStage* __restrict__ stages, const FcSeg* __restrict__ segs,
                const int* __restrict__ cta_seg_begin, TickState* ts, int S, int phase, int par, int publish,
                int* __restrict__ label_ring, float* __restrict__ losses, long long t_base,

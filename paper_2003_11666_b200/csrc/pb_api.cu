@@ -194,7 +194,7 @@ void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSe
         total += (double)main_rows[f] * st.in_dim * 8.0;
     }
     if (total <= 0) return;
-    int ncta = 2 * h->num_sms - fused_ctas;       // two resident blocks per SM
+    int ncta = kFcBlocksPerSM * h->num_sms - fused_ctas;       // one wave of resident blocks
     const int by_size = (int)(total / (48.0 * 1024)) + 1;      // at least 48 KB of weights per block
     if (ncta > by_size) ncta = by_size;
     if (ncta < 1) ncta = 1;
