@@ -99,6 +99,8 @@ struct PostChunk { int stage, grp, cl0, ncl, p0, np, idx, nidx, bundle; };   // 
 struct GroupRef { int stage, grp; };
 struct PostBundle { int stage, grp0, ngrp, nchunks, ftile0, nftiles, btile0, nbtiles; };
 constexpr int kUpdChunk = 4096;
+// stream priorities of a conv tick's side chains (1 = the device's highest, 0 = default)
+constexpr int kPrioBwd = 1, kPrioAux = 1, kPrioSide = 0;
 
 #ifdef __CUDACC__
 // Quotient a / b for 0 <= a < 2^21 and b <= 2^13 from the float reciprocal of b: the

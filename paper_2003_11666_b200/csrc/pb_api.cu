@@ -862,12 +862,20 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     up(h->d_tc, h->h_tc.data(), h->h_tc.size() * sizeof(ConvGemmTC));
     for (int q = 0; q < 3; ++q) up(h->d_tctiles[q], h->h_tctiles[q].data(), h->h_tctiles[q].size() * sizeof(GemmTile));
     if (e == cudaSuccess && !h->all_fc) {
-        e = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking);
+        // The backward chain (normalisation backward -> data gradients) is the longest of the
+        // tick's chains and the update waits for it.  In small networks, whose launches do not
+        // fill the GPU, giving its streams the higher priority shortens the tick (measured:
+        // VGG-11 200 -> 186 us, ResNet-20 69 -> 66 us); in ResNet-50 it starves the forward
+        // convolutions (597 -> 613 us), so large networks keep equal priorities.
+        int prio_least = 0, prio_greatest = 0;
+        cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest);
+        auto prio = [&](int level) { return (level && h->post_fuse) ? prio_greatest : prio_least; };
+        e = cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, prio(kPrioSide));
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->bwd, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&h->bwd, cudaStreamNonBlocking, prio(kPrioBwd));
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_bjoin, cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&h->aux, cudaStreamNonBlocking, prio(kPrioAux));
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_dz, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_wjoin, cudaEventDisableTiming);
     }
