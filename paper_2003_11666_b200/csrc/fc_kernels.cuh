@@ -369,6 +369,14 @@ fc_tick_kernel(const FcStage* __restrict__ stages, const FcSeg* __restrict__ seg
                float* __restrict__ in_ring, int in_slots, int elems) {
     __shared__ FcShared sh;
     __shared__ FcStage sst;
+    // Programmatic dependent launch: when the host launches consecutive ticks with that
+    // attribute, the next tick's blocks may become resident as soon as every block of
+    // this one has started, and they stop here until this grid has finished and its
+    // stores are visible.  Only the constant tables are read before the wait.  (Without
+    // the attribute both instructions do nothing.)
+    if (kFcEarlyTrigger) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int seg_begin = cta_seg_begin[blockIdx.x], seg_end = cta_seg_begin[blockIdx.x + 1];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const long long t = ts->cnt[par];
     float* loss_out = losses ? losses + (t - t_base) : nullptr;
     const float* x_now = nullptr;
@@ -381,7 +389,7 @@ fc_tick_kernel(const FcStage* __restrict__ stages, const FcSeg* __restrict__ seg
         for (int k = blockIdx.x * kFcThreads + threadIdx.x; k < elems; k += gridDim.x * kFcThreads) dst[k] = x_now[k];
         if (blockIdx.x == 0 && threadIdx.x == 0) label_ring[t % S] = label_now;
     }
-    for (int q = cta_seg_begin[blockIdx.x]; q < cta_seg_begin[blockIdx.x + 1]; ++q) {
+    for (int q = seg_begin; q < seg_end; ++q) {
         const FcSeg seg = segs[q];
         // the stage descriptor goes through shared memory: the kernel stores to global
         // memory in its loops, so fields behind a global reference would be re-read

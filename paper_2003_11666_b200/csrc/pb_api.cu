@@ -660,9 +660,18 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
         if (h->all_fc) {
             // one launch: ingest + every stage (two when the last stage needs its own)
             prof_begin(h, 0);
-            fc_tick_kernel<<<h->nctaA, kFcThreads, 0, h->stream>>>(h->d_fc, h->d_segA, h->d_ctaA, h->d_ts, h->S, 0, par,
-                                                                  fused_last ? 1 : 0, h->label_ring, dev_losses, t_base,
-                                                                  dev_xs, dev_labels, label_value, h->in_ring, h->in_slots, elems);
+            {
+                // consecutive ticks overlap their launch latency (see the kernel's first lines)
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(h->nctaA); cfg.blockDim = dim3(kFcThreads); cfg.dynamicSmemBytes = 0; cfg.stream = h->stream;
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+                attr[0].val.programmaticStreamSerializationAllowed = 1;
+                cfg.attrs = attr; cfg.numAttrs = (fused_last && !h->profile) ? 1 : 0;
+                cudaLaunchKernelEx(&cfg, fc_tick_kernel, (const FcStage*)h->d_fc, (const FcSeg*)h->d_segA, (const int*)h->d_ctaA, h->d_ts,
+                                   h->S, 0, par, fused_last ? 1 : 0, h->label_ring, dev_losses, t_base,
+                                   dev_xs, dev_labels, label_value, h->in_ring, h->in_slots, elems);
+            }
             prof_end(h);
             h->last_launches += 1;
             if (!fused_last) {

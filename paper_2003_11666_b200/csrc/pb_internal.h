@@ -10,6 +10,10 @@ constexpr int kFcThreads = 256;
 constexpr int kFcWarps = kFcThreads / 32;
 constexpr int kFcMaxSegRows = 256;  // rows of one FC segment (bounds shared memory)
 constexpr int kFcChunksPerSweep = 2;
+// FC tick kernel: signal the next tick's launch at the START of this one (its blocks then wait
+// resident) instead of at block exit.  Measured slower on the 4-stage MLP (14.7 vs 13.2 us/tick),
+// equal on the deep one: off.
+constexpr bool kFcEarlyTrigger = false;
 constexpr int kFcBlocksPerSM = 2;         // resident blocks per SM of the FC tick kernel (register budget) = blocks of the first wave
 constexpr double kFcTailFraction = 0.10;  // share of a large stage's rows left to short second-wave blocks
 constexpr int kFcTailRows = 16;           // rows of one such block
