@@ -725,9 +725,23 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             // current weights, so it runs on its own stream beside the forward chain; only the
             // update, which overwrites the predicted weights the forward reads, waits for both.
             cudaStream_t bs = h->bwd ? h->bwd : h->stream;
-            cudaStreamWaitEvent(bs, h->ev_fork, 0);
+            // In the three-launch form the first backward step touches no parameter and no
+            // gradient table: it reads rings that were filled at least two ticks ago, the
+            // hand-offs that the previous tick's backward chain (this stream), its FC stage (side
+            // stream) and nobody else wrote, and it overwrites the scratch that the previous
+            // tick's weight gradients (third stream) were the last to read.  So it need not wait
+            // for the previous tick's update: it starts as soon as those two streams are done and
+            // runs beside the update and the ingest; the merge that follows waits for the fork.
+            const bool early_bwd = !h->post_fuse && kEarlyBackward && h->bwd && h->aux && h->side;
+            if (early_bwd) {
+                cudaStreamWaitEvent(bs, h->ev_join, 0);      // as recorded by the previous tick
+                cudaStreamWaitEvent(bs, h->ev_wjoin, 0);
+            } else {
+                cudaStreamWaitEvent(bs, h->ev_fork, 0);
+            }
             prof_begin(h, 6, bs);
             conv_bwd_post_kernel<<<post_grid, kPostThreads, 0, bs>>>(h->d_cs, h->d_pchunks, npc, h->d_bundles, h->d_ptiles[1], h->d_bcnt[1], h->d_ts, h->S, par);
+            if (early_bwd) cudaStreamWaitEvent(bs, h->ev_fork, 0);
             if (ngr > 0)
                 conv_group_merge_kernel<<<ceil_div(ngr, 8), 256, 0, bs>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 1);
             if (!h->h_dtiles[1].empty())
