@@ -99,6 +99,7 @@ struct PostChunk { int stage, grp, cl0, ncl, p0, np, idx, nidx, bundle; };   // 
 struct GroupRef { int stage, grp; };
 struct PostBundle { int stage, grp0, ngrp, nchunks, ftile0, nftiles, btile0, nbtiles; };
 constexpr int kUpdChunk = 4096;
+constexpr bool kEarlyIngest = true;        // conv networks: the sample of tick t+1 is copied in beside the update of tick t
 constexpr bool kEarlyBackward = true;      // large networks: the first backward step of tick t+1 runs beside the update of tick t
 // stream priorities of a conv tick's side chains (1 = the device's highest, 0 = default)
 constexpr int kPrioBwd = 1, kPrioAux = 1, kPrioSide = 0;

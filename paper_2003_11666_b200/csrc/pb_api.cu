@@ -683,11 +683,28 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
                 h->last_launches += 1;
             }
         } else {
-            ingest_kernel<<<ingest_blocks, 256, 0, h->stream>>>(h->d_ts, par, dev_xs, dev_labels, label_value, h->in_ring,
-                                                                h->in_slots, elems, h->label_ring, h->S, t_base);
+            // The new sample goes into the ring slot that the previous tick's weight gradient of
+            // stage 0 was the last to read, and its label into the slot the previous tick's loss
+            // read: the copy waits for those two only (side stream, after the FC stage of the
+            // previous tick) and so runs beside the previous tick's update.  The caller's buffers
+            // are ordered behind the caller's stream once per call.
+            cudaStream_t fs = h->side ? h->side : h->stream;
+            if (kEarlyIngest && h->side && h->ev_inputs) {
+                if (k == 0) {
+                    cudaEventRecord(h->ev_inputs, h->stream);
+                    cudaStreamWaitEvent(fs, h->ev_inputs, 0);
+                }
+                cudaStreamWaitEvent(fs, h->ev_wjoin, 0);         // as recorded by the previous tick
+                ingest_kernel<<<ingest_blocks, 256, 0, fs>>>(h->d_ts, par, dev_xs, dev_labels, label_value, h->in_ring,
+                                                             h->in_slots, elems, h->label_ring, h->S, t_base);
+                cudaEventRecord(h->ev_ingest, fs);
+                cudaStreamWaitEvent(h->stream, h->ev_ingest, 0);
+            } else {
+                ingest_kernel<<<ingest_blocks, 256, 0, h->stream>>>(h->d_ts, par, dev_xs, dev_labels, label_value, h->in_ring,
+                                                                    h->in_slots, elems, h->label_ring, h->S, t_base);
+            }
             // The FC stages of this tick depend only on what earlier ticks left in the rings
             // (and on the label just ingested): they run on a side stream beside the conv chain.
-            cudaStream_t fs = h->side ? h->side : h->stream;
             cudaEventRecord(h->ev_fork, h->stream);
             cudaStreamWaitEvent(fs, h->ev_fork, 0);
             prof_begin(h, 0, fs);
@@ -895,6 +912,8 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
         auto prio = [&](int level) { return (level && h->post_fuse) ? prio_greatest : prio_least; };
         e = cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, prio(kPrioSide));
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_inputs, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_ingest, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&h->bwd, cudaStreamNonBlocking, prio(kPrioBwd));
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_bjoin, cudaEventDisableTiming);
@@ -1082,6 +1101,8 @@ void pb_destroy(pb_handle* h) {
     if (h->ev_dz) cudaEventDestroy(h->ev_dz);
     if (h->ev_wjoin) cudaEventDestroy(h->ev_wjoin);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_inputs) cudaEventDestroy(h->ev_inputs);
+    if (h->ev_ingest) cudaEventDestroy(h->ev_ingest);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->staging) cudaFree(h->staging);
     cudaFree(h->arena);

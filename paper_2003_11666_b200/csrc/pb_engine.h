@@ -55,6 +55,7 @@ struct pb_handle {
     cudaStream_t aux = nullptr;                 // weight gradients, beside the data gradients
     cudaEvent_t ev_dz = nullptr, ev_wjoin = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_bjoin = nullptr;
+    cudaEvent_t ev_inputs = nullptr, ev_ingest = nullptr;   // caller's inputs ordered once per call; the sample's copy done
     int device = 0, num_sms = 0;
     unsigned flags = 0;
     float lr = 0, momentum = 0;
