@@ -136,6 +136,29 @@ def test_last_stage_too_large_to_fuse_uses_its_own_launch():
     e.destroy()
 
 
+def test_long_run_equals_single_ticks_bit_for_bit():
+    # 203 ticks through pb_run (no host involvement between ticks) against 203 pb_tick calls,
+    # with the mitigations on and in fill-and-drain mode: losses (NaN positions included),
+    # weights and velocities must be identical
+    import torch
+    for update_size in (0, 5):
+        wl = mlp([96, 80, 64, 48, 7], lr=0.002, seed=12)
+        n = 203
+        x, y = make_inputs(wl.seed, n, wl.sample_elems, wl.n_classes)
+        xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+        a, b = make_engine(wl), make_engine(wl)
+        if update_size:
+            a.set_update_size(update_size); b.set_update_size(update_size)
+        la = torch.zeros(n, device="cuda")
+        a.run(xd, yd, n, la)
+        a.sync()
+        one = np.array([b.tick(xd[t], int(y[t])) for t in range(n)], dtype=np.float32)
+        np.testing.assert_array_equal(la.cpu().numpy(), one)
+        np.testing.assert_array_equal(a.get_weights(), b.get_weights())
+        np.testing.assert_array_equal(a.get_velocity(), b.get_velocity())
+        a.destroy(); b.destroy()
+
+
 def test_consecutive_runs_and_ticks_form_one_stream_and_zero_ticks_is_a_no_op():
     import torch
     wl = mlp([48, 40, 24, 5], lr=0.003, seed=10)
