@@ -32,7 +32,7 @@ constexpr int kTcStageBytes = 16384 * 2;      // A tile + B tile
 constexpr int kTcStages = 3;                  // shared-memory stages of the operand pipeline
 constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + 1024;
 constexpr int kTcWaitLimit = 1 << 22;
-constexpr int kTcMaxK = 2048;                 // longest K loop of one tile before K is sliced
+constexpr int kTcMaxK = 3072;                 // longest K loop of one tile before K is sliced
 
 struct ConvGemmTC {
     int mode, M, N, K;
