@@ -233,9 +233,9 @@ def main():
         alg_bytes, kernel = 28.0 * (P - p_last), "update_kernel"
     # DRAM bytes per launch of that kernel from the ncu capture summarised under profiles/
     # (dram__bytes_read.sum + dram__bytes_write.sum, steady-state tick); None where not captured
-    # (profiles/fc_tick_kernel_mlp16x2048.md: 508.16 MB read + 451.67 MB written; the update
-    # kernel was captured on ResNet-50's parameters only, profiles/tick_kernels_resnet50.md)
-    traffic = {"mlp16x2048": 959.83e6, "resnet50": 508.10e6, "resnet50_112": 508.10e6}.get(args.workload)
+    # (FC tick kernel on the deep MLP: 508.17 MB read + 453.10 MB written; the update kernel
+    # was captured on ResNet-50's parameters only: 282.8 MB read + 225.3 MB written)
+    traffic = {"mlp16x2048": 961.27e6, "resnet50": 508.10e6, "resnet50_112": 508.10e6}.get(args.workload)
     achieved = alg_bytes / (k_ms / k_n * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind,
