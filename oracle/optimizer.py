@@ -43,7 +43,20 @@ class StageOptimizer:
         self.a, self.b = dtype(a), dtype(b)
         self.T = dtype(horizon if use_lwp else 0)
         self.w_form = bool(w_form)
+        self.use_sc, self.use_lwp = bool(use_sc), bool(use_lwp)
         self.version = 0        # number of updates applied so far
+
+    def set_mitigation(self, sc_delay, horizon):
+        """Other compensation strengths from now on (generalized Spike
+        Compensation with the coefficients of another delay, e.g. SC_2D;
+        Appendix "Extended Weight Prediction Horizons": T = alpha D).  The
+        state (w, v) is untouched: the next prediction uses the new T, the
+        next update the new a, b."""
+        if self.use_sc:
+            a, b = sc_coefficients(float(self.m), sc_delay)
+            self.a, self.b = self.dtype(a), self.dtype(b)
+        if self.use_lwp:
+            self.T = self.dtype(horizon)
 
     def predicted(self):
         """Weights the forward pass uses (Eq. "LWP velocity form":

@@ -241,6 +241,14 @@ class PBOracle:
             if self.record:
                 self.history[st.index].append((self.opt[-1].w.copy(), self.opt[-1].v.copy()))
 
+    def set_mitigation(self, sc_delay_scale, horizon_scale):
+        """Stage s uses the SC coefficients of delay sc_delay_scale * D_s and the
+        horizon T = horizon_scale * D_s from the next tick on."""
+        self.sc_delay_scale, self.horizon_scale = sc_delay_scale, horizon_scale
+        for st, op in zip(self.stages, self.opt):
+            D = self.delay(st.index)
+            op.set_mitigation(sc_delay_scale * D, horizon_scale * D)
+
     def get_weights(self):
         return np.concatenate([o.w for o in self.opt])
 

@@ -204,6 +204,32 @@ def test_compensation_scales_set_the_stage_constants():
         assert opt.a / 0.1 + opt.b == pytest.approx(10.0, rel=1e-12)     # total contribution unchanged
 
 
+def test_switching_the_compensation_between_ticks_changes_constants_not_state():
+    # Other strengths from some tick on: (w, v) stay as they are, the constants become those
+    # of the closed forms, and the very next prediction is w - lr (alpha_T D) v by hand.
+    wl = mlp([6, 5, 4, 3], lr=0.05)
+    o = _oracle(wl)
+    x, y = make_inputs(wl.seed, 12, wl.sample_elems, wl.n_classes)
+    for t in range(9):
+        o.tick(x[t], y[t])
+    w, v = o.get_weights().copy(), o.get_velocity().copy()
+    assert v.any()
+    o.set_mitigation(2, 0.5)
+    np.testing.assert_array_equal(o.get_weights(), w)
+    np.testing.assert_array_equal(o.get_velocity(), v)
+    for s, opt in enumerate(o.opt):
+        D = 2 * (o.S - 1 - s)
+        assert opt.a == pytest.approx(0.9 ** (2 * D), rel=1e-12)
+        assert opt.b == pytest.approx((1 - 0.9 ** (2 * D)) / 0.1, rel=1e-12, abs=1e-15)
+        np.testing.assert_allclose(opt.predicted(), opt.w - 0.05 * (0.5 * D) * opt.v, rtol=1e-14, atol=0)
+    # switched at tick 0 it is the same machine as one built with those scales
+    a = _oracle(wl); a.set_mitigation(2, 0.5)
+    b = _oracle(wl, sc_delay_scale=2, horizon_scale=0.5)
+    for t in range(12):
+        assert a.tick(x[t], y[t]) == b.tick(x[t], y[t]) or t < o.S - 1
+    np.testing.assert_array_equal(a.get_weights(), b.get_weights())
+
+
 @pytest.mark.parametrize("make,N", [(lambda: mlp([10, 8, 6, 4], lr=0.05), 3), (tiny_cnn, 4),
                                     (tiny_resnet, 2), (lambda: tiny_resnet(bottleneck=True), 5),
                                     (lambda: mlp([9, 5], lr=0.05), 1)])
