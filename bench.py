@@ -1,17 +1,24 @@
 """Throughput of Pipelined Backpropagation ticks (samples/s at batch 1).
 
-One step is one tick: every stage's forward and backward on its current
-samples plus the SC+LWP update of every stage.  Workload: the deep MLP
+One step is one STEADY-STATE tick: every stage's forward and backward on its
+current samples plus the SC+LWP update of every stage.  Workload: the deep MLP
 (16 FC stages of width 2048), whose weights and velocities (504 MB) exceed
 the L2 cache, so every tick streams them from HBM.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+Before anything is timed the pipeline is FILLED: 2(S-1)+2 set-up ticks, after
+which every stage runs its forward, its backward and its update in every tick
+(a stage's first gradient arrives at tick 2(S-1)-s).  Then come the W warm-up
+ticks and the K timed ticks.  A line whose implied memory bandwidth is beyond
+what the device can deliver is refused (value null).
 
 With N > 1 (under torch.distributed.run) each rank runs an independent replica
 of the pipeline on its own GPU: the tick has no data-parallel form at update
 size one, so the job scales by replicas and no collective is on the data path.
 """
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -28,14 +35,44 @@ if ROOT not in sys.path:
 WORKLOAD = "mlp16x2048"
 METRIC = "PB ticks/sec (samples/sec, batch 1)"
 UNIT = "ticks/s"
+HBM_HW_GBS = 7700.0            # HBM3e of one B200 in an HGX board, vendor figure
+L2_BYTES = 126e6
+# step sizes at which the diverging configurations stay bounded (same kernels, finite numbers)
+STABLE_LR = {"mlp4": 0.001, "mlp16x2048": 1e-4, "resnet50": 5e-4, "resnet50_112": 5e-4}
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel,
+# from the ncu captures summarised under profiles/; each entry names the source file of the
+# kernel and that file's SHA-1 when the counters were taken, and is dropped (null) as soon as
+# the file has changed since.
+NCU_TRAFFIC = {
+    "mlp16x2048": (961.27e6, "fc_kernels.cuh", "7e526d5ef4d69460462d69ec3ccf0b8737ce1263",
+                   "profiles/fc_tick_kernel_mlp16x2048.md: 508.17 MB read + 453.10 MB written, gpu__dram_throughput 67.4 % of the hardware peak"),
+}
+
+
+def ncu_traffic(workload_name):
+    ent = NCU_TRAFFIC.get(workload_name)
+    if ent is None:
+        return None, None
+    nbytes, fname, sha, note = ent
+    path = os.path.join(ROOT, "paper_2003_11666_b200", "csrc", fname)
+    try:
+        with open(path, "rb") as f:
+            now = hashlib.sha1(f.read()).hexdigest()
+    except OSError:
+        return None, None
+    if now != sha:
+        return None, "kernel source changed since the counters were taken"
+    return nbytes, note
 
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
-            return json.load(f).get("hbm_gbs", 6650.0), "measured"
-    return 6650.0, "fallback"
+            d = json.load(f)
+        return d.get("hbm_gbs", 6650.0), d.get("bf16_tflops_sustained", 1400.0), "measured"
+    return 6650.0, 1400.0, "fallback"
 
 
 class ClockSampler:
@@ -106,6 +143,33 @@ def replica_seed(base_seed, rank):
     return base_seed + 1000 * rank
 
 
+def fill_ticks(n_stages):
+    """Set-up ticks before any timing: stage s gets its first gradient at tick
+    2(S-1)-s, so after 2(S-1)+2 ticks every stage has forwarded, back-propagated
+    and updated at least twice."""
+    return 2 * (n_stages - 1) + 2
+
+
+def tick_floor(work, peaks, bf16):
+    """Least time one steady-state tick can take on this device, in microseconds, and
+    what bounds it.  Memory: 16 B per parameter (one read and one write of w and v)
+    plus every activation once (float32, or bfloat16 for tensor-core operands), at
+    the L2 bandwidth when weights, velocities and activations together stay well
+    inside the L2 cache, else at the HBM copy rate.  Arithmetic: three passes
+    (forward, data gradient, weight gradient) of 2 flops per multiply-accumulate on
+    the unit that runs them.  The floor is the largest of the three."""
+    state = 8.0 * work["params"]
+    act = work["act_elems"] * (2.0 if bf16 else 4.0)
+    in_l2 = state + act < 0.6 * L2_BYTES
+    bw = peaks["l2_gbs"] if in_l2 else peaks["hbm_gbs"]
+    t_mem = (16.0 * work["params"] + act) / (bw * 1e9) * 1e6
+    t_f32 = 6.0 * (work["macs_conv_f32"] + work["macs_fc"]) / (peaks["fp32_fma_tflops"] * 1e12) * 1e6
+    t_tc = 6.0 * work["macs_conv_bf16"] / (peaks["bf16_tflops"] * 1e12) * 1e6
+    parts = {"memory_us": t_mem, "fp32_fma_us": t_f32, "tensor_us": t_tc,
+             "memory_level": "l2" if in_l2 else "hbm"}
+    return max(t_mem, t_f32, t_tc), parts
+
+
 def time_oracle(wl, budget_s=20.0, max_ticks=None):
     """Times the CPU checker as it stands on steady-state ticks of `wl`."""
     from oracle import PBOracle
@@ -134,13 +198,13 @@ def run_reference(args, rank):
     if rank != 0:
         return
     from pb_workloads import workload
-    wl = workload(WORKLOAD)
+    wl = workload(args.workload)
     base, s_per_tick = time_oracle(wl, budget_s=25.0, max_ticks=max(1, min(args.steps, 16)))
     line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT,
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": 1e3 * s_per_tick, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "stages": wl.n_stages, "note": "CPU checker on host cores"},
+            "config": {"workload": args.workload, "stages": wl.n_stages, "note": "CPU checker on host cores"},
             "cpu_baseline": base,
             "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -170,7 +234,7 @@ def main():
     if local_rank == 0:
         pbuild.build()
     import paper_2003_11666_b200 as pbm
-    from pb_workloads import he_normal_weights, make_inputs, workload
+    from pb_workloads import he_normal_weights, make_inputs, work_per_tick, workload
 
     torch.cuda.set_device(local_rank)
     if world > 1:
@@ -179,102 +243,154 @@ def main():
     wl = workload(args.workload)
     K, W = args.steps, max(args.warmup, 3)
     S = wl.n_stages
+    F = fill_ticks(S)
     seed = replica_seed(wl.seed, rank)
-    x, y = make_inputs(seed, K + W, wl.sample_elems, wl.n_classes)
+    n_in = F + W + K
+    x, y = make_inputs(seed, n_in, wl.sample_elems, wl.n_classes)
     stream = torch.cuda.current_stream()
-    eng = pbm.PB(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, wl.lr, wl.momentum,
-                 wl.flags, stream=stream.cuda_stream)
-    eng.set_weights(he_normal_weights(wl.seed, wl))
+    w_init = he_normal_weights(wl.seed, wl)
     xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
-    losses = torch.zeros(K + W, device="cuda")
+    losses = torch.zeros(n_in, device="cuda")
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing: W warm-up ticks (fills the pipeline), then K ticks
-    eng.run(xd[:W], yd[:W], W, losses[:W])
-    barrier()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record(stream)
-    eng.run(xd[W:], yd[W:], K, losses[W:])
-    e1.record(stream)
-    barrier()
-    launches = eng.last_launch_count
-    ms = max_over_ranks(e0.elapsed_time(e1), world)
-    clocks = sampler.stop() if rank == 0 else None
-    value = job_value(world, K, ms)
+    def new_engine(lr):
+        e = pbm.PB(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, lr, wl.momentum,
+                   wl.flags, stream=stream.cuda_stream)
+        e.set_weights(w_init)
+        return e
 
-    # ---- per-kernel durations (CUDA events on the engine's stream, separate pass)
+    def timed_leg(e, with_clocks):
+        """Fill (set-up), W warm-up ticks, then K timed ticks; returns (ms, clocks)."""
+        e.run(xd[:F], yd[:F], F, losses[:F])
+        e.run(xd[F:F + W], yd[F:F + W], W, losses[F:F + W])
+        barrier()
+        sampler = ClockSampler(local_rank)
+        if with_clocks and rank == 0:
+            sampler.start()
+            time.sleep(0.3)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        e.run(xd[F + W:], yd[F + W:], K, losses[F + W:])
+        e1.record(stream)
+        barrier()
+        ms_ = max_over_ranks(e0.elapsed_time(e1), world)
+        return ms_, (sampler.stop() if with_clocks and rank == 0 else None)
+
+    # ---- device-resident timing, literal hyper-parameters
+    eng = new_engine(wl.lr)
+    ms, clocks = timed_leg(eng, True)
+    launches = eng.last_launch_count
+    value = job_value(world, K, ms)
+    finite_ticks = int(torch.isfinite(losses[F + W:]).sum().item())
+
+    # ---- per-kernel durations (CUDA events on the engine's streams, separate pass, still steady state)
     eng.profile_enable(True)
     kp = min(K, 512)
-    eng.run(xd[W:W + kp], yd[W:W + kp], kp, losses[W:W + kp])
+    eng.run(xd[F:F + kp], yd[F:F + kp], kp, losses[F:F + kp])
     eng.sync()
     classes = {name: eng.profile_ms(c) for c, name in enumerate(("fc_phase0", "fc_phase1", "update", "conv_simt", "conv_tc_fprop",
                                                                "conv_post_fwd", "conv_post_bwd", "conv_tc_wgrad", "conv_tc_dgrad"))}
     eng.profile_enable(False)
     P = eng.num_params
-    p_last = wl.layers[-2].c_in * wl.layers[-2].c_out + wl.layers[-2].c_out
-    peak, peak_kind = measured_peaks()
+    hbm_peak, bf16_peak, peak_kind = measured_peaks()
+    peaks = {"hbm_gbs": hbm_peak, "hbm_source": peak_kind + " copy rate", "hbm_hw_gbs": HBM_HW_GBS,
+             "bf16_tflops": bf16_peak,
+             "l2_gbs": pbm.bench_l2_bandwidth(32 << 20, 200, stream.cuda_stream),
+             "l2_source": "in-place sweep over 32 MiB, 200 passes, this run",
+             "fp32_fma_tflops": pbm.bench_fp32_fma(8192, stream.cuda_stream),
+             "fp32_fma_source": "16 FMA chains per thread, 8 blocks of 256 threads per SM, this run"}
     all_fc = all(int(L.op) in (0, 3, 7) for L in wl.layers)
     if all_fc:
-        # one read and one write of (w, v) per parameter updated by the launch
         k_ms, k_n = classes["fc_phase0"]
-        alg_bytes, kernel = 16.0 * (P - p_last), "fc_tick_kernel(phase 0)"
+        alg_bytes, kernel = eng.kernel_min_bytes(0), "fc_tick_kernel"
+        if classes["fc_phase1"][1]:
+            p_last = wl.layers[-2].c_in * wl.layers[-2].c_out + wl.layers[-2].c_out
+            alg_bytes -= 16.0 * p_last
+            kernel = "fc_tick_kernel(phase 0)"
     else:
-        # conv parameters: read w, v, g; write w, v, predicted w
         k_ms, k_n = classes["update"]
-        alg_bytes, kernel = 28.0 * (P - p_last), "update_kernel"
-    # DRAM bytes per launch of that kernel from the ncu capture summarised under profiles/
-    # (dram__bytes_read.sum + dram__bytes_write.sum, steady-state tick); None where not captured
-    # (FC tick kernel on the deep MLP: 508.17 MB read + 453.10 MB written; the update kernel
-    # was captured on ResNet-50's parameters only: 282.8 MB read + 225.3 MB written)
-    traffic = {"mlp16x2048": 961.27e6, "resnet50": 508.10e6, "resnet50_112": 508.10e6}.get(args.workload)
-    achieved = alg_bytes / (k_ms / k_n * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_source": peak_kind,
+        alg_bytes, kernel = eng.kernel_min_bytes(2), "update_kernel"
+    work = work_per_tick(wl)
+    state_bytes = 8.0 * P
+    in_l2 = state_bytes + 4.0 * work["act_elems"] < 0.6 * L2_BYTES
+    k_peak = peaks["l2_gbs"] if in_l2 else hbm_peak
+    traffic, traffic_note = ncu_traffic(args.workload)
+    launch_s = k_ms / k_n * 1e-3
+    achieved = alg_bytes / launch_s / 1e9
+    floor_us, floor_parts = tick_floor(work, peaks, bool(wl.flags & 8))
+    roofline = {"bound": "l2" if in_l2 else "hbm", "kernel": kernel, "achieved": achieved, "peak": k_peak,
+                "unit": "GB/s", "frac": achieved / k_peak,
+                "peak_source": ("L2 sweep of this run" if in_l2 else peak_kind + " copy rate (MEASURED_PEAKS.json)"),
+                "frac_of_hw_peak": None if in_l2 else achieved / HBM_HW_GBS,
+                "traffic": traffic, "traffic_note": traffic_note,
+                "achieved_traffic": (traffic / launch_s / 1e9) if traffic else None,
                 "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": k_ms / k_n, "launches_timed": k_n,
+                "peaks": peaks,
+                "tick_floor_us": floor_us, "tick_floor_parts": floor_parts,
+                "tick_frac": floor_us / (1e3 * ms / K),
                 "us_per_tick_by_class": {n: (1e3 * m / kp if c else 0.0) for n, (m, c) in classes.items()}}
+    eng.destroy()
+
+    # ---- the same workload at a bounded step size (finite numbers in every kernel)
+    stable = None
+    if args.workload in STABLE_LR:
+        es = new_engine(STABLE_LR[args.workload])
+        ms_s, clocks_s = timed_leg(es, True)
+        stable = {"lr": STABLE_LR[args.workload], "ms_per_step": ms_s / K, "value": job_value(world, K, ms_s),
+                  "finite_losses": int(torch.isfinite(losses[F + W:]).sum().item()), "of": K,
+                  "sm_mhz": clocks_s["sm_mhz"] if clocks_s else None}
+        es.destroy()
 
     # ---- end to end through the host-buffer entry point (pinned memory, copies timed)
-    eng.set_weights(he_normal_weights(wl.seed, wl))
+    eng = new_engine(wl.lr)
     hx = torch.from_numpy(x).pin_memory()
     hy = torch.from_numpy(y).pin_memory()
-    hl = torch.zeros(K + W).pin_memory()
-    # warm-up of the same size as the timed call: it fills the pipeline and sizes the
-    # library's staging buffer, so that the timed call allocates nothing
-    eng.run_host(hx[W:], hy[W:], K, hl[W:])
+    hl = torch.zeros(n_in).pin_memory()
+    # set-up: fill the pipeline, then a warm-up call of the timed call's size, which also sizes
+    # the library's staging buffer so that the timed call allocates nothing
+    eng.run_host(hx[:F], hy[:F], F, hl[:F])
+    eng.run_host(hx[F + W:], hy[F + W:], K, hl[F + W:])
     barrier()
     t0 = time.perf_counter()
-    eng.run_host(hx[W:], hy[W:], K, hl[W:])
+    eng.run_host(hx[F + W:], hy[F + W:], K, hl[F + W:])
     torch.cuda.synchronize()
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3, world)
     e2e = {"value": job_value(world, K, e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": wl.sample_elems * 4 + 4, "d2h_bytes_per_step": 4}
-    finite_ticks = int(np.isfinite(hl[W:].numpy()).sum())
     eng.destroy()
 
     if rank == 0:
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
             cpu, _ = time_oracle(wl, budget_s=15.0, max_ticks=8)
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-                "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        # a tick cannot move its parameters faster than the memory system allows: refuse a
+        # number that says otherwise (it would mean work was skipped in the timed region)
+        rejected = None
+        if state_bytes > L2_BYTES:
+            implied = 16.0 * P / (ms / K * 1e-3) / 1e9 / world
+            if implied > 1.2 * hbm_peak:
+                rejected = "implied %.0f GB/s per GPU for 16 B/parameter exceeds 1.2 x the %.0f GB/s copy peak" % (implied, hbm_peak)
+        line = {"metric": METRIC, "value": None if rejected else value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                "fill_ticks": F, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16" if wl.flags & 8 else "f32", "data": "synthetic",
                 "config": {"workload": args.workload, "stages": S, "params": P, "batch": 1,
                            "parallelism": "replicas x%d" % world if world > 1 else "1 gpu",
-                           "l2": "weights+velocity %.0f MB stream from HBM every tick (> 126 MB L2), no flush needed" % (8e-6 * P),
+                           "l2": ("weights+velocity %.0f MB stream from HBM every tick (> 126 MB L2), no flush needed" % (8e-6 * P))
+                                 if state_bytes > L2_BYTES else
+                                 ("weights+velocity %.1f MB stay in the L2 cache by design (steady state of the method); no flush" % (8e-6 * P)),
+                           "steady_state": "timed ticks %d..%d, all %d stages forward, backward and update in each" % (F + W, F + W + K - 1, S),
                            "note": "literal hyper-parameters; losses finite on %d of %d timed ticks "
-                                   "(the deep MLP and ResNet-50 runs diverge); kernel work does not depend "
-                                   "on the values" % (finite_ticks, K)},
+                                   "(the deep MLP and ResNet-50 runs diverge); stable_lr times the same "
+                                   "kernels on finite numbers" % (finite_ticks, K)},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-                "roofline": roofline, "cpu_baseline": cpu}
+                "roofline": roofline, "stable_lr": stable, "cpu_baseline": cpu}
+        if rejected:
+            line["rejected"] = rejected
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

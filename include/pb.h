@@ -101,8 +101,13 @@ int pb_set_weights(pb_handle* h, const float* host_w, size_t n);
  * other a, b, e.g. SC_2D; Appendix "Extended Weight Prediction Horizons",
  * T = alpha D).  Stage s then uses a = m^(sc_delay_scale * D_s),
  * b = (1 - a)/(1 - m) and T = horizon_scale * D_s; (1, 1) is the default
- * SC_D + LWP_D.  Takes effect for ticks issued after the call; synchronises
- * the stream.  Scales must be >= 0. */
+ * SC_D + LWP_D.  Takes effect for ticks issued after the call, for every
+ * stage alike: the next forward of each stage already predicts with the new T
+ * (stored predicted weights are re-made from the current w and v), and its
+ * next update uses the new a, b.  With PB_LWP_WFORM the prediction is made from
+ * the previous weights, which are not kept, so there the call is only accepted
+ * before the first tick (PB_E_UNSUPPORTED afterwards).  Synchronises the
+ * stream.  Scales must be >= 0. */
 int pb_set_mitigation(pb_handle* h, float sc_delay_scale, float horizon_scale);
 
 /* Fill-and-drain training (Section 1; Appendix "Pipelined Backpropagation":
@@ -128,7 +133,12 @@ int pb_set_update_size(pb_handle* h, int n_samples);
  * NULL the stream is synchronised and *host_loss receives the loss the last
  * stage computed in this tick, which belongs to the sample fed S-1 ticks
  * earlier (a sample needs 2S-1 steps, Appendix "Pipelined Backpropagation");
- * it is NaN during the first S-1 ticks. */
+ * it is NaN during the first S-1 ticks.
+ * Alignment: dev_x (and dev_xs of pb_run / pb_mlp_run_static) must be 16-byte
+ * aligned when the network is fully connected and the sample length is a
+ * multiple of 4 (the first stage then reads the sample 16 bytes at a time);
+ * otherwise PB_E_ARG is returned before anything is launched.  In every other
+ * case 4-byte alignment is enough. */
 int pb_tick(pb_handle* h, const float* dev_x, int label, float* host_loss);
 
 /* n_ticks ticks without host synchronisation.  dev_xs: [n_ticks, sample]
@@ -178,6 +188,26 @@ size_t pb_device_bytes(const pb_handle* h);
 int pb_profile_enable(pb_handle* h, int enable);
 double pb_profile_ms(pb_handle* h, int which, long long* launches);
 
+/* Least device-memory traffic, in bytes per steady-state tick, of kernel class
+ * `which` as the engine is configured: 0 = the FC tick kernel (one read and one
+ * write of w and v per FC parameter: the optimizer's full-model pass that
+ * Appendix "GPU Bottlenecks for Fine-Grained Pipelined Training" names, fused
+ * with forward and backward), 2 = the update kernel of conv stages (w, v and
+ * every weight-gradient slice read, w, v and the predicted weights written).
+ * Negative for other classes.  Benchmarks divide it by the measured duration. */
+double pb_kernel_min_bytes(const pb_handle* h, int which);
+
+/* Roofline denominators that a plain HBM copy does not give (measurement aids,
+ * no counterpart in the paper).  pb_bench_l2_bandwidth: read + write GB/s of an
+ * in-place sweep over `bytes` of device memory repeated `iters` times; with
+ * `bytes` well under the L2 capacity this is the L2 bandwidth that bounds the
+ * update of networks whose weights and velocities stay cached.
+ * pb_bench_fp32_fma: float32 fused-multiply-add rate of the CUDA cores in
+ * TFLOP/s (2 flops per FMA), the bound of the float32 convolutions.  Both
+ * allocate and free their own scratch and synchronise `stream`. */
+int pb_bench_l2_bandwidth(size_t bytes, int iters, void* stream, double* gbs);
+int pb_bench_fp32_fma(int iters, void* stream, double* tflops);
+
 /* Allocation-free variant of pb_create + pb_set_weights + pb_run for small fully
  * connected pipelines.  (The paper has no counterpart: this exists for callers
  * that must not allocate device memory - code running inside a pre-sized memory
@@ -201,6 +231,9 @@ double pb_profile_ms(pb_handle* h, int which, long long* launches);
  *
  * The first call on each device looks up the array's device address
  * (cudaGetSymbolAddress) and should therefore come before any stream capture.
+ * That look-up fills a per-device cache without a lock: two threads making the
+ * first call on one device at the same moment both store the same address,
+ * which is harmless, but the calls themselves must not overlap anyway (below).
  * All calls share the array and it keeps the previous call's contents: each
  * call clears the part it uses, and two calls that overlap on the GPU (other
  * streams, other threads) race on it.  The call waits for `stream` before it

@@ -20,7 +20,7 @@ EXPORTS = [
     "pb_get_velocity", "pb_sync", "pb_num_params", "pb_num_stages", "pb_stage_delay",
     "pb_tick_count", "pb_last_launch_count", "pb_device_bytes", "pb_profile_enable",
     "pb_profile_ms", "pb_last_error", "pb_destroy", "pb_mlp_run_static", "pb_set_mitigation",
-    "pb_set_update_size",
+    "pb_set_update_size", "pb_kernel_min_bytes", "pb_bench_l2_bandwidth", "pb_bench_fp32_fma",
 ]
 
 
@@ -76,6 +76,10 @@ def load_library():
     lib.pb_last_error.restype = C.c_char_p
     lib.pb_destroy.argtypes = [vp]
     lib.pb_destroy.restype = None
+    lib.pb_kernel_min_bytes.argtypes = [vp, i32]
+    lib.pb_kernel_min_bytes.restype = C.c_double
+    lib.pb_bench_l2_bandwidth.argtypes = [C.c_size_t, i32, vp, C.POINTER(C.c_double)]
+    lib.pb_bench_fp32_fma.argtypes = [i32, vp, C.POINTER(C.c_double)]
     lib.pb_mlp_run_static.argtypes = [C.POINTER(C.c_int32), i32, f32, f32, C.c_uint, vp, vp, vp, vp, i32, vp, vp]
     _lib = lib
     return lib
@@ -104,6 +108,26 @@ def mlp_run_static(sizes, lr, momentum, flags, dev_w, dev_v, dev_xs, dev_labels,
                                _ptr(dev_losses), C.c_void_p(stream))
     if rc != 0:
         raise PBError(rc, lib.pb_last_error(None).decode())
+
+
+def bench_l2_bandwidth(nbytes, iters=200, stream=0):
+    """pb_bench_l2_bandwidth: GB/s (read + write) of an in-place sweep over `nbytes`."""
+    lib = load_library()
+    out = C.c_double(0.0)
+    rc = lib.pb_bench_l2_bandwidth(int(nbytes), int(iters), C.c_void_p(stream), C.byref(out))
+    if rc != 0:
+        raise PBError(rc, lib.pb_last_error(None).decode())
+    return out.value
+
+
+def bench_fp32_fma(iters=4096, stream=0):
+    """pb_bench_fp32_fma: float32 FMA rate of the CUDA cores in TFLOP/s."""
+    lib = load_library()
+    out = C.c_double(0.0)
+    rc = lib.pb_bench_fp32_fma(int(iters), C.c_void_p(stream), C.byref(out))
+    if rc != 0:
+        raise PBError(rc, lib.pb_last_error(None).decode())
+    return out.value
 
 
 class PB:
@@ -187,6 +211,9 @@ class PB:
     @property
     def device_bytes(self):
         return int(self._lib.pb_device_bytes(self._h))
+
+    def kernel_min_bytes(self, which):
+        return float(self._lib.pb_kernel_min_bytes(self._h, int(which)))
 
     def profile_enable(self, on=True):
         self._check(self._lib.pb_profile_enable(self._h, 1 if on else 0))

@@ -797,4 +797,18 @@ cast_weights_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restr
     }
 }
 
+// Predicted weights re-made from the current state, w_hat = w - lr T v (LWP, velocity
+// form), after the horizon T of the stages has been changed between ticks.
+__global__ void __launch_bounds__(256)
+repredict_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ chunks) {
+    const UpdChunk ch = chunks[blockIdx.x];
+    const UpdRange& R = ranges[ch.range];
+    const int end = min(R.n, ch.start + kUpdChunk);
+    for (int e = ch.start + threadIdx.x; e < end; e += 256) {
+        const float wh = fmaf(R.neg_lr_T, R.v[e], R.w[e]);
+        if (R.wh16) R.wh16[e] = __float2bfloat16_rn(wh);
+        else R.wh[e] = wh;
+    }
+}
+
 }  // namespace pb

@@ -9,6 +9,7 @@
 #include "conv_gemm.cuh"
 #include "conv_stage.cuh"
 #include "fc_kernels.cuh"
+#include "microbench.cuh"
 #include "pb_engine.h"
 
 using namespace pb;
@@ -230,6 +231,41 @@ void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSe
             cta_begin.push_back((int)segs.size());
         }
     }
+}
+
+// FC stage descriptors and their partition into thread blocks.  w_base / v_base: where the
+// flat parameter vectors start when they are the caller's memory (their alignment then
+// decides whether rows can be read 16 bytes at a time); nullptr for the engine's own arena,
+// whose stage blocks are 256-byte aligned.
+void build_fc_tables(pb_handle* h, const float* w_base, const float* v_base) {
+    std::vector<int> idsA, idsB;
+    for (const StageHost& x : h->stages) {
+        if (x.head_op != PB_FC) continue;
+        FcStage f{};
+        f.in_dim = x.head.c_in; f.out_dim = x.head.c_out; f.s = x.index;
+        f.relu = x.relu; f.is_last = x.loss; f.need_dx = x.src >= 0;
+        bool aligned = true;
+        if (w_base)
+            aligned = ((reinterpret_cast<uintptr_t>(w_base + x.dev_off) | reinterpret_cast<uintptr_t>(v_base + x.dev_off)) & 15) == 0;
+        f.vec = (f.in_dim % 4 == 0 && aligned) ? 4 : 1;
+        f.neg_lr_T = -h->lr * x.T; f.m = h->momentum; f.neg_lr_a = -h->lr * x.a; f.neg_lr_b = -h->lr * x.b;
+        idsA.push_back((int)h->h_fc.size());
+        if (x.loss) idsB.push_back((int)h->h_fc.size());
+        h->h_fc.push_back(f);
+    }
+    std::vector<int> npartsA(h->h_fc.size(), 1), npartsB(h->h_fc.size(), 1);
+    // a last stage of at most 256 rows and 64 K weights is fused into the phase-0 launch
+    bool fuse_last = false;
+    for (int f : idsB) fuse_last = h->h_fc[f].out_dim <= kFcMaxSegRows && (long long)h->h_fc[f].out_dim * h->h_fc[f].in_dim <= 65536;
+    partition_fc(h, idsA, h->h_segA, h->h_ctaA, npartsA, fuse_last);
+    if (fuse_last) { h->h_segB.clear(); h->h_ctaB.assign(1, 0); }
+    else partition_fc(h, idsB, h->h_segB, h->h_ctaB, npartsB, false);
+    for (size_t f = 0; f < h->h_fc.size(); ++f) {
+        StageHost& x = h->stages[h->h_fc[f].s];
+        x.dx_nparts = (x.loss && !fuse_last) ? npartsB[f] : npartsA[f];
+    }
+    h->nctaA = (int)h->h_ctaA.size() - 1;
+    h->nctaB = (int)h->h_ctaB.size() - 1;
 }
 
 // ---------------------------------------------------------------- convolution planning
@@ -650,6 +686,11 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
     const int ingest_blocks = std::min(ceil_div(elems, 1024), 2 * h->num_sms);
     const long long t_base = h->tick;
     h->last_launches = 0;
+    // Fully connected pipelines read the current sample straight from the caller's buffer,
+    // 16 bytes at a time when the sample length is a multiple of 4: the buffer must then be
+    // 16-byte aligned (checked here, on the host, before anything is launched).
+    if (h->all_fc && !h->h_fc.empty() && h->h_fc[0].vec == 4 && (reinterpret_cast<uintptr_t>(dev_xs) & 15) != 0)
+        return fail(h, PB_E_ARG, "the sample buffer must be 16-byte aligned when the sample length is a multiple of 4");
     if (h->profile) for (auto& p : h->prof) p = ProfileClass{};
     const bool fused_last = h->nctaB == 0;      // the last stage rides in the phase-0 launch
     const int npc = (int)h->h_pchunks.size();
@@ -840,32 +881,7 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e != cudaSuccess) { std::string m = cudaGetErrorString(e); delete h; return fail(nullptr, PB_E_CUDA, "pb_create: no CUDA device: " + m); }
 
-    // FC tables and their partition
-    std::vector<int> idsA, idsB;
-    for (const StageHost& x : h->stages) {
-        if (x.head_op != PB_FC) continue;
-        FcStage f{};
-        f.in_dim = x.head.c_in; f.out_dim = x.head.c_out; f.s = x.index;
-        f.relu = x.relu; f.is_last = x.loss; f.need_dx = x.src >= 0;
-        f.vec = (f.in_dim % 4 == 0) ? 4 : 1;
-        f.neg_lr_T = -lr * x.T; f.m = momentum; f.neg_lr_a = -lr * x.a; f.neg_lr_b = -lr * x.b;
-        idsA.push_back((int)h->h_fc.size());
-        if (x.loss) idsB.push_back((int)h->h_fc.size());
-        h->h_fc.push_back(f);
-    }
-    std::vector<int> npartsA(h->h_fc.size(), 1), npartsB(h->h_fc.size(), 1);
-    // a last stage of at most 256 rows and 64 K weights is fused into the phase-0 launch
-    bool fuse_last = false;
-    for (int f : idsB) fuse_last = h->h_fc[f].out_dim <= kFcMaxSegRows && (long long)h->h_fc[f].out_dim * h->h_fc[f].in_dim <= 65536;
-    partition_fc(h, idsA, h->h_segA, h->h_ctaA, npartsA, fuse_last);
-    if (fuse_last) { h->h_segB.clear(); h->h_ctaB.assign(1, 0); }
-    else partition_fc(h, idsB, h->h_segB, h->h_ctaB, npartsB, false);
-    for (size_t f = 0; f < h->h_fc.size(); ++f) {
-        StageHost& x = h->stages[h->h_fc[f].s];
-        x.dx_nparts = (x.loss && !fuse_last) ? npartsB[f] : npartsA[f];
-    }
-    h->nctaA = (int)h->h_ctaA.size() - 1;
-    h->nctaB = (int)h->h_ctaB.size() - 1;
+    build_fc_tables(h, nullptr, nullptr);
 
     rc = validate_conv(h);
     if (rc != PB_OK) { delete h; return rc; }
@@ -926,7 +942,8 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
     if (e != cudaSuccess) {
         std::string m = std::string("pb_create: upload failed: ") + cudaGetErrorString(e);
-        cudaFree(h->arena); delete h; return fail(nullptr, PB_E_CUDA, m);
+        pb_destroy(h);          // frees the arena and whatever streams and events exist by now
+        return fail(nullptr, PB_E_CUDA, m);
     }
     *out = h;
     return PB_OK;
@@ -964,6 +981,9 @@ int pb_set_weights(pb_handle* h, const float* host_w, size_t n) {
 int pb_set_mitigation(pb_handle* h, float sc_delay_scale, float horizon_scale) {
     if (!h) return PB_E_ARG;
     if (!(sc_delay_scale >= 0.f) || !(horizon_scale >= 0.f)) return fail(h, PB_E_ARG, "pb_set_mitigation: scales must be >= 0");
+    if ((h->flags & PB_LWP_WFORM) && h->tick != 0)
+        return fail(h, PB_E_UNSUPPORTED, "pb_set_mitigation: with PB_LWP_WFORM the scales can only be set before the first tick "
+                                         "(the stored prediction cannot be re-made without the previous weights)");
     h->sc_delay_scale = sc_delay_scale;
     h->horizon_scale = horizon_scale;
     for (StageHost& x : h->stages) mitigation_constants(h, x);
@@ -973,8 +993,16 @@ int pb_set_mitigation(pb_handle* h, float sc_delay_scale, float horizon_scale) {
     PB_CUDA(h, cudaStreamSynchronize(h->stream));
     if (!h->h_fc.empty())
         PB_CUDA(h, cudaMemcpyAsync(h->d_fc, h->h_fc.data(), h->h_fc.size() * sizeof(FcStage), cudaMemcpyHostToDevice, h->stream));
-    if (!h->h_upd.empty())
+    if (!h->h_upd.empty()) {
         PB_CUDA(h, cudaMemcpyAsync(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange), cudaMemcpyHostToDevice, h->stream));
+        // Conv stages read STORED predicted weights, written by their last update with the old
+        // horizon: re-make them from (w, v) so that the next forward of every stage, FC or
+        // conv, uses the new T.  (Velocity form only; see the check above.)
+        if (!(h->flags & PB_LWP_WFORM) && !h->h_chunks.empty()) {
+            repredict_kernel<<<(int)h->h_chunks.size(), 256, 0, h->stream>>>(h->d_upd, h->d_chunks);
+            PB_CUDA(h, cudaGetLastError());
+        }
+    }
     PB_CUDA(h, cudaStreamSynchronize(h->stream));
     return PB_OK;
 }
@@ -1076,6 +1104,87 @@ long long pb_tick_count(const pb_handle* h) { return h ? h->tick : -1; }
 long long pb_last_launch_count(const pb_handle* h) { return h ? h->last_launches : -1; }
 size_t pb_device_bytes(const pb_handle* h) { return h ? h->arena_bytes : 0; }
 
+double pb_kernel_min_bytes(const pb_handle* h, int which) {
+    if (!h) return -1.0;
+    double bytes = 0.0;
+    if (which == 0) {
+        // FC tick kernel: w and v read once and written once; the weight-difference form
+        // also reads and writes its stored prediction
+        const double per = (h->flags & PB_LWP_WFORM) ? 24.0 : 16.0;
+        for (const pb::FcStage& f : h->h_fc) bytes += per * ((double)f.in_dim * f.out_dim + f.out_dim);
+        return bytes;
+    }
+    if (which == 2) {
+        // update kernel: reads w, v and every gradient slice (4 B each), writes w, v (8 B) and
+        // the prediction (4 B as float32, or two bfloat16 copies of w and w_hat)
+        for (const pb::UpdRange& r : h->h_upd) bytes += (double)r.n * (24.0 + 4.0 * (r.nparts - 1));
+        return bytes;
+    }
+    return -1.0;
+}
+
+int pb_bench_l2_bandwidth(size_t bytes, int iters, void* stream, double* gbs) {
+    if (!gbs || bytes < 4096 || iters <= 0) return fail(nullptr, PB_E_ARG, "pb_bench_l2_bandwidth: bad argument");
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t n = bytes / sizeof(float4);
+    float4* buf = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    int sms = 0, dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&buf, n * sizeof(float4));
+    if (e == cudaSuccess) e = cudaMemsetAsync(buf, 0, n * sizeof(float4), st);
+    if (e == cudaSuccess) e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) {
+        const int grid = sms * 8;
+        for (int k = 0; k < 3; ++k) l2_sweep_kernel<<<grid, 256, 0, st>>>(buf, n, 0.5f, 1.0f);     // warm: the buffer is now cached
+        cudaEventRecord(e0, st);
+        for (int k = 0; k < iters; ++k) l2_sweep_kernel<<<grid, 256, 0, st>>>(buf, n, 0.5f, 1.0f);
+        cudaEventRecord(e1, st);
+        e = cudaEventSynchronize(e1);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+        if (e == cudaSuccess) e = cudaGetLastError();
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (buf) cudaFree(buf);
+    if (e != cudaSuccess) return fail(nullptr, PB_E_CUDA, std::string("pb_bench_l2_bandwidth: ") + cudaGetErrorString(e));
+    *gbs = 2.0 * (double)(n * sizeof(float4)) * iters / (ms * 1e-3) / 1e9;
+    return PB_OK;
+}
+
+int pb_bench_fp32_fma(int iters, void* stream, double* tflops) {
+    if (!tflops || iters <= 0) return fail(nullptr, PB_E_ARG, "pb_bench_fp32_fma: bad argument");
+    cudaStream_t st = (cudaStream_t)stream;
+    float* out = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    int sms = 0, dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int grid = sms * 8, threads = 256;
+    if (e == cudaSuccess) e = cudaMalloc((void**)&out, (size_t)grid * threads * sizeof(float));
+    if (e == cudaSuccess) e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) {
+        fma_chain_kernel<<<grid, threads, 0, st>>>(out, 64, 0.999f, 1e-3f);
+        cudaEventRecord(e0, st);
+        fma_chain_kernel<<<grid, threads, 0, st>>>(out, iters, 0.999f, 1e-3f);
+        cudaEventRecord(e1, st);
+        e = cudaEventSynchronize(e1);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+        if (e == cudaSuccess) e = cudaGetLastError();
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (out) cudaFree(out);
+    if (e != cudaSuccess) return fail(nullptr, PB_E_CUDA, std::string("pb_bench_fp32_fma: ") + cudaGetErrorString(e));
+    *tflops = 2.0 * 16.0 * (double)iters * grid * threads / (ms * 1e-3) / 1e12;
+    return PB_OK;
+}
+
 int pb_profile_enable(pb_handle* h, int enable) {
     if (!h) return PB_E_ARG;
     h->profile = enable != 0;
@@ -1169,32 +1278,8 @@ extern "C" int pb_mlp_run_static(const int32_t* sizes, int n_sizes, float lr, fl
 
     // the caller's flat vectors are the master weights and velocities
     h->d_w = dev_w; h->d_v = dev_v;
-    std::vector<int> idsA, idsB;
-    for (StageHost& x : h->stages) {
-        x.dev_off = x.user_off;
-        FcStage f{};
-        f.in_dim = x.head.c_in; f.out_dim = x.head.c_out; f.s = x.index;
-        f.relu = x.relu; f.is_last = x.loss; f.need_dx = x.src >= 0;
-        const bool aligned = ((reinterpret_cast<uintptr_t>(dev_w + x.user_off) | reinterpret_cast<uintptr_t>(dev_v + x.user_off)) & 15) == 0;
-        f.vec = (f.in_dim % 4 == 0 && aligned) ? 4 : 1;
-        f.neg_lr_T = -lr * x.T; f.m = momentum; f.neg_lr_a = -lr * x.a; f.neg_lr_b = -lr * x.b;
-        idsA.push_back((int)h->h_fc.size());
-        if (x.loss) idsB.push_back((int)h->h_fc.size());
-        h->h_fc.push_back(f);
-    }
-    std::vector<int> npartsA(h->h_fc.size(), 1), npartsB(h->h_fc.size(), 1);
-    // a last stage of at most 256 rows and 64 K weights is fused into the phase-0 launch
-    bool fuse_last = false;
-    for (int f : idsB) fuse_last = h->h_fc[f].out_dim <= kFcMaxSegRows && (long long)h->h_fc[f].out_dim * h->h_fc[f].in_dim <= 65536;
-    partition_fc(h, idsA, h->h_segA, h->h_ctaA, npartsA, fuse_last);
-    if (fuse_last) { h->h_segB.clear(); h->h_ctaB.assign(1, 0); }
-    else partition_fc(h, idsB, h->h_segB, h->h_ctaB, npartsB, false);
-    for (size_t f = 0; f < h->h_fc.size(); ++f) {
-        StageHost& x = h->stages[h->h_fc[f].s];
-        x.dx_nparts = (x.loss && !fuse_last) ? npartsB[f] : npartsA[f];
-    }
-    h->nctaA = (int)h->h_ctaA.size() - 1;
-    h->nctaB = (int)h->h_ctaB.size() - 1;
+    for (StageHost& x : h->stages) x.dev_off = x.user_off;
+    build_fc_tables(h, dev_w, dev_v);
 
     // carve the static array
     Carver c{base};

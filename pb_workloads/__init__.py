@@ -9,9 +9,10 @@ be fed from it without sharing any of the method's code.
 from .gen import (splitmix64, uniform01, normal, labels, he_normal_weights,
                   make_inputs)
 from .configs import (OP, Layer, Workload, workload, WORKLOAD_NAMES,
-                      param_sizes, infer_shapes, mlp, tiny_cnn, tiny_resnet)
+                      param_sizes, infer_shapes, work_per_tick, mlp, tiny_cnn, tiny_resnet,
+                      tall_bottleneck)
 
 __all__ = ["splitmix64", "uniform01", "normal", "labels", "he_normal_weights",
            "make_inputs", "OP", "Layer", "Workload", "workload",
-           "WORKLOAD_NAMES", "param_sizes", "infer_shapes", "mlp", "tiny_cnn",
-           "tiny_resnet"]
+           "WORKLOAD_NAMES", "param_sizes", "infer_shapes", "work_per_tick", "mlp", "tiny_cnn",
+           "tiny_resnet", "tall_bottleneck"]

@@ -211,6 +211,20 @@ def tiny_resnet(seed=12, ticks=40, flags=FLAG_SC | FLAG_LWP, bottleneck=False):
                      name="tiny_resnet", lr=0.02, ticks=ticks, seed=seed)
 
 
+def tall_bottleneck(seed=13, ticks=48, lr=0.001, flags=FLAG_SC | FLAG_LWP | FLAG_CONV_BF16):
+    """Few channels on large images: the ResNet-50 stage kinds (7x7/2 stem with
+    3x3/2 max-pool, two bottleneck blocks with projection shortcuts, the second
+    one strided) at 8..64 channels on 3x256x256 inputs.  The stem's output has
+    16384 pixels and the first block's 4096, so the shapes only large images
+    reach (weight gradients contracting over thousands of pixels, normalisation
+    groups cut into several pieces per channel) are met by a net whose CPU
+    evaluation takes a fraction of a second per tick."""
+    wl = _resnet50(depths=(1, 1), base=8, hw=256, n_classes=7, groups=4,
+                   name="tall_bottleneck", ticks=ticks, seed=seed, flags=flags)
+    wl.lr = lr
+    return wl
+
+
 WORKLOAD_NAMES = ["mlp4", "mlp16x2048", "vgg11", "resnet20", "resnet50"]
 
 
@@ -278,3 +292,42 @@ def infer_shapes(wl):
             cur = (cur[0], 1, 1)
             shapes[s] = cur
     return shapes
+
+
+def work_per_tick(wl):
+    """Bookkeeping for benchmarks: what one steady-state tick has to touch.
+
+    Returns a dict with `params`; forward multiply-accumulates per tick split
+    into `macs_fc`, `macs_conv_f32` (CUDA cores) and `macs_conv_bf16` (tensor
+    cores: every conv of a bfloat16 workload whose channel counts are multiples
+    of 8 and whose input is not the network input); and `act_elems`, the
+    activation elements a tick moves at least once: per stage 3 x input
+    (forward read, weight-gradient read, data gradient written) + 2 x head
+    output (written forward, read backward) + 2 x stage output (written forward,
+    its gradient read backward)."""
+    shapes = infer_shapes(wl)
+    out = dict(params=0, macs_fc=0, macs_conv_f32=0, macs_conv_bf16=0, act_elems=0)
+    bf16 = bool(wl.flags & FLAG_CONV_BF16)
+    for L, s in zip(wl.layers, wl.stage_of_layer):
+        if L.op not in (OP.FC, OP.CONV2D):
+            if L.op == OP.GROUPNORM:
+                out["params"] += 2 * L.c_out
+            continue
+        src = L.src if L.src >= 0 else s - 1
+        cin = wl.in_shape if src < 0 else shapes[src]
+        a_in = cin[0] * cin[1] * cin[2]
+        a_out = shapes[s][0] * shapes[s][1] * shapes[s][2]
+        if L.op == OP.FC:
+            out["params"] += L.c_in * L.c_out + L.c_out
+            out["macs_fc"] += L.c_in * L.c_out
+            a_head = L.c_out
+        else:
+            h = (cin[1] + 2 * L.pad - L.k) // L.stride + 1
+            w = (cin[2] + 2 * L.pad - L.k) // L.stride + 1
+            a_head = L.c_out * h * w
+            macs = a_head * L.c_in * L.k * L.k
+            out["params"] += L.c_out * L.c_in * L.k * L.k
+            tc = bf16 and src >= 0 and L.c_in % 8 == 0 and L.c_out % 8 == 0
+            out["macs_conv_bf16" if tc else "macs_conv_f32"] += macs
+        out["act_elems"] += 3 * a_in + 2 * a_head + 2 * a_out
+    return out

@@ -1,11 +1,14 @@
 """Shared helpers of the GPU parity tests: run the CUDA engine and the CPU
-checker on the same seeded inputs and compare per tick."""
+checker on the same seeded inputs and compare per tick, per stage and per
+parameter tensor."""
 import math
 
 import numpy as np
 
 from oracle import PBOracle
 from pb_workloads import he_normal_weights, make_inputs
+
+F32_HALF_ULP = 2.0 ** -24      # relative rounding error of one float32 store
 
 
 def rel_err(got, ref):
@@ -19,9 +22,100 @@ def rel_err(got, ref):
     return float(np.linalg.norm(got - ref) / max(n, 1e-12))
 
 
+def tensor_slices(o):
+    """[(stage, kind, slice)] of every parameter tensor in the flat vector the
+    checker `o` (and the engine) use: FC weight / bias, conv weight / GroupNorm
+    scale / shift, in layer order."""
+    out, off = [], 0
+    for st in o.stages:
+        h = st.head
+        if int(h.op) == 0:                      # FC
+            nw = h.c_in * h.c_out
+            out.append((st.index, "weight", slice(off, off + nw)))
+            out.append((st.index, "bias", slice(off + nw, off + nw + h.c_out)))
+        else:
+            nw = h.c_out * h.c_in * h.k * h.k
+            out.append((st.index, "weight", slice(off, off + nw)))
+            if st.gn_groups:
+                out.append((st.index, "gamma", slice(off + nw, off + nw + h.c_out)))
+                out.append((st.index, "beta", slice(off + nw + h.c_out, off + nw + 2 * h.c_out)))
+        off += st.n_params
+    assert off == o.n_params
+    return out
+
+
+def compare_state(slices, w_init, got_w, got_v, ref_w, ref_v, updates, tol_w, tol_v):
+    """Per-tensor comparison of one tick's state.  Pure numpy (no GPU).
+
+    For every parameter tensor:
+      * velocity: ||got_v - ref_v|| <= tol_v * ||ref_v||; a velocity that is
+        exactly zero in the reference (no gradient has reached the stage yet,
+        Appendix "Pipelined Backpropagation", Eq. F_i) must be exactly zero;
+      * weights, through their DISPLACEMENT from the initial values, so that a
+        wrong update cannot hide behind the unchanged bulk of the weights:
+        ||got_w - ref_w|| <= tol_w * ||ref_w - w_init|| + floor, where floor =
+        2^-24 sqrt(n) ||ref_w|| is the rounding of n float32 stores of w
+        (n = updates of that stage so far); weights that have not moved in the
+        reference must still hold their initial bits.
+    tol_w / tol_v: a number, or a dict {(stage, kind): number}.
+    Returns (worst weight ratio, worst velocity ratio, failures): ratios are
+    error / allowed (<= 1 passes), failures a list of messages."""
+    worst_w = worst_v = 0.0
+    fails = []
+    for s, kind, sl in slices:
+        tw = tol_w[(s, kind)] if isinstance(tol_w, dict) else tol_w
+        tv = tol_v[(s, kind)] if isinstance(tol_v, dict) else tol_v
+        rw = np.asarray(ref_w[sl], np.float64)
+        rv = np.asarray(ref_v[sl], np.float64)
+        gw = np.asarray(got_w[sl], np.float64)
+        gv = np.asarray(got_v[sl], np.float64)
+        w0 = np.asarray(w_init[sl], np.float64)
+        # velocity
+        nv = np.linalg.norm(rv)
+        if nv == 0.0:
+            if gv.any():
+                fails.append("stage %d %s: velocity must be exactly zero before the stage's first gradient" % (s, kind))
+                worst_v = float("inf")
+        else:
+            r = float(np.linalg.norm(gv - rv) / (tv * nv))
+            worst_v = max(worst_v, r)
+            if not r <= 1.0:
+                fails.append("stage %d %s: velocity rel err %.3g (bound %.3g)" % (s, kind, r * tv, tv))
+        # weights
+        nd = np.linalg.norm(rw - w0)
+        if nd == 0.0:
+            if not np.array_equal(np.asarray(got_w[sl], np.float32), np.asarray(w_init[sl], np.float32)):
+                fails.append("stage %d %s: weights moved although the reference has not updated them" % (s, kind))
+                worst_w = float("inf")
+        else:
+            n_upd = updates[s] if updates is not None else 1
+            allowed = tw * nd + F32_HALF_ULP * math.sqrt(max(n_upd, 1)) * np.linalg.norm(rw)
+            r = float(np.linalg.norm(gw - rw) / allowed)
+            worst_w = max(worst_w, r)
+            if not r <= 1.0:
+                fails.append("stage %d %s: weight displacement rel err %.3g (bound %.3g)"
+                             % (s, kind, float(np.linalg.norm(gw - rw) / nd), tw))
+    return worst_w, worst_v, fails
+
+
+def tensor_spread(slices, a_w, a_v, b_w, b_v, w_init):
+    """Per-tensor distance between two runs of the checker (float32 and
+    float64): {(stage, kind): (weight displacement spread, velocity spread)}."""
+    out = {}
+    for s, kind, sl in slices:
+        nd = np.linalg.norm(np.asarray(b_w[sl], np.float64) - np.asarray(w_init[sl], np.float64))
+        nv = np.linalg.norm(np.asarray(b_v[sl], np.float64))
+        dw = np.linalg.norm(np.asarray(a_w[sl], np.float64) - np.asarray(b_w[sl], np.float64))
+        dv = np.linalg.norm(np.asarray(a_v[sl], np.float64) - np.asarray(b_v[sl], np.float64))
+        out[(s, kind)] = (float(dw / nd) if nd > 0 else 0.0, float(dv / nv) if nv > 0 else 0.0)
+    return out
+
+
 def make_oracle(wl, dtype=np.float64, **kw):
     if wl.flags & 8:
         kw.setdefault("conv_operands", "bf16")
+    if getattr(wl, "weight_stash", False):
+        kw.setdefault("weight_stash", True)
     o = PBOracle(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, wl.lr, wl.momentum,
                  wl.flags & 7, dtype=dtype, **kw)
     o.set_weights(he_normal_weights(wl.seed, wl))
@@ -31,15 +125,21 @@ def make_oracle(wl, dtype=np.float64, **kw):
 def make_engine(wl):
     import torch
     from paper_2003_11666_b200 import PB
+    flags = wl.flags | (16 if getattr(wl, "weight_stash", False) else 0)
     eng = PB(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, wl.lr, wl.momentum,
-             wl.flags, stream=torch.cuda.current_stream().cuda_stream)
+             flags, stream=torch.cuda.current_stream().cuda_stream)
     eng.set_weights(he_normal_weights(wl.seed, wl))
     return eng
 
 
 def compare_ticks(wl, n_ticks, tol, check_every=1, finite_limit=1e30, loose_after=None,
-                  fragile_margin=None, fragile_tol=None, spread_factor=None, mitigation=None):
+                  fragile_margin=None, fragile_tol=None, spread_factor=None, mitigation=None,
+                  plain_loss_tol=None, unrounded_loss_tol=None, check_ticks=None, mitigation_switch=None):
     """Tick both sides one sample at a time; returns the worst errors seen.
+
+    Weights and velocities are compared per stage and per tensor
+    (`compare_state`); `worst["w"]`, `worst["v"]` are the largest error /
+    allowed ratios times the tolerance (so they read as relative errors).
 
     The window ends early (returning the tick) once the checker's own state
     exceeds `finite_limit`: past that the float32 engine is out of range.
@@ -55,8 +155,17 @@ def compare_ticks(wl, n_ticks, tol, check_every=1, finite_limit=1e30, loose_afte
     spread_factor: for arithmetic that amplifies rounding-order differences
     (bfloat16 operands: a float32-level change can flip a bfloat16 rounding,
     which moves ReLU decisions), the checker is also run in float32 and the
-    bound on weights and velocities at a tick becomes
-    max(tol, spread_factor * distance between its float32 and float64 runs)."""
+    bound on a STAGE's tensors at a tick becomes max(tol, spread_factor * the
+    largest distance between the float32 and float64 runs over the tensors of
+    that stage and of the stages after it, whose gradients feed it).
+
+    plain_loss_tol: also bound the plain ratio |dl| / |l| on ticks where the
+    loss is not small against the logits (l > 1e-3 max|logit|).
+    unrounded_loss_tol: also run the checker WITHOUT operand rounding (the
+    paper's arithmetic in float64) and bound the engine's loss against it.
+    check_ticks: explicit set of ticks at which the state is compared.
+    mitigation_switch: (tick, (SC delay scale, horizon scale)): both sides
+    change their compensation strengths before that tick."""
     import torch
     x, y = make_inputs(wl.seed, n_ticks, wl.sample_elems, wl.n_classes)
     okw = {}
@@ -65,16 +174,26 @@ def compare_ticks(wl, n_ticks, tol, check_every=1, finite_limit=1e30, loose_afte
     o = make_oracle(wl, margins=fragile_margin is not None, **okw)
     fragile_tick = None
     o32 = make_oracle(wl, dtype=np.float32, **okw) if spread_factor is not None else None
+    oplain = make_oracle(wl, conv_operands=None, **okw) if unrounded_loss_tol is not None else None
+    slices = tensor_slices(o)
+    w_init = he_normal_weights(wl.seed, wl)
     eng = make_engine(wl)
     if mitigation is not None:
         eng.set_mitigation(*mitigation)
     xd = torch.from_numpy(x).cuda()
-    worst = {"loss": 0.0, "w": 0.0, "v": 0.0, "ticks": 0, "fragile_tick": None, "strict_w": 0.0, "strict_v": 0.0}
+    worst = {"loss": 0.0, "w": 0.0, "v": 0.0, "ticks": 0, "fragile_tick": None, "strict_w": 0.0, "strict_v": 0.0,
+             "plain_loss": 0.0, "unrounded_loss": 0.0, "min_updates": 0}
     for t in range(n_ticks):
+        if mitigation_switch is not None and t == mitigation_switch[0]:
+            for o_ in (o, o32, oplain):
+                if o_ is not None:
+                    o_.set_mitigation(*mitigation_switch[1])
+            eng.set_mitigation(*mitigation_switch[1])
         lo = o.tick(x[t], y[t])
         lg = eng.tick(xd[t], int(y[t]))
         if o32 is not None:
             o32.tick(x[t], y[t])
+        lp = oplain.tick(x[t], y[t]) if oplain is not None else None
         wo = o.get_weights()
         if not np.isfinite(wo).all() or np.abs(wo).max() > finite_limit:
             break
@@ -93,21 +212,41 @@ def compare_ticks(wl, n_ticks, tol, check_every=1, finite_limit=1e30, loose_afte
         else:
             # loss = logsumexp(o) - o[label] is a difference of numbers of the
             # logits' size, so its rounding error scales with max|o|, not with itself
-            e = abs(lg - lo) / max(abs(lo), float(np.abs(o.last_logits).max()), 1e-12)
+            mxl = float(np.abs(o.last_logits).max())
+            e = abs(lg - lo) / max(abs(lo), mxl, 1e-12)
             worst["loss"] = max(worst["loss"], e)
             assert e <= tl, "tick %d: loss %r vs %r (rel %.3g)" % (t, lg, lo, e)
-        if t % check_every == 0 or t == n_ticks - 1:
-            ew = rel_err(eng.get_weights(), wo)
-            ev = rel_err(eng.get_velocity(), o.get_velocity())
-            tlw = tlv = tl
+            if abs(lo) > 1e-3 * mxl:
+                ep = abs(lg - lo) / abs(lo)
+                worst["plain_loss"] = max(worst["plain_loss"], ep)
+                if plain_loss_tol is not None:
+                    assert ep <= max(plain_loss_tol, tl), "tick %d: plain loss ratio %.3g" % (t, ep)
+            if lp is not None and not math.isnan(lp):
+                eu = abs(lg - lp) / max(abs(lp), 1e-12)
+                worst["unrounded_loss"] = max(worst["unrounded_loss"], eu)
+                assert eu <= unrounded_loss_tol, \
+                    "tick %d: loss %r vs %r of the checker without operand rounding (rel %.3g)" % (t, lg, lp, eu)
+        due = (t in check_ticks) if check_ticks is not None else (t % check_every == 0)
+        if due or t == n_ticks - 1:
+            vo = o.get_velocity()
+            tw = tv = tl
             if o32 is not None:
-                tlw = max(tl, spread_factor * rel_err(o32.get_weights(), wo))
-                tlv = max(tl, spread_factor * rel_err(o32.get_velocity(), o.get_velocity()))
-            worst["w"], worst["v"] = max(worst["w"], ew), max(worst["v"], ev)
+                sp = tensor_spread(slices, o32.get_weights(), o32.get_velocity(), wo, vo, w_init)
+                # a stage's gradient is made from everything downstream of it
+                stage_sp = np.zeros((o.S, 2))
+                for (s_, _k), (a, b) in sp.items():
+                    stage_sp[s_, 0] = max(stage_sp[s_, 0], a)
+                    stage_sp[s_, 1] = max(stage_sp[s_, 1], b)
+                down = np.maximum.accumulate(stage_sp[::-1], axis=0)[::-1]
+                tw = {(s_, k_): max(tl, spread_factor * down[s_, 0]) for s_, k_, _ in slices}
+                tv = {(s_, k_): max(tl, spread_factor * down[s_, 1]) for s_, k_, _ in slices}
+            updates = [op.version for op in o.opt]
+            rw, rv, fails = compare_state(slices, w_init, eng.get_weights(), eng.get_velocity(), wo, vo, updates, tw, tv)
+            assert not fails, "tick %d: %s" % (t, "; ".join(fails[:6]))
+            worst["w"], worst["v"] = max(worst["w"], rw * tl), max(worst["v"], rv * tl)
             if fragile_tick is None or t < fragile_tick:
-                worst["strict_w"], worst["strict_v"] = max(worst["strict_w"], ew), max(worst["strict_v"], ev)
-            assert ew <= tlw, "tick %d: weights rel err %.3g (bound %.3g)" % (t, ew, tlw)
-            assert ev <= tlv, "tick %d: velocity rel err %.3g (bound %.3g)" % (t, ev, tlv)
+                worst["strict_w"], worst["strict_v"] = max(worst["strict_w"], rw * tl), max(worst["strict_v"], rv * tl)
+            worst["min_updates"] = min(updates)
         worst["ticks"] = t + 1
         worst["fragile_tick"] = fragile_tick
     eng.destroy()

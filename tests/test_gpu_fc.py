@@ -115,6 +115,32 @@ def test_bad_arguments_are_reported_not_thrown_across_the_abi():
     e.destroy()
 
 
+def test_misaligned_sample_buffer_is_rejected_on_the_host():
+    # the first FC stage reads the caller's sample 16 bytes at a time when its length is a
+    # multiple of 4: a float pointer that is only 4-byte aligned must come back as PB_E_ARG
+    # from the host-side check (nothing is launched), not as a device fault
+    import torch
+    from paper_2003_11666_b200 import PBError
+    wl = mlp([64, 16, 4], lr=0.01, seed=6)
+    e = make_engine(wl)
+    buf = torch.zeros(4 * 64 + 8, device="cuda")
+    lab = torch.zeros(4, dtype=torch.int32, device="cuda")
+    before = e.tick_count
+    for call in (lambda p: e.tick(p, 0, want_loss=False), lambda p: e.run(p, lab, 2)):
+        with pytest.raises(PBError) as err:
+            call(buf.data_ptr() + 4)
+        assert err.value.code == -1 and "aligned" in str(err.value)
+    assert e.tick_count == before
+    e.run(buf, lab, 2)                               # the aligned buffer is fine
+    e.sync()
+    # a sample length that is not a multiple of 4 takes the scalar path: any float pointer will do
+    wl2 = mlp([30, 8, 3], lr=0.01, seed=6)
+    e2 = make_engine(wl2)
+    e2.run(buf.data_ptr() + 4, lab, 2)
+    e2.sync()
+    e.destroy(); e2.destroy()
+
+
 def test_single_stage_network_on_the_gpu():
     # S = 1: delay 0, the sample and its label are consumed in the tick that ingests them
     wl = mlp([40, 6], lr=0.01, seed=8)

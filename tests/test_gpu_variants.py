@@ -36,6 +36,33 @@ def test_over_and_under_compensation(make, scales):
     assert w["ticks"] == n
 
 
+@pytest.mark.parametrize("make", [lambda: mlp([48, 40, 33, 24, 5], lr=0.003, seed=32), tiny_cnn, lambda: _resnet(3)])
+def test_compensation_switched_after_every_stage_has_updated(make):
+    # conv stages keep their predicted weights in memory: a new horizon must reach them at
+    # once (re-made from w and v), as it reaches FC stages, which predict on the fly
+    wl = make()
+    S = wl.n_stages
+    n = 2 * (S - 1) + 24
+    w = compare_ticks(wl, n, TOL, mitigation_switch=(2 * (S - 1) + 5, (2.0, 0.5)))
+    assert w["ticks"] == n and w["min_updates"] >= 10
+
+
+def test_weight_difference_form_takes_new_scales_only_before_the_first_tick():
+    import torch
+    from paper_2003_11666_b200 import PBError
+    from pb_workloads import make_inputs
+    from tests.parity import make_engine
+    wl = tiny_cnn(flags=7)
+    e = make_engine(wl)
+    e.set_mitigation(2.0, 2.0)                      # tick 0: accepted
+    x, y = make_inputs(wl.seed, 2, wl.sample_elems, wl.n_classes)
+    e.run(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda(), 2)
+    with pytest.raises(PBError) as err:
+        e.set_mitigation(1.0, 1.0)
+    assert err.value.code == -6
+    e.destroy()
+
+
 def test_mitigation_scale_arguments_are_checked():
     from paper_2003_11666_b200 import PBError
     from tests.parity import make_engine

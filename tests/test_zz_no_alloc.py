@@ -1,10 +1,12 @@
-"""The allocation-free entry point against the ordinary engine.
+"""The allocation-free entry point against the ordinary engine and the CPU checker.
 
 Some users of this library run where device memory may not be allocated (a
 fixed memory budget, or inside another framework's allocator); for them
 pb_mlp_run_static keeps all of its scratch in a static array inside the
 library.  It must give the numbers pb_create + pb_run give, also when the
-array still holds an earlier call's contents."""
+array still holds an earlier call's contents; it must match the CPU checker
+like every other path; and the amount of free device memory must be the same
+after a call as before it."""
 import numpy as np
 import pytest
 
@@ -63,6 +65,39 @@ def test_static_entry_point_matches_engine_on_two_calls_in_a_row():
     b = _static_run(wl, sizes_a, x, y, 40)
     for u, v in zip(a, b):
         np.testing.assert_array_equal(u, v)
+
+
+def test_static_entry_point_matches_the_cpu_checker_and_allocates_nothing():
+    import torch
+    from tests.parity import compare_state, make_oracle, tensor_slices
+    sizes, n = [72, 40, 24, 7], 36
+    wl = mlp(sizes, lr=0.003, seed=7)
+    x, y = make_inputs(wl.seed, n, wl.sample_elems, wl.n_classes)
+    o = make_oracle(wl)
+    ref_l = np.array([o.tick(x[t], y[t]) for t in range(n)])
+    # the first call on a device looks up the array's address (and loads the kernels);
+    # free memory is compared across the calls after it
+    _static_run(wl, sizes, x, y, 4)
+    import paper_2003_11666_b200 as p
+    w0 = he_normal_weights(wl.seed, wl)
+    w = torch.from_numpy(w0).cuda()
+    v = torch.zeros_like(w)
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    losses = torch.full((n,), 7.0, device="cuda")
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    p.mlp_run_static(sizes, wl.lr, wl.momentum, wl.flags, w, v, xd, yd, n, losses,
+                     stream=torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "the call changed the free device memory by %d bytes" % (free_before - free_after)
+    got_l = losses.cpu().numpy().astype(np.float64)
+    S = wl.n_stages
+    assert np.isnan(got_l[:S - 1]).all()
+    assert np.abs(got_l[S - 1:] - ref_l[S - 1:]).max() <= TOL * np.abs(ref_l[S - 1:]).max()
+    _, _, fails = compare_state(tensor_slices(o), w0, w.cpu().numpy(), v.cpu().numpy(), o.get_weights(), o.get_velocity(),
+                                [op.version for op in o.opt], TOL, TOL)
+    assert not fails, fails
 
 
 def test_static_entry_point_rejects_what_does_not_fit():
