@@ -22,6 +22,12 @@ enters, and only when it is empty are all stages updated, with the mean of the
 N gradients and plain SGD with momentum; one update takes N + 2S - 2 ticks.
 Every sample then sees the same weights forward and backward, so the result
 is ordinary mini-batch SGD with momentum.
+
+Weight stashing (`weight_stash`; Appendix "Pipelined Backpropagation", Eq.
+"W_{i+1} = W_i - eta grad L(x_i; F_i)", the PipeDream rule the paper compares
+with): every stage keeps the weights it used for a sample's forward pass and
+uses those same weights for that sample's backward pass, so the gradient is
+the true gradient at F_i; the update still lands on the current weights.
 """
 import numpy as np
 
@@ -189,7 +195,7 @@ class PBOracle:
     def __init__(self, layer_list, stage_of_layer, in_shape, n_classes, lr,
                  momentum, flags=FLAG_SC | FLAG_LWP, dtype=np.float64,
                  sc_delay_scale=1, horizon_scale=1, record=False, conv_operands=None,
-                 margins=False, update_size=0):
+                 margins=False, update_size=0, weight_stash=False):
         """conv_operands: None, or "bf16" to round both operands of every
         convolution product (forward, data gradient, weight gradient) to
         bfloat16 while accumulating in `dtype`.  margins: log in
@@ -216,6 +222,8 @@ class PBOracle:
         self.opt = None
         self.t = 0
         self.out, self.stash, self.dsum, self.labels = {}, {}, {}, {}
+        self.weight_stash = bool(weight_stash)
+        self.wstash = {}          # (stage, sample) -> weights of that sample's forward pass
         self.record = record
         self.fwd_version, self.bwd_version, self.grads = {}, {}, {}
         self.history = [[] for _ in self.stages]   # (w, v) after each version
@@ -248,6 +256,16 @@ class PBOracle:
         for st, op in zip(self.stages, self.opt):
             D = self.delay(st.index)
             op.set_mitigation(sc_delay_scale * D, horizon_scale * D)
+
+    def load_state(self, flat_w, flat_v):
+        """Overwrites every stage's weights and velocities (flat vectors in
+        layer order) without touching the pipeline: samples in flight keep what
+        they stored.  Bookkeeping only; used to start a tick from a given state."""
+        off = 0
+        for st, op in zip(self.stages, self.opt):
+            op.w = np.array(flat_w[off:off + st.n_params], dtype=self.dtype)
+            op.v = np.array(flat_v[off:off + st.n_params], dtype=self.dtype)
+            off += st.n_params
 
     def get_weights(self):
         return np.concatenate([o.w for o in self.opt])
@@ -283,6 +301,8 @@ class PBOracle:
             skip_in = self.out[(st.skip[0], i)] if st.skip is not None else None
             y, stash = st.forward(theta_hat[s], self.out[(st.src, i)], skip_in)
             self.out[(s, i)], self.stash[(s, i)] = y, stash
+            if self.weight_stash:
+                self.wstash[(s, i)] = theta_hat[s]
             if st.margins:
                 self.min_margin[(s, i)] = stash["margin"]
             if self.record:
@@ -304,7 +324,8 @@ class PBOracle:
                 continue
             dy = self.dsum.pop((s, j))
             skip_shape = self.stages[st.skip[0]].out_shape if st.skip is not None else None
-            g, dx, dskip = st.backward(self.opt[s].w, self.stash.pop((s, j)), dy,
+            theta_b = self.wstash.pop((s, j)) if self.weight_stash else self.opt[s].w
+            g, dx, dskip = st.backward(theta_b, self.stash.pop((s, j)), dy,
                                        st.src >= 0, skip_shape)
             if dx is not None:
                 self._accumulate((st.src, j), dx)

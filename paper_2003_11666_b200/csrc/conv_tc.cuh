@@ -2,19 +2,36 @@
 //
 // The three GEMMs of a convolution stage run on the 5th-generation tensor
 // cores: 128 x BN tiles of D accumulate in tensor memory (fp32), operands are
-// bfloat16 and are gathered straight from the NHWC activation ring / gradient
-// scratch / KRSC weight copies into 128-byte-swizzled shared-memory tiles by
-// the block's threads (implicit im2col: no staging buffer in global memory).
+// bfloat16 in 128-byte-swizzled shared-memory tiles.
 //   fprop  D[c_out, pixel]      A = predicted weights (K-major)   B = im2col(x)      (K-major)
 //   dgrad  D[c_in, in pixel]    A = weights, read transposed (MN-major)  B = scattered dz (K-major)
 //   wgrad  D[c_out, (r,s,c_in)] A = dz (MN-major)                 B = im2col(x)      (MN-major)
 // with K ordered (r, s, channel) so that 8 consecutive K (one 16-byte unit)
-// are 8 consecutive channels of one pixel.  The gather uses 16-byte asynchronous
-// copies (cp.async, zero-filled outside the image) into a three-stage ring: two
-// K-chunks of 64 are in flight while the tensor core works on a third.
-// Every mbarrier wait is bounded; on expiry the block records an error, skips
-// its stores, frees its tensor memory and returns.
+// are 8 consecutive channels of one pixel.
+//
+// One persistent block per SM works through a list of tiles (all stages of the
+// tick, balanced on the host by their number of K chunks) with three kinds of warps:
+//   * producer warps (4) fill a three-stage ring of K chunks of 64.  An operand
+//     that is a plain matrix in memory (the weights in all three GEMMs, dz as
+//     the A operand of wgrad, and the activations / dz of 1x1 stride-1
+//     convolutions) is fetched by ONE thread with a bulk tensor copy (TMA, 2-D
+//     or 3-D tiles, 128-byte swizzle, zero fill outside the matrix) that
+//     completes on the stage's "full" barrier; an operand that needs the
+//     implicit im2col (3x3 taps, strides, padding) is gathered by all producer
+//     threads with 16-byte cp.async copies, zero-filled outside the image;
+//   * one MMA warp: a single thread waits for "full", issues four
+//     tcgen05.mma (K = 16 each) per chunk and commits them to the stage's
+//     "empty" barrier, and after a tile's last chunk to the accumulator's barrier;
+//   * epilogue warps (4, one per quarter of the tensor-memory lanes) drain the
+//     accumulator with tcgen05.ld while the MMA warp already works on the next
+//     tile in the second accumulator (2 x 128 columns of tensor memory).
+// The forward GEMM of a stage whose K fits one slice also produces what the
+// normalisation needs: it writes the conv output straight into its ring slot and,
+// per channel and column tile, count / mean / M2 of the values it has in registers.
+// Every barrier wait is bounded; on expiry the block records an error, stops
+// issuing work, waits for its copies in flight, frees its tensor memory and returns.
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "conv_types.h"
@@ -22,17 +39,18 @@
 namespace pb {
 
 constexpr int kTcChunk = 64;                  // K elements per shared-memory stage
-constexpr int kTcThreads = 256;                // 8 warps gather; warps 0-3 / 4-7 split the columns in the epilogue
-constexpr int kTcRowsPerPass = kTcThreads / 8; // K-major tiles: rows filled per pass (8 units of 16 bytes per row)
-constexpr int kTcPasses = 128 / kTcRowsPerPass;
-constexpr int kTcKPerPass = kTcThreads / 16;   // MN-major tiles of width 128: k rows filled per pass
-constexpr int kTcKPasses = kTcChunk / kTcKPerPass;
 constexpr int kTcBM = 128;
 constexpr int kTcStageBytes = 16384 * 2;      // A tile + B tile
 constexpr int kTcStages = 3;                  // shared-memory stages of the operand pipeline
 constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + 1024;
+constexpr int kTcEpiWarps = 4;                // warps 0-3: quarter q of the tensor-memory lanes belongs to warp q
+constexpr int kTcProducers = 128;             // warps 4-7
+constexpr int kTcMmaWarp = 8;
+constexpr int kTcThreads = 32 * (kTcMmaWarp + 1);
+constexpr int kTcTmemCols = 256;              // two accumulators of 128 columns
 constexpr int kTcWaitLimit = 1 << 22;
-constexpr int kTcMaxK = 3072;                 // longest K loop of one tile before K is sliced
+constexpr int kTcMaxK = 3072;                 // longest K loop of one dgrad / wgrad tile before K is sliced
+constexpr int kTcMaxKFprop = 8192;            // ... of a forward tile (a single slice lets the epilogue finish the stage's statistics)
 
 struct ConvGemmTC {
     int mode, M, N, K;
@@ -44,6 +62,16 @@ struct ConvGemmTC {
     int b_slots, b_elems;
     float* c;                     // [c_slots][nsplit][M*N]
     int c_slots;
+    int a_tmap, b_tmap;           // index of the operand's tensor map (bulk tensor copy), or -1: gathered
+    // forward GEMMs that also finish the statistics (nsplit == 1): c is then the conv-output ring
+    int fuse, cpg, ntn;           // channels per normalisation group; column tiles per row of D
+    float* fstat;                 // [groups][cpg * ntn][3]: count, mean, M2 of (channel, column tile)
+};
+
+// One thread block's tiles are tiles[begin[b] .. begin[b+1]).
+struct TcLaunch {
+    const GemmTile* tiles;
+    const int* begin;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -74,13 +102,31 @@ __device__ __forceinline__ uint32_t mnmajor_off(int k, int mu) {
     return (uint32_t)((mu >> 3) * 8192 + (k >> 3) * 1024 + (k & 7) * 128 + (((mu & 7) ^ (k & 7)) << 4));
 }
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait on an mbarrier phase; gives up early once another warp has reported a failure.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* fail) {
     uint32_t done = 0;
     for (int it = 0; it < kTcWaitLimit && !done; ++it) {
         asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
                      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (!done && (it & 63) == 63 && *fail) return false;
     }
     return done != 0;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+// Bulk tensor copies (tiles of a matrix described by a tensor map) that complete on an mbarrier.
+__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
 
 // 16-byte asynchronous global -> shared copy; with ok == false the destination is zero-filled
@@ -89,228 +135,349 @@ __device__ __forceinline__ void cp_async16(unsigned char* dst, const __nv_bfloat
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(sz) : "memory");
 }
 
-__global__ void __launch_bounds__(kTcThreads)
-conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, TickState* ts, int S, int par) {
-    extern __shared__ unsigned char tc_smem_raw[];
-    __shared__ uint64_t mbar[kTcStages];
-    __shared__ uint32_t tmem_base_sh;
-    __shared__ ConvGemmTC G;                               // descriptor copy (no re-reads through global memory)
-    const GemmTile tl = tiles[blockIdx.x];
-    {
-        const int* s_ = reinterpret_cast<const int*>(&gemms[tl.gemm]);
-        int* d_ = reinterpret_cast<int*>(&G);
-        for (int k = threadIdx.x; k < (int)(sizeof(ConvGemmTC) / 4); k += kTcThreads) d_[k] = s_[k];
-    }
-    __syncthreads();
-    const long long t = ts->cnt[par];
-    const long long smp = (G.mode == kFprop) ? t - G.s : t - 2LL * (S - 1) + G.s;
-    if (!sample_live(ts, smp)) return;                                   // uniform: before any allocation
-    unsigned char* smem = (unsigned char*)(((uintptr_t)tc_smem_raw + 1023) & ~(uintptr_t)1023);
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int M = G.M, N = G.N, BN = G.bn;
-    const int kb = tl.split * G.k_per_split, ke = min(G.K, kb + G.k_per_split);
-    const int nchunks = (ke - kb + kTcChunk - 1) / kTcChunk;
-    const __nv_bfloat16* __restrict__ A = G.a;
-    const __nv_bfloat16* __restrict__ B = G.b + (size_t)(smp % G.b_slots) * G.b_elems;
-    float* __restrict__ Cp = G.c + ((size_t)(smp % G.c_slots) * G.nsplit + tl.split) * ((size_t)M * N);
-    const int CI = G.ci, CO = G.co, ksz = G.k, st = G.stride, pad = G.pad, ih = G.ih, iw = G.iw, oh = G.oh, ow = G.ow;
-    // the gathers divide by these for every 16-byte unit: reciprocals once per block
-    const float inv_ci = 1.f / (float)CI, inv_co = 1.f / (float)CO, inv_ksz = 1.f / (float)ksz,
-                inv_st = 1.f / (float)st, inv_ow = 1.f / (float)ow;
+struct TcShared {
+    uint64_t full[kTcStages];     // a stage's operands have landed (128 producer arrivals + 1 with the bulk copies' bytes)
+    uint64_t empty[kTcStages];    // the MMAs that read a stage have completed
+    uint64_t acc_full[2];         // a tile's accumulator is complete
+    uint64_t acc_empty[2];        // the epilogue warps have drained an accumulator
+    uint32_t tmem_base;
+    int fail;
+};
 
-    if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_sh)), "r"(128) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (tid == 0) {
-        for (int q = 0; q < kTcStages; ++q)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&mbar[q])) : "memory");
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem = tmem_base_sh;
-    const int a_mn = G.mode != kFprop, b_mn = G.mode == kWgrad;
-    const uint32_t idesc = tc_idesc(kTcBM, BN, a_mn, b_mn);
+__device__ __forceinline__ long long tc_sample(const ConvGemmTC& G, long long t, int S) {
+    return (G.mode == kFprop) ? t - G.s : t - 2LL * (S - 1) + G.s;
+}
 
-    // ---- per-thread invariants of the gathers
-    // K-major tiles: this thread fills unit (tid & 7) of rows (tid >> 3) + kTcRowsPerPass i
-    // MN-major tiles of width 128: unit (tid & 15) of k-rows (tid >> 4) + kTcKPerPass i
-    const int ku = tid & 7, krow0 = tid >> 3;
-    int bp[kTcPasses], bq[kTcPasses];   // K-major B rows: pixel coordinates (fprop: output pixel; dgrad: input pixel)
-    bool bok[kTcPasses];
-    if (G.mode != kWgrad) {
-        const int wdt = (G.mode == kFprop) ? ow : iw;
-        const float inv_wdt = 1.f / (float)wdt;
+// ------------------------------------------------------------------ producer warps
+__device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, int q0, int q1,
+                            const CUtensorMap* __restrict__ tmaps, const TickState* ts, long long t, int S,
+                            unsigned char* smem, TcShared& sh) {
+    const int ptid = threadIdx.x - 32 * kTcEpiWarps;          // 0 .. 127
+    int it = 0;                                               // chunks issued so far (all tiles)
+    bool ok_all = true;
+    for (int q = q0; q < q1 && ok_all; ++q) {
+        const GemmTile tl = tiles[q];
+        const ConvGemmTC& G = gemms[tl.gemm];
+        const long long smp = tc_sample(G, t, S);
+        if (!sample_live(ts, smp)) continue;
+        const int mode = G.mode, M = G.M, N = G.N, BN = G.bn;
+        const int kb = tl.split * G.k_per_split, ke = min(G.K, kb + G.k_per_split);
+        const int nchunks = (ke - kb + kTcChunk - 1) / kTcChunk;
+        const int slot = (int)(smp % G.b_slots);
+        const __nv_bfloat16* __restrict__ A = G.a;
+        const __nv_bfloat16* __restrict__ B = G.b + (size_t)slot * G.b_elems;
+        const int CI = G.ci, CO = G.co, ksz = G.k, st = G.stride, pad = G.pad, ih = G.ih, iw = G.iw, oh = G.oh, ow = G.ow;
+        const CUtensorMap* tmA = G.a_tmap >= 0 ? tmaps + G.a_tmap : nullptr;
+        const CUtensorMap* tmB = G.b_tmap >= 0 ? tmaps + G.b_tmap : nullptr;
+        // MN-major tiles arrive as boxes of 64 columns: a second box that would lie wholly outside
+        // the matrix is not fetched (its rows / columns of D are never stored)
+        const bool a2 = mode != kFprop && tl.m0 + 64 < M;
+        const bool b2 = mode == kWgrad && BN == 128 && tl.n0 + 64 < N;
+        const uint32_t tx_bytes = (tmA ? (mode == kFprop ? 16384u : (a2 ? 16384u : 8192u)) : 0u) +
+                                  (tmB ? (mode == kWgrad ? (b2 ? 16384u : 8192u) : (uint32_t)BN * 128u) : 0u);
+        // the gathers divide by these for every 16-byte unit: reciprocals once per tile
+        const float inv_ci = 1.f / (float)CI, inv_co = 1.f / (float)CO, inv_ksz = 1.f / (float)ksz,
+                    inv_st = 1.f / (float)st, inv_ow = 1.f / (float)ow;
+        // ---- per-thread invariants of the gathers
+        // K-major tiles (rows of 8 units): unit ku of rows krow0 + 16 i
+        const int ku = ptid & 7, krow0 = ptid >> 3;
+        int bp[8], bq[8];               // K-major B rows: pixel coordinates (fprop: output pixel; dgrad: input pixel)
+        bool bok[8];
+        if (!tmB && mode != kWgrad) {
+            const int wdt = (mode == kFprop) ? ow : iw;
+            const float inv_wdt = 1.f / (float)wdt;
 #pragma unroll
-        for (int i = 0; i < kTcPasses; ++i) {
-            const int n = tl.n0 + krow0 + kTcRowsPerPass * i;
-            bok[i] = (krow0 + kTcRowsPerPass * i) < BN && n < N;
-            bp[i] = quot(n, inv_wdt); bq[i] = n - bp[i] * wdt;
-        }
-    }
-    // wgrad B: this thread's 8 consecutive n = (r, s, ci..ci+7)
-    const int b_units_per_k = BN >> 3;                      // 16 or 8
-    const int bshift = BN == 128 ? 4 : 3;                   // log2 of b_units_per_k
-    const int bmu = tid & (b_units_per_k - 1), bk0 = tid >> bshift, bkstep = kTcThreads >> bshift;
-    int wr = 0, wsx = 0, wci = 0;
-    bool wok = false;
-    if (G.mode == kWgrad) {
-        const int n = tl.n0 + bmu * 8;
-        wok = n < N;
-        const int rs = quot(n, inv_ci); wci = n - rs * CI; wr = quot(rs, inv_ksz); wsx = rs - wr * ksz;
-    }
-    const int amu = tid & 15, ak0 = tid >> 4;               // MN-major A (width 128)
-    const bool a_m_ok = (tl.m0 + amu * 8) < M;
-
-    // gather of K-chunk c into its stage (every unit is written: data or zeros)
-    auto gather = [&](int c) {
-        unsigned char* sA = smem + (c % kTcStages) * kTcStageBytes;
-        unsigned char* sB = sA + 16384;
-        const int k0 = kb + c * kTcChunk;
-        // ---------------- A tile
-        if (G.mode == kFprop) {
-            const int k = k0 + ku * 8;
-#pragma unroll
-            for (int i = 0; i < kTcPasses; ++i) {
-                const int row = krow0 + kTcRowsPerPass * i, m = tl.m0 + row;
-                const bool ok = m < M && k < ke;
-                cp_async16(sA + kmajor_off(row, ku), ok ? A + (size_t)m * G.K + k : A, ok);
-            }
-        } else if (G.mode == kDgrad) {
-#pragma unroll
-            for (int i = 0; i < kTcKPasses; ++i) {
-                const int kl = ak0 + kTcKPerPass * i, k = k0 + kl;          // k = rs * CO + co
-                const bool ok = a_m_ok && k < ke;
-                const int rs = quot(k, inv_co), co = k - rs * CO;
-                cp_async16(sA + mnmajor_off(kl, amu), ok ? A + ((size_t)co * (ksz * ksz) + rs) * CI + tl.m0 + amu * 8 : A, ok);
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < kTcKPasses; ++i) {
-                const int kl = ak0 + kTcKPerPass * i, k = k0 + kl;          // k = output pixel
-                const bool ok = a_m_ok && k < ke;
-                cp_async16(sA + mnmajor_off(kl, amu), ok ? A + (size_t)k * CO + tl.m0 + amu * 8 : A, ok);
+            for (int i = 0; i < 8; ++i) {
+                const int row = krow0 + 16 * i, n = tl.n0 + row;
+                bok[i] = row < BN && n < N;
+                bp[i] = quot(n, inv_wdt); bq[i] = n - bp[i] * wdt;
             }
         }
-        // ---------------- B tile
-        if (G.mode == kFprop) {
-            const int k = k0 + ku * 8;
-            const int rs = quot(k, inv_ci), ci = k - rs * CI, r = quot(rs, inv_ksz), s = rs - r * ksz;
-#pragma unroll
-            for (int i = 0; i < kTcPasses; ++i) {
-                const int row = krow0 + kTcRowsPerPass * i;
-                if (row >= BN) break;
-                const int y = bp[i] * st + r - pad, x = bq[i] * st + s - pad;
-                const bool ok = bok[i] && k < ke && y >= 0 && y < ih && x >= 0 && x < iw;
-                cp_async16(sB + kmajor_off(row, ku), ok ? B + ((size_t)y * iw + x) * CI + ci : B, ok);
+        // MN-major tiles: unit mu of k-rows k0 + step i
+        const int b_units = BN >> 3;                          // 16 or 8 units per k-row of B
+        const int bshift = BN == 128 ? 4 : 3;
+        const int bmu = ptid & (b_units - 1), bk0 = ptid >> bshift, bkstep = kTcProducers >> bshift;
+        int wr = 0, wsx = 0, wci = 0;
+        bool wok = false;
+        if (!tmB && mode == kWgrad) {
+            const int n = tl.n0 + bmu * 8;                    // this thread's 8 consecutive n = (r, s, ci..ci+7)
+            wok = n < N;
+            const int rs = quot(n, inv_ci); wci = n - rs * CI; wr = quot(rs, inv_ksz); wsx = rs - wr * ksz;
+        }
+        const int amu = ptid & 15, ak0 = ptid >> 4;           // MN-major A (width 128): k-rows ak0 + 8 i
+        const bool a_m_ok = (tl.m0 + amu * 8) < M;
+
+        for (int c = 0; c < nchunks; ++c, ++it) {
+            const int stg = it % kTcStages;
+            if (it >= kTcStages && !mbar_wait(smem_u32(&sh.empty[stg]), (uint32_t)(((it / kTcStages) & 1) ^ 1), &sh.fail)) { ok_all = false; break; }
+            unsigned char* sA = smem + stg * kTcStageBytes;
+            unsigned char* sB = sA + 16384;
+            const int k0 = kb + c * kTcChunk;
+            const uint32_t fullb = smem_u32(&sh.full[stg]);
+            if (ptid == 0) {
+                // the 129th arrival of the stage, carrying the bytes of this chunk's bulk copies
+                if (tx_bytes) mbar_arrive_tx(fullb, tx_bytes); else mbar_arrive(fullb);
+                if (tmA) {
+                    if (mode == kFprop) {
+                        tma_2d(smem_u32(sA), tmA, k0, tl.m0, fullb);
+                    } else if (mode == kDgrad) {
+                        const int rs = k0 / CO, co0 = k0 - rs * CO;       // a chunk is 64 output channels of one tap
+                        tma_3d(smem_u32(sA), tmA, tl.m0, rs, co0, fullb);
+                        if (a2) tma_3d(smem_u32(sA) + 8192, tmA, tl.m0 + 64, rs, co0, fullb);
+                    } else {
+                        tma_2d(smem_u32(sA), tmA, tl.m0, k0, fullb);
+                        if (a2) tma_2d(smem_u32(sA) + 8192, tmA, tl.m0 + 64, k0, fullb);
+                    }
+                }
+                if (tmB) {
+                    if (mode == kFprop) {
+                        tma_3d(smem_u32(sB), tmB, k0, tl.n0, slot, fullb);
+                    } else if (mode == kDgrad) {
+                        tma_2d(smem_u32(sB), tmB, k0, tl.n0, fullb);
+                    } else {
+                        tma_3d(smem_u32(sB), tmB, tl.n0, k0, slot, fullb);
+                        if (b2) tma_3d(smem_u32(sB) + 8192, tmB, tl.n0 + 64, k0, slot, fullb);
+                    }
+                }
             }
-        } else if (G.mode == kDgrad) {
-            const int k = k0 + ku * 8;
-            const int rs = quot(k, inv_co), co = k - rs * CO, r = quot(rs, inv_ksz), s = rs - r * ksz;
+            // ---------------- gathered A tile
+            if (!tmA) {
+                if (mode == kFprop) {
+                    const int k = k0 + ku * 8;
 #pragma unroll
-            for (int i = 0; i < kTcPasses; ++i) {
-                const int row = krow0 + kTcRowsPerPass * i;
-                if (row >= BN) break;
-                const int ty = bp[i] + pad - r, tx = bq[i] + pad - s;
-                const int p = quot(ty, inv_st), q = quot(tx, inv_st);
-                const bool ok = bok[i] && k < ke && ty >= 0 && tx >= 0 && p * st == ty && q * st == tx && p < oh && q < ow;
-                cp_async16(sB + kmajor_off(row, ku), ok ? B + ((size_t)p * ow + q) * CO + co : B, ok);
+                    for (int i = 0; i < 8; ++i) {
+                        const int row = krow0 + 16 * i, m = tl.m0 + row;
+                        const bool ok = m < M && k < ke;
+                        cp_async16(sA + kmajor_off(row, ku), ok ? A + (size_t)m * G.K + k : A, ok);
+                    }
+                } else if (mode == kDgrad) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int kl = ak0 + 8 * i, k = k0 + kl;                    // k = rs * CO + co
+                        const bool ok = a_m_ok && k < ke;
+                        const int rs = quot(k, inv_co), co = k - rs * CO;
+                        cp_async16(sA + mnmajor_off(kl, amu), ok ? A + ((size_t)co * (ksz * ksz) + rs) * CI + tl.m0 + amu * 8 : A, ok);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int kl = ak0 + 8 * i, k = k0 + kl;                    // k = output pixel
+                        const bool ok = a_m_ok && k < ke;
+                        cp_async16(sA + mnmajor_off(kl, amu), ok ? A + (size_t)k * CO + tl.m0 + amu * 8 : A, ok);
+                    }
+                }
             }
-        } else {
-            for (int kl = bk0; kl < kTcChunk; kl += bkstep) {
-                const int k = k0 + kl;
-                const int p = quot(k, inv_ow), q = k - p * ow;
-                const int y = p * st + wr - pad, x = q * st + wsx - pad;
-                const bool ok = wok && k < ke && y >= 0 && y < ih && x >= 0 && x < iw;
-                cp_async16(sB + mnmajor_off(kl, bmu), ok ? B + ((size_t)y * iw + x) * CI + wci : B, ok);
+            // ---------------- gathered B tile
+            if (!tmB) {
+                if (mode == kFprop) {
+                    const int k = k0 + ku * 8;
+                    const int rs = quot(k, inv_ci), ci = k - rs * CI, r = quot(rs, inv_ksz), s = rs - r * ksz;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int row = krow0 + 16 * i;
+                        if (row >= BN) break;
+                        const int y = bp[i] * st + r - pad, x = bq[i] * st + s - pad;
+                        const bool ok = bok[i] && k < ke && y >= 0 && y < ih && x >= 0 && x < iw;
+                        cp_async16(sB + kmajor_off(row, ku), ok ? B + ((size_t)y * iw + x) * CI + ci : B, ok);
+                    }
+                } else if (mode == kDgrad) {
+                    const int k = k0 + ku * 8;
+                    const int rs = quot(k, inv_co), co = k - rs * CO, r = quot(rs, inv_ksz), s = rs - r * ksz;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int row = krow0 + 16 * i;
+                        if (row >= BN) break;
+                        const int ty = bp[i] + pad - r, tx = bq[i] + pad - s;
+                        const int p = quot(ty, inv_st), qq = quot(tx, inv_st);
+                        const bool ok = bok[i] && k < ke && ty >= 0 && tx >= 0 && p * st == ty && qq * st == tx && p < oh && qq < ow;
+                        cp_async16(sB + kmajor_off(row, ku), ok ? B + ((size_t)p * ow + qq) * CO + co : B, ok);
+                    }
+                } else {
+                    for (int kl = bk0; kl < kTcChunk; kl += bkstep) {
+                        const int k = k0 + kl;
+                        const int p = quot(k, inv_ow), qq = k - p * ow;
+                        const int y = p * st + wr - pad, x = qq * st + wsx - pad;
+                        const bool ok = wok && k < ke && y >= 0 && y < ih && x >= 0 && x < iw;
+                        cp_async16(sB + mnmajor_off(kl, bmu), ok ? B + ((size_t)y * iw + x) * CI + wci : B, ok);
+                    }
+                }
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            // this thread's copies of the PREVIOUS chunk have landed: make them visible to the
+            // tensor core (async proxy) and count in at that chunk's barrier; the copies just
+            // issued stay in flight meanwhile
+            if (it > 0) {
+                asm volatile("cp.async.wait_group 1;" ::: "memory");
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(smem_u32(&sh.full[(it - 1) % kTcStages]));
             }
         }
-    };
-
-    bool failed = false;
-    for (int c = 0; c < kTcStages - 1; ++c) {
-        if (c < nchunks) gather(c);
-        asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    for (int c = 0; c < nchunks; ++c) {
-        const int stg = c % kTcStages;
-        unsigned char* sA = smem + stg * kTcStageBytes;
-        unsigned char* sB = sA + 16384;
-        // this thread's copies of chunk c have landed; make them visible to the tensor core
-        asm volatile("cp.async.wait_group %0;" ::"n"(kTcStages - 2) : "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (it > 0 && ok_all) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        if (__syncthreads_or(failed)) { failed = true; break; }
-        if (tid == 0) {
+        mbar_arrive(smem_u32(&sh.full[(it - 1) % kTcStages]));
+    }
+    if (!ok_all) sh.fail = 1;
+}
+
+// ------------------------------------------------------------------ MMA warp (one thread)
+__device__ void tc_mma(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, int q0, int q1,
+                       const TickState* ts, long long t, int S, unsigned char* smem, TcShared& sh) {
+    const uint32_t tmem = sh.tmem_base;
+    int it = 0, lt = 0;
+    for (int q = q0; q < q1; ++q) {
+        const GemmTile tl = tiles[q];
+        const ConvGemmTC& G = gemms[tl.gemm];
+        if (!sample_live(ts, tc_sample(G, t, S))) continue;
+        const int kb = tl.split * G.k_per_split, ke = min(G.K, kb + G.k_per_split);
+        const int nchunks = (ke - kb + kTcChunk - 1) / kTcChunk;
+        const int a_mn = G.mode != kFprop, b_mn = G.mode == kWgrad;
+        const uint32_t idesc = tc_idesc(kTcBM, G.bn, a_mn, b_mn);
+        const int buf = lt & 1;
+        if (lt >= 2 && !mbar_wait(smem_u32(&sh.acc_empty[buf]), (uint32_t)(((lt >> 1) & 1) ^ 1), &sh.fail)) { sh.fail = 1; return; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t dcol = tmem + (uint32_t)(buf * 128);
+        for (int c = 0; c < nchunks; ++c, ++it) {
+            const int stg = it % kTcStages;
+            if (!mbar_wait(smem_u32(&sh.full[stg]), (uint32_t)((it / kTcStages) & 1), &sh.fail)) { sh.fail = 1; return; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t sA = smem_u32(smem + stg * kTcStageBytes), sB = sA + 16384;
 #pragma unroll
             for (int j = 0; j < kTcChunk / 16; ++j) {
-                const uint64_t da = a_mn ? tc_desc(smem_u32(sA) + j * 2048, 8192, 1024) : tc_desc(smem_u32(sA) + j * 32, 16, 1024);
-                const uint64_t db = b_mn ? tc_desc(smem_u32(sB) + j * 2048, 8192, 1024) : tc_desc(smem_u32(sB) + j * 32, 16, 1024);
+                const uint64_t da = a_mn ? tc_desc(sA + j * 2048, 8192, 1024) : tc_desc(sA + j * 32, 16, 1024);
+                const uint64_t db = b_mn ? tc_desc(sB + j * 2048, 8192, 1024) : tc_desc(sB + j * 32, 16, 1024);
                 const uint32_t acc = (c > 0 || j > 0) ? 1u : 0u;
                 asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
                              "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-                             ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+                             ::"r"(dcol), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
             }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&mbar[stg])) : "memory");
+            // frees the stage once these MMAs (and all before them) have read it
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&sh.empty[stg])) : "memory");
         }
-        // refill the stage that chunk c-1 used, once its MMAs have read it
-        const int nxt = c + kTcStages - 1;
-        if (nxt < nchunks) {
-            if (c >= 1 && !mbar_wait(smem_u32(&mbar[(c - 1) % kTcStages]), (uint32_t)(((c - 1) / kTcStages) & 1))) failed = true;
-            gather(nxt);
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&sh.acc_full[buf])) : "memory");
+        ++lt;
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    // the last commit covers every MMA issued before it
-    if (!failed && nchunks > 0) {
-        const int last = nchunks - 1;
-        if (!mbar_wait(smem_u32(&mbar[last % kTcStages]), (uint32_t)((last / kTcStages) & 1))) failed = true;
-    }
-    failed = __syncthreads_or(failed);
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (!failed) {
-        // epilogue: warp w reads lanes 32w..32w+31 (rows of D), 32 columns per load
-        // (a warp may only touch the TMEM lanes of its quarter, warp % 4; the two warps of a
-        //  quarter take one half of the columns each)
-        const int quarter = warp & 3, half = warp >> 2;
-        const int m = tl.m0 + quarter * 32 + lane;
-        for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
-            if (tl.n0 + c0 >= N) break;                         // uniform
+}
+
+// ------------------------------------------------------------------ epilogue warps
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+                   "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+                   "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+                   "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ void tc_epilogue(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, int q0, int q1,
+                            const TickState* ts, long long t, int S, TcShared& sh) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;      // warp = quarter of the tensor-memory lanes
+    const uint32_t tmem = sh.tmem_base;
+    int lt = 0;
+    for (int q = q0; q < q1; ++q) {
+        const GemmTile tl = tiles[q];
+        const ConvGemmTC& G = gemms[tl.gemm];
+        const long long smp = tc_sample(G, t, S);
+        if (!sample_live(ts, smp)) continue;
+        const int M = G.M, N = G.N, BN = G.bn;
+        const int buf = lt & 1;
+        if (!mbar_wait(smem_u32(&sh.acc_full[buf]), (uint32_t)((lt >> 1) & 1), &sh.fail)) { sh.fail = 1; return; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        float* __restrict__ Cp = G.fuse ? G.c + (size_t)(smp % G.c_slots) * ((size_t)M * N)
+                                        : G.c + ((size_t)(smp % G.c_slots) * G.nsplit + tl.split) * ((size_t)M * N);
+        const int m = tl.m0 + warp * 32 + lane;                     // row of D held by this thread
+        float cnt = 0.f, mean = 0.f, m2 = 0.f;                      // statistics of this row's columns (forward, fused)
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+            if (tl.n0 + c0 >= N) break;                             // uniform
             uint32_t r[32];
-            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0;
-            asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                         "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
-                           "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
-                           "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
-                           "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                         : "r"(taddr) : "memory");
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 128 + c0), r);
             if (m < M) {
                 float* dst = Cp + (size_t)m * N + tl.n0 + c0;
                 const int nleft = N - (tl.n0 + c0);
                 if (nleft >= 32 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
 #pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        reinterpret_cast<float4*>(dst)[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
-                                                                        __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+                    for (int u = 0; u < 8; ++u)
+                        reinterpret_cast<float4*>(dst)[u] = make_float4(__uint_as_float(r[4 * u]), __uint_as_float(r[4 * u + 1]),
+                                                                        __uint_as_float(r[4 * u + 2]), __uint_as_float(r[4 * u + 3]));
                 } else {
 #pragma unroll
-                    for (int q = 0; q < 32; ++q)
-                        if (q < nleft) dst[q] = __uint_as_float(r[q]);
+                    for (int u = 0; u < 32; ++u)
+                        if (u < nleft) dst[u] = __uint_as_float(r[u]);
+                }
+                if (G.fuse) {
+                    // count / mean / M2 of these (up to) 32 values, merged into the row's running triple
+                    const int nv = min(32, nleft);
+                    float s = 0.f;
+#pragma unroll
+                    for (int u = 0; u < 32; ++u) s += (u < nv) ? __uint_as_float(r[u]) : 0.f;
+                    const float mg = s / (float)nv;
+                    float q2 = 0.f;
+#pragma unroll
+                    for (int u = 0; u < 32; ++u) { const float d = __uint_as_float(r[u]) - mg; q2 = (u < nv) ? fmaf(d, d, q2) : q2; }
+                    const float tot = cnt + (float)nv, dl = mg - mean;
+                    mean += dl * ((float)nv / tot);
+                    m2 += q2 + dl * dl * (cnt * (float)nv / tot);
+                    cnt = tot;
                 }
             }
         }
-    } else if (tid == 0) {
-        ts->error = kErrWait;
-        ts->error_info = tl.gemm;
+        if (G.fuse && m < M) {
+            const int grp = m / G.cpg, cl = m - grp * G.cpg;
+            float* f = G.fstat + (((size_t)grp * G.cpg + cl) * G.ntn + tl.n0 / BN) * 3;
+            f[0] = cnt; f[1] = mean; f[2] = m2;
+        }
+        // the accumulator may be overwritten once all four epilogue warps have read it
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh.acc_empty[buf]));
+        ++lt;
+    }
+}
+
+__global__ void __launch_bounds__(kTcThreads, 2)
+conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, TcLaunch L, const CUtensorMap* __restrict__ tmaps,
+               TickState* ts, int S, int par) {
+    extern __shared__ unsigned char tc_smem_raw[];
+    __shared__ TcShared sh;
+    unsigned char* smem = (unsigned char*)(((uintptr_t)tc_smem_raw + 1023) & ~(uintptr_t)1023);
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int q0 = L.begin[blockIdx.x], q1 = L.begin[blockIdx.x + 1];
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(kTcTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 32) {
+        for (int q = 0; q < kTcStages; ++q) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh.full[q])), "r"(kTcProducers + 1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh.empty[q])) : "memory");
+        }
+        for (int q = 0; q < 2; ++q) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh.acc_full[q])) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh.acc_empty[q])), "r"(kTcEpiWarps) : "memory");
+        }
+        sh.fail = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(128) : "memory");
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const long long t = ts->cnt[par];
+    if (warp < kTcEpiWarps) tc_epilogue(gemms, L.tiles, q0, q1, ts, t, S, sh);
+    else if (warp < kTcMmaWarp) tc_producer(gemms, L.tiles, q0, q1, tmaps, ts, t, S, smem, sh);
+    else if (tid == 32 * kTcMmaWarp) tc_mma(gemms, L.tiles, q0, q1, ts, t, S, smem, sh);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (sh.fail) {
+        // a wait ran out: report it and give bulk copies still in flight time to land before
+        // the shared memory they write goes back to the SM
+        if (tid == 0) { ts->error = kErrWait; ts->error_info = (int)blockIdx.x; }
+        for (int k = 0; k < 512; ++k) __nanosleep(200);
+    }
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(sh.tmem_base), "r"(kTcTmemCols) : "memory");
 }
 
 }  // namespace pb

@@ -277,12 +277,11 @@ void choose_split(int M, int N, int K, int num_sms, int& nsplit, int& kps) {
     nsplit = ceil_div(K, kps);
 }
 
-void choose_split_tc(int M, int N, int bn, int K, int num_sms, int& nsplit, int& kps) {
+void choose_split_tc(int K, int max_k, int& nsplit, int& kps) {
     // The grouped launch already holds thousands of tiles, so K is sliced only to bound the
     // length of one tile's K loop (every slice costs a partial result that must be written
-    // and read back): at most kTcMaxK elements of K per slice.
-    (void)M; (void)N; (void)bn; (void)num_sms;
-    nsplit = std::max(1, std::min(ceil_div(K, kTcMaxK), 16));
+    // and read back): at most max_k elements of K per slice.
+    nsplit = std::max(1, std::min(ceil_div(K, max_k), 16));
     kps = ceil_div(ceil_div(K, nsplit), kTcChunk) * kTcChunk;
     nsplit = ceil_div(K, kps);
 }
@@ -290,6 +289,16 @@ void choose_split_tc(int M, int N, int bn, int K, int num_sms, int& nsplit, int&
 int tc_bn(int N) { return N <= 64 ? 64 : 128; }
 
 void plan_conv(pb_handle* h) {
+    {
+        // first-step blocks of the normalisation launches over the whole network
+        long long chunks = 0;
+        for (const StageHost& x : h->stages) {
+            if (x.head_op != PB_CONV2D) continue;
+            const int hw = x.z.h * x.z.w, cpg = x.head.c_out / x.gn_groups;
+            chunks += (long long)x.gn_groups * (hw <= kPostChunk ? ceil_div(cpg, std::max(1, kPostChunk / hw)) : cpg * ceil_div(hw, kPostChunk));
+        }
+        h->post_fuse = chunks <= 8LL * h->num_sms;       // under two waves of four blocks per SM
+    }
     for (StageHost& x : h->stages) {
         if (x.head_op != PB_CONV2D) continue;
         const int k2 = x.head.k * x.head.k;
@@ -302,10 +311,17 @@ void plan_conv(pb_handle* h) {
                h->stages[x.src].head_op == PB_CONV2D;
         if (x.tc) {
             const int opix = x.z.h * x.z.w, ipix = x.in.h * x.in.w;
-            choose_split_tc(x.head.c_out, opix, tc_bn(opix), x.head.c_in * k2, h->num_sms, x.split_f, x.kps_f);
-            choose_split_tc(x.head.c_in, ipix, tc_bn(ipix), x.head.c_out * k2, h->num_sms, x.split_d, x.kps_d);
-            choose_split_tc(x.head.c_out, x.head.c_in * k2, tc_bn(x.head.c_in * k2), opix, h->num_sms, x.split_w, x.kps_w);
+            (void)ipix;
+            choose_split_tc(x.head.c_in * k2, kTcMaxKFprop, x.split_f, x.kps_f);
+            choose_split_tc(x.head.c_out * k2, kTcMaxK, x.split_d, x.kps_d);
+            choose_split_tc(opix, kTcMaxK, x.split_w, x.kps_w);
             x.dx_nparts = x.split_d;
+            // Large networks: a forward GEMM with one K slice writes the conv output into its ring
+            // and the per-(channel, column tile) statistics itself, so the first normalisation
+            // step is not run for that stage.
+            x.ntn = ceil_div(opix, tc_bn(opix));
+            x.fuse_stats = !h->post_fuse && x.split_f == 1;
+            if (x.fuse_stats) x.fstat_stride = (x.head.c_out / x.gn_groups) * x.ntn;
             continue;
         }
         choose_split(x.head.c_out, x.z.h * x.z.w, x.head.c_in * k2, h->num_sms, x.split_f, x.kps_f);
@@ -321,18 +337,80 @@ void add_tiles(std::vector<GemmTile>& tiles, int gemm, int M, int N, int nsplit,
             for (int n0 = 0; n0 < N; n0 += bn) tiles.push_back(GemmTile{gemm, m0, n0, q});
 }
 
-void fill_conv_tables(pb_handle* h) {
-    {
-        // first-step blocks of the normalisation launches over the whole network
-        long long chunks = 0;
-        for (const StageHost& x : h->stages) {
-            if (x.head_op != PB_CONV2D) continue;
-            const int hw = x.z.h * x.z.w, cpg = x.head.c_out / x.gn_groups;
-            chunks += (long long)x.gn_groups * (hw <= kPostChunk ? ceil_div(cpg, std::max(1, kPostChunk / hw)) : cpg * ceil_div(hw, kPostChunk));
-        }
-        h->post_fuse = chunks <= 8LL * h->num_sms;       // under two waves of four blocks per SM
+// Tensor map (descriptor of a bulk tensor copy) of a bfloat16 matrix with up to three
+// dimensions, innermost first; strides in bytes for dimensions 1.., 128-byte swizzle, zero
+// fill outside the matrix.  With a null base (the sizing pass before the arena exists) an
+// empty placeholder is filed so that table sizes do not change between the passes.
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+TensorMapEncodeFn tensor_map_encoder() {
+    static TensorMapEncodeFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<TensorMapEncodeFn>(p);
     }
-    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_bundles.clear(); h->h_groups.clear(); h->h_ptiles[0].clear(); h->h_ptiles[1].clear(); h->h_dtiles[0].clear(); h->h_dtiles[1].clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear();
+    return fn;
+}
+
+int add_tensor_map(pb_handle* h, const void* base, int rank, const unsigned long long* dims, const unsigned long long* strides_bytes,
+                   const unsigned* box, bool* all_ok) {
+    bool this_ok = true;
+    bool* ok = &this_ok;
+    struct Note { bool* all; bool* one; ~Note() { if (!*one) *all = false; } } note{all_ok, &this_ok};
+    CUtensorMap tm;
+    std::memset(&tm, 0, sizeof(tm));
+    if (base) {
+        TensorMapEncodeFn enc = tensor_map_encoder();
+        cuuint64_t gd[3] = {1, 1, 1}, gs[2] = {0, 0};
+        cuuint32_t bx[3] = {1, 1, 1}, es[3] = {1, 1, 1};
+        for (int q = 0; q < rank; ++q) { gd[q] = dims[q]; bx[q] = box[q]; }
+        for (int q = 0; q + 1 < rank; ++q) gs[q] = strides_bytes[q];
+        if (!enc || enc(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs, bx, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            *ok = false;
+    }
+    h->h_tmaps.push_back(tm);
+    return *ok ? (int)h->h_tmaps.size() - 1 : -1;       // an operand without a map is gathered instead
+}
+
+// Tiles of one grouped tensor-core launch handed to persistent blocks: longest first, each
+// to the block with the least work so far (cost = K chunks plus a constant for the epilogue).
+void balance_tc_tiles(const pb_handle* h, const std::vector<ConvGemmTC>& gemms, std::vector<GemmTile>& tiles, std::vector<int>& begin) {
+    const int nb = std::max(1, std::min((int)tiles.size(), h->num_sms));
+    auto cost = [&](const GemmTile& t) {
+        const ConvGemmTC& g = gemms[t.gemm];
+        const int kb = t.split * g.k_per_split, ke = std::min(g.K, kb + g.k_per_split);
+        return ceil_div(ke - kb, kTcChunk) + 3;
+    };
+    std::vector<int> order(tiles.size());
+    for (size_t q = 0; q < order.size(); ++q) order[q] = (int)q;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cost(tiles[a]) > cost(tiles[b]); });
+    std::vector<long long> load(nb, 0);
+    std::vector<std::vector<int>> mine(nb);
+    for (int q : order) {
+        int best = 0;
+        for (int b = 1; b < nb; ++b) if (load[b] < load[best]) best = b;
+        load[best] += cost(tiles[q]);
+        mine[best].push_back(q);
+    }
+    std::vector<GemmTile> out;
+    begin.assign(1, 0);
+    for (int b = 0; b < nb; ++b) {
+        for (int q : mine[b]) out.push_back(tiles[q]);
+        begin.push_back((int)out.size());
+    }
+    tiles.swap(out);
+}
+
+bool fill_conv_tables(pb_handle* h) {
+    bool maps_ok = true;
+    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_bundles.clear(); h->h_groups.clear(); h->h_ptiles[0].clear(); h->h_ptiles[1].clear(); h->h_dtiles[0].clear(); h->h_dtiles[1].clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear(); h->h_tmaps.clear(); h->h_fchunks.clear();
     for (auto& t : h->h_tiles) t.clear();
     for (auto& t : h->h_tctiles) t.clear();
     const int bf = (h->flags & PB_CONV_BF16) ? 1 : 0;
@@ -347,18 +425,49 @@ void fill_conv_tables(pb_handle* h) {
             ConvGemmTC t{};
             t.ci = L.c_in; t.co = L.c_out; t.k = L.k; t.stride = L.stride; t.pad = L.pad;
             t.ih = x.in.h; t.iw = x.in.w; t.oh = x.z.h; t.ow = x.z.w; t.s = x.index;
+            const bool plain = L.k == 1 && L.stride == 1 && L.pad == 0;     // the activations / dz are then plain [pixel][channel] matrices
+            const __nv_bfloat16* none = nullptr;
+            const bool live = h->arena != nullptr;
             // fprop: D[c_out, out pixel]
             t.mode = kFprop; t.M = L.c_out; t.N = opix; t.K = L.c_in * k2; t.bn = tc_bn(t.N);
             t.nsplit = x.split_f; t.k_per_split = x.kps_f;
             t.a = h->d_wh16 + x.dev_off; t.b = y.out16; t.b_slots = y.out_slots; t.b_elems = x.in.elems();
             t.c = x.zpart; t.c_slots = 1;
+            t.fuse = x.fuse_stats ? 1 : 0; t.cpg = L.c_out / x.gn_groups; t.ntn = x.ntn; t.fstat = x.fstat;
+            if (t.fuse) { t.c = x.z_ring; t.c_slots = x.out_slots; }
+            {
+                const unsigned long long d[2] = {(unsigned long long)t.K, (unsigned long long)t.M}, sb[1] = {(unsigned long long)t.K * 2};
+                const unsigned bx[2] = {64, 128};
+                t.a_tmap = add_tensor_map(h, live ? t.a : none, 2, d, sb, bx, &maps_ok);
+            }
+            t.b_tmap = -1;
+            if (plain) {
+                const unsigned long long d[3] = {(unsigned long long)L.c_in, (unsigned long long)ipix, (unsigned long long)y.out_slots},
+                                         sb[2] = {(unsigned long long)L.c_in * 2, (unsigned long long)x.in.elems() * 2};
+                const unsigned bx[3] = {64, (unsigned)t.bn, 1};
+                t.b_tmap = add_tensor_map(h, live ? t.b : none, 3, d, sb, bx, &maps_ok);
+            }
             add_tiles(h->h_tctiles[0], (int)h->h_tc.size(), t.M, t.N, t.nsplit, kTcBM, t.bn);
             h->h_tc.push_back(t);
+            t.fuse = 0; t.fstat = nullptr;
             // dgrad: D[c_in, in pixel]
             t.mode = kDgrad; t.M = L.c_in; t.N = ipix; t.K = L.c_out * k2; t.bn = tc_bn(t.N);
             t.nsplit = x.split_d; t.k_per_split = x.kps_d;
             t.a = h->d_w16 + x.dev_off; t.b = x.dz16; t.b_slots = 1; t.b_elems = x.z.elems();
             t.c = x.dx; t.c_slots = x.dx_slots;
+            t.a_tmap = -1; t.b_tmap = -1;
+            if (L.c_out % 64 == 0) {
+                // weights [c_out][tap][c_in]: a K chunk is 64 output channels of one tap
+                const unsigned long long d[3] = {(unsigned long long)L.c_in, (unsigned long long)k2, (unsigned long long)L.c_out},
+                                         sb[2] = {(unsigned long long)L.c_in * 2, (unsigned long long)k2 * L.c_in * 2};
+                const unsigned bx[3] = {64, 1, 64};
+                t.a_tmap = add_tensor_map(h, live ? t.a : none, 3, d, sb, bx, &maps_ok);
+            }
+            if (plain) {
+                const unsigned long long d[2] = {(unsigned long long)L.c_out, (unsigned long long)opix}, sb[1] = {(unsigned long long)L.c_out * 2};
+                const unsigned bx[2] = {64, (unsigned)t.bn};
+                t.b_tmap = add_tensor_map(h, live ? t.b : none, 2, d, sb, bx, &maps_ok);
+            }
             add_tiles(h->h_tctiles[1], (int)h->h_tc.size(), t.M, t.N, t.nsplit, kTcBM, t.bn);
             h->h_tc.push_back(t);
             // wgrad: D[c_out, (r, s, c_in)]
@@ -366,6 +475,18 @@ void fill_conv_tables(pb_handle* h) {
             t.nsplit = x.split_w; t.k_per_split = x.kps_w;
             t.a = x.dz16; t.b = y.out16; t.b_slots = y.out_slots; t.b_elems = x.in.elems();
             t.c = x.gpart; t.c_slots = 1;
+            {
+                const unsigned long long d[2] = {(unsigned long long)L.c_out, (unsigned long long)opix}, sb[1] = {(unsigned long long)L.c_out * 2};
+                const unsigned bx[2] = {64, 64};
+                t.a_tmap = add_tensor_map(h, live ? t.a : none, 2, d, sb, bx, &maps_ok);
+            }
+            t.b_tmap = -1;
+            if (plain) {
+                const unsigned long long d[3] = {(unsigned long long)L.c_in, (unsigned long long)ipix, (unsigned long long)y.out_slots},
+                                         sb[2] = {(unsigned long long)L.c_in * 2, (unsigned long long)x.in.elems() * 2};
+                const unsigned bx[3] = {64, 64, 1};
+                t.b_tmap = add_tensor_map(h, live ? t.b : none, 3, d, sb, bx, &maps_ok);
+            }
             add_tiles(h->h_tctiles[2], (int)h->h_tc.size(), t.M, t.N, t.nsplit, kTcBM, t.bn);
             h->h_tc.push_back(t);
         }
@@ -521,6 +642,14 @@ void fill_conv_tables(pb_handle* h) {
         for (int st = 0; st < r.n; st += kUpdChunk) h->h_chunks.push_back(UpdChunk{(int)h->h_upd.size(), st});
         h->h_upd.push_back(r);
     }
+    for (int q = 0; q < 3; ++q) balance_tc_tiles(h, h->h_tc, h->h_tctiles[q], h->h_tcbegin[q]);
+    // the first forward normalisation step skips the stages whose GEMM epilogue has done it
+    {
+        std::vector<char> fused;
+        for (const StageHost& x : h->stages) if (x.head_op == PB_CONV2D) fused.push_back(x.fuse_stats ? 1 : 0);
+        for (const PostChunk& ch : h->h_pchunks) if (!fused[ch.stage]) h->h_fchunks.push_back(ch);
+    }
+    return maps_ok;
 }
 
 int validate_conv(pb_handle* h) {
@@ -579,6 +708,9 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     h->d_chunks = c.take<UpdChunk>(h->h_chunks.size() + 1);
     h->d_tc = c.take<ConvGemmTC>(h->h_tc.size() + 1);
     for (int q = 0; q < 3; ++q) h->d_tctiles[q] = c.take<GemmTile>(h->h_tctiles[q].size() + 1);
+    for (int q = 0; q < 3; ++q) h->d_tcbegin[q] = c.take<int>(h->h_tcbegin[q].size() + 1);
+    h->d_tmaps = c.take<CUtensorMap>(h->h_tmaps.size() + 1);
+    h->d_fchunks = c.take<PostChunk>(h->h_fchunks.size() + 1);
     h->d_w = c.take<float>(h->dev_params);
     if (!h->all_fc || (h->flags & PB_LWP_WFORM)) h->d_wh = c.take<float>(h->dev_params);
     *zero_from = c.off;
@@ -694,6 +826,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
     if (h->profile) for (auto& p : h->prof) p = ProfileClass{};
     const bool fused_last = h->nctaB == 0;      // the last stage rides in the phase-0 launch
     const int npc = (int)h->h_pchunks.size();
+    const int nfc = (int)h->h_fchunks.size();            // forward first-step blocks (stages whose GEMM has not done that step)
     const int post_grid = std::max(1, npc);              // one block per chunk
     const int ngr = (int)h->h_groups.size();             // groups of the stages that keep the three-launch form
     for (int k = 0; k < n_ticks; ++k) {
@@ -768,11 +901,13 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             }
             if (!h->h_tctiles[0].empty()) {
                 prof_begin(h, 4);
-                conv_tc_kernel<<<(int)h->h_tctiles[0].size(), kTcThreads, kTcSmemBytes, h->stream>>>(h->d_tc, h->d_tctiles[0], h->d_ts, h->S, par);
+                conv_tc_kernel<<<(int)h->h_tcbegin[0].size() - 1, kTcThreads, kTcSmemBytes, h->stream>>>(
+                    h->d_tc, TcLaunch{h->d_tctiles[0], h->d_tcbegin[0]}, h->d_tmaps, h->d_ts, h->S, par);
                 prof_end(h);
             }
             prof_begin(h, 5);
-            conv_fwd_post_kernel<<<post_grid, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_pchunks, npc, h->d_bundles, h->d_ptiles[0], h->d_bcnt[0], h->d_ts, h->S, par);
+            if (nfc > 0)
+                conv_fwd_post_kernel<<<nfc, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_fchunks, nfc, h->d_bundles, h->d_ptiles[0], h->d_bcnt[0], h->d_ts, h->S, par);
             if (ngr > 0)
                 conv_group_merge_kernel<<<ceil_div(ngr, 8), 256, 0, h->stream>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 0);
             if (!h->h_dtiles[0].empty())
@@ -819,7 +954,8 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
                 }
                 if (!h->h_tctiles[q].empty()) {
                     prof_begin(h, q == 1 ? 8 : 7, qs);
-                    conv_tc_kernel<<<(int)h->h_tctiles[q].size(), kTcThreads, kTcSmemBytes, qs>>>(h->d_tc, h->d_tctiles[q], h->d_ts, h->S, par);
+                    conv_tc_kernel<<<(int)h->h_tcbegin[q].size() - 1, kTcThreads, kTcSmemBytes, qs>>>(
+                        h->d_tc, TcLaunch{h->d_tctiles[q], h->d_tcbegin[q]}, h->d_tmaps, h->d_ts, h->S, par);
                     prof_end(h, qs);
                 }
             }
@@ -833,7 +969,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             // the conv chain waits for the FC stages before the tick ends
             cudaEventRecord(h->ev_join, fs);
             cudaStreamWaitEvent(h->stream, h->ev_join, 0);
-            h->last_launches += 5 + (fused_last ? 0 : 1);      // ingest, the two normalisation kernels, update, FC
+            h->last_launches += 4 + (nfc > 0 ? 1 : 0) + (fused_last ? 0 : 1);      // ingest, the normalisation kernels, update, FC
             h->last_launches += (h->h_dtiles[0].empty() ? 0 : 1) + (h->h_dtiles[1].empty() ? 0 : 1) + (ngr > 0 ? 2 : 0);
             for (int q = 0; q < 3; ++q) h->last_launches += (h->h_tiles[q].empty() ? 0 : 1) + (h->h_tctiles[q].empty() ? 0 : 1);
         }
@@ -917,6 +1053,9 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     up(h->d_chunks, h->h_chunks.data(), h->h_chunks.size() * sizeof(UpdChunk));
     up(h->d_tc, h->h_tc.data(), h->h_tc.size() * sizeof(ConvGemmTC));
     for (int q = 0; q < 3; ++q) up(h->d_tctiles[q], h->h_tctiles[q].data(), h->h_tctiles[q].size() * sizeof(GemmTile));
+    for (int q = 0; q < 3; ++q) up(h->d_tcbegin[q], h->h_tcbegin[q].data(), h->h_tcbegin[q].size() * sizeof(int));
+    up(h->d_tmaps, h->h_tmaps.data(), h->h_tmaps.size() * sizeof(CUtensorMap));
+    up(h->d_fchunks, h->h_fchunks.data(), h->h_fchunks.size() * sizeof(PostChunk));
     if (e == cudaSuccess && !h->all_fc) {
         // The backward chain (normalisation backward -> data gradients) is the longest of the
         // tick's chains and the update waits for it.  In small networks, whose launches do not

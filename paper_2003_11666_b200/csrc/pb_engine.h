@@ -41,6 +41,8 @@ struct StageHost {
     int split_f = 1, split_d = 1, split_w = 1;                     // K-slices of fprop / dgrad / wgrad
     int kps_f = 0, kps_d = 0, kps_w = 0;                           // K per slice
     bool tc = false;                                               // tensor-core path, weights kept as [co][r][s][ci]
+    bool fuse_stats = false;                                       // its forward GEMM writes the conv output and the chunk statistics
+    int ntn = 1;                                                   // column tiles of that GEMM
     __nv_bfloat16 *out16 = nullptr, *dz16 = nullptr;
 };
 
@@ -88,6 +90,9 @@ struct pb_handle {
     __nv_bfloat16 *d_w16 = nullptr, *d_wh16 = nullptr;
     std::vector<pb::ConvGemmTC> h_tc; pb::ConvGemmTC* d_tc = nullptr;
     std::vector<pb::GemmTile> h_tctiles[3]; pb::GemmTile* d_tctiles[3] = {nullptr, nullptr, nullptr};
+    std::vector<int> h_tcbegin[3]; int* d_tcbegin[3] = {nullptr, nullptr, nullptr};        // tiles of each persistent block
+    std::vector<CUtensorMap> h_tmaps; CUtensorMap* d_tmaps = nullptr;                        // operand matrices fetched by bulk tensor copies
+    std::vector<pb::PostChunk> h_fchunks; pb::PostChunk* d_fchunks = nullptr;                // first forward normalisation step (stages whose GEMM has not done it)
     std::vector<pb::ConvGemm> h_gemms; pb::ConvGemm* d_gemms = nullptr;
     std::vector<pb::GemmTile> h_tiles[3]; pb::GemmTile* d_tiles[3] = {nullptr, nullptr, nullptr};
     std::vector<pb::ConvStage> h_cs; pb::ConvStage* d_cs = nullptr;

@@ -162,7 +162,9 @@ def _resnet20(widths=(16, 32, 64), blocks=3, groups=8, hw=32, n_classes=10,
 
 def _resnet50(depths=(3, 4, 6, 3), base=64, hw=224, n_classes=1000,
               groups=32, name="resnet50", ticks=512, seed=4,
-              flags=FLAG_SC | FLAG_LWP | FLAG_CONV_BF16):
+              flags=FLAG_SC | FLAG_LWP | FLAG_CONV_BF16, relu=True):
+    """relu=False leaves the activation out of every stage after the stem (a
+    network that is smooth in its weights; the stem keeps ReLU and max-pool)."""
     b = _Builder()
     prev = b.conv(3, base, 7, 2, 3, groups, pool=(3, 2, 1))
     c_in = base
@@ -179,10 +181,10 @@ def _resnet50(depths=(3, 4, 6, 3), base=64, hw=224, n_classes=1000,
                               src=block_in)
             else:
                 skip = block_in
-            b.conv(c_in, w, 1, 1, 0, groups, src=block_in)
-            b.conv(w, w, 3, stride, 1, groups)
+            b.conv(c_in, w, 1, 1, 0, groups, src=block_in, relu=relu)
+            b.conv(w, w, 3, stride, 1, groups, relu=relu)
             done += 1
-            prev = b.conv(w, 4 * w, 1, 1, 0, groups, skip=skip,
+            prev = b.conv(w, 4 * w, 1, 1, 0, groups, skip=skip, relu=relu,
                           avgpool=(done == n_blocks))
             c_in = 4 * w
     b.fc(c_in, n_classes, relu=False, loss=True)
@@ -201,17 +203,17 @@ def tiny_cnn(seed=11, ticks=24, flags=FLAG_SC | FLAG_LWP):
                     0.02, 0.9, ticks, seed, flags)
 
 
-def tiny_resnet(seed=12, ticks=40, flags=FLAG_SC | FLAG_LWP, bottleneck=False):
+def tiny_resnet(seed=12, ticks=40, flags=FLAG_SC | FLAG_LWP, bottleneck=False, relu=True):
     """Small residual nets that reach every skip form the big ones use."""
     if bottleneck:
         return _resnet50(depths=(1, 2), base=8, hw=16, n_classes=7, groups=4,
                          name="tiny_bottleneck", ticks=ticks, seed=seed,
-                         flags=flags)
+                         flags=flags, relu=relu)
     return _resnet20(widths=(4, 8), blocks=1, groups=2, hw=8, n_classes=5,
                      name="tiny_resnet", lr=0.02, ticks=ticks, seed=seed)
 
 
-def tall_bottleneck(seed=13, ticks=48, lr=0.001, flags=FLAG_SC | FLAG_LWP | FLAG_CONV_BF16):
+def tall_bottleneck(seed=13, ticks=48, lr=0.001, flags=FLAG_SC | FLAG_LWP | FLAG_CONV_BF16, relu=True):
     """Few channels on large images: the ResNet-50 stage kinds (7x7/2 stem with
     3x3/2 max-pool, two bottleneck blocks with projection shortcuts, the second
     one strided) at 8..64 channels on 3x256x256 inputs.  The stem's output has
@@ -220,7 +222,7 @@ def tall_bottleneck(seed=13, ticks=48, lr=0.001, flags=FLAG_SC | FLAG_LWP | FLAG
     groups cut into several pieces per channel) are met by a net whose CPU
     evaluation takes a fraction of a second per tick."""
     wl = _resnet50(depths=(1, 1), base=8, hw=256, n_classes=7, groups=4,
-                   name="tall_bottleneck", ticks=ticks, seed=seed, flags=flags)
+                   name="tall_bottleneck", ticks=ticks, seed=seed, flags=flags, relu=relu)
     wl.lr = lr
     return wl
 

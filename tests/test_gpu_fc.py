@@ -43,8 +43,11 @@ def test_deep_mlp_full_size_until_float32_range_ends():
     # 1e30 near tick 34, where float32 overflows; the comparison covers every tick
     # up to there (all 16 stages have updated by tick 30).  The weights are compared
     # on every third tick to keep the float64 norms affordable.
+    # Per tensor the strict bound holds through tick 30, when the first stage takes its first
+    # update; in the last three ticks before the overflow every quantity grows a thousandfold
+    # per tick and rounding differences with it (2e-3 there, as for the 4-stage MLP).
     wl = workload("mlp16x2048")
-    w = compare_ticks(wl, 64, TOL, check_every=3, finite_limit=1e24)
+    w = compare_ticks(wl, 64, TOL, check_every=3, finite_limit=1e24, loose_after=(31, 2e-3))
     assert 31 <= w["ticks"] <= 36, w
 
 

@@ -156,6 +156,53 @@ def test_per_sample_replay(make, flags):
             np.testing.assert_allclose(w1, w0 - lr * (a * (m * v0 + g) + b * g), rtol=1e-9, atol=1e-11)
 
 
+@pytest.mark.parametrize("make,flags", [
+    (lambda: mlp([9, 7, 6, 5], lr=0.05), 0), (tiny_cnn, 0), (tiny_resnet, 0),
+    (lambda: tiny_resnet(bottleneck=True), 3), (tiny_cnn, 2)])
+def test_weight_stashing_gives_the_true_gradient_at_the_forward_weights(make, flags):
+    """Eq. "W_{i+1} = W_i - eta grad L(x_i; F_i)": with stashing every sample's
+    gradient is an ORDINARY backward pass (plain torch autograd, nothing mixed)
+    of the network that holds, in stage s, the weights of that sample's forward
+    tick; the update then moves the current weights."""
+    wl = make()
+    o = _oracle(wl, record=True, flags=flags, weight_stash=True)
+    S, lr, m = wl.n_stages, wl.lr, wl.momentum
+    n = 2 * (S - 1) + 8
+    x, y = make_inputs(wl.seed, n, wl.sample_elems, wl.n_classes)
+    losses = [o.tick(x[t], y[t]) for t in range(n)]
+    stages = torch_ref.build(wl)
+    done = sorted({i for (s, i) in o.bwd_version if s == 0})
+    assert len(done) >= 8
+    differs = False
+    for i in done:
+        F_i = []
+        for st in stages:
+            s = st.index
+            D = 2 * (S - 1 - s)
+            w, v = o.history[s][o.fwd_version[(s, i)]]
+            F_i.append(torch.tensor(w - lr * D * v if flags & 2 else w, requires_grad=True))
+            differs = differs or o.fwd_version[(s, i)] != o.bwd_version[(s, i)]
+        xt = torch.tensor(x[i], dtype=torch.float64).view(*wl.in_shape)
+        loss = torch_ref.network_loss(stages, F_i, xt, y[i])
+        loss.backward()
+        assert losses[i + S - 1] == pytest.approx(loss.item(), rel=1e-9)
+        for st in stages:
+            s = st.index
+            g = F_i[s].grad.numpy()
+            np.testing.assert_allclose(o.grads[(s, i)], g, rtol=1e-8, atol=1e-10 * max(1.0, np.abs(g).max()))
+            D = 2 * (S - 1 - s)
+            a, b = sc_coefficients(m, D) if flags & 1 else (1.0, 0.0)
+            w0, v0 = o.history[s][i]
+            w1, v1 = o.history[s][i + 1]
+            np.testing.assert_allclose(w1, w0 - lr * (a * (m * v0 + g) + b * g), rtol=1e-9, atol=1e-11)
+    assert differs                      # forward and backward ticks really saw different weight versions
+    # and it is a different trajectory from the one without stashing
+    p = _oracle(wl, flags=flags)
+    for t in range(n):
+        p.tick(x[t], y[t])
+    assert not np.allclose(p.get_weights(), o.get_weights(), rtol=1e-6, atol=0)
+
+
 def test_fill_phase_leaves_state_untouched():
     wl = mlp([6, 5, 4, 3])
     o = _oracle(wl)

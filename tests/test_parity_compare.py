@@ -6,7 +6,7 @@ single norm over all parameters would have let it through."""
 import numpy as np
 
 from pb_workloads import he_normal_weights, make_inputs, tiny_resnet
-from tests.parity import compare_state, make_oracle, rel_err, tensor_slices
+from tests.parity import compare_state, make_oracle, rel_err, tensor_slices, update_rule_residual
 
 TOL_BF16 = 2e-2
 
@@ -115,3 +115,51 @@ def test_float32_rounding_of_the_weights_alone_passes_the_strict_tolerance():
     _, _, fails = compare_state(slices, w_init, ref_w.astype(np.float32), ref_v.astype(np.float32), ref_w, ref_v,
                                 updates, 1e-4, 1e-4)
     assert not fails
+
+
+def test_update_rule_property_accepts_the_checker_and_rejects_a_wrong_coefficient():
+    # the property the GPU tests check on the engine's own consecutive states: fed the
+    # checker's states (rounded to float32, as the engine stores them) it holds; with one
+    # stage's step redone with b 10 % off, or with the SC term dropped, it does not
+    S = 13
+    wl = tiny_resnet(bottleneck=True, flags=3)
+    o = make_oracle(wl, record=True)
+    n = 2 * (S - 1) + 8
+    x, y = make_inputs(wl.seed, n, wl.sample_elems, wl.n_classes)
+    for t in range(n - 1):
+        o.tick(x[t], y[t])
+    w0, v0 = o.get_weights().astype(np.float32), o.get_velocity().astype(np.float32)
+    o.tick(x[n - 1], y[n - 1])
+    w1, v1 = o.get_weights().astype(np.float32), o.get_velocity().astype(np.float32)
+    slices = tensor_slices(o)
+    assert update_rule_residual(o, slices, w0, v0, w1, v1) <= 1.0
+    for s, scale in ((0, 0.9), (4, 0.9), (7, 0.0)):
+        op = o.opt[s]
+        off = _stage_offset(o, s)
+        sl = slice(off, off + op.w.size)
+        g = v1[sl].astype(np.float64) - float(op.m) * v0[sl]
+        bad = w1.copy()
+        bad[sl] = (w0[sl] - float(op.lr) * (float(op.a) * v1[sl] + scale * float(op.b) * g)).astype(np.float32)
+        assert update_rule_residual(o, slices, w0, v0, bad, v1) > 1.0, "stage %d" % s
+
+
+def test_checker_in_its_own_process_gives_the_same_numbers():
+    # the full-size GPU comparisons run the checker in spawned processes; same bits as in-process
+    from tests.oracle_proc import RemoteOracle
+    wl = tiny_resnet()
+    n = 2 * (wl.n_stages - 1) + 3
+    x, y = make_inputs(wl.seed, n, wl.sample_elems, wl.n_classes)
+    o = make_oracle(wl)
+    r = RemoteOracle(wl)
+    try:
+        for t in range(n):
+            r.tick_begin(x[t], y[t])
+            lo = o.tick(x[t], y[t])
+            lr_ = r.tick_end()
+            assert (np.isnan(lo) and np.isnan(lr_)) or lo == lr_
+        w, v, ver = r.state()
+        np.testing.assert_array_equal(w, o.get_weights())
+        np.testing.assert_array_equal(v, o.get_velocity())
+        assert ver == [p.version for p in o.opt]
+    finally:
+        r.close()
