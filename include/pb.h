@@ -78,8 +78,17 @@ typedef struct {
  * form w_hat = w + T (w - w_previous) instead of the velocity form; the two
  * differ once SC is on (Section "Combined Mitigation").  PB_CONV_BF16:
  * convolutions multiply bf16 operands with fp32 accumulation; master weights,
- * velocity and everything else stay fp32. */
-enum { PB_SC = 1, PB_LWP = 2, PB_LWP_WFORM = 4, PB_CONV_BF16 = 8 };
+ * velocity and everything else stay fp32.
+ * PB_WEIGHT_STASH: the comparison mode of Appendix "Pipelined Backpropagation"
+ * (Eq. W_{i+1} = W_i - eta grad L(x_i; F_i), PipeDream's weight stashing):
+ * every stage keeps, per sample in flight, the weights its forward pass used
+ * (D_s + 1 versions) and takes that sample's backward pass with them instead
+ * of the current weights; the update still moves the current weights.  It
+ * costs (D_s + 1) copies of every stage's weights in device memory and one more
+ * read and write of the weights per tick, and can be combined with the other
+ * flags.  pb_create returns PB_E_UNSUPPORTED when the copies would need more
+ * than 16 GiB. */
+enum { PB_SC = 1, PB_LWP = 2, PB_LWP_WFORM = 4, PB_CONV_BF16 = 8, PB_WEIGHT_STASH = 16 };
 
 /* Builds the engine.  layers/stage_of_layer: host arrays of n_layers entries,
  * stage indices non-decreasing from 0.  (in_c, in_h, in_w): shape of one

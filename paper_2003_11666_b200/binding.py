@@ -13,7 +13,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpb_b200.so")
 
-PB_SC, PB_LWP, PB_LWP_WFORM, PB_CONV_BF16 = 1, 2, 4, 8
+PB_SC, PB_LWP, PB_LWP_WFORM, PB_CONV_BF16, PB_WEIGHT_STASH = 1, 2, 4, 8, 16
 
 EXPORTS = [
     "pb_create", "pb_set_weights", "pb_tick", "pb_run", "pb_run_host", "pb_get_weights",

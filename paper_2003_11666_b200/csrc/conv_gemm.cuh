@@ -36,7 +36,7 @@ __device__ void gemm_tile(const ConvGemm& G, const GemmTile& tl, long long smp, 
     const int M = G.M, N = G.N;
     const int kb = tl.split * G.k_per_split;
     const int ke = min(G.K, kb + G.k_per_split);
-    const float* __restrict__ A = G.a;
+    const float* __restrict__ A = G.a + (size_t)(smp % G.a_slots) * G.a_elems;
     const float* __restrict__ B = G.b + (size_t)(smp % G.b_slots) * G.b_elems;
     float* __restrict__ Cp = G.c + ((size_t)(smp % G.c_slots) * G.nsplit + tl.split) * ((size_t)M * N);
     const int ksz = G.k, st = G.stride, pad = G.pad, ih = G.ih, iw = G.iw, oh = G.oh, ow = G.ow;

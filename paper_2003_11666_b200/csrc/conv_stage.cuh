@@ -456,7 +456,8 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
     const size_t zelems = (size_t)st.co * hw;
     const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
     const float* __restrict__ stat = st.stat_ring + (size_t)slot * st.groups * 2;
-    const float* __restrict__ gam = st.w + st.nw;      // the CURRENT scale
+    // the CURRENT scale (with weight stashing: the one the sample's forward used)
+    const float* __restrict__ gam = st.gstash ? st.gstash + (size_t)slot_of(j, st.gstash_slots) * st.co : st.w + st.nw;
     float* __restrict__ dz = st.dz;
     const bool transposed = st.dz16 && (ch.ncl & 7) == 0 && ch.ncl <= kPostTileChannels && (ch.cl0 & 7) == 0 && (st.co & 7) == 0;
     int cc[U], pp[U];
@@ -543,9 +544,9 @@ __device__ __forceinline__ void group_merge_fwd(const ConvStage& st, int grp, lo
 
 // backward: per-chunk channel sums -> gradients of scale and shift, and the two group
 // means the gradient at the conv output needs (with the CURRENT scale).
-__device__ __forceinline__ void group_merge_bwd(const ConvStage& st, int grp, int lane) {
+__device__ __forceinline__ void group_merge_bwd(const ConvStage& st, int grp, int lane, long long j) {
     const int hw = st.oh * st.ow, cpg = st.cpg, c0 = grp * cpg;
-    const float* __restrict__ gam = st.w + st.nw;
+    const float* __restrict__ gam = st.gstash ? st.gstash + (size_t)slot_of(j, st.gstash_slots) * st.co : st.w + st.nw;
     const int np = st.npieces;
     float m1 = 0.f, m2 = 0.f;
     if (np >= 8) {
@@ -619,7 +620,7 @@ __device__ __noinline__ void close_bundle_bwd(const ConvStage* __restrict__ stag
                                               const PostChunk* __restrict__ tiles, long long t, const TickState* ts, int S, __nv_bfloat16* t16) {
     const PostBundle bd = bundles[bundle];
     const ConvStage& st = stages[bd.stage];
-    for (int g = threadIdx.x >> 5; g < bd.ngrp; g += kPostWarps) group_merge_bwd(st, bd.grp0 + g, threadIdx.x & 31);
+    for (int g = threadIdx.x >> 5; g < bd.ngrp; g += kPostWarps) group_merge_bwd(st, bd.grp0 + g, threadIdx.x & 31, t - 2LL * (S - 1) + st.s);
     __syncthreads();
     for (int q = 0; q < bd.nbtiles; ++q) {
         const PostChunk tl = tiles[bd.btile0 + q];
@@ -683,7 +684,7 @@ conv_group_merge_kernel(const ConvStage* __restrict__ stages, const GroupRef* __
     if (mode == 0) {
         if (sample_live(ts, t - st.s)) group_merge_fwd(st, gr.grp, t, threadIdx.x & 31);
     } else {
-        if (sample_live(ts, t - 2LL * (S - 1) + st.s)) group_merge_bwd(st, gr.grp, threadIdx.x & 31);
+        if (sample_live(ts, t - 2LL * (S - 1) + st.s)) group_merge_bwd(st, gr.grp, threadIdx.x & 31, t - 2LL * (S - 1) + st.s);
     }
 }
 
@@ -795,6 +796,27 @@ cast_weights_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restr
         R.w16[e] = b;
         R.wh16[e] = b;
     }
+}
+
+// Weight stashing: files the weights (and normalisation scale) that this tick's forward
+// of every stage has used under the forward sample's ring slot, before the update
+// overwrites them.  16-byte copies (every tensor and slot starts on a 16-byte boundary).
+__global__ void __launch_bounds__(256)
+stash_copy_kernel(const StashRange* __restrict__ ranges, const StashChunk* __restrict__ chunks,
+                  const TickState* __restrict__ ts, int par) {
+    const StashChunk ch = chunks[blockIdx.x];
+    const StashRange R = ranges[ch.range];
+    const long long i = ts->cnt[par] - R.s;
+    if (!sample_live(ts, i)) return;
+    const long long bytes = R.n * R.esize;
+    const char* src = static_cast<const char*>(R.src);
+    char* dst = static_cast<char*>(R.ring) + (size_t)slot_of(i, R.slots) * (size_t)((bytes + 15) / 16 * 16);
+    const long long end = min(bytes, ch.start + (long long)kStashChunkBytes);
+    long long b = ch.start + 16LL * threadIdx.x;
+    for (; b + 16 <= end; b += 16LL * 256) *reinterpret_cast<uint4*>(dst + b) = *reinterpret_cast<const uint4*>(src + b);
+    // ragged tail of the tensor (fewer than 16 bytes), byte by byte, by the thread whose turn it is
+    if (b < end && b + 16 > end)
+        for (long long q = b; q < end; ++q) dst[q] = src[q];
 }
 
 // Predicted weights re-made from the current state, w_hat = w - lr T v (LWP, velocity

@@ -58,6 +58,7 @@ struct ConvGemmTC {
     int s, bn;                    // stage index; N-tile width (64 or 128)
     int nsplit, k_per_split;      // k_per_split is a multiple of kTcChunk
     const __nv_bfloat16* a;       // fprop: predicted weights; dgrad: weights; wgrad: dz (NHWC)
+    int a_slots, a_elems;         // ring geometry of a: 1 slot, or the stashed forward weights of dgrad (then gathered, no tensor map)
     const __nv_bfloat16* b;       // fprop/wgrad: NHWC activation ring; dgrad: dz (NHWC)
     int b_slots, b_elems;
     float* c;                     // [c_slots][nsplit][M*N]
@@ -164,7 +165,7 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
         const int kb = tl.split * G.k_per_split, ke = min(G.K, kb + G.k_per_split);
         const int nchunks = (ke - kb + kTcChunk - 1) / kTcChunk;
         const int slot = (int)(smp % G.b_slots);
-        const __nv_bfloat16* __restrict__ A = G.a;
+        const __nv_bfloat16* __restrict__ A = G.a + (size_t)(smp % G.a_slots) * G.a_elems;
         const __nv_bfloat16* __restrict__ B = G.b + (size_t)slot * G.b_elems;
         const int CI = G.ci, CO = G.co, ksz = G.k, st = G.stride, pad = G.pad, ih = G.ih, iw = G.iw, oh = G.oh, ow = G.ow;
         const CUtensorMap* tmA = G.a_tmap >= 0 ? tmaps + G.a_tmap : nullptr;

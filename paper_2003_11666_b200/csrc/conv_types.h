@@ -31,7 +31,8 @@ struct ConvGemm {
     int bf16;                    // round both operands to bfloat16 before multiplying
     int tm, tn;                  // per-thread patch (1 or 4): the tile is (16 tm) x (16 tn)
     int nsplit, k_per_split;
-    const float* a;              // fprop: w_hat; dgrad: w; wgrad: dz
+    const float* a;              // fprop: w_hat; dgrad: w (or the ring of stashed forward weights); wgrad: dz
+    int a_slots, a_elems;        // ring geometry of a (1 slot unless the weights are stashed per sample)
     const float* b;              // fprop/wgrad: ring of the input activations; dgrad: dz
     int b_slots, b_elems;        // ring geometry of b (1 slot for dz)
     float* c;                    // [c_slots][nsplit][M*N]
@@ -46,6 +47,7 @@ struct ConvStage {
     int co, oh, ow;              // conv output (z) shape
     int groups, cpg;             // GroupNorm groups, channels per group
     int relu, avgpool;
+    int need_out32;              // somebody reads the float32 output ring (a skip add, a CUDA-core or FC consumer)
     int vec4;                    // oh*ow is a multiple of 4: the element kernels use 4-wide accesses
     int pool_k, pool_stride, pool_pad;   // pool_k == 0: no max-pool
     int out_h, out_w;            // stage output spatial shape (after pooling)
@@ -70,6 +72,7 @@ struct ConvStage {
     float* dskip; int dskip_slots;       // gradient handed to the skip source [slots][skip elems]
     // backward
     int n_dsrc; DeltaSrc dsrc[kMaxDeltaSrc];
+    const float* gstash; int gstash_slots;   // weight stashing: ring [slots][co] of the scale each forward used (or nullptr)
     float* dz;                   // scratch [co*oh*ow]
     __nv_bfloat16* dz16;         // scratch [oh*ow][co] bfloat16 NHWC copy (or nullptr)
 };
@@ -86,6 +89,11 @@ struct UpdRange {
     float T_w; int wform;        // weight-difference form: w_hat = w_new + T (w_new - w_old)
 };
 struct UpdChunk { int range, start; };
+// Weight stashing: one tensor whose forward copy (src) is filed under the forward sample's
+// slot of a ring, n elements of esize bytes each.
+struct StashRange { const void* src; void* ring; int slots, s, esize; long long n; };
+struct StashChunk { int range; long long start; };
+constexpr int kStashChunkBytes = 32768;
 
 // One block's share of the normalisation kernels: channels [cl0, cl0+ncl) of group `grp`
 // (relative to the group), pixels [p0, p0+np); chunk `idx` of `nidx` in its group.

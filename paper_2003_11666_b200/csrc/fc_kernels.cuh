@@ -109,7 +109,11 @@ __device__ __forceinline__ float gather_delta(const FcStage& st, int r, long lon
 // phase 0: every stage's forward, and backward + update of every stage but the
 //          last (whose gradient only exists once its own forward is done);
 // phase 1: the last stage's loss, backward and update.
-template <int VEC, bool WF>
+// ST: weight stashing (the comparison mode of Appendix "Pipelined Backpropagation",
+//     Eq. W_{i+1} = W_i - eta grad L(x_i; F_i)): the forward files the weights it used in
+//     a ring slot of its sample, and the data gradient of the backward sample is taken
+//     with the weights filed at THAT sample's forward instead of the current ones.
+template <int VEC, bool WF, bool ST>
 __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int S, int phase,
                            const int* __restrict__ label_ring, float* __restrict__ loss_out,
                            FcShared& sh, TickState* ts, const float* __restrict__ x_now, int label_now) {
@@ -198,6 +202,9 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
     float m, nla, gsc;
     step_coefficients(ts, j, st.m, st.neg_lr_a, m, nla, gsc);
     const bool want_dx = do_bwd && st.need_dx;
+    const size_t wcount = (size_t)out * in;
+    float* __restrict__ stash_f = ST ? st.stash + (size_t)ring_slot(i < 0 ? 0 : i, st.stash_slots) * wcount : nullptr;
+    const float* __restrict__ stash_b = ST ? st.stash + (size_t)ring_slot(j < 0 ? 0 : j, st.stash_slots) * wcount : nullptr;
 
     for (int c0 = 0; c0 < nchunks; c0 += ncg * kFcChunksPerSweep) {
         int col[kFcChunksPerSweep];
@@ -224,26 +231,28 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
         const int step = nrs * 2;
         // (WF: the weight-difference form keeps its predicted weights in memory; they ride
         //  in the slot of the velocity operand's twin `hv`)
+        // (ST: the stashed weights of the backward sample ride in `sv`)
         auto load_pair = [&](float (&wv)[2][kFcChunksPerSweep][VEC], float (&vv)[2][kFcChunksPerSweep][VEC],
-                             float (&hv)[2][kFcChunksPerSweep][VEC], int r0) {
+                             float (&hv)[2][kFcChunksPerSweep][VEC], float (&sv)[2][kFcChunksPerSweep][VEC], int r0) {
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
                 const int r = r0 + u;
 #pragma unroll
                 for (int c = 0; c < kFcChunksPerSweep; ++c) {
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) { wv[u][c][e] = 0.f; vv[u][c][e] = 0.f; if (WF) hv[u][c][e] = 0.f; }
+                    for (int e = 0; e < VEC; ++e) { wv[u][c][e] = 0.f; vv[u][c][e] = 0.f; if (WF) hv[u][c][e] = 0.f; if (ST) sv[u][c][e] = 0.f; }
                     if (r < rows && cok[c]) {
                         const size_t off = (size_t)(seg.row0 + r) * in + col[c];
                         vload_stream<VEC>(wv[u][c], st.w + off);
                         if (do_bwd) vload_stream<VEC>(vv[u][c], st.v + off);
                         if (WF && do_fwd) vload_stream<VEC>(hv[u][c], st.wh + off);
+                        if (ST && want_dx) vload_stream<VEC>(sv[u][c], stash_b + off);
                     }
                 }
             }
         };
         auto use_pair = [&](float (&wv)[2][kFcChunksPerSweep][VEC], float (&vv)[2][kFcChunksPerSweep][VEC],
-                            float (&hv)[2][kFcChunksPerSweep][VEC], int r0) {
+                            float (&hv)[2][kFcChunksPerSweep][VEC], float (&sv)[2][kFcChunksPerSweep][VEC], int r0) {
             float facc[2];
 #pragma unroll
             for (int u = 0; u < 2; ++u) {
@@ -252,18 +261,21 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
                 const float d = (do_bwd && r < rows) ? sh.delta[r] : 0.f;
 #pragma unroll
                 for (int c = 0; c < kFcChunksPerSweep; ++c) {
-                    float wn[VEC], vn[VEC], hn[VEC];
+                    float wn[VEC], vn[VEC], hn[VEC], wf[VEC];
 #pragma unroll
                     for (int e = 0; e < VEC; ++e) {
                         const float w = wv[u][c][e], v = vv[u][c][e];
                         const float what = WF ? hv[u][c][e] : fmaf(nlT, v, w);   // w_hat = w - lr T v (or the stored prediction)
+                        wf[e] = what;
                         facc[u] = fmaf(what, xfr[c][e], facc[u]);     // forward  (W_hat x)
-                        cacc[c][e] = fmaf(w, d, cacc[c][e]);          // backward (W^T delta)
+                        cacc[c][e] = fmaf(ST ? sv[u][c][e] : w, d, cacc[c][e]);   // backward (W^T delta; stashed forward weights when ST)
                         const float g = d * xbr[c][e];                // rank-1 gradient (xbr carries the 1/N of a mini-batch mean)
                         vn[e] = fmaf(m, v, g);                        // v <- m v + g
                         wn[e] = fmaf(nla, vn[e], fmaf(nlb, g, w));    // w <- w - lr (a v + b g)
                         hn[e] = fmaf(Tw, wn[e] - w, wn[e]);           // w_hat = w_new + T (w_new - w_old)
                     }
+                    if (ST && do_fwd && r < rows && cok[c])
+                        vstore_stream<VEC>(stash_f + (size_t)(seg.row0 + r) * in + col[c], wf);
                     if (do_bwd && r < rows && cok[c]) {
                         const size_t off = (size_t)(seg.row0 + r) * in + col[c];
                         vstore_stream<VEC>(st.w + off, wn);
@@ -291,15 +303,15 @@ __device__ void fc_segment(const FcStage& st, const FcSeg& seg, long long t, int
         };
         {
             // (ha / hb are only touched when WF is set; otherwise they cost nothing)
-            float wa[2][kFcChunksPerSweep][VEC], va[2][kFcChunksPerSweep][VEC], ha[2][kFcChunksPerSweep][VEC];
-            float wb[2][kFcChunksPerSweep][VEC], vb[2][kFcChunksPerSweep][VEC], hb[2][kFcChunksPerSweep][VEC];
+            float wa[2][kFcChunksPerSweep][VEC], va[2][kFcChunksPerSweep][VEC], ha[2][kFcChunksPerSweep][VEC], sa[2][kFcChunksPerSweep][VEC];
+            float wb[2][kFcChunksPerSweep][VEC], vb[2][kFcChunksPerSweep][VEC], hb[2][kFcChunksPerSweep][VEC], sb[2][kFcChunksPerSweep][VEC];
             int r0 = rs * 2;
-            load_pair(wa, va, ha, r0);
+            load_pair(wa, va, ha, sa, r0);
             for (; r0 < rows; r0 += 2 * step) {
-                load_pair(wb, vb, hb, r0 + step);
-                use_pair(wa, va, ha, r0);
-                load_pair(wa, va, ha, r0 + 2 * step);
-                use_pair(wb, vb, hb, r0 + step);
+                load_pair(wb, vb, hb, sb, r0 + step);
+                use_pair(wa, va, ha, sa, r0);
+                load_pair(wa, va, ha, sa, r0 + 2 * step);
+                use_pair(wb, vb, hb, sb, r0 + step);
             }
         }
         // column partials: combine the row splits in a fixed order, then store
@@ -404,12 +416,21 @@ fc_tick_kernel(const FcStage* __restrict__ stages, const FcSeg* __restrict__ seg
         const int nph = seg.fused ? 2 : 1;
         for (int ph = 0; ph < nph; ++ph) {
             const int phs = seg.fused ? ph : phase;
-            if (st.wh) {
-                if (st.vec == 4) fc_segment<4, true>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
-                else fc_segment<1, true>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+            if (st.stash) {
+                // the comparison mode: scalar or vector, both prediction forms, in one instantiation each
+                if (st.wh) {
+                    if (st.vec == 4) fc_segment<4, true, true>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+                    else fc_segment<1, true, true>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+                } else {
+                    if (st.vec == 4) fc_segment<4, false, true>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+                    else fc_segment<1, false, true>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+                }
+            } else if (st.wh) {
+                if (st.vec == 4) fc_segment<4, true, false>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+                else fc_segment<1, true, false>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
             } else {
-                if (st.vec == 4) fc_segment<4, false>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
-                else fc_segment<1, false>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+                if (st.vec == 4) fc_segment<4, false, false>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
+                else fc_segment<1, false, false>(st, seg, t, S, phs, label_ring, loss_out, sh, ts, x_now, label_now);
             }
             __syncthreads();      // the logits written by phase 0 are read by phase 1
         }

@@ -331,6 +331,20 @@ void plan_conv(pb_handle* h) {
     }
 }
 
+// Weight stashing: ring geometry of the weight versions a stage keeps (D_s + 1 of them; a stage
+// with delay 0 takes forward and backward of a sample in the same tick and keeps nothing).
+void plan_stash(pb_handle* h) {
+    if (!(h->flags & PB_WEIGHT_STASH)) return;
+    for (StageHost& x : h->stages) {
+        if (x.delay <= 0) continue;
+        x.stash_slots = x.delay + 1;
+        const size_t nw = x.head_op == PB_FC ? (size_t)x.head.c_in * x.head.c_out
+                                             : (size_t)x.head.c_out * x.head.c_in * x.head.k * x.head.k;
+        x.wstash_stride = x.head_op == PB_FC ? nw * 4 : align_up(nw * (x.tc ? 2 : 4), 16);
+        if (x.head_op == PB_CONV2D) x.gstash_stride = align_up((size_t)x.head.c_out * 4, 16);
+    }
+}
+
 void add_tiles(std::vector<GemmTile>& tiles, int gemm, int M, int N, int nsplit, int bm = kBM, int bn = kBN) {
     for (int q = 0; q < nsplit; ++q)
         for (int m0 = 0; m0 < M; m0 += bm)
@@ -410,7 +424,7 @@ void balance_tc_tiles(const pb_handle* h, const std::vector<ConvGemmTC>& gemms, 
 
 bool fill_conv_tables(pb_handle* h) {
     bool maps_ok = true;
-    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_bundles.clear(); h->h_groups.clear(); h->h_ptiles[0].clear(); h->h_ptiles[1].clear(); h->h_dtiles[0].clear(); h->h_dtiles[1].clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear(); h->h_tmaps.clear(); h->h_fchunks.clear();
+    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_bundles.clear(); h->h_groups.clear(); h->h_ptiles[0].clear(); h->h_ptiles[1].clear(); h->h_dtiles[0].clear(); h->h_dtiles[1].clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear(); h->h_tmaps.clear(); h->h_fchunks.clear(); h->h_stash.clear(); h->h_stashchunks.clear(); h->h_gblocks.clear();
     for (auto& t : h->h_tiles) t.clear();
     for (auto& t : h->h_tctiles) t.clear();
     const int bf = (h->flags & PB_CONV_BF16) ? 1 : 0;
@@ -425,6 +439,7 @@ bool fill_conv_tables(pb_handle* h) {
             ConvGemmTC t{};
             t.ci = L.c_in; t.co = L.c_out; t.k = L.k; t.stride = L.stride; t.pad = L.pad;
             t.ih = x.in.h; t.iw = x.in.w; t.oh = x.z.h; t.ow = x.z.w; t.s = x.index;
+            t.a_slots = 1; t.a_elems = 0;
             const bool plain = L.k == 1 && L.stride == 1 && L.pad == 0;     // the activations / dz are then plain [pixel][channel] matrices
             const __nv_bfloat16* none = nullptr;
             const bool live = h->arena != nullptr;
@@ -456,7 +471,10 @@ bool fill_conv_tables(pb_handle* h) {
             t.a = h->d_w16 + x.dev_off; t.b = x.dz16; t.b_slots = 1; t.b_elems = x.z.elems();
             t.c = x.dx; t.c_slots = x.dx_slots;
             t.a_tmap = -1; t.b_tmap = -1;
-            if (L.c_out % 64 == 0) {
+            if (x.stash_slots > 0) {
+                // the weights of the sample's forward, one ring slot per sample: gathered
+                t.a = x.wstash16; t.a_slots = x.stash_slots; t.a_elems = (int)(x.wstash_stride / 2);
+            } else if (L.c_out % 64 == 0) {
                 // weights [c_out][tap][c_in]: a K chunk is 64 output channels of one tap
                 const unsigned long long d[3] = {(unsigned long long)L.c_in, (unsigned long long)k2, (unsigned long long)L.c_out},
                                          sb[2] = {(unsigned long long)L.c_in * 2, (unsigned long long)k2 * L.c_in * 2};
@@ -471,6 +489,7 @@ bool fill_conv_tables(pb_handle* h) {
             add_tiles(h->h_tctiles[1], (int)h->h_tc.size(), t.M, t.N, t.nsplit, kTcBM, t.bn);
             h->h_tc.push_back(t);
             // wgrad: D[c_out, (r, s, c_in)]
+            t.a_slots = 1; t.a_elems = 0;
             t.mode = kWgrad; t.M = L.c_out; t.N = L.c_in * k2; t.K = opix; t.bn = tc_bn(t.N);
             t.nsplit = x.split_w; t.k_per_split = x.kps_w;
             t.a = x.dz16; t.b = y.out16; t.b_slots = y.out_slots; t.b_elems = x.in.elems();
@@ -497,6 +516,7 @@ bool fill_conv_tables(pb_handle* h) {
         g.mode = kFprop; g.M = L.c_out; g.N = opix; g.K = L.c_in * k2; g.nsplit = x.split_f; g.k_per_split = x.kps_f;
         g.a = h->d_wh + x.dev_off; g.b = xin; g.b_slots = xin_slots; g.b_elems = x.in.elems();
         g.c = x.zpart; g.c_slots = 1;
+        g.a_slots = 1; g.a_elems = 0;
         g.tm = g.M <= 16 ? 1 : 4; g.tn = g.N <= 16 ? 1 : 4;        // small problems take small tiles
         if (!x.tc) add_tiles(h->h_tiles[0], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
         h->h_gemms.push_back(g);
@@ -504,6 +524,7 @@ bool fill_conv_tables(pb_handle* h) {
         if (x.src >= 0) {
             g.mode = kDgrad; g.M = L.c_in; g.N = ipix; g.K = L.c_out * k2; g.nsplit = x.split_d; g.k_per_split = x.kps_d;
             g.a = h->d_w + x.dev_off; g.b = x.dz; g.b_slots = 1; g.b_elems = x.z.elems();
+            if (!x.tc && x.stash_slots > 0) { g.a = x.wstash; g.a_slots = x.stash_slots; g.a_elems = (int)(x.wstash_stride / 4); }   // the forward's weights
             g.c = x.dx; g.c_slots = x.dx_slots;
             g.tm = g.M <= 16 ? 1 : 4; g.tn = g.N <= 16 ? 1 : 4;
             if (!x.tc) add_tiles(h->h_tiles[1], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
@@ -512,6 +533,7 @@ bool fill_conv_tables(pb_handle* h) {
         // wgrad
         g.mode = kWgrad; g.M = L.c_out; g.N = L.c_in * k2; g.K = opix; g.nsplit = x.split_w; g.k_per_split = x.kps_w;
         g.a = x.dz; g.b = xin; g.b_slots = xin_slots; g.b_elems = x.in.elems();
+        g.a_slots = 1; g.a_elems = 0;
         g.c = x.gpart; g.c_slots = 1;
         g.tm = g.M <= 16 ? 1 : 4; g.tn = g.N <= 16 ? 1 : 4;
         if (!x.tc) add_tiles(h->h_tiles[2], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
@@ -521,6 +543,8 @@ bool fill_conv_tables(pb_handle* h) {
         c.s = x.index; c.co = L.c_out; c.oh = x.z.h; c.ow = x.z.w;
         c.groups = x.gn_groups; c.cpg = L.c_out / x.gn_groups;
         c.relu = x.relu; c.avgpool = x.avgpool;
+        c.need_out32 = x.consumers_skip.empty() ? 0 : 1;
+        for (int q : x.consumers_main) if (!h->stages[q].tc) c.need_out32 = 1;
         c.vec4 = ((x.z.h * x.z.w) % 4 == 0) ? 1 : 0;
         c.pool_k = x.has_pool ? x.pool_k : 0; c.pool_stride = x.pool_stride; c.pool_pad = x.pool_pad;
         c.out_h = x.out.h; c.out_w = x.out.w;
@@ -539,6 +563,8 @@ bool fill_conv_tables(pb_handle* h) {
         for (int q : x.consumers_main) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dx, y.dx_slots, y.dx_nparts}; }
         for (int q : x.consumers_skip) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dskip, y.dskip_slots, 1}; }
         c.dz = x.dz;
+        c.gstash = x.gstash; c.gstash_slots = x.stash_slots;
+        if (x.gstash && x.gstash_stride != (size_t)L.c_out * 4) c.gstash = nullptr;     // (channel counts are multiples of 4 in every supported stash layout; see validate_conv)
         c.fstat = x.fstat; c.fstat_stride = x.fstat_stride; c.bsum = x.bsum; c.npieces = x.npieces; c.gsum = x.gsum;
         {
             // Chunks of the first step: whole channels while they fit, else pieces of one channel.
@@ -554,6 +580,16 @@ bool fill_conv_tables(pb_handle* h) {
             const int hw = x.z.h * x.z.w, cpg = c.cpg, stage_idx = (int)h->h_cs.size();
             const bool need16 = x.tc && L.c_out % 8 == 0 && 8 % cpg == 0;
             const int gpb = need16 && cpg < 8 ? 8 / cpg : 1;           // groups per bundle
+            // Large networks: a tensor-core stage whose bundles fit in shared memory is normalised by
+            // one block per bundle, forward and backward (conv_group.cuh), and leaves the lists below.
+            const bool resident = x.fuse_stats && need16 && !x.has_pool && !x.avgpool && x.gn_groups % gpb == 0 &&
+                                  gpb * cpg <= kGroupMaxChannels && (long long)gpb * cpg * hw <= kGroupMaxElems;
+            if (resident) {
+                for (int g0 = 0; g0 < x.gn_groups; g0 += gpb) h->h_gblocks.push_back(GroupBlock{stage_idx, g0, gpb});
+                h->group_smem_fwd = std::max(h->group_smem_fwd, (size_t)gpb * cpg * (hw + 2) * 2);
+                h->group_smem_bwd = std::max(h->group_smem_bwd, (size_t)gpb * cpg * (hw + 4) * 4);
+            }
+            if (!resident) {
             const bool pooled = x.has_pool || x.avgpool;
             auto tile_shape = [&](int channels, int& CT, int& PT) {
                 CT = std::min(kPostTileChannels, std::max(8, (kPostChunk / std::min(hw, kPostTilePixels)) / 8 * 8));
@@ -626,6 +662,7 @@ bool fill_conv_tables(pb_handle* h) {
                         h->h_dtiles[1].push_back(tch);
                     }
             }
+            }   // !resident
         }
         h->h_cs.push_back(c);
 
@@ -641,6 +678,15 @@ bool fill_conv_tables(pb_handle* h) {
         r.g = h->d_g + x.dev_off + nw; r.nparts = 1; r.part_stride = 0; r.n = 2 * L.c_out;
         for (int st = 0; st < r.n; st += kUpdChunk) h->h_chunks.push_back(UpdChunk{(int)h->h_upd.size(), st});
         h->h_upd.push_back(r);
+        if (x.stash_slots > 0) {
+            auto add = [&](const void* src, void* ring, int esize, long long n) {
+                for (long long b0 = 0; b0 < n * esize; b0 += kStashChunkBytes) h->h_stashchunks.push_back(StashChunk{(int)h->h_stash.size(), b0});
+                h->h_stash.push_back(StashRange{src, ring, x.stash_slots, x.index, esize, n});
+            };
+            if (x.tc) add(h->d_wh16 + x.dev_off, x.wstash16, 2, nw);
+            else add(h->d_wh + x.dev_off, x.wstash, 4, nw);
+            add(h->d_wh + x.dev_off + nw, x.gstash, 4, L.c_out);
+        }
     }
     for (int q = 0; q < 3; ++q) balance_tc_tiles(h, h->h_tc, h->h_tctiles[q], h->h_tcbegin[q]);
     // the first forward normalisation step skips the stages whose GEMM epilogue has done it
@@ -660,6 +706,7 @@ int validate_conv(pb_handle* h) {
         if (x.has_pool && x.avgpool) return fail(nullptr, PB_E_UNSUPPORTED, "max-pool and average pool in one stage");
         if (x.avgpool && x.z.h * x.z.w > kPostChunk) return fail(nullptr, PB_E_UNSUPPORTED, "global average pool over more than 2048 pixels");
         if ((int)(x.consumers_main.size() + x.consumers_skip.size()) > kMaxDeltaSrc) return fail(nullptr, PB_E_UNSUPPORTED, "too many consumers of one stage");
+        if ((h->flags & PB_WEIGHT_STASH) && x.head.c_out % 4) return fail(nullptr, PB_E_UNSUPPORTED, "weight stashing needs channel counts that are multiples of 4");
     }
     for (const StageHost& x : h->stages)
         if (x.head_op == PB_FC && (x.has_skip || x.has_pool || x.avgpool || x.gn_groups)) return fail(nullptr, PB_E_UNSUPPORTED, "FC stages take only RELU or SOFTMAX_CE");
@@ -706,6 +753,9 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     for (int q = 0; q < 2; ++q) h->d_dtiles[q] = c.take<PostChunk>(h->h_dtiles[q].size() + 1);
     h->d_upd = c.take<UpdRange>(h->h_upd.size() + 1);
     h->d_chunks = c.take<UpdChunk>(h->h_chunks.size() + 1);
+    h->d_gblocks = c.take<GroupBlock>(h->h_gblocks.size() + 1);
+    h->d_stash = c.take<StashRange>(h->h_stash.size() + 1);
+    h->d_stashchunks = c.take<StashChunk>(h->h_stashchunks.size() + 1);
     h->d_tc = c.take<ConvGemmTC>(h->h_tc.size() + 1);
     for (int q = 0; q < 3; ++q) h->d_tctiles[q] = c.take<GemmTile>(h->h_tctiles[q].size() + 1);
     for (int q = 0; q < 3; ++q) h->d_tcbegin[q] = c.take<int>(h->h_tcbegin[q].size() + 1);
@@ -753,6 +803,11 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
                 x.dz16 = c.take<__nv_bfloat16>(ze);
             }
         }
+        if (x.stash_slots > 0) {
+            if (x.tc) x.wstash16 = reinterpret_cast<__nv_bfloat16*>(c.take<char>(x.wstash_stride * x.stash_slots));
+            else x.wstash = reinterpret_cast<float*>(c.take<char>(x.wstash_stride * x.stash_slots));
+            if (x.head_op == PB_CONV2D) x.gstash = reinterpret_cast<float*>(c.take<char>(x.gstash_stride * x.stash_slots));
+        }
     }
     return c.off;
 }
@@ -765,6 +820,7 @@ void fill_fc_tables(pb_handle* h) {
         f.neg_lr_T = -h->lr * x.T; f.m = h->momentum; f.neg_lr_a = -h->lr * x.a; f.neg_lr_b = -h->lr * x.b;
         f.T_w = x.T;
         f.wh = ((h->flags & PB_LWP_WFORM) && h->d_wh) ? h->d_wh + x.dev_off : nullptr;
+        f.stash = x.wstash; f.stash_slots = x.stash_slots;      // slots of exactly out*in floats
         if (x.src < 0) { f.xin = h->in_ring; f.xin_slots = h->in_slots; }
         else { f.xin = h->stages[x.src].out_ring; f.xin_slots = h->stages[x.src].out_slots; }
         f.out = x.out_ring; f.out_slots = x.out_slots;
@@ -826,6 +882,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
     if (h->profile) for (auto& p : h->prof) p = ProfileClass{};
     const bool fused_last = h->nctaB == 0;      // the last stage rides in the phase-0 launch
     const int npc = (int)h->h_pchunks.size();
+    const int ngb = (int)h->h_gblocks.size();             // bundles normalised by one block each (large networks)
     const int nfc = (int)h->h_fchunks.size();            // forward first-step blocks (stages whose GEMM has not done that step)
     const int post_grid = std::max(1, npc);              // one block per chunk
     const int ngr = (int)h->h_groups.size();             // groups of the stages that keep the three-launch form
@@ -912,6 +969,8 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
                 conv_group_merge_kernel<<<ceil_div(ngr, 8), 256, 0, h->stream>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 0);
             if (!h->h_dtiles[0].empty())
                 conv_apply_fwd_kernel<<<(int)h->h_dtiles[0].size(), kPostThreads, 0, h->stream>>>(h->d_cs, h->d_dtiles[0], (int)h->h_dtiles[0].size(), h->d_ts, h->S, par);
+            if (ngb > 0)
+                conv_group_fwd_kernel<<<ngb, kGroupThreads, h->group_smem_fwd, h->stream>>>(h->d_cs, h->d_gblocks, ngb, h->d_ts, h->S, par);
             prof_end(h);
             // Backward chain: through pool/ReLU/GroupNorm -> data and weight gradients.  It reads
             // what earlier ticks stored (other ring slots than the forward chain writes) and the
@@ -939,6 +998,8 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
                 conv_group_merge_kernel<<<ceil_div(ngr, 8), 256, 0, bs>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 1);
             if (!h->h_dtiles[1].empty())
                 conv_bwd_dz_kernel<<<(int)h->h_dtiles[1].size(), kPostThreads, 0, bs>>>(h->d_cs, h->d_dtiles[1], (int)h->h_dtiles[1].size(), h->d_ts, h->S, par);
+            if (ngb > 0)
+                conv_group_bwd_kernel<<<ngb, kGroupThreads, h->group_smem_bwd, bs>>>(h->d_cs, h->d_gblocks, ngb, h->d_ts, h->S, par);
             prof_end(h, bs);
             // data gradients (dgrad) and weight gradients (wgrad) both start from dz and write
             // different buffers: wgrad goes to a stream of its own
@@ -963,6 +1024,11 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             cudaStreamWaitEvent(h->stream, h->ev_wjoin, 0);
             cudaEventRecord(h->ev_bjoin, bs);
             cudaStreamWaitEvent(h->stream, h->ev_bjoin, 0);
+            if (!h->h_stashchunks.empty()) {
+                // weight stashing: this tick's forward weights go to their sample's slot before the update replaces them
+                stash_copy_kernel<<<(int)h->h_stashchunks.size(), 256, 0, h->stream>>>(h->d_stash, h->d_stashchunks, h->d_ts, par);
+                h->last_launches += 1;
+            }
             prof_begin(h, 2);
             update_kernel<<<(int)h->h_chunks.size(), 256, 0, h->stream>>>(h->d_upd, h->d_chunks, h->d_ts, h->S, par);
             prof_end(h);
@@ -970,6 +1036,7 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             cudaEventRecord(h->ev_join, fs);
             cudaStreamWaitEvent(h->stream, h->ev_join, 0);
             h->last_launches += 4 + (nfc > 0 ? 1 : 0) + (fused_last ? 0 : 1);      // ingest, the normalisation kernels, update, FC
+            h->last_launches += (ngb > 0 ? 2 : 0);
             h->last_launches += (h->h_dtiles[0].empty() ? 0 : 1) + (h->h_dtiles[1].empty() ? 0 : 1) + (ngr > 0 ? 2 : 0);
             for (int q = 0; q < 3; ++q) h->last_launches += (h->h_tiles[q].empty() ? 0 : 1) + (h->h_tctiles[q].empty() ? 0 : 1);
         }
@@ -1001,7 +1068,7 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     if (!layers || !stage_of_layer || !out || n_layers <= 0 || in_c <= 0 || in_h <= 0 || in_w <= 0 || n_classes <= 0)
         return fail(nullptr, PB_E_ARG, "pb_create: NULL pointer or non-positive size");
     if (!(momentum >= 0.f && momentum < 1.f) || !(lr >= 0.f)) return fail(nullptr, PB_E_ARG, "pb_create: need 0 <= momentum < 1 and lr >= 0");
-    if (flags & ~(unsigned)(PB_SC | PB_LWP | PB_LWP_WFORM | PB_CONV_BF16)) return fail(nullptr, PB_E_ARG, "pb_create: unknown flag");
+    if (flags & ~(unsigned)(PB_SC | PB_LWP | PB_LWP_WFORM | PB_CONV_BF16 | PB_WEIGHT_STASH)) return fail(nullptr, PB_E_ARG, "pb_create: unknown flag");
     if ((flags & PB_LWP_WFORM) && !(flags & PB_LWP)) return fail(nullptr, PB_E_ARG, "pb_create: PB_LWP_WFORM needs PB_LWP");
     for (int q = 1; q < n_layers; ++q)
         if (stage_of_layer[q] < stage_of_layer[q - 1]) return fail(nullptr, PB_E_ARG, "pb_create: stage indices must not decrease");
@@ -1022,9 +1089,18 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     rc = validate_conv(h);
     if (rc != PB_OK) { delete h; return rc; }
     plan_conv(h);
+    plan_stash(h);
     fill_conv_tables(h);     // sizes only; pointers are filled in after the layout
     size_t zero_from = 0;
     h->arena_bytes = layout(h, nullptr, &zero_from);
+    if (flags & PB_WEIGHT_STASH) {
+        size_t stash_bytes = 0;
+        for (const StageHost& x : h->stages) stash_bytes += (x.wstash_stride + x.gstash_stride) * (size_t)x.stash_slots;
+        if (stash_bytes > (16ull << 30)) {
+            std::string m = "pb_create: weight stashing would keep " + std::to_string(stash_bytes) + " bytes of weight versions (limit 16 GiB)";
+            delete h; return fail(nullptr, PB_E_UNSUPPORTED, m);
+        }
+    }
     e = cudaMalloc((void**)&h->arena, h->arena_bytes);
     if (e != cudaSuccess) {
         std::string m = "pb_create: cudaMalloc of " + std::to_string(h->arena_bytes) + " bytes failed: " + cudaGetErrorString(e);
@@ -1051,6 +1127,9 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     for (int q = 0; q < 2; ++q) up(h->d_dtiles[q], h->h_dtiles[q].data(), h->h_dtiles[q].size() * sizeof(PostChunk));
     up(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange));
     up(h->d_chunks, h->h_chunks.data(), h->h_chunks.size() * sizeof(UpdChunk));
+    up(h->d_gblocks, h->h_gblocks.data(), h->h_gblocks.size() * sizeof(GroupBlock));
+    up(h->d_stash, h->h_stash.data(), h->h_stash.size() * sizeof(StashRange));
+    up(h->d_stashchunks, h->h_stashchunks.data(), h->h_stashchunks.size() * sizeof(StashChunk));
     up(h->d_tc, h->h_tc.data(), h->h_tc.size() * sizeof(ConvGemmTC));
     for (int q = 0; q < 3; ++q) up(h->d_tctiles[q], h->h_tctiles[q].data(), h->h_tctiles[q].size() * sizeof(GemmTile));
     for (int q = 0; q < 3; ++q) up(h->d_tcbegin[q], h->h_tcbegin[q].data(), h->h_tcbegin[q].size() * sizeof(int));
@@ -1078,6 +1157,10 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     }
     if (e == cudaSuccess && !h->h_tc.empty())
         e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
+    if (e == cudaSuccess && !h->h_gblocks.empty()) {
+        e = cudaFuncSetAttribute(conv_group_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->group_smem_fwd);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(conv_group_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->group_smem_bwd);
+    }
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
     if (e != cudaSuccess) {
         std::string m = std::string("pb_create: upload failed: ") + cudaGetErrorString(e);
@@ -1249,7 +1332,7 @@ double pb_kernel_min_bytes(const pb_handle* h, int which) {
     if (which == 0) {
         // FC tick kernel: w and v read once and written once; the weight-difference form
         // also reads and writes its stored prediction
-        const double per = (h->flags & PB_LWP_WFORM) ? 24.0 : 16.0;
+        const double per = ((h->flags & PB_LWP_WFORM) ? 24.0 : 16.0) + ((h->flags & PB_WEIGHT_STASH) ? 8.0 : 0.0);
         for (const pb::FcStage& f : h->h_fc) bytes += per * ((double)f.in_dim * f.out_dim + f.out_dim);
         return bytes;
     }

@@ -7,6 +7,7 @@
 #include "pb_internal.h"
 #include "conv_types.h"
 #include "conv_tc.cuh"
+#include "conv_group.cuh"
 
 namespace pb {
 
@@ -41,6 +42,9 @@ struct StageHost {
     int split_f = 1, split_d = 1, split_w = 1;                     // K-slices of fprop / dgrad / wgrad
     int kps_f = 0, kps_d = 0, kps_w = 0;                           // K per slice
     bool tc = false;                                               // tensor-core path, weights kept as [co][r][s][ci]
+    // weight stashing: rings of the weights (and normalisation scale) each forward used
+    float* wstash = nullptr; __nv_bfloat16* wstash16 = nullptr; float* gstash = nullptr;
+    int stash_slots = 0; size_t wstash_stride = 0, gstash_stride = 0;       // strides in bytes, multiples of 16
     bool fuse_stats = false;                                       // its forward GEMM writes the conv output and the chunk statistics
     int ntn = 1;                                                   // column tiles of that GEMM
     __nv_bfloat16 *out16 = nullptr, *dz16 = nullptr;
@@ -105,6 +109,10 @@ struct pb_handle {
     std::vector<pb::PostChunk> h_ptiles[2]; pb::PostChunk* d_ptiles[2] = {nullptr, nullptr};   // tiles of the elementwise kernels: forward, backward
     std::vector<pb::UpdRange> h_upd; pb::UpdRange* d_upd = nullptr;
     std::vector<pb::UpdChunk> h_chunks; pb::UpdChunk* d_chunks = nullptr;
+    std::vector<pb::GroupBlock> h_gblocks; pb::GroupBlock* d_gblocks = nullptr;             // bundles normalised by one block each
+    size_t group_smem_fwd = 0, group_smem_bwd = 0;
+    std::vector<pb::StashRange> h_stash; pb::StashRange* d_stash = nullptr;
+    std::vector<pb::StashChunk> h_stashchunks; pb::StashChunk* d_stashchunks = nullptr;
 
     long long tick = 0, last_launches = 0;
     bool profile = false;

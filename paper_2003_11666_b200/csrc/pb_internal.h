@@ -47,6 +47,8 @@ struct FcStage {
     float neg_lr_T;        // -lr * T      (LWP horizon)
     float T_w;             // T itself, for the weight-difference form
     float* wh;             // stored predicted weights (weight-difference form only), else nullptr
+    float* stash;          // weight stashing: ring [stash_slots][out*in] of the weights each forward used, else nullptr
+    int stash_slots;
     float m;               // momentum
     float neg_lr_a;        // -lr * a      (spike compensation)
     float neg_lr_b;        // -lr * b

@@ -304,19 +304,22 @@ def compare_ticks(wl, n_ticks, tol, check_every=1, finite_limit=1e30, loose_afte
                 mxl = main.last_max_logit
                 e = abs(lg - lo) / max(abs(lo), mxl, 1e-12)
                 worst["loss"] = max(worst["loss"], e)
-                tll = tl
+                # flipped units move the trajectory, hence later losses (float32 runs: only once a
+                # decision that either side may take differently is in play)
+                ff = float(flip_floor.max()) if (fragile_margin is None or (fragile_tick is not None and t >= fragile_tick)) else 0.0
+                tll = max(tl, ff)
                 if lo32 is not None and not math.isnan(lo32):
                     # late in a long bfloat16 run two correct evaluations have drifted apart: the
                     # checker's own float32 run tells by how much (largest distance so far: the
                     # drift grows with the tick, a single tick's distance can be small by chance)
                     loss_spread = max(loss_spread, abs(lo32 - lo) / max(abs(lo), mxl, 1e-12))
-                    tll = max(tl, spread_factor * loss_spread)
+                    tll = max(tll, spread_factor * loss_spread)
                 assert e <= tll, "tick %d: loss %r vs %r (rel %.3g, bound %.3g)" % (t, lg, lo, e, tll)
                 if abs(lo) > 1e-3 * mxl:
                     ep = abs(lg - lo) / abs(lo)
                     worst["plain_loss"] = max(worst["plain_loss"], ep)
                     if plain_loss_tol is not None:
-                        tlp = max(plain_loss_tol, tl)
+                        tlp = max(plain_loss_tol, tl, ff)
                         if lo32 is not None and not math.isnan(lo32):
                             plain_spread = max(plain_spread, abs(lo32 - lo) / abs(lo))
                             tlp = max(tlp, spread_factor * plain_spread)

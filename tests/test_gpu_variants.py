@@ -78,3 +78,44 @@ def test_wform_needs_lwp():
     wl = mlp([8, 6, 4])
     with pytest.raises(PBError):
         PB(wl.layers, wl.stage_of_layer, wl.in_shape, wl.n_classes, 0.1, 0.9, flags=4)
+
+
+def _stashed(wl):
+    wl.weight_stash = True
+    return wl
+
+
+@pytest.mark.parametrize("make,tol", [
+    (lambda: mlp([48, 40, 33, 24, 5], lr=0.003, seed=33), TOL),
+    (lambda: mlp([64, 48, 32, 6], lr=0.003, seed=34, flags=0), TOL),
+    (tiny_cnn, TOL), (lambda: tiny_cnn(flags=0), TOL), (lambda: _resnet(3), TOL),
+    (lambda: tiny_resnet(bottleneck=True, flags=3), TOL),
+    (lambda: tiny_resnet(bottleneck=True, flags=3 | 8, relu=False), 2e-2)])
+def test_weight_stashing(make, tol):
+    # the comparison mode of the paper's appendix (PipeDream's rule): the backward pass of a
+    # sample uses the weights of its own forward pass; FC stages, CUDA-core and tensor-core
+    # convolutions, with and without the mitigations
+    wl = _stashed(make())
+    n = 2 * (wl.n_stages - 1) + 20
+    w = compare_ticks(wl, n, tol)
+    assert w["ticks"] == n and w["min_updates"] >= 20
+
+
+def test_weight_stashing_changes_the_trajectory():
+    # (so that the test above cannot pass with the flag ignored on both sides)
+    import numpy as np
+    import torch
+    from pb_workloads import make_inputs
+    from tests.parity import make_engine
+    outs = []
+    for stash in (False, True):
+        wl = tiny_cnn()
+        wl.weight_stash = stash
+        e = make_engine(wl)
+        n = 2 * (wl.n_stages - 1) + 12
+        x, y = make_inputs(wl.seed, n, wl.sample_elems, wl.n_classes)
+        e.run(torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda(), n)
+        e.sync()
+        outs.append(e.get_weights())
+        e.destroy()
+    assert not np.allclose(outs[0], outs[1], rtol=1e-6, atol=0)
