@@ -197,6 +197,53 @@ size_t pb_device_bytes(const pb_handle* h);
 int pb_profile_enable(pb_handle* h, int enable);
 double pb_profile_ms(pb_handle* h, int which, long long* launches);
 
+/* ---- Stage split over several GPUs (Section 2.1: stages split over GPUs, one
+ * host thread per GPU; Appendix "Batch Parallel vs Pipeline Parallel
+ * Computation": neighbours exchange one activation forward and one gradient
+ * backward per tick, nothing else).  Fully connected networks only.
+ *
+ * pb_split_plan: contiguous stage ranges [lo[r], hi[r]) for n_ranks ranks that
+ * minimise the largest per-tick weight traffic (16 bytes per parameter) of any
+ * rank.  Host arithmetic only (no device is touched).  lo / hi: n_ranks ints.
+ *
+ * pb_create_split: as pb_create, but the handle runs only the stages of `rank`
+ * in that plan, on the device current at the call.  Every rank is fed the same
+ * tick stream: pb_tick / pb_run use dev_x only on the rank that owns stage 0
+ * (elsewhere it may be NULL) and the label only on the rank that owns the last
+ * stage, whose loss is the tick's loss (other ranks return NaN).
+ * pb_set_weights takes the whole network's vector on every rank and keeps its
+ * own stages' part; pb_get_weights / pb_get_velocity return the own stages'
+ * values and zeros elsewhere (the caller adds the ranks' vectors up).
+ *
+ * Hand-off: pb_split_ports gives the device addresses where THIS rank receives
+ * (its copy of the previous rank's boundary activation ring, of the next
+ * rank's boundary gradient buffer, and their tick stamps); pb_split_connect is
+ * given the neighbours' ports (NULL where there is no neighbour).  At the end
+ * of every tick a rank writes its boundary tensors and the stamp t + 1 into
+ * its neighbours' ports with plain stores (the ranks' devices must have peer
+ * access to each other when they differ; nothing else is required), and at the
+ * start of tick t it waits, for at most one second, until both of its own
+ * stamps have reached t; an expired wait is reported as PB_E_DEVICE by the next
+ * synchronising call.  Ranks may therefore run at most one tick apart.  On ONE
+ * device (testing), tick the ranks in turn with pb_tick, rank 0 first: then
+ * every stamp is already in place when it is looked at and nothing waits. */
+typedef struct {
+    void* act;          /* boundary activation ring [slots][dim] floats          */
+    void* act_stamp;    /* int64 tick stamp                                      */
+    void* grad;         /* boundary gradient buffer [2][dim] floats              */
+    void* grad_stamp;   /* int64 tick stamp                                      */
+} pb_split_port;
+
+int pb_split_plan(const pb_layer* layers, int n_layers, const int32_t* stage_of_layer,
+                  int in_c, int in_h, int in_w, int n_classes, int n_ranks, int32_t* lo, int32_t* hi);
+int pb_create_split(const pb_layer* layers, int n_layers, const int32_t* stage_of_layer,
+                    int in_c, int in_h, int in_w, int n_classes,
+                    float lr, float momentum, unsigned flags, void* stream,
+                    int rank, int n_ranks, pb_handle** out);
+int pb_split_range(const pb_handle* h, int32_t* lo, int32_t* hi);
+int pb_split_ports(pb_handle* h, pb_split_port* mine);
+int pb_split_connect(pb_handle* h, const pb_split_port* prev_rank, const pb_split_port* next_rank);
+
 /* Least device-memory traffic, in bytes per steady-state tick, of kernel class
  * `which` as the engine is configured: 0 = the FC tick kernel (one read and one
  * write of w and v per FC parameter: the optimizer's full-model pass that

@@ -21,12 +21,17 @@ EXPORTS = [
     "pb_tick_count", "pb_last_launch_count", "pb_device_bytes", "pb_profile_enable",
     "pb_profile_ms", "pb_last_error", "pb_destroy", "pb_mlp_run_static", "pb_set_mitigation",
     "pb_set_update_size", "pb_kernel_min_bytes", "pb_bench_l2_bandwidth", "pb_bench_fp32_fma",
+    "pb_split_plan", "pb_create_split", "pb_split_range", "pb_split_ports", "pb_split_connect",
 ]
 
 
 class pb_layer(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("op", "c_in", "c_out", "k", "stride", "pad", "groups", "src", "skip_mode")]
+
+
+class pb_split_port(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("act", "act_stamp", "grad", "grad_stamp")]
 
 
 class PBError(RuntimeError):
@@ -80,6 +85,13 @@ def load_library():
     lib.pb_kernel_min_bytes.restype = C.c_double
     lib.pb_bench_l2_bandwidth.argtypes = [C.c_size_t, i32, vp, C.POINTER(C.c_double)]
     lib.pb_bench_fp32_fma.argtypes = [i32, vp, C.POINTER(C.c_double)]
+    lib.pb_split_plan.argtypes = [C.POINTER(pb_layer), i32, C.POINTER(C.c_int32), i32, i32, i32, i32, i32,
+                                  C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.pb_create_split.argtypes = [C.POINTER(pb_layer), i32, C.POINTER(C.c_int32), i32, i32, i32, i32,
+                                    f32, f32, C.c_uint, vp, i32, i32, C.POINTER(vp)]
+    lib.pb_split_range.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.pb_split_ports.argtypes = [vp, C.POINTER(pb_split_port)]
+    lib.pb_split_connect.argtypes = [vp, C.POINTER(pb_split_port), C.POINTER(pb_split_port)]
     lib.pb_mlp_run_static.argtypes = [C.POINTER(C.c_int32), i32, f32, f32, C.c_uint, vp, vp, vp, vp, i32, vp, vp]
     _lib = lib
     return lib
@@ -110,6 +122,26 @@ def mlp_run_static(sizes, lr, momentum, flags, dev_w, dev_v, dev_xs, dev_labels,
         raise PBError(rc, lib.pb_last_error(None).decode())
 
 
+def _layer_arrays(layers, stage_of_layer):
+    arr = (pb_layer * len(layers))()
+    for q, L in enumerate(layers):
+        arr[q] = pb_layer(*L.astuple()) if hasattr(L, "astuple") else pb_layer(*L)
+    st = (C.c_int32 * len(layers))(*[int(s) for s in stage_of_layer])
+    return arr, st
+
+
+def split_plan(layers, stage_of_layer, in_shape, n_classes, n_ranks):
+    """pb_split_plan: [(lo, hi)] stage ranges of the ranks (host arithmetic only)."""
+    lib = load_library()
+    arr, st = _layer_arrays(layers, stage_of_layer)
+    lo, hi = (C.c_int32 * n_ranks)(), (C.c_int32 * n_ranks)()
+    rc = lib.pb_split_plan(arr, len(layers), st, int(in_shape[0]), int(in_shape[1]), int(in_shape[2]),
+                           int(n_classes), int(n_ranks), lo, hi)
+    if rc != 0:
+        raise PBError(rc, lib.pb_last_error(None).decode())
+    return [(int(a), int(b)) for a, b in zip(lo, hi)]
+
+
 def bench_l2_bandwidth(nbytes, iters=200, stream=0):
     """pb_bench_l2_bandwidth: GB/s (read + write) of an in-place sweep over `nbytes`."""
     lib = load_library()
@@ -134,16 +166,19 @@ class PB:
     """Owner of one pb_handle.  Methods mirror the C calls one to one."""
 
     def __init__(self, layers, stage_of_layer, in_shape, n_classes, lr, momentum,
-                 flags=PB_SC | PB_LWP, stream=0):
+                 flags=PB_SC | PB_LWP, stream=0, rank=None, n_ranks=None):
+        """rank / n_ranks given: pb_create_split (this handle runs one rank's stages)."""
         self._lib = load_library()
         self._h = C.c_void_p()
-        arr = (pb_layer * len(layers))()
-        for q, L in enumerate(layers):
-            arr[q] = pb_layer(*L.astuple()) if hasattr(L, "astuple") else pb_layer(*L)
-        st = (C.c_int32 * len(layers))(*[int(s) for s in stage_of_layer])
-        rc = self._lib.pb_create(arr, len(layers), st, int(in_shape[0]), int(in_shape[1]),
-                                 int(in_shape[2]), int(n_classes), float(lr), float(momentum),
-                                 int(flags), C.c_void_p(stream), C.byref(self._h))
+        arr, st = _layer_arrays(layers, stage_of_layer)
+        if n_ranks is None:
+            rc = self._lib.pb_create(arr, len(layers), st, int(in_shape[0]), int(in_shape[1]),
+                                     int(in_shape[2]), int(n_classes), float(lr), float(momentum),
+                                     int(flags), C.c_void_p(stream), C.byref(self._h))
+        else:
+            rc = self._lib.pb_create_split(arr, len(layers), st, int(in_shape[0]), int(in_shape[1]),
+                                           int(in_shape[2]), int(n_classes), float(lr), float(momentum),
+                                           int(flags), C.c_void_p(stream), int(rank), int(n_ranks), C.byref(self._h))
         if rc != 0:
             raise PBError(rc, self._lib.pb_last_error(None).decode())
         self.sample_elems = int(in_shape[0]) * int(in_shape[1]) * int(in_shape[2])
@@ -211,6 +246,21 @@ class PB:
     @property
     def device_bytes(self):
         return int(self._lib.pb_device_bytes(self._h))
+
+    def split_range(self):
+        lo, hi = C.c_int32(0), C.c_int32(0)
+        self._check(self._lib.pb_split_range(self._h, C.byref(lo), C.byref(hi)))
+        return int(lo.value), int(hi.value)
+
+    def split_ports(self):
+        port = pb_split_port()
+        self._check(self._lib.pb_split_ports(self._h, C.byref(port)))
+        return port
+
+    def split_connect(self, prev_rank_port, next_rank_port):
+        self._check(self._lib.pb_split_connect(
+            self._h, C.byref(prev_rank_port) if prev_rank_port is not None else None,
+            C.byref(next_rank_port) if next_rank_port is not None else None))
 
     def kernel_min_bytes(self, which):
         return float(self._lib.pb_kernel_min_bytes(self._h, int(which)))

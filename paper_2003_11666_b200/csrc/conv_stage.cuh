@@ -800,7 +800,7 @@ cast_weights_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restr
 
 // Weight stashing: files the weights (and normalisation scale) that this tick's forward
 // of every stage has used under the forward sample's ring slot, before the update
-// overwrites them.  16-byte copies (every tensor and slot starts on a 16-byte boundary).
+// overwrites them.  16-byte copies where source, ring and slot stride allow, else word by word.
 __global__ void __launch_bounds__(256)
 stash_copy_kernel(const StashRange* __restrict__ ranges, const StashChunk* __restrict__ chunks,
                   const TickState* __restrict__ ts, int par) {
@@ -810,13 +810,21 @@ stash_copy_kernel(const StashRange* __restrict__ ranges, const StashChunk* __res
     if (!sample_live(ts, i)) return;
     const long long bytes = R.n * R.esize;
     const char* src = static_cast<const char*>(R.src);
-    char* dst = static_cast<char*>(R.ring) + (size_t)slot_of(i, R.slots) * (size_t)((bytes + 15) / 16 * 16);
+    char* dst = static_cast<char*>(R.ring) + (size_t)slot_of(i, R.slots) * (size_t)R.stride;
     const long long end = min(bytes, ch.start + (long long)kStashChunkBytes);
-    long long b = ch.start + 16LL * threadIdx.x;
-    for (; b + 16 <= end; b += 16LL * 256) *reinterpret_cast<uint4*>(dst + b) = *reinterpret_cast<const uint4*>(src + b);
-    // ragged tail of the tensor (fewer than 16 bytes), byte by byte, by the thread whose turn it is
-    if (b < end && b + 16 > end)
-        for (long long q = b; q < end; ++q) dst[q] = src[q];
+    const bool wide = ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) == 0;
+    long long b = ch.start;                       // chunk starts are multiples of 16 bytes
+    if (wide) {
+        const long long full = ch.start + (end - ch.start) / 16 * 16;
+        for (long long q = b + 16LL * threadIdx.x; q < full; q += 16LL * 256)
+            *reinterpret_cast<uint4*>(dst + q) = *reinterpret_cast<const uint4*>(src + q);
+        b = full;
+    }
+    // the rest (everything when not 16-byte aligned) in elements of 2 or 4 bytes
+    if (R.esize == 4)
+        for (long long q = b + 4LL * threadIdx.x; q < end; q += 4LL * 256) *reinterpret_cast<float*>(dst + q) = *reinterpret_cast<const float*>(src + q);
+    else
+        for (long long q = b + 2LL * threadIdx.x; q < end; q += 2LL * 256) *reinterpret_cast<unsigned short*>(dst + q) = *reinterpret_cast<const unsigned short*>(src + q);
 }
 
 // Predicted weights re-made from the current state, w_hat = w - lr T v (LWP, velocity

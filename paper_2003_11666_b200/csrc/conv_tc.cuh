@@ -48,7 +48,7 @@ constexpr int kTcProducers = 128;             // warps 4-7
 constexpr int kTcMmaWarp = 8;
 constexpr int kTcThreads = 32 * (kTcMmaWarp + 1);
 constexpr int kTcTmemCols = 256;              // two accumulators of 128 columns
-constexpr int kTcWaitLimit = 1 << 22;
+constexpr long long kTcWaitNs = 200LL * 1000 * 1000;   // a barrier wait gives up after 0.2 s
 constexpr int kTcMaxK = 3072;                 // longest K loop of one dgrad / wgrad tile before K is sliced
 constexpr int kTcMaxKFprop = 8192;            // ... of a forward tile (a single slice lets the epilogue finish the stage's statistics)
 
@@ -104,14 +104,25 @@ __device__ __forceinline__ uint32_t mnmajor_off(int k, int mu) {
 }
 
 // Bounded wait on an mbarrier phase; gives up early once another warp has reported a failure.
+__device__ __forceinline__ long long global_ns() {
+    long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* fail) {
     uint32_t done = 0;
-    for (int it = 0; it < kTcWaitLimit && !done; ++it) {
+    long long t0 = 0;
+    for (int it = 0; !done; ++it) {
         asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
                      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (!done && (it & 63) == 63 && *fail) return false;
+        if (!done && (it & 63) == 63) {
+            if (*fail) return false;
+            const long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kTcWaitNs) return false;
+        }
     }
-    return done != 0;
+    return true;
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");

@@ -91,7 +91,7 @@ struct UpdRange {
 struct UpdChunk { int range, start; };
 // Weight stashing: one tensor whose forward copy (src) is filed under the forward sample's
 // slot of a ring, n elements of esize bytes each.
-struct StashRange { const void* src; void* ring; int slots, s, esize; long long n; };
+struct StashRange { const void* src; void* ring; int slots, s, esize; long long n, stride; };   // stride: bytes between ring slots
 struct StashChunk { int range; long long start; };
 constexpr int kStashChunkBytes = 32768;
 

@@ -240,7 +240,7 @@ void partition_fc(pb_handle* h, const std::vector<int>& fc_ids, std::vector<FcSe
 void build_fc_tables(pb_handle* h, const float* w_base, const float* v_base) {
     std::vector<int> idsA, idsB;
     for (const StageHost& x : h->stages) {
-        if (x.head_op != PB_FC) continue;
+        if (x.head_op != PB_FC || !h->owns(x.index)) continue;
         FcStage f{};
         f.in_dim = x.head.c_in; f.out_dim = x.head.c_out; f.s = x.index;
         f.relu = x.relu; f.is_last = x.loss; f.need_dx = x.src >= 0;
@@ -341,7 +341,7 @@ void plan_stash(pb_handle* h) {
         const size_t nw = x.head_op == PB_FC ? (size_t)x.head.c_in * x.head.c_out
                                              : (size_t)x.head.c_out * x.head.c_in * x.head.k * x.head.k;
         x.wstash_stride = x.head_op == PB_FC ? nw * 4 : align_up(nw * (x.tc ? 2 : 4), 16);
-        if (x.head_op == PB_CONV2D) x.gstash_stride = align_up((size_t)x.head.c_out * 4, 16);
+        if (x.head_op == PB_CONV2D) x.gstash_stride = (size_t)x.head.c_out * 4;       // slots of exactly c_out floats
     }
 }
 
@@ -564,7 +564,6 @@ bool fill_conv_tables(pb_handle* h) {
         for (int q : x.consumers_skip) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dskip, y.dskip_slots, 1}; }
         c.dz = x.dz;
         c.gstash = x.gstash; c.gstash_slots = x.stash_slots;
-        if (x.gstash && x.gstash_stride != (size_t)L.c_out * 4) c.gstash = nullptr;     // (channel counts are multiples of 4 in every supported stash layout; see validate_conv)
         c.fstat = x.fstat; c.fstat_stride = x.fstat_stride; c.bsum = x.bsum; c.npieces = x.npieces; c.gsum = x.gsum;
         {
             // Chunks of the first step: whole channels while they fit, else pieces of one channel.
@@ -679,13 +678,13 @@ bool fill_conv_tables(pb_handle* h) {
         for (int st = 0; st < r.n; st += kUpdChunk) h->h_chunks.push_back(UpdChunk{(int)h->h_upd.size(), st});
         h->h_upd.push_back(r);
         if (x.stash_slots > 0) {
-            auto add = [&](const void* src, void* ring, int esize, long long n) {
+            auto add = [&](const void* src, void* ring, int esize, long long n, size_t stride) {
                 for (long long b0 = 0; b0 < n * esize; b0 += kStashChunkBytes) h->h_stashchunks.push_back(StashChunk{(int)h->h_stash.size(), b0});
-                h->h_stash.push_back(StashRange{src, ring, x.stash_slots, x.index, esize, n});
+                h->h_stash.push_back(StashRange{src, ring, x.stash_slots, x.index, esize, n, (long long)stride});
             };
-            if (x.tc) add(h->d_wh16 + x.dev_off, x.wstash16, 2, nw);
-            else add(h->d_wh + x.dev_off, x.wstash, 4, nw);
-            add(h->d_wh + x.dev_off + nw, x.gstash, 4, L.c_out);
+            if (x.tc) add(h->d_wh16 + x.dev_off, x.wstash16, 2, nw, x.wstash_stride);
+            else add(h->d_wh + x.dev_off, x.wstash, 4, nw, x.wstash_stride);
+            add(h->d_wh + x.dev_off + nw, x.gstash, 4, L.c_out, x.gstash_stride);
         }
     }
     for (int q = 0; q < 3; ++q) balance_tc_tiles(h, h->h_tc, h->h_tctiles[q], h->h_tcbegin[q]);
@@ -706,7 +705,6 @@ int validate_conv(pb_handle* h) {
         if (x.has_pool && x.avgpool) return fail(nullptr, PB_E_UNSUPPORTED, "max-pool and average pool in one stage");
         if (x.avgpool && x.z.h * x.z.w > kPostChunk) return fail(nullptr, PB_E_UNSUPPORTED, "global average pool over more than 2048 pixels");
         if ((int)(x.consumers_main.size() + x.consumers_skip.size()) > kMaxDeltaSrc) return fail(nullptr, PB_E_UNSUPPORTED, "too many consumers of one stage");
-        if ((h->flags & PB_WEIGHT_STASH) && x.head.c_out % 4) return fail(nullptr, PB_E_UNSUPPORTED, "weight stashing needs channel counts that are multiples of 4");
     }
     for (const StageHost& x : h->stages)
         if (x.head_op == PB_FC && (x.has_skip || x.has_pool || x.avgpool || x.gn_groups)) return fail(nullptr, PB_E_UNSUPPORTED, "FC stages take only RELU or SOFTMAX_CE");
@@ -764,6 +762,7 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     h->d_w = c.take<float>(h->dev_params);
     if (!h->all_fc || (h->flags & PB_LWP_WFORM)) h->d_wh = c.take<float>(h->dev_params);
     *zero_from = c.off;
+    h->d_stamps = c.take<long long>(2);
     h->d_v = c.take<float>(h->dev_params);
     for (int q = 0; q < 2; ++q) h->d_bcnt[q] = c.take<int>(h->h_bundles.size() + 1);   // bundle counters (zero between launches)
     if (!h->all_fc) h->d_g = c.take<float>(h->dev_params);
@@ -867,6 +866,41 @@ void prof_collect(pb_handle* h) {
     h->ev_used = 0;
 }
 
+// ---------------------------------------------------------------- stage split
+// Contiguous ranges of stages for n ranks that minimise the largest per-rank sum of `cost`
+// (dynamic programme over the cut positions; every rank gets at least one stage).
+bool split_ranges(const std::vector<double>& cost, int n, std::vector<int>& lo, std::vector<int>& hi) {
+    const int S = (int)cost.size();
+    if (n < 1 || n > S) return false;
+    std::vector<double> pre(S + 1, 0.0);
+    for (int s = 0; s < S; ++s) pre[s + 1] = pre[s] + cost[s];
+    const double inf = 1e300;
+    std::vector<std::vector<double>> best(n + 1, std::vector<double>(S + 1, inf));
+    std::vector<std::vector<int>> cut(n + 1, std::vector<int>(S + 1, 0));
+    best[0][0] = 0.0;
+    for (int r = 1; r <= n; ++r)
+        for (int e = r; e <= S; ++e)
+            for (int b = r - 1; b < e; ++b) {
+                const double v = std::max(best[r - 1][b], pre[e] - pre[b]);
+                if (v < best[r][e]) { best[r][e] = v; cut[r][e] = b; }
+            }
+    lo.assign(n, 0); hi.assign(n, 0);
+    int e = S;
+    for (int r = n; r >= 1; --r) { hi[r - 1] = e; lo[r - 1] = cut[r][e]; e = cut[r][e]; }
+    return true;
+}
+
+int plan_split(pb_handle* h, int n_ranks, std::vector<int>& lo, std::vector<int>& hi) {
+    for (const StageHost& x : h->stages) {
+        if (x.head_op != PB_FC || x.has_skip) return fail(nullptr, PB_E_UNSUPPORTED, "the stage split supports fully connected networks only");
+        if (x.src != x.index - 1) return fail(nullptr, PB_E_UNSUPPORTED, "the stage split needs every stage to read the stage before it");
+    }
+    std::vector<double> cost;
+    for (const StageHost& x : h->stages) cost.push_back(16.0 * (double)x.n_params);      // one read and one write of w and v per tick
+    if (!split_ranges(cost, n_ranks, lo, hi)) return fail(nullptr, PB_E_ARG, "need 1 <= n_ranks <= number of stages");
+    return PB_OK;
+}
+
 // ---------------------------------------------------------------- ticks
 int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int label_value,
               int n_ticks, float* dev_losses) {
@@ -877,7 +911,9 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
     // Fully connected pipelines read the current sample straight from the caller's buffer,
     // 16 bytes at a time when the sample length is a multiple of 4: the buffer must then be
     // 16-byte aligned (checked here, on the host, before anything is launched).
-    if (h->all_fc && !h->h_fc.empty() && h->h_fc[0].vec == 4 && (reinterpret_cast<uintptr_t>(dev_xs) & 15) != 0)
+    const bool split = h->split_n > 1;
+    if (split && !h->split_connected) return fail(h, PB_E_ARG, "a split handle must be connected to its neighbours first (pb_split_connect)");
+    if (h->all_fc && h->owns(0) && !h->h_fc.empty() && h->h_fc[0].vec == 4 && (reinterpret_cast<uintptr_t>(dev_xs) & 15) != 0)
         return fail(h, PB_E_ARG, "the sample buffer must be 16-byte aligned when the sample length is a multiple of 4");
     if (h->profile) for (auto& p : h->prof) p = ProfileClass{};
     const bool fused_last = h->nctaB == 0;      // the last stage rides in the phase-0 launch
@@ -890,6 +926,15 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
         const int par = (int)((t_base + k) & 1);
         if (h->all_fc) {
             // one launch: ingest + every stage (two when the last stage needs its own)
+            const float* xs_mine = h->owns(0) ? dev_xs : nullptr;       // only the rank with stage 0 ingests the sample
+            if (split) {
+                // wait for the neighbours' previous tick; ranks without stage 0 file the label here,
+                // ranks without the last stage report NaN as this tick's loss
+                split_wait_kernel<<<1, 32, 0, h->stream>>>(h->links, h->d_ts, par, h->owns(0) ? nullptr : h->label_ring, h->S,
+                                                           dev_labels, label_value, t_base,
+                                                           (!h->owns(h->S - 1) && dev_losses) ? dev_losses : nullptr);
+                h->last_launches += 1;
+            }
             prof_begin(h, 0);
             {
                 // consecutive ticks overlap their launch latency (see the kernel's first lines)
@@ -898,10 +943,10 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
                 cudaLaunchAttribute attr[1];
                 attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
                 attr[0].val.programmaticStreamSerializationAllowed = 1;
-                cfg.attrs = attr; cfg.numAttrs = (fused_last && !h->profile) ? 1 : 0;
+                cfg.attrs = attr; cfg.numAttrs = (fused_last && !h->profile && !split) ? 1 : 0;
                 cudaLaunchKernelEx(&cfg, fc_tick_kernel, (const FcStage*)h->d_fc, (const FcSeg*)h->d_segA, (const int*)h->d_ctaA, h->d_ts,
                                    h->S, 0, par, fused_last ? 1 : 0, h->label_ring, dev_losses, t_base,
-                                   dev_xs, dev_labels, label_value, h->in_ring, h->in_slots, elems);
+                                   xs_mine, dev_labels, label_value, h->in_ring, h->in_slots, elems);
             }
             prof_end(h);
             h->last_launches += 1;
@@ -911,6 +956,10 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
                                                                       h->label_ring, dev_losses, t_base,
                                                                       nullptr, nullptr, 0, nullptr, 0, 0);
                 prof_end(h);
+                h->last_launches += 1;
+            }
+            if (split) {
+                split_handoff_kernel<<<1, 256, 0, h->stream>>>(h->links, h->d_ts, par, h->S);
                 h->last_launches += 1;
             }
         } else {
@@ -1059,11 +1108,10 @@ int check_device_error(pb_handle* h) {
 }  // namespace
 
 // ---------------------------------------------------------------- C interface
-extern "C" {
-
-int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_layer, int in_c, int in_h,
-              int in_w, int n_classes, float lr, float momentum, unsigned flags, void* stream,
-              pb_handle** out) {
+namespace {
+int create_engine(const pb_layer* layers, int n_layers, const int32_t* stage_of_layer, int in_c, int in_h,
+                  int in_w, int n_classes, float lr, float momentum, unsigned flags, void* stream,
+                  int rank, int n_ranks, pb_handle** out) {
     if (out) *out = nullptr;
     if (!layers || !stage_of_layer || !out || n_layers <= 0 || in_c <= 0 || in_h <= 0 || in_w <= 0 || n_classes <= 0)
         return fail(nullptr, PB_E_ARG, "pb_create: NULL pointer or non-positive size");
@@ -1080,6 +1128,13 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     int rc = parse_layers(h, layers, n_layers, stage_of_layer);
     if (rc != PB_OK) { delete h; return rc; }
     schedule_constants(h);
+    h->s_lo = 0; h->s_hi = h->S;
+    if (n_ranks > 1) {
+        std::vector<int> lo, hi;
+        rc = plan_split(h, n_ranks, lo, hi);
+        if (rc != PB_OK) { delete h; return rc; }
+        h->split_rank = rank; h->split_n = n_ranks; h->s_lo = lo[rank]; h->s_hi = hi[rank];
+    }
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e != cudaSuccess) { std::string m = cudaGetErrorString(e); delete h; return fail(nullptr, PB_E_CUDA, "pb_create: no CUDA device: " + m); }
@@ -1170,6 +1225,82 @@ int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_laye
     *out = h;
     return PB_OK;
 }
+}  // namespace
+
+extern "C" {
+
+int pb_create(const pb_layer* layers, int n_layers, const int32_t* stage_of_layer, int in_c, int in_h,
+              int in_w, int n_classes, float lr, float momentum, unsigned flags, void* stream,
+              pb_handle** out) {
+    return create_engine(layers, n_layers, stage_of_layer, in_c, in_h, in_w, n_classes, lr, momentum, flags, stream, 0, 1, out);
+}
+
+int pb_create_split(const pb_layer* layers, int n_layers, const int32_t* stage_of_layer, int in_c, int in_h,
+                    int in_w, int n_classes, float lr, float momentum, unsigned flags, void* stream,
+                    int rank, int n_ranks, pb_handle** out) {
+    if (out) *out = nullptr;
+    if (n_ranks < 1 || rank < 0 || rank >= n_ranks) return fail(nullptr, PB_E_ARG, "pb_create_split: need 0 <= rank < n_ranks");
+    return create_engine(layers, n_layers, stage_of_layer, in_c, in_h, in_w, n_classes, lr, momentum, flags, stream, rank, n_ranks, out);
+}
+
+int pb_split_plan(const pb_layer* layers, int n_layers, const int32_t* stage_of_layer, int in_c, int in_h, int in_w,
+                  int n_classes, int n_ranks, int32_t* lo, int32_t* hi) {
+    if (!layers || !stage_of_layer || !lo || !hi || n_layers <= 0 || in_c <= 0 || in_h <= 0 || in_w <= 0 || n_classes <= 0)
+        return fail(nullptr, PB_E_ARG, "pb_split_plan: NULL pointer or non-positive size");
+    for (int q = 1; q < n_layers; ++q)
+        if (stage_of_layer[q] < stage_of_layer[q - 1]) return fail(nullptr, PB_E_ARG, "pb_split_plan: stage indices must not decrease");
+    pb_handle hs;                       // host bookkeeping only
+    hs.n_classes = n_classes; hs.in_shape = Shape{in_c, in_h, in_w};
+    int rc = parse_layers(&hs, layers, n_layers, stage_of_layer);
+    if (rc != PB_OK) return rc;
+    std::vector<int> l, u;
+    rc = plan_split(&hs, n_ranks, l, u);
+    if (rc != PB_OK) return rc;
+    for (int r = 0; r < n_ranks; ++r) { lo[r] = l[r]; hi[r] = u[r]; }
+    return PB_OK;
+}
+
+int pb_split_range(const pb_handle* h, int32_t* lo, int32_t* hi) {
+    if (!h || !lo || !hi) return PB_E_ARG;
+    *lo = h->split_n > 1 ? h->s_lo : 0; *hi = h->split_n > 1 ? h->s_hi : h->S;
+    return PB_OK;
+}
+
+int pb_split_ports(pb_handle* h, pb_split_port* mine) {
+    if (!h || !mine) return PB_E_ARG;
+    if (h->split_n <= 1) return fail(h, PB_E_ARG, "pb_split_ports: not a split handle");
+    // the neighbours' boundary tensors land in this handle's own copies of the neighbour stages' rings
+    mine->act = h->s_lo > 0 ? (void*)h->stages[h->s_lo - 1].out_ring : nullptr;
+    mine->act_stamp = h->s_lo > 0 ? (void*)(h->d_stamps + 0) : nullptr;
+    mine->grad = h->s_hi < h->S ? (void*)h->stages[h->s_hi].dx : nullptr;
+    mine->grad_stamp = h->s_hi < h->S ? (void*)(h->d_stamps + 1) : nullptr;
+    return PB_OK;
+}
+
+int pb_split_connect(pb_handle* h, const pb_split_port* prev_rank, const pb_split_port* next_rank) {
+    if (!h) return PB_E_ARG;
+    if (h->split_n <= 1) return fail(h, PB_E_ARG, "pb_split_connect: not a split handle");
+    if ((h->s_lo > 0) != (prev_rank != nullptr) || (h->s_hi < h->S) != (next_rank != nullptr))
+        return fail(h, PB_E_ARG, "pb_split_connect: a port is needed for exactly the neighbours that exist");
+    SplitLinks L{};
+    if (prev_rank) {
+        if (!prev_rank->grad || !prev_rank->grad_stamp) return fail(h, PB_E_ARG, "pb_split_connect: the previous rank's gradient port is empty");
+        const StageHost& x = h->stages[h->s_lo];                 // own first stage: its input gradient goes back
+        L.act_stamp = h->d_stamps + 0;
+        L.grad_src = x.dx; L.grad_slots = x.dx_slots; L.grad_nparts = x.dx_nparts; L.grad_dim = x.in.elems(); L.grad_stage = x.index;
+        L.grad_dst = static_cast<float*>(prev_rank->grad); L.grad_dst_stamp = static_cast<long long*>(prev_rank->grad_stamp);
+    }
+    if (next_rank) {
+        if (!next_rank->act || !next_rank->act_stamp) return fail(h, PB_E_ARG, "pb_split_connect: the next rank's activation port is empty");
+        const StageHost& x = h->stages[h->s_hi - 1];             // own last stage: its output goes forward
+        L.grad_stamp = h->d_stamps + 1;
+        L.act_src = x.out_ring; L.act_slots = x.out_slots; L.act_dim = x.out.elems(); L.act_stage = x.index;
+        L.act_dst = static_cast<float*>(next_rank->act); L.act_dst_stamp = static_cast<long long*>(next_rank->act_stamp);
+    }
+    h->links = L;
+    h->split_connected = true;
+    return PB_OK;
+}
 
 int pb_set_weights(pb_handle* h, const float* host_w, size_t n) {
     if (!h) return PB_E_ARG;
@@ -1248,7 +1379,7 @@ int pb_set_update_size(pb_handle* h, int n_samples) {
 
 int pb_tick(pb_handle* h, const float* dev_x, int label, float* host_loss) {
     if (!h) return PB_E_ARG;
-    if (!dev_x || label < 0 || label >= h->n_classes) return fail(h, PB_E_ARG, "pb_tick: NULL input or label out of range");
+    if ((!dev_x && h->owns(0)) || label < 0 || label >= h->n_classes) return fail(h, PB_E_ARG, "pb_tick: NULL input or label out of range");
     int rc = run_ticks(h, dev_x, nullptr, label, 1, h->d_loss1);
     if (rc != PB_OK) return rc;
     if (host_loss) {
@@ -1261,7 +1392,7 @@ int pb_tick(pb_handle* h, const float* dev_x, int label, float* host_loss) {
 int pb_run(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int n_ticks, float* dev_losses) {
     if (!h) return PB_E_ARG;
     if (n_ticks == 0) return PB_OK;         // nothing to do; the pointers are not looked at
-    if (!dev_xs || !dev_labels || n_ticks < 0) return fail(h, PB_E_ARG, "pb_run: NULL pointer or negative count");
+    if ((!dev_xs && h->owns(0)) || !dev_labels || n_ticks < 0) return fail(h, PB_E_ARG, "pb_run: NULL pointer or negative count");
     return run_ticks(h, dev_xs, dev_labels, 0, n_ticks, dev_losses);
 }
 
@@ -1296,8 +1427,10 @@ int pb_run_host(pb_handle* h, const float* host_xs, const int32_t* host_labels, 
 static int get_params(pb_handle* h, const float* dev, float* host, size_t n, const char* who) {
     if (!h) return PB_E_ARG;
     if (!host || n != h->n_params) return fail(h, PB_E_ARG, std::string(who) + ": need pb_num_params() floats");
-    for (const StageHost& x : h->stages)
+    for (const StageHost& x : h->stages) {
+        if (!h->owns(x.index)) { std::memset(host + x.user_off, 0, x.n_params * sizeof(float)); continue; }   // that stage lives on another rank
         PB_CUDA(h, cudaMemcpyAsync(host + x.user_off, dev + x.dev_off, x.n_params * sizeof(float), cudaMemcpyDeviceToHost, h->stream));
+    }
     int rc = check_device_error(h);
     if (rc != PB_OK) return rc;
     std::vector<float> tmp;

@@ -8,6 +8,7 @@
 #include "conv_types.h"
 #include "conv_tc.cuh"
 #include "conv_group.cuh"
+#include "split.cuh"
 
 namespace pb {
 
@@ -113,6 +114,13 @@ struct pb_handle {
     size_t group_smem_fwd = 0, group_smem_bwd = 0;
     std::vector<pb::StashRange> h_stash; pb::StashRange* d_stash = nullptr;
     std::vector<pb::StashChunk> h_stashchunks; pb::StashChunk* d_stashchunks = nullptr;
+
+    // stage split over several GPUs: this handle runs stages [s_lo, s_hi) (the whole network when n_ranks == 1)
+    int split_rank = 0, split_n = 1, s_lo = 0, s_hi = 0;
+    long long* d_stamps = nullptr;              // [0]: previous rank's activation stamp, [1]: next rank's gradient stamp
+    pb::SplitLinks links{};
+    bool split_connected = false;
+    bool owns(int s) const { return split_n <= 1 || (s >= s_lo && s < s_hi); }
 
     long long tick = 0, last_launches = 0;
     bool profile = false;

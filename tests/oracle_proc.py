@@ -36,12 +36,29 @@ def _serve(conn, wl, dtype_name, kw):
             return
 
 
+# Several instances run side by side, each with its own BLAS thread pool: unbounded pools
+# oversubscribe the cores (busy-waiting threads) and make every instance many times slower.
+MAX_SIDE_BY_SIDE = 3
+_THREAD_VARS = ("OMP_NUM_THREADS", "OPENBLAS_NUM_THREADS", "MKL_NUM_THREADS")
+
+
 class RemoteOracle:
     def __init__(self, wl, dtype=np.float64, **kw):
+        import os
         ctx = mp.get_context("spawn")
         self.conn, child = ctx.Pipe()
         self.proc = ctx.Process(target=_serve, args=(child, wl, np.dtype(dtype).name, kw), daemon=True)
-        self.proc.start()
+        threads = str(max(1, ((os.cpu_count() or 4) - 1) // MAX_SIDE_BY_SIDE))
+        saved = {v: os.environ.get(v) for v in _THREAD_VARS}
+        os.environ.update({v: threads for v in _THREAD_VARS})      # inherited by the spawned interpreter
+        try:
+            self.proc.start()
+        finally:
+            for v, old in saved.items():
+                if old is None:
+                    os.environ.pop(v, None)
+                else:
+                    os.environ[v] = old
         child.close()
         self.last_max_logit = 0.0
 

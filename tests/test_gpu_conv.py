@@ -55,6 +55,9 @@ def test_tiny_bottleneck_projection_shortcuts_float32():
 #     engine's own step must satisfy the update rule exactly (a property that no decision
 #     can blur).  ReLU masks and max-pool winners themselves are pinned at 1e-4 by the
 #     float32 tests, which run the same normalisation / activation / pooling kernels.
+#     (The tiny bottleneck net is not run with ReLU on this path: its smallest activation
+#     has 64 units, so ONE flipped unit is an eighth of a layer's gradient and the bound
+#     4/sqrt(64) would say nothing; the net with 16384-unit activations below does.)
 BF16_STATISTICAL = dict(spread_factor=3.0, flip_allowance=4.0, check_update_rule=True)
 
 
@@ -62,13 +65,6 @@ def test_tiny_bottleneck_bf16_smooth_is_within_2e_2_on_every_tensor():
     wl = tiny_resnet(bottleneck=True, flags=3 | 8, relu=False)
     n = 2 * (wl.n_stages - 1) + 24
     w = compare_ticks(wl, n, TOL_BF16, check_update_rule=True)
-    assert w["ticks"] == n and w["min_updates"] >= 24
-
-
-def test_tiny_bottleneck_bf16_operands():
-    wl = tiny_resnet(bottleneck=True, flags=3 | 8)
-    n = 2 * (wl.n_stages - 1) + 24
-    w = compare_ticks(wl, n, TOL_BF16, **BF16_STATISTICAL)
     assert w["ticks"] == n and w["min_updates"] >= 24
 
 
