@@ -4,8 +4,11 @@
 // or differentiated (backward).  For the stages of a deep bottleneck network a
 // group - and even a bundle of groups that together span 8 channels, the unit
 // of the bfloat16 [pixel][channel] copies - is at most a hundred kilobytes, so
-// ONE thread block takes a bundle through both steps with the intermediate in
-// shared memory, in one launch and with one pass over memory per direction:
+// a CLUSTER of four thread blocks takes a bundle through both steps with the
+// intermediate in shared memory, in one launch and with one pass over memory per
+// direction; each block of the cluster owns a quarter of the pixels (so that many
+// blocks fit on an SM) and the per-channel sums cross the cluster through
+// distributed shared memory:
 //   forward   merge the (channel, column tile) statistics that the GEMM epilogue
 //             left -> group mean and 1/std -> normalise, add the skip input,
 //             ReLU -> float32 output (only where somebody reads it), ReLU mask,
@@ -19,6 +22,8 @@
 // Reductions have a fixed order (lanes over pixels, then a warp shuffle tree), so
 // results do not depend on scheduling.
 #pragma once
+#include <cooperative_groups.h>
+
 #include "conv_stage.cuh"
 
 namespace pb {
@@ -27,6 +32,7 @@ constexpr int kGroupThreads = 256;
 constexpr int kGroupWarps = kGroupThreads / 32;
 constexpr int kGroupMaxElems = 25088;          // elements of a bundle that stay in shared memory (98 KB as float32)
 constexpr int kGroupMaxChannels = 64;
+constexpr int kGroupSplit = 4;                 // blocks (one cluster) that share a bundle's pixels
 
 // One block's bundle: groups [grp0, grp0 + ngrp) of one stage.
 struct GroupBlock { int stage, grp0, ngrp; };
@@ -36,37 +42,71 @@ struct GroupShared {
     float mean[kGroupMaxChannels], rstd[kGroupMaxChannels];   // per channel copy of its group's statistics
     float s1[kGroupMaxChannels], s2[kGroupMaxChannels];       // per channel sums of dn and dn * zhat
     float m1[kGroupMaxChannels], m2[kGroupMaxChannels];       // per channel copy of its group's means
+    float t1[kGroupMaxChannels], t2[kGroupMaxChannels];       // the sums over the whole cluster
 };
+
+// Pixel units [lo, hi) of block `rank` of a bundle's cluster (npu units of VEC pixels per channel).
+__device__ __forceinline__ void group_range(int npu, int rank, int& lo, int& hi) {
+    lo = (int)((long long)npu * rank / kGroupSplit);
+    hi = (int)((long long)npu * (rank + 1) / kGroupSplit);
+}
 
 // ---------------------------------------------------------------- forward
 template <int VEC>
-__device__ void group_forward(const ConvStage& st, const GroupBlock gb, long long t, float* buf, GroupShared& sh) {
+__device__ void group_forward(const ConvStage& st, const GroupBlock gb, int rank, long long t, float* buf, GroupShared& sh) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long i = t - st.s;
     const int slot = slot_of(i, st.slots);
     const int hw = st.oh * st.ow, cpg = st.cpg, c0 = gb.grp0 * cpg, nch = gb.ngrp * cpg;
     const size_t zelems = (size_t)st.co * hw;
-    // ---- group statistics from the GEMM epilogue's partials (count, mean, M2 per channel and column tile)
-    for (int g = warp; g < gb.ngrp; g += kGroupWarps) {
+    // ---- group statistics from the GEMM epilogue's partials (count, mean, M2 per channel and column
+    // tile): every thread folds the entries k = tid, tid + 256, ... of a group into one triple (all its
+    // loads are independent: one memory latency), then the triples are merged along a fixed tree
+    for (int g = 0; g < gb.ngrp; ++g) {
         const int grp = gb.grp0 + g, nidx = st.fstat_stride;
         const float* f = st.fstat + (size_t)grp * nidx * 3;
-        float tot = 0.f, wsum = 0.f;
-        for (int k = lane; k < nidx; k += 32) { const float n = f[3 * k]; tot += n; wsum = fmaf(n, f[3 * k + 1], wsum); }
-        tot = warp_sum(tot);
-        const float mean = warp_sum(wsum) / tot;
-        float m2 = 0.f;
-        for (int k = lane; k < nidx; k += 32) { const float d = f[3 * k + 1] - mean; m2 += f[3 * k + 2] + f[3 * k] * d * d; }
-        const float rstd = rsqrtf(warp_sum(m2) / tot + kGnEps);
-        if (lane == 0) {
-            st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0] = mean;
-            st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 1] = rstd;
+        float n = 0.f, mean = 0.f, m2 = 0.f;
+        for (int k = tid; k < nidx; k += kGroupThreads) {
+            const float nb = f[3 * k], mb = f[3 * k + 1], qb = f[3 * k + 2];
+            const float tot = n + nb, dl = mb - mean;
+            if (tot > 0.f) { mean += dl * (nb / tot); m2 += qb + dl * dl * (n * nb / tot); }
+            n = tot;
         }
-        for (int cl = lane; cl < cpg; cl += 32) {
-            const int c = c0 + g * cpg + cl;
-            sh.gs[g * cpg + cl] = st.wh[st.nw + c] * rstd;
-            sh.bb[g * cpg + cl] = st.wh[st.nw + st.co + c];
-            sh.mean[g * cpg + cl] = mean;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float nb = __shfl_xor_sync(0xffffffffu, n, o), mb = __shfl_xor_sync(0xffffffffu, mean, o), qb = __shfl_xor_sync(0xffffffffu, m2, o);
+            // (both partners compute the same merged triple: a and b enter symmetrically up to the sign of dl)
+            const bool low = (lane & o) == 0;
+            const float na = low ? n : nb, ma = low ? mean : mb, qa = low ? m2 : qb;
+            const float nc = low ? nb : n, mc = low ? mb : mean, qc = low ? qb : m2;
+            const float tot = na + nc, dl = mc - ma;
+            if (tot > 0.f) { mean = ma + dl * (nc / tot); m2 = qa + qc + dl * dl * (na * nc / tot); } else { mean = 0.f; m2 = 0.f; }
+            n = tot;
         }
+        if (lane == 0) { sh.s1[warp] = n; sh.s2[warp] = mean; sh.t1[warp] = m2; }
+        __syncthreads();
+        if (tid == 0) {
+            float na = sh.s1[0], ma = sh.s2[0], qa = sh.t1[0];
+            for (int w = 1; w < kGroupWarps; ++w) {
+                const float nc = sh.s1[w], mc = sh.s2[w], qc = sh.t1[w];
+                const float tot = na + nc, dl = mc - ma;
+                if (tot > 0.f) { ma += dl * (nc / tot); qa += qc + dl * dl * (na * nc / tot); }
+                na = tot;
+            }
+            const float rstd = rsqrtf(qa / na + kGnEps);
+            sh.m1[g] = ma; sh.m2[g] = rstd;
+            if (rank == 0) {                   // (every block of the bundle computes the same numbers)
+                st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0] = ma;
+                st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 1] = rstd;
+            }
+        }
+        __syncthreads();
+    }
+    for (int cl = tid; cl < nch; cl += kGroupThreads) {
+        const int g = cl / cpg, c = c0 + cl;
+        sh.gs[cl] = st.wh[st.nw + c] * sh.m2[g];
+        sh.bb[cl] = st.wh[st.nw + st.co + c];
+        sh.mean[cl] = sh.m1[g];
     }
     __syncthreads();
     const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
@@ -74,66 +114,73 @@ __device__ void group_forward(const ConvStage& st, const GroupBlock gb, long lon
         ? st.skip_ring + (size_t)slot_of(i, st.skip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
     unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems;
     float* __restrict__ out = st.out_ring + (size_t)slot * zelems;
-    __nv_bfloat16* t16 = reinterpret_cast<__nv_bfloat16*>(buf);          // [nch][hw + 2]
-    const int rs = hw + 2;
     const int npu = hw / VEC;
-    // ---- normalise, skip, ReLU: a warp per channel, lanes over the pixels
-    for (int cl = warp; cl < nch; cl += kGroupWarps) {
-        const int c = c0 + cl;
+    int u_lo, u_hi;
+    group_range(npu, rank, u_lo, u_hi);
+    const int p_lo = u_lo * VEC, np = (u_hi - u_lo) * VEC;               // this block's pixels
+    __nv_bfloat16* t16 = reinterpret_cast<__nv_bfloat16*>(buf);          // [nch][np + 2]
+    const int rs = np + 2;
+    // ---- normalise, skip, ReLU: the bundle's (channel, pixel unit) pairs spread flat over the
+    // block, four units of a thread in flight at a time (a channel's share of the pixels can be
+    // a dozen pixels: per-channel loops would wait one memory latency per channel)
+    const int upc = u_hi - u_lo, total = nch * upc;
+    const float inv_upc = 1.f / (float)max(upc, 1);
+#pragma unroll 4
+    for (int idx = tid; idx < total; idx += kGroupThreads) {
+        const int cl = quot(idx, inv_upc), u = u_lo + idx - cl * upc;
+        const int c = c0 + cl, p = u * VEC;
         const float gs = sh.gs[cl], bb = sh.bb[cl], mean = sh.mean[cl];
         const size_t base = (size_t)c * hw;
-        for (int u = lane; u < npu; u += 32) {
-            const int p = u * VEC;
-            float zv[VEC], sv[VEC], a[VEC];
-            unsigned char cd[VEC];
-            vload<VEC>(zv, z + base + p);
-            if (!sk) {
+        float zv[VEC], sv[VEC], a[VEC];
+        unsigned char cd[VEC];
+        vload<VEC>(zv, z + base + p);
+        if (!sk) {
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) sv[e] = 0.f;
-            } else if (st.skip_mode == 0) {
-                vload<VEC>(sv, sk + base + p);
-            } else {
+            for (int e = 0; e < VEC; ++e) sv[e] = 0.f;
+        } else if (st.skip_mode == 0) {
+            vload<VEC>(sv, sk + base + p);
+        } else {
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) sv[e] = skip_value(st, sk, c, (p + e) / st.ow, (p + e) % st.ow);
-            }
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-                const float v = fmaf(gs, zv[e] - mean, bb) + sv[e];
-                const bool pass = st.relu ? v > 0.f : true;
-                cd[e] = pass ? 1 : 0;
-                a[e] = pass ? v : 0.f;
-                t16[cl * rs + p + e] = __float2bfloat16_rn(a[e]);
-            }
-            stb<VEC>(code + base + p, cd);
-            if (st.need_out32) vstore<VEC>(out + base + p, a);
+            for (int e = 0; e < VEC; ++e) sv[e] = skip_value(st, sk, c, (p + e) / st.ow, (p + e) % st.ow);
         }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            const float v = fmaf(gs, zv[e] - mean, bb) + sv[e];
+            const bool pass = st.relu ? v > 0.f : true;
+            cd[e] = pass ? 1 : 0;
+            a[e] = pass ? v : 0.f;
+            t16[cl * rs + p - p_lo + e] = __float2bfloat16_rn(a[e]);
+        }
+        stb<VEC>(code + base + p, cd);
+        if (st.need_out32) vstore<VEC>(out + base + p, a);
     }
     __syncthreads();
     // ---- bfloat16 [pixel][channel] copy: 16-byte runs of 8 channels (bundles span multiples of 8 channels)
     __nv_bfloat16* __restrict__ out16 = st.out16 + (size_t)slot * zelems;
     const int ng = nch >> 3;
     const unsigned short* s16 = reinterpret_cast<const unsigned short*>(t16);
-    for (int idx = tid; idx < ng * hw; idx += kGroupThreads) {
-        const int u = idx / hw, p = idx - u * hw;           // pixels fastest: conflict-free shared-memory reads
+    for (int idx = tid; idx < ng * np; idx += kGroupThreads) {
+        const int u = idx / np, p = idx - u * np;           // pixels fastest: conflict-free shared-memory reads
         const unsigned short* src = s16 + (size_t)(u * 8) * rs + p;
         uint4 v;
         v.x = src[0] | ((unsigned)src[rs] << 16);
         v.y = src[2 * rs] | ((unsigned)src[3 * rs] << 16);
         v.z = src[4 * rs] | ((unsigned)src[5 * rs] << 16);
         v.w = src[6 * rs] | ((unsigned)src[7 * rs] << 16);
-        *reinterpret_cast<uint4*>(out16 + (size_t)p * st.co + c0 + u * 8) = v;
+        *reinterpret_cast<uint4*>(out16 + (size_t)(p_lo + p) * st.co + c0 + u * 8) = v;
     }
 }
 
-__global__ void __launch_bounds__(kGroupThreads, 2)
+__global__ void __launch_bounds__(kGroupThreads, 4)
 conv_group_fwd_kernel(const ConvStage* __restrict__ stages, const GroupBlock* __restrict__ blocks, int nblocks,
                       const TickState* __restrict__ ts, int S, int par) {
     extern __shared__ __align__(16) float group_buf[];
     __shared__ GroupShared sh;
     __shared__ ConvStage st;
     (void)S;
-    if ((int)blockIdx.x >= nblocks) return;
-    const GroupBlock gb = blocks[blockIdx.x];
+    if ((int)blockIdx.x >= nblocks * kGroupSplit) return;
+    const GroupBlock gb = blocks[blockIdx.x / kGroupSplit];
+    const int rank = blockIdx.x % kGroupSplit;
     {
         const int* s_ = reinterpret_cast<const int*>(&stages[gb.stage]);
         int* d_ = reinterpret_cast<int*>(&st);
@@ -142,13 +189,16 @@ conv_group_fwd_kernel(const ConvStage* __restrict__ stages, const GroupBlock* __
     __syncthreads();
     const long long t = ts->cnt[par];
     if (!sample_live(ts, t - st.s)) return;
-    if (st.vec4) group_forward<4>(st, gb, t, group_buf, sh);
-    else group_forward<1>(st, gb, t, group_buf, sh);
+    if (st.vec4) group_forward<4>(st, gb, rank, t, group_buf, sh);
+    else group_forward<1>(st, gb, rank, t, group_buf, sh);
 }
 
 // ---------------------------------------------------------------- backward
 template <int VEC>
 __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long long j, float* dn, GroupShared& sh) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int slot = slot_of(j, st.slots);
     const int hw = st.oh * st.ow, cpg = st.cpg, c0 = gb.grp0 * cpg, nch = gb.ngrp * cpg;
@@ -156,8 +206,12 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
     const float* __restrict__ z = st.z_ring + (size_t)slot * zelems;
     const unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems;
     const float* __restrict__ gam = st.gstash ? st.gstash + (size_t)slot_of(j, st.gstash_slots) * st.co : st.w + st.nw;
-    const int rs = hw + 4;                                   // row pitch of dn in shared memory (a multiple of 4 when hw is)
     const int npu = hw / VEC;
+    int u_lo, u_hi;
+    group_range(npu, rank, u_lo, u_hi);
+    const int p_lo = u_lo * VEC, np = (u_hi - u_lo) * VEC;   // this block's pixels
+    const int rs = np + 4;                                   // row pitch of dn and zhat in shared memory
+    float* zh = dn + (size_t)nch * rs;                       // normalised conv output, kept beside dn
     for (int cl = tid; cl < nch; cl += kGroupThreads) {
         const int grp = (c0 + cl) / cpg;
         sh.mean[cl] = st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0];
@@ -165,40 +219,71 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
         sh.gs[cl] = gam[c0 + cl];
     }
     __syncthreads();
-    // ---- gradient at the normalised activation and its per-channel sums: a warp per channel
-    for (int cl = warp; cl < nch; cl += kGroupWarps) {
+    // where each consumer's partial rows for this sample start (the same for the whole block)
+    const float* dptr[kMaxDeltaSrc];
+    int dnp[kMaxDeltaSrc];
+#pragma unroll
+    for (int q = 0; q < kMaxDeltaSrc; ++q) {
+        const bool on = q < st.n_dsrc;
+        dnp[q] = on ? st.dsrc[q].nparts : 0;
+        dptr[q] = on ? st.dsrc[q].ptr + (size_t)slot_of(j, st.dsrc[q].slots) * st.dsrc[q].nparts * zelems : nullptr;
+    }
+    // ---- gradient at the normalised activation, and the normalised conv output, into shared
+    // memory: the bundle's (channel, pixel unit) pairs spread flat over the block, several units
+    // of a thread in flight at a time
+    const int upc = u_hi - u_lo, total = nch * upc;
+    const float inv_upc = 1.f / (float)max(upc, 1);
+#pragma unroll 2
+    for (int idx = tid; idx < total; idx += kGroupThreads) {
+        const int cl = quot(idx, inv_upc), u = u_lo + idx - cl * upc;
+        const int p = u * VEC;
         const size_t base = (size_t)(c0 + cl) * hw;
         const float mean = sh.mean[cl], rstd = sh.rstd[cl];
+        float d[VEC], zv[VEC];
+        unsigned char cd[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) d[e] = 0.f;
+        vload<VEC>(zv, z + base + p);
+        ldb<VEC>(cd, code + base + p);
+#pragma unroll
+        for (int q = 0; q < kMaxDeltaSrc; ++q) {
+            const float* bp = dptr[q] + base + p;
+            for (int kp = 0; kp < dnp[q]; ++kp, bp += zelems) {
+                float r[VEC];
+                vload<VEC>(r, bp);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) d[e] += r[e];
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            dn[cl * rs + p - p_lo + e] = cd[e] ? d[e] : 0.f;
+            zh[cl * rs + p - p_lo + e] = (zv[e] - mean) * rstd;
+        }
+    }
+    __syncthreads();
+    // ---- per-channel sums of dn and dn * zhat over this block's pixels: a warp per channel, from shared memory
+    for (int cl = warp; cl < nch; cl += kGroupWarps) {
         float a1 = 0.f, a2 = 0.f;
-        for (int u = lane; u < npu; u += 32) {
-            const int p = u * VEC;
-            float d[VEC], zv[VEC];
-            unsigned char cd[VEC];
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) d[e] = 0.f;
-            vload<VEC>(zv, z + base + p);
-            ldb<VEC>(cd, code + base + p);
-            for (int q = 0; q < st.n_dsrc; ++q) {
-                const float* bp = st.dsrc[q].ptr + (size_t)slot_of(j, st.dsrc[q].slots) * st.dsrc[q].nparts * zelems + base + p;
-                for (int kp = 0; kp < st.dsrc[q].nparts; ++kp, bp += zelems) {
-                    float r[VEC];
-                    vload<VEC>(r, bp);
-#pragma unroll
-                    for (int e = 0; e < VEC; ++e) d[e] += r[e];
-                }
-            }
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-                d[e] = cd[e] ? d[e] : 0.f;
-                a1 += d[e];
-                a2 = fmaf(d[e], (zv[e] - mean) * rstd, a2);
-                dn[cl * rs + p + e] = d[e];
-            }
+        for (int p = lane; p < np; p += 32) {
+            const float d = dn[cl * rs + p];
+            a1 += d;
+            a2 = fmaf(d, zh[cl * rs + p], a2);
         }
         a1 = warp_sum(a1);
         a2 = warp_sum(a2);
-        if (lane == 0) {
-            sh.s1[cl] = a1; sh.s2[cl] = a2;
+        if (lane == 0) { sh.s1[cl] = a1; sh.s2[cl] = a2; }   // this block's pixels only
+    }
+    // ---- the cluster's blocks add their sums up in rank order (distributed shared memory)
+    cluster.sync();
+    for (int cl = tid; cl < nch; cl += kGroupThreads) {
+        float a1 = 0.f, a2 = 0.f;
+        for (int r = 0; r < kGroupSplit; ++r) {
+            const GroupShared* peer = cluster.map_shared_rank(&sh, r);
+            a1 += peer->s1[cl]; a2 += peer->s2[cl];
+        }
+        sh.t1[cl] = a1; sh.t2[cl] = a2;
+        if (rank == 0) {
             st.g[st.nw + c0 + cl] = a2;                      // gradient of the scale
             st.g[st.nw + st.co + c0 + cl] = a1;              // gradient of the shift
         }
@@ -208,8 +293,8 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
     for (int g = tid; g < gb.ngrp; g += kGroupThreads) {
         float m1 = 0.f, m2 = 0.f;
         for (int cl = 0; cl < cpg; ++cl) {
-            m1 = fmaf(sh.gs[g * cpg + cl], sh.s1[g * cpg + cl], m1);
-            m2 = fmaf(sh.gs[g * cpg + cl], sh.s2[g * cpg + cl], m2);
+            m1 = fmaf(sh.gs[g * cpg + cl], sh.t1[g * cpg + cl], m1);
+            m2 = fmaf(sh.gs[g * cpg + cl], sh.t2[g * cpg + cl], m2);
         }
         m1 /= (float)(cpg * hw); m2 /= (float)(cpg * hw);
         for (int cl = 0; cl < cpg; ++cl) { sh.m1[g * cpg + cl] = m1; sh.m2[g * cpg + cl] = m2; }
@@ -218,63 +303,60 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
     // ---- gradient at the conv output (kept in place of dn), gradient of the skip input
     float* __restrict__ dsk = st.dskip
         ? st.dskip + (size_t)slot_of(j, st.dskip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
-    for (int cl = warp; cl < nch; cl += kGroupWarps) {
-        const int c = c0 + cl;
+#pragma unroll 2
+    for (int idx = tid; idx < total; idx += kGroupThreads) {
+        const int cl = quot(idx, inv_upc), u = u_lo + idx - cl * upc;
+        const int c = c0 + cl, p = u * VEC;
         const size_t base = (size_t)c * hw;
-        const float mean = sh.mean[cl], rstd = sh.rstd[cl], gv = sh.gs[cl], m1 = sh.m1[cl], m2 = sh.m2[cl];
-        for (int u = lane; u < npu; u += 32) {
-            const int p = u * VEC;
-            float zv[VEC], d[VEC];
-            vload<VEC>(zv, z + base + p);
+        const float rstd = sh.rstd[cl], gv = sh.gs[cl], m1 = sh.m1[cl], m2 = sh.m2[cl];
+        float d[VEC];
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) d[e] = dn[cl * rs + p + e];
-            if (dsk) {
-                // the skip input joined after the normalisation: it receives dn itself
-                if (st.skip_mode == 0) {
-                    vstore<VEC>(dsk + base + p, d);
-                } else if (c < st.skip_c) {
+        for (int e = 0; e < VEC; ++e) d[e] = dn[cl * rs + p - p_lo + e];
+        if (dsk) {
+            // the skip input joined after the normalisation: it receives dn itself
+            if (st.skip_mode == 0) {
+                vstore<VEC>(dsk + base + p, d);
+            } else if (c < st.skip_c) {
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) {
-                        const int y = (p + e) / st.ow, x = (p + e) % st.ow;
-                        for (int dy = 0; dy < 2; ++dy)
-                            for (int dx = 0; dx < 2; ++dx) {
-                                const int ys = 2 * y + dy, xs = 2 * x + dx;
-                                if (ys < st.skip_h && xs < st.skip_w)
-                                    dsk[((size_t)c * st.skip_h + ys) * st.skip_w + xs] = (dy | dx) ? 0.f : d[e];
-                            }
-                    }
+                for (int e = 0; e < VEC; ++e) {
+                    const int y = (p + e) / st.ow, x = (p + e) % st.ow;
+                    for (int dy = 0; dy < 2; ++dy)
+                        for (int dx = 0; dx < 2; ++dx) {
+                            const int ys = 2 * y + dy, xs = 2 * x + dx;
+                            if (ys < st.skip_h && xs < st.skip_w)
+                                dsk[((size_t)c * st.skip_h + ys) * st.skip_w + xs] = (dy | dx) ? 0.f : d[e];
+                        }
                 }
             }
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) {
-                const float zh = (zv[e] - mean) * rstd;
-                dn[cl * rs + p + e] = rstd * (fmaf(d[e], gv, -m1) - zh * m2);
-            }
         }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e)
+            dn[cl * rs + p - p_lo + e] = rstd * (fmaf(d[e], gv, -m1) - zh[cl * rs + p - p_lo + e] * m2);
     }
     __syncthreads();
     // ---- bfloat16 [pixel][channel] operand of dgrad / wgrad
     const int ng = nch >> 3;
-    for (int idx = tid; idx < ng * hw; idx += kGroupThreads) {
-        const int u = idx / hw, p = idx - u * hw;
+    for (int idx = tid; idx < ng * np; idx += kGroupThreads) {
+        const int u = idx / np, p = idx - u * np;
         const float* src = dn + (size_t)(u * 8) * rs + p;
         __nv_bfloat162 b0 = __floats2bfloat162_rn(src[0], src[rs]), b1 = __floats2bfloat162_rn(src[2 * rs], src[3 * rs]);
         __nv_bfloat162 b2 = __floats2bfloat162_rn(src[4 * rs], src[5 * rs]), b3 = __floats2bfloat162_rn(src[6 * rs], src[7 * rs]);
         uint4 v;
         v.x = *reinterpret_cast<unsigned*>(&b0); v.y = *reinterpret_cast<unsigned*>(&b1);
         v.z = *reinterpret_cast<unsigned*>(&b2); v.w = *reinterpret_cast<unsigned*>(&b3);
-        *reinterpret_cast<uint4*>(st.dz16 + (size_t)p * st.co + c0 + u * 8) = v;
+        *reinterpret_cast<uint4*>(st.dz16 + (size_t)(p_lo + p) * st.co + c0 + u * 8) = v;
     }
+    cluster.sync();          // no block leaves while another may still read its sums
 }
 
-__global__ void __launch_bounds__(kGroupThreads, 2)
+__global__ void __cluster_dims__(kGroupSplit, 1, 1) __launch_bounds__(kGroupThreads, 3)
 conv_group_bwd_kernel(const ConvStage* __restrict__ stages, const GroupBlock* __restrict__ blocks, int nblocks,
                       const TickState* __restrict__ ts, int S, int par) {
     extern __shared__ __align__(16) float group_buf[];
     __shared__ GroupShared sh;
     __shared__ ConvStage st;
-    if ((int)blockIdx.x >= nblocks) return;
-    const GroupBlock gb = blocks[blockIdx.x];
+    if ((int)blockIdx.x >= nblocks * kGroupSplit) return;       // (uniform over a cluster: the grid is nblocks clusters)
+    const GroupBlock gb = blocks[blockIdx.x / kGroupSplit];
     {
         const int* s_ = reinterpret_cast<const int*>(&stages[gb.stage]);
         int* d_ = reinterpret_cast<int*>(&st);

@@ -379,14 +379,15 @@ __device__ void conv_bwd_dn_chunk(const ConvStage& st, const PostChunk& ch, long
                 const int p = p0 + e;
                 const int y = p / st.ow, x = p % st.ow;
                 float a = 0.f;
-                for (int r = 0; r < kk; ++r) {
+                // only window offsets congruent to the element's position modulo the stride can hold it
+                for (int r = (y + pp) % ps; r < kk; r += ps) {
                     const int ty = y + pp - r;
-                    if (ty < 0 || ty % ps) continue;
+                    if (ty < 0) break;
                     const int py = ty / ps;
                     if (py >= st.out_h) continue;
-                    for (int s = 0; s < kk; ++s) {
+                    for (int s = (x + pp) % ps; s < kk; s += ps) {
                         const int tx = x + pp - s;
-                        if (tx < 0 || tx % ps) continue;
+                        if (tx < 0) break;
                         const int px = tx / ps;
                         if (px >= st.out_w) continue;
                         const size_t o = (size_t)c * ohw + py * st.out_w + px;

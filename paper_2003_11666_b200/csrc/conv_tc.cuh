@@ -9,7 +9,7 @@
 // with K ordered (r, s, channel) so that 8 consecutive K (one 16-byte unit)
 // are 8 consecutive channels of one pixel.
 //
-// One persistent block per SM works through a list of tiles (all stages of the
+// Two persistent blocks per SM work through lists of tiles (all stages of the
 // tick, balanced on the host by their number of K chunks) with three kinds of warps:
 //   * producer warps (4) fill a three-stage ring of K chunks of 64.  An operand
 //     that is a plain matrix in memory (the weights in all three GEMMs, dz as
@@ -41,11 +41,17 @@ namespace pb {
 constexpr int kTcChunk = 64;                  // K elements per shared-memory stage
 constexpr int kTcBM = 128;
 constexpr int kTcStageBytes = 16384 * 2;      // A tile + B tile
-constexpr int kTcStages = 3;                  // shared-memory stages of the operand pipeline
+constexpr int kTcStages = 3;                  // shared-memory stages of the operand pipeline (97 KB: two blocks per SM)
 constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + 1024;
 constexpr int kTcEpiWarps = 4;                // warps 0-3: quarter q of the tensor-memory lanes belongs to warp q
-constexpr int kTcProducers = 128;             // warps 4-7
-constexpr int kTcMmaWarp = 8;
+constexpr int kTcProdWarps = 4;               // warps 4-7
+constexpr int kTcProducers = 32 * kTcProdWarps;
+constexpr int kTcRowStep = kTcProducers / 8;  // K-major tiles: rows between two units of one thread (8 units per row)
+constexpr int kTcRowIters = 128 / kTcRowStep;
+constexpr int kTcKStep = kTcProducers / 16;   // MN-major tiles of width 128: k rows between two units of one thread
+constexpr int kTcKIters = kTcChunk / kTcKStep;
+constexpr int kTcLag = 1;                     // chunks a producer thread keeps in flight behind the one it is issuing (< kTcStages - 1)
+constexpr int kTcMmaWarp = kTcEpiWarps + kTcProdWarps;
 constexpr int kTcThreads = 32 * (kTcMmaWarp + 1);
 constexpr int kTcTmemCols = 256;              // two accumulators of 128 columns
 constexpr long long kTcWaitNs = 200LL * 1000 * 1000;   // a barrier wait gives up after 0.2 s
@@ -64,6 +70,8 @@ struct ConvGemmTC {
     float* c;                     // [c_slots][nsplit][M*N]
     int c_slots;
     int a_tmap, b_tmap;           // index of the operand's tensor map (bulk tensor copy), or -1: gathered
+    int b_rect, b_bytes;          // B of a 3x3 stride-1 convolution fetched as boxes of whole image rows, one tap per K chunk
+                                  // (b_rect = image width of the boxed tensor); bytes of one B box
     // forward GEMMs that also finish the statistics (nsplit == 1): c is then the conv-output ring
     int fuse, cpg, ntn;           // channels per normalisation group; column tiles per row of D
     float* fstat;                 // [groups][cpg * ntn][3]: count, mean, M2 of (channel, column tile)
@@ -141,6 +149,11 @@ __device__ __forceinline__ void tma_3d(uint32_t dst, const CUtensorMap* tm, int 
                  ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
 
+__device__ __forceinline__ void tma_4d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+
 // 16-byte asynchronous global -> shared copy; with ok == false the destination is zero-filled
 __device__ __forceinline__ void cp_async16(unsigned char* dst, const __nv_bfloat16* src, bool ok) {
     const int sz = ok ? 16 : 0;
@@ -148,7 +161,7 @@ __device__ __forceinline__ void cp_async16(unsigned char* dst, const __nv_bfloat
 }
 
 struct TcShared {
-    uint64_t full[kTcStages];     // a stage's operands have landed (128 producer arrivals + 1 with the bulk copies' bytes)
+    uint64_t full[kTcStages];     // a stage's operands have landed (one arrival per producer thread + 1 with the bulk copies' bytes)
     uint64_t empty[kTcStages];    // the MMAs that read a stage have completed
     uint64_t acc_full[2];         // a tile's accumulator is complete
     uint64_t acc_empty[2];        // the epilogue warps have drained an accumulator
@@ -164,7 +177,7 @@ __device__ __forceinline__ long long tc_sample(const ConvGemmTC& G, long long t,
 __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, int q0, int q1,
                             const CUtensorMap* __restrict__ tmaps, const TickState* ts, long long t, int S,
                             unsigned char* smem, TcShared& sh) {
-    const int ptid = threadIdx.x - 32 * kTcEpiWarps;          // 0 .. 127
+    const int ptid = threadIdx.x - 32 * kTcEpiWarps;          // 0 .. kTcProducers - 1
     int it = 0;                                               // chunks issued so far (all tiles)
     bool ok_all = true;
     for (int q = q0; q < q1 && ok_all; ++q) {
@@ -186,21 +199,21 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
         const bool a2 = mode != kFprop && tl.m0 + 64 < M;
         const bool b2 = mode == kWgrad && BN == 128 && tl.n0 + 64 < N;
         const uint32_t tx_bytes = (tmA ? (mode == kFprop ? 16384u : (a2 ? 16384u : 8192u)) : 0u) +
-                                  (tmB ? (mode == kWgrad ? (b2 ? 16384u : 8192u) : (uint32_t)BN * 128u) : 0u);
+                                  (tmB ? (mode == kWgrad ? (b2 ? 16384u : 8192u) : (uint32_t)G.b_bytes) : 0u);
         // the gathers divide by these for every 16-byte unit: reciprocals once per tile
         const float inv_ci = 1.f / (float)CI, inv_co = 1.f / (float)CO, inv_ksz = 1.f / (float)ksz,
                     inv_st = 1.f / (float)st, inv_ow = 1.f / (float)ow;
         // ---- per-thread invariants of the gathers
-        // K-major tiles (rows of 8 units): unit ku of rows krow0 + 16 i
+        // K-major tiles (rows of 8 units): unit ku of rows krow0 + kTcRowStep i
         const int ku = ptid & 7, krow0 = ptid >> 3;
-        int bp[8], bq[8];               // K-major B rows: pixel coordinates (fprop: output pixel; dgrad: input pixel)
-        bool bok[8];
+        int bp[kTcRowIters], bq[kTcRowIters];               // K-major B rows: pixel coordinates (fprop: output pixel; dgrad: input pixel)
+        bool bok[kTcRowIters];
         if (!tmB && mode != kWgrad) {
             const int wdt = (mode == kFprop) ? ow : iw;
             const float inv_wdt = 1.f / (float)wdt;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int row = krow0 + 16 * i, n = tl.n0 + row;
+            for (int i = 0; i < kTcRowIters; ++i) {
+                const int row = krow0 + kTcRowStep * i, n = tl.n0 + row;
                 bok[i] = row < BN && n < N;
                 bp[i] = quot(n, inv_wdt); bq[i] = n - bp[i] * wdt;
             }
@@ -216,7 +229,7 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
             wok = n < N;
             const int rs = quot(n, inv_ci); wci = n - rs * CI; wr = quot(rs, inv_ksz); wsx = rs - wr * ksz;
         }
-        const int amu = ptid & 15, ak0 = ptid >> 4;           // MN-major A (width 128): k-rows ak0 + 8 i
+        const int amu = ptid & 15, ak0 = ptid >> 4;           // MN-major A (width 128): k-rows ak0 + kTcKStep i
         const bool a_m_ok = (tl.m0 + amu * 8) < M;
 
         for (int c = 0; c < nchunks; ++c, ++it) {
@@ -227,7 +240,7 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
             const int k0 = kb + c * kTcChunk;
             const uint32_t fullb = smem_u32(&sh.full[stg]);
             if (ptid == 0) {
-                // the 129th arrival of the stage, carrying the bytes of this chunk's bulk copies
+                // the extra arrival of the stage, carrying the bytes of this chunk's bulk copies
                 if (tx_bytes) mbar_arrive_tx(fullb, tx_bytes); else mbar_arrive(fullb);
                 if (tmA) {
                     if (mode == kFprop) {
@@ -242,7 +255,16 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
                     }
                 }
                 if (tmB) {
-                    if (mode == kFprop) {
+                    if (G.b_rect) {
+                        // 3x3, stride 1: the chunk is 64 channels of ONE tap (r, s); the tile's pixels are whole
+                        // image rows, so its operand is the same box of the image shifted by the tap
+                        // (rows and columns outside the image arrive as zeros)
+                        const int C = mode == kFprop ? CI : CO;
+                        const int rs = k0 / C, c0 = k0 - rs * C, r = rs / ksz, sx = rs - r * ksz;
+                        const int row0 = tl.n0 / G.b_rect;
+                        if (mode == kFprop) tma_4d(smem_u32(sB), tmB, c0, sx - pad, row0 + r - pad, slot, fullb);
+                        else tma_3d(smem_u32(sB), tmB, c0, pad - sx, row0 + pad - r, fullb);
+                    } else if (mode == kFprop) {
                         tma_3d(smem_u32(sB), tmB, k0, tl.n0, slot, fullb);
                     } else if (mode == kDgrad) {
                         tma_2d(smem_u32(sB), tmB, k0, tl.n0, fullb);
@@ -257,23 +279,23 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
                 if (mode == kFprop) {
                     const int k = k0 + ku * 8;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int row = krow0 + 16 * i, m = tl.m0 + row;
+                    for (int i = 0; i < kTcRowIters; ++i) {
+                        const int row = krow0 + kTcRowStep * i, m = tl.m0 + row;
                         const bool ok = m < M && k < ke;
                         cp_async16(sA + kmajor_off(row, ku), ok ? A + (size_t)m * G.K + k : A, ok);
                     }
                 } else if (mode == kDgrad) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int kl = ak0 + 8 * i, k = k0 + kl;                    // k = rs * CO + co
+                    for (int i = 0; i < kTcKIters; ++i) {
+                        const int kl = ak0 + kTcKStep * i, k = k0 + kl;                    // k = rs * CO + co
                         const bool ok = a_m_ok && k < ke;
                         const int rs = quot(k, inv_co), co = k - rs * CO;
                         cp_async16(sA + mnmajor_off(kl, amu), ok ? A + ((size_t)co * (ksz * ksz) + rs) * CI + tl.m0 + amu * 8 : A, ok);
                     }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int kl = ak0 + 8 * i, k = k0 + kl;                    // k = output pixel
+                    for (int i = 0; i < kTcKIters; ++i) {
+                        const int kl = ak0 + kTcKStep * i, k = k0 + kl;                    // k = output pixel
                         const bool ok = a_m_ok && k < ke;
                         cp_async16(sA + mnmajor_off(kl, amu), ok ? A + (size_t)k * CO + tl.m0 + amu * 8 : A, ok);
                     }
@@ -285,8 +307,8 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
                     const int k = k0 + ku * 8;
                     const int rs = quot(k, inv_ci), ci = k - rs * CI, r = quot(rs, inv_ksz), s = rs - r * ksz;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int row = krow0 + 16 * i;
+                    for (int i = 0; i < kTcRowIters; ++i) {
+                        const int row = krow0 + kTcRowStep * i;
                         if (row >= BN) break;
                         const int y = bp[i] * st + r - pad, x = bq[i] * st + s - pad;
                         const bool ok = bok[i] && k < ke && y >= 0 && y < ih && x >= 0 && x < iw;
@@ -296,8 +318,8 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
                     const int k = k0 + ku * 8;
                     const int rs = quot(k, inv_co), co = k - rs * CO, r = quot(rs, inv_ksz), s = rs - r * ksz;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int row = krow0 + 16 * i;
+                    for (int i = 0; i < kTcRowIters; ++i) {
+                        const int row = krow0 + kTcRowStep * i;
                         if (row >= BN) break;
                         const int ty = bp[i] + pad - r, tx = bq[i] + pad - s;
                         const int p = quot(ty, inv_st), qq = quot(tx, inv_st);
@@ -315,20 +337,21 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
                 }
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
-            // this thread's copies of the PREVIOUS chunk have landed: make them visible to the
-            // tensor core (async proxy) and count in at that chunk's barrier; the copies just
-            // issued stay in flight meanwhile
-            if (it > 0) {
-                asm volatile("cp.async.wait_group 1;" ::: "memory");
+            // this thread's copies of the chunk issued kTcLag iterations ago have landed: make them
+            // visible to the tensor core (async proxy) and count in at that chunk's barrier; the
+            // copies of the kTcLag chunks issued since stay in flight meanwhile
+            if (it >= kTcLag) {
+                asm volatile("cp.async.wait_group %0;" ::"n"(kTcLag) : "memory");
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_arrive(smem_u32(&sh.full[(it - 1) % kTcStages]));
+                mbar_arrive(smem_u32(&sh.full[(it - kTcLag) % kTcStages]));
             }
         }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (it > 0 && ok_all) {
+    if (ok_all) {
+        // the chunks still owed an arrival, oldest first
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(smem_u32(&sh.full[(it - 1) % kTcStages]));
+        for (int c = max(0, it - kTcLag); c < it; ++c) mbar_arrive(smem_u32(&sh.full[c % kTcStages]));
     }
     if (!ok_all) sh.fail = 1;
 }
@@ -408,7 +431,7 @@ __device__ void tc_epilogue(const ConvGemmTC* __restrict__ gemms, const GemmTile
             tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 128 + c0), r);
             if (m < M) {
                 float* dst = Cp + (size_t)m * N + tl.n0 + c0;
-                const int nleft = N - (tl.n0 + c0);
+                const int nleft = min(N - (tl.n0 + c0), BN - c0);      // columns of this tile that exist (a tile may be narrower than 32 k)
                 if (nleft >= 32 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
 #pragma unroll
                     for (int u = 0; u < 8; ++u)

@@ -272,7 +272,7 @@ void build_fc_tables(pb_handle* h, const float* w_base, const float* v_base) {
 void choose_split(int M, int N, int K, int num_sms, int& nsplit, int& kps) {
     // as for the tensor-core path: slices only bound the K loop of one tile
     (void)M; (void)N; (void)num_sms;
-    nsplit = std::max(1, std::min(ceil_div(K, kSimtMaxK), 32));
+    nsplit = std::max(1, std::min(ceil_div(K, kSimtMaxK), 64));
     kps = ceil_div(ceil_div(K, nsplit), kBK) * kBK;
     nsplit = ceil_div(K, kps);
 }
@@ -287,6 +287,20 @@ void choose_split_tc(int K, int max_k, int& nsplit, int& kps) {
 }
 
 int tc_bn(int N) { return N <= 64 ? 64 : 128; }
+
+// Column tiles made of whole image rows (for operands fetched as boxes of the image): the
+// largest number of rows whose pixels fit one tile and are a multiple of 16 (the MMA's N
+// granularity); a small image is one tile.  Returns the rows of a box (0: no such tiling)
+// and the tile width in bn.
+int rect_rows(int w, int hgt, int& bn) {
+    if (w > 128) return 0;
+    if (w * hgt <= 64) { bn = 64; return hgt; }
+    for (int r = 128 / w; r >= 1; --r)
+        if ((r * w) % 16 == 0) { bn = r * w; return r; }
+    return 0;
+}
+// 3x3 stride-1 convolutions whose channel count lets a K chunk of 64 sit inside one tap
+bool rect_conv(const pb_layer& L, int channels) { return L.k == 3 && L.stride == 1 && L.pad == 1 && channels % 64 == 0; }
 
 void plan_conv(pb_handle* h) {
     {
@@ -319,7 +333,11 @@ void plan_conv(pb_handle* h) {
             // Large networks: a forward GEMM with one K slice writes the conv output into its ring
             // and the per-(channel, column tile) statistics itself, so the first normalisation
             // step is not run for that stage.
-            x.ntn = ceil_div(opix, tc_bn(opix));
+            {
+                int bn = tc_bn(opix), rbn = 0;
+                if (rect_conv(x.head, x.head.c_in) && rect_rows(x.z.w, x.z.h, rbn) > 0) bn = rbn;
+                x.ntn = ceil_div(opix, bn);
+            }
             x.fuse_stats = !h->post_fuse && x.split_f == 1;
             if (x.fuse_stats) x.fstat_stride = (x.head.c_out / x.gn_groups) * x.ntn;
             continue;
@@ -328,6 +346,16 @@ void plan_conv(pb_handle* h) {
         choose_split(x.head.c_in, x.in.h * x.in.w, x.head.c_out * k2, h->num_sms, x.split_d, x.kps_d);
         choose_split(x.head.c_out, x.head.c_in * k2, x.z.h * x.z.w, h->num_sms, x.split_w, x.kps_w);
         x.dx_nparts = x.split_d;
+        // 3x3 / stride 1 / pad 1 on a 4x4 or 2x2 image: a weight-streaming problem, run by the fused
+        // tick kernel of conv_gemv.cuh (forward, both gradients and the update in one pass over w, v)
+        x.gemv = x.head.k == 3 && x.head.stride == 1 && x.head.pad == 1 && x.src >= 0 && x.in.h == x.in.w &&
+                 (x.in.h == 4 || x.in.h == 2) && x.z.h == x.in.h && x.head.c_in % 32 == 0 &&
+                 !(h->flags & (PB_LWP_WFORM | PB_WEIGHT_STASH));
+        if (x.gemv) {
+            x.split_f = 1; x.kps_f = ceil_div(x.head.c_in * k2, kBK) * kBK;
+            x.split_w = 1; x.kps_w = ceil_div(x.z.h * x.z.w, kBK) * kBK;
+            x.dx_nparts = ceil_div(x.head.c_out, kGemvRows);
+        }
     }
 }
 
@@ -396,7 +424,7 @@ int add_tensor_map(pb_handle* h, const void* base, int rank, const unsigned long
 // Tiles of one grouped tensor-core launch handed to persistent blocks: longest first, each
 // to the block with the least work so far (cost = K chunks plus a constant for the epilogue).
 void balance_tc_tiles(const pb_handle* h, const std::vector<ConvGemmTC>& gemms, std::vector<GemmTile>& tiles, std::vector<int>& begin) {
-    const int nb = std::max(1, std::min((int)tiles.size(), h->num_sms));
+    const int nb = std::max(1, std::min((int)tiles.size(), 2 * h->num_sms));       // two resident blocks per SM
     auto cost = [&](const GemmTile& t) {
         const ConvGemmTC& g = gemms[t.gemm];
         const int kb = t.split * g.k_per_split, ke = std::min(g.K, kb + g.k_per_split);
@@ -424,7 +452,7 @@ void balance_tc_tiles(const pb_handle* h, const std::vector<ConvGemmTC>& gemms, 
 
 bool fill_conv_tables(pb_handle* h) {
     bool maps_ok = true;
-    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_bundles.clear(); h->h_groups.clear(); h->h_ptiles[0].clear(); h->h_ptiles[1].clear(); h->h_dtiles[0].clear(); h->h_dtiles[1].clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear(); h->h_tmaps.clear(); h->h_fchunks.clear(); h->h_stash.clear(); h->h_stashchunks.clear(); h->h_gblocks.clear();
+    h->h_gemms.clear(); h->h_cs.clear(); h->h_pchunks.clear(); h->h_bundles.clear(); h->h_groups.clear(); h->h_ptiles[0].clear(); h->h_ptiles[1].clear(); h->h_dtiles[0].clear(); h->h_dtiles[1].clear(); h->h_upd.clear(); h->h_chunks.clear(); h->h_tc.clear(); h->h_tmaps.clear(); h->h_fchunks.clear(); h->h_stash.clear(); h->h_stashchunks.clear(); h->h_gblocks.clear(); h->h_gemv.clear(); h->h_gemvblocks.clear();
     for (auto& t : h->h_tiles) t.clear();
     for (auto& t : h->h_tctiles) t.clear();
     const int bf = (h->flags & PB_CONV_BF16) ? 1 : 0;
@@ -455,12 +483,24 @@ bool fill_conv_tables(pb_handle* h) {
                 const unsigned bx[2] = {64, 128};
                 t.a_tmap = add_tensor_map(h, live ? t.a : none, 2, d, sb, bx, &maps_ok);
             }
-            t.b_tmap = -1;
+            t.b_tmap = -1; t.b_rect = 0; t.b_bytes = t.bn * 128;
             if (plain) {
                 const unsigned long long d[3] = {(unsigned long long)L.c_in, (unsigned long long)ipix, (unsigned long long)y.out_slots},
                                          sb[2] = {(unsigned long long)L.c_in * 2, (unsigned long long)x.in.elems() * 2};
                 const unsigned bx[3] = {64, (unsigned)t.bn, 1};
                 t.b_tmap = add_tensor_map(h, live ? t.b : none, 3, d, sb, bx, &maps_ok);
+            } else {
+                int rbn = 0;
+                const int rows = rect_conv(L, L.c_in) ? rect_rows(x.z.w, x.z.h, rbn) : 0;
+                if (rows > 0) {
+                    // input image [slot][y][x][c_in] (same size as the output: stride 1, pad 1)
+                    const unsigned long long d[4] = {(unsigned long long)L.c_in, (unsigned long long)x.in.w, (unsigned long long)x.in.h, (unsigned long long)y.out_slots},
+                                             sb[3] = {(unsigned long long)L.c_in * 2, (unsigned long long)x.in.w * L.c_in * 2, (unsigned long long)x.in.elems() * 2};
+                    const unsigned bx[4] = {64, (unsigned)x.in.w, (unsigned)rows, 1};
+                    const int m = add_tensor_map(h, live ? t.b : none, 4, d, sb, bx, &maps_ok);
+                    t.bn = rbn;                                  // the tiling holds whether or not the map could be made
+                    if (m >= 0) { t.b_tmap = m; t.b_rect = x.in.w; t.b_bytes = 128 * x.in.w * rows; }
+                }
             }
             add_tiles(h->h_tctiles[0], (int)h->h_tc.size(), t.M, t.N, t.nsplit, kTcBM, t.bn);
             h->h_tc.push_back(t);
@@ -481,15 +521,28 @@ bool fill_conv_tables(pb_handle* h) {
                 const unsigned bx[3] = {64, 1, 64};
                 t.a_tmap = add_tensor_map(h, live ? t.a : none, 3, d, sb, bx, &maps_ok);
             }
+            t.b_rect = 0; t.b_bytes = t.bn * 128;
             if (plain) {
                 const unsigned long long d[2] = {(unsigned long long)L.c_out, (unsigned long long)opix}, sb[1] = {(unsigned long long)L.c_out * 2};
                 const unsigned bx[2] = {64, (unsigned)t.bn};
                 t.b_tmap = add_tensor_map(h, live ? t.b : none, 2, d, sb, bx, &maps_ok);
+            } else {
+                int rbn = 0;
+                const int rows = rect_conv(L, L.c_out) ? rect_rows(x.in.w, x.in.h, rbn) : 0;
+                if (rows > 0) {
+                    // gradient image [y][x][c_out] (same size as the input: stride 1, pad 1)
+                    const unsigned long long d[3] = {(unsigned long long)L.c_out, (unsigned long long)x.z.w, (unsigned long long)x.z.h},
+                                             sb[2] = {(unsigned long long)L.c_out * 2, (unsigned long long)x.z.w * L.c_out * 2};
+                    const unsigned bx[3] = {64, (unsigned)x.z.w, (unsigned)rows};
+                    const int m = add_tensor_map(h, live ? t.b : none, 3, d, sb, bx, &maps_ok);
+                    t.bn = rbn;
+                    if (m >= 0) { t.b_tmap = m; t.b_rect = x.z.w; t.b_bytes = 128 * x.z.w * rows; }
+                }
             }
             add_tiles(h->h_tctiles[1], (int)h->h_tc.size(), t.M, t.N, t.nsplit, kTcBM, t.bn);
             h->h_tc.push_back(t);
             // wgrad: D[c_out, (r, s, c_in)]
-            t.a_slots = 1; t.a_elems = 0;
+            t.a_slots = 1; t.a_elems = 0; t.b_rect = 0;
             t.mode = kWgrad; t.M = L.c_out; t.N = L.c_in * k2; t.K = opix; t.bn = tc_bn(t.N);
             t.nsplit = x.split_w; t.k_per_split = x.kps_w;
             t.a = x.dz16; t.b = y.out16; t.b_slots = y.out_slots; t.b_elems = x.in.elems();
@@ -518,7 +571,7 @@ bool fill_conv_tables(pb_handle* h) {
         g.c = x.zpart; g.c_slots = 1;
         g.a_slots = 1; g.a_elems = 0;
         g.tm = g.M <= 16 ? 1 : 4; g.tn = g.N <= 16 ? 1 : 4;        // small problems take small tiles
-        if (!x.tc) add_tiles(h->h_tiles[0], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
+        if (!x.tc && !x.gemv) add_tiles(h->h_tiles[0], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
         h->h_gemms.push_back(g);
         // dgrad (not for the first stage: nobody needs the gradient of the input)
         if (x.src >= 0) {
@@ -527,7 +580,7 @@ bool fill_conv_tables(pb_handle* h) {
             if (!x.tc && x.stash_slots > 0) { g.a = x.wstash; g.a_slots = x.stash_slots; g.a_elems = (int)(x.wstash_stride / 4); }   // the forward's weights
             g.c = x.dx; g.c_slots = x.dx_slots;
             g.tm = g.M <= 16 ? 1 : 4; g.tn = g.N <= 16 ? 1 : 4;
-            if (!x.tc) add_tiles(h->h_tiles[1], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
+            if (!x.tc && !x.gemv) add_tiles(h->h_tiles[1], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
             h->h_gemms.push_back(g);
         }
         // wgrad
@@ -536,7 +589,7 @@ bool fill_conv_tables(pb_handle* h) {
         g.a_slots = 1; g.a_elems = 0;
         g.c = x.gpart; g.c_slots = 1;
         g.tm = g.M <= 16 ? 1 : 4; g.tn = g.N <= 16 ? 1 : 4;
-        if (!x.tc) add_tiles(h->h_tiles[2], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
+        if (!x.tc && !x.gemv) add_tiles(h->h_tiles[2], (int)h->h_gemms.size(), g.M, g.N, g.nsplit, 16 * g.tm, 16 * g.tn);
         h->h_gemms.push_back(g);
 
         ConvStage c{};
@@ -581,12 +634,16 @@ bool fill_conv_tables(pb_handle* h) {
             const int gpb = need16 && cpg < 8 ? 8 / cpg : 1;           // groups per bundle
             // Large networks: a tensor-core stage whose bundles fit in shared memory is normalised by
             // one block per bundle, forward and backward (conv_group.cuh), and leaves the lists below.
-            const bool resident = x.fuse_stats && need16 && !x.has_pool && !x.avgpool && x.gn_groups % gpb == 0 &&
+            // (a bundle spans whole 8-channel units: groups of 1, 2, 4 channels are bundled, groups of 8, 16, ... stand alone)
+            const bool units_ok = x.tc && L.c_out % 8 == 0 && (cpg < 8 ? 8 % cpg == 0 : cpg % 8 == 0);
+            const bool resident = x.fuse_stats && units_ok && !x.has_pool && !x.avgpool && x.gn_groups % gpb == 0 &&
                                   gpb * cpg <= kGroupMaxChannels && (long long)gpb * cpg * hw <= kGroupMaxElems;
             if (resident) {
                 for (int g0 = 0; g0 < x.gn_groups; g0 += gpb) h->h_gblocks.push_back(GroupBlock{stage_idx, g0, gpb});
-                h->group_smem_fwd = std::max(h->group_smem_fwd, (size_t)gpb * cpg * (hw + 2) * 2);
-                h->group_smem_bwd = std::max(h->group_smem_bwd, (size_t)gpb * cpg * (hw + 4) * 4);
+                // each of the kGroupSplit blocks of a bundle holds a quarter of the pixels (rounded up to whole units of 4)
+                const size_t np = (size_t)(ceil_div(ceil_div(hw, 4), kGroupSplit) + 1) * 4;
+                h->group_smem_fwd = std::max(h->group_smem_fwd, (size_t)gpb * cpg * (np + 2) * 2);
+                h->group_smem_bwd = std::max(h->group_smem_bwd, (size_t)2 * gpb * cpg * (np + 4) * 4);      // dn and zhat
             }
             if (!resident) {
             const bool pooled = x.has_pool || x.avgpool;
@@ -671,8 +728,23 @@ bool fill_conv_tables(pb_handle* h) {
         r.w = h->d_w + x.dev_off; r.v = h->d_v + x.dev_off; r.wh = h->d_wh + x.dev_off;
         r.g = x.gpart; r.nparts = x.split_w; r.part_stride = nw; r.n = nw;
         if (x.tc) { r.w16 = h->d_w16 + x.dev_off; r.wh16 = h->d_wh16 + x.dev_off; }
+        if (x.gemv) {
+            // its conv weights are updated inside the fused kernel (and predicted on the fly)
+            ConvGemvStage gs{};
+            gs.w = h->d_w + x.dev_off; gs.v = h->d_v + x.dev_off;
+            gs.ci = L.c_in; gs.co = L.c_out; gs.hw = x.in.h; gs.s = x.index;
+            gs.xin = xin; gs.xin_slots = xin_slots;
+            gs.dz = x.dz; gs.z = x.zpart;
+            gs.dx = x.dx; gs.dx_slots = x.dx_slots; gs.dx_nparts = x.dx_nparts;
+            gs.neg_lr_T = -h->lr * x.T; gs.m = h->momentum; gs.neg_lr_a = -h->lr * x.a; gs.neg_lr_b = -h->lr * x.b;
+            for (int r0 = 0, part = 0; r0 < L.c_out; r0 += kGemvRows, ++part) h->h_gemvblocks.push_back(GemvBlock{(int)h->h_gemv.size(), r0, part});
+            h->h_gemv.push_back(gs);
+            const int P = x.in.h * x.in.w;
+            h->gemv_smem = std::max(h->gemv_smem, sizeof(float) * ((size_t)2 * L.c_in * (P + 1) + (size_t)(1 + kGemvWarps) * kGemvRows * P + (size_t)kGemvWarps * 576 + 4));
+        } else {
         for (int st = 0; st < r.n; st += kUpdChunk) h->h_chunks.push_back(UpdChunk{(int)h->h_upd.size(), st});
         h->h_upd.push_back(r);
+        }
         r.w += nw; r.v += nw; r.wh += nw; r.w16 = nullptr; r.wh16 = nullptr;
         r.g = h->d_g + x.dev_off + nw; r.nparts = 1; r.part_stride = 0; r.n = 2 * L.c_out;
         for (int st = 0; st < r.n; st += kUpdChunk) h->h_chunks.push_back(UpdChunk{(int)h->h_upd.size(), st});
@@ -752,6 +824,8 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
     h->d_upd = c.take<UpdRange>(h->h_upd.size() + 1);
     h->d_chunks = c.take<UpdChunk>(h->h_chunks.size() + 1);
     h->d_gblocks = c.take<GroupBlock>(h->h_gblocks.size() + 1);
+    h->d_gemv = c.take<ConvGemvStage>(h->h_gemv.size() + 1);
+    h->d_gemvblocks = c.take<GemvBlock>(h->h_gemvblocks.size() + 1);
     h->d_stash = c.take<StashRange>(h->h_stash.size() + 1);
     h->d_stashchunks = c.take<StashChunk>(h->h_stashchunks.size() + 1);
     h->d_tc = c.take<ConvGemmTC>(h->h_tc.size() + 1);
@@ -1011,16 +1085,6 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
                     h->d_tc, TcLaunch{h->d_tctiles[0], h->d_tcbegin[0]}, h->d_tmaps, h->d_ts, h->S, par);
                 prof_end(h);
             }
-            prof_begin(h, 5);
-            if (nfc > 0)
-                conv_fwd_post_kernel<<<nfc, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_fchunks, nfc, h->d_bundles, h->d_ptiles[0], h->d_bcnt[0], h->d_ts, h->S, par);
-            if (ngr > 0)
-                conv_group_merge_kernel<<<ceil_div(ngr, 8), 256, 0, h->stream>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 0);
-            if (!h->h_dtiles[0].empty())
-                conv_apply_fwd_kernel<<<(int)h->h_dtiles[0].size(), kPostThreads, 0, h->stream>>>(h->d_cs, h->d_dtiles[0], (int)h->h_dtiles[0].size(), h->d_ts, h->S, par);
-            if (ngb > 0)
-                conv_group_fwd_kernel<<<ngb, kGroupThreads, h->group_smem_fwd, h->stream>>>(h->d_cs, h->d_gblocks, ngb, h->d_ts, h->S, par);
-            prof_end(h);
             // Backward chain: through pool/ReLU/GroupNorm -> data and weight gradients.  It reads
             // what earlier ticks stored (other ring slots than the forward chain writes) and the
             // current weights, so it runs on its own stream beside the forward chain; only the
@@ -1048,8 +1112,32 @@ int run_ticks(pb_handle* h, const float* dev_xs, const int32_t* dev_labels, int 
             if (!h->h_dtiles[1].empty())
                 conv_bwd_dz_kernel<<<(int)h->h_dtiles[1].size(), kPostThreads, 0, bs>>>(h->d_cs, h->d_dtiles[1], (int)h->h_dtiles[1].size(), h->d_ts, h->S, par);
             if (ngb > 0)
-                conv_group_bwd_kernel<<<ngb, kGroupThreads, h->group_smem_bwd, bs>>>(h->d_cs, h->d_gblocks, ngb, h->d_ts, h->S, par);
+                conv_group_bwd_kernel<<<ngb * kGroupSplit, kGroupThreads, h->group_smem_bwd, bs>>>(h->d_cs, h->d_gblocks, ngb, h->d_ts, h->S, par);     // clusters of kGroupSplit
             prof_end(h, bs);
+            const int ngv_ = (int)h->h_gemvblocks.size();
+            if (ngv_ > 0) {
+                // 3x3 stages on tiny images: forward, both gradients and the update in one pass over (w, v)
+                prof_begin(h, 3, bs);
+                conv_gemv_kernel<<<ngv_, kGemvThreads, h->gemv_smem, bs>>>(h->d_gemv, h->d_gemvblocks, h->d_ts, h->S, par);
+                prof_end(h, bs);
+                cudaEventRecord(h->ev_gemv, bs);
+                h->last_launches += 1;
+            }
+            // forward normalisation (issued here, after the kernel above has been queued: it waits for it)
+            const int ngv = (int)h->h_gemvblocks.size();
+            prof_begin(h, 5);
+            // (stages run by the fused tiny-image kernel get their conv output from it: that kernel sits
+            //  in the backward chain, behind the gradient it also needs, so the forward normalisation waits for it)
+            if (ngv > 0) cudaStreamWaitEvent(h->stream, h->ev_gemv, 0);
+            if (nfc > 0)
+                conv_fwd_post_kernel<<<nfc, kPostThreads, 0, h->stream>>>(h->d_cs, h->d_fchunks, nfc, h->d_bundles, h->d_ptiles[0], h->d_bcnt[0], h->d_ts, h->S, par);
+            if (ngr > 0)
+                conv_group_merge_kernel<<<ceil_div(ngr, 8), 256, 0, h->stream>>>(h->d_cs, h->d_groups, ngr, h->d_ts, h->S, par, 0);
+            if (!h->h_dtiles[0].empty())
+                conv_apply_fwd_kernel<<<(int)h->h_dtiles[0].size(), kPostThreads, 0, h->stream>>>(h->d_cs, h->d_dtiles[0], (int)h->h_dtiles[0].size(), h->d_ts, h->S, par);
+            if (ngb > 0)
+                conv_group_fwd_kernel<<<ngb * kGroupSplit, kGroupThreads, h->group_smem_fwd, h->stream>>>(h->d_cs, h->d_gblocks, ngb, h->d_ts, h->S, par);
+            prof_end(h);
             // data gradients (dgrad) and weight gradients (wgrad) both start from dz and write
             // different buffers: wgrad goes to a stream of its own
             cudaStream_t ws = h->aux ? h->aux : bs;
@@ -1183,6 +1271,8 @@ int create_engine(const pb_layer* layers, int n_layers, const int32_t* stage_of_
     up(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange));
     up(h->d_chunks, h->h_chunks.data(), h->h_chunks.size() * sizeof(UpdChunk));
     up(h->d_gblocks, h->h_gblocks.data(), h->h_gblocks.size() * sizeof(GroupBlock));
+    up(h->d_gemv, h->h_gemv.data(), h->h_gemv.size() * sizeof(ConvGemvStage));
+    up(h->d_gemvblocks, h->h_gemvblocks.data(), h->h_gemvblocks.size() * sizeof(GemvBlock));
     up(h->d_stash, h->h_stash.data(), h->h_stash.size() * sizeof(StashRange));
     up(h->d_stashchunks, h->h_stashchunks.data(), h->h_stashchunks.size() * sizeof(StashChunk));
     up(h->d_tc, h->h_tc.data(), h->h_tc.size() * sizeof(ConvGemmTC));
@@ -1212,6 +1302,10 @@ int create_engine(const pb_layer* layers, int n_layers, const int32_t* stage_of_
     }
     if (e == cudaSuccess && !h->h_tc.empty())
         e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemBytes);
+    if (e == cudaSuccess && !h->h_gemvblocks.empty()) {
+        e = cudaFuncSetAttribute(conv_gemv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->gemv_smem);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_gemv, cudaEventDisableTiming);
+    }
     if (e == cudaSuccess && !h->h_gblocks.empty()) {
         e = cudaFuncSetAttribute(conv_group_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->group_smem_fwd);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(conv_group_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->group_smem_bwd);
@@ -1346,6 +1440,8 @@ int pb_set_mitigation(pb_handle* h, float sc_delay_scale, float horizon_scale) {
     PB_CUDA(h, cudaStreamSynchronize(h->stream));
     if (!h->h_fc.empty())
         PB_CUDA(h, cudaMemcpyAsync(h->d_fc, h->h_fc.data(), h->h_fc.size() * sizeof(FcStage), cudaMemcpyHostToDevice, h->stream));
+    if (!h->h_gemv.empty())
+        PB_CUDA(h, cudaMemcpyAsync(h->d_gemv, h->h_gemv.data(), h->h_gemv.size() * sizeof(ConvGemvStage), cudaMemcpyHostToDevice, h->stream));
     if (!h->h_upd.empty()) {
         PB_CUDA(h, cudaMemcpyAsync(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange), cudaMemcpyHostToDevice, h->stream));
         // Conv stages read STORED predicted weights, written by their last update with the old
@@ -1371,6 +1467,8 @@ int pb_set_update_size(pb_handle* h, int n_samples) {
     PB_CUDA(h, cudaStreamSynchronize(h->stream));
     if (!h->h_fc.empty())
         PB_CUDA(h, cudaMemcpyAsync(h->d_fc, h->h_fc.data(), h->h_fc.size() * sizeof(FcStage), cudaMemcpyHostToDevice, h->stream));
+    if (!h->h_gemv.empty())
+        PB_CUDA(h, cudaMemcpyAsync(h->d_gemv, h->h_gemv.data(), h->h_gemv.size() * sizeof(ConvGemvStage), cudaMemcpyHostToDevice, h->stream));
     if (!h->h_upd.empty())
         PB_CUDA(h, cudaMemcpyAsync(h->d_upd, h->h_upd.data(), h->h_upd.size() * sizeof(UpdRange), cudaMemcpyHostToDevice, h->stream));
     if (reset_tick_state(h) != PB_OK) return fail(h, PB_E_CUDA, "pb_set_update_size: could not write the tick state");
@@ -1563,6 +1661,7 @@ void pb_destroy(pb_handle* h) {
     if (h->ev_bjoin) cudaEventDestroy(h->ev_bjoin);
     if (h->aux) { cudaStreamSynchronize(h->aux); cudaStreamDestroy(h->aux); }
     if (h->ev_dz) cudaEventDestroy(h->ev_dz);
+    if (h->ev_gemv) cudaEventDestroy(h->ev_gemv);
     if (h->ev_wjoin) cudaEventDestroy(h->ev_wjoin);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_inputs) cudaEventDestroy(h->ev_inputs);

@@ -9,6 +9,7 @@
 #include "conv_tc.cuh"
 #include "conv_group.cuh"
 #include "split.cuh"
+#include "conv_gemv.cuh"
 
 namespace pb {
 
@@ -46,6 +47,7 @@ struct StageHost {
     // weight stashing: rings of the weights (and normalisation scale) each forward used
     float* wstash = nullptr; __nv_bfloat16* wstash16 = nullptr; float* gstash = nullptr;
     int stash_slots = 0; size_t wstash_stride = 0, gstash_stride = 0;       // strides in bytes, multiples of 16
+    bool gemv = false;                                             // 3x3 stage on a tiny image: one fused pass over (w, v) per tick
     bool fuse_stats = false;                                       // its forward GEMM writes the conv output and the chunk statistics
     int ntn = 1;                                                   // column tiles of that GEMM
     __nv_bfloat16 *out16 = nullptr, *dz16 = nullptr;
@@ -110,6 +112,10 @@ struct pb_handle {
     std::vector<pb::PostChunk> h_ptiles[2]; pb::PostChunk* d_ptiles[2] = {nullptr, nullptr};   // tiles of the elementwise kernels: forward, backward
     std::vector<pb::UpdRange> h_upd; pb::UpdRange* d_upd = nullptr;
     std::vector<pb::UpdChunk> h_chunks; pb::UpdChunk* d_chunks = nullptr;
+    std::vector<pb::ConvGemvStage> h_gemv; pb::ConvGemvStage* d_gemv = nullptr;             // stages run by the fused tiny-image kernel
+    std::vector<pb::GemvBlock> h_gemvblocks; pb::GemvBlock* d_gemvblocks = nullptr;
+    size_t gemv_smem = 0;
+    cudaEvent_t ev_gemv = nullptr;
     std::vector<pb::GroupBlock> h_gblocks; pb::GroupBlock* d_gblocks = nullptr;             // bundles normalised by one block each
     size_t group_smem_fwd = 0, group_smem_bwd = 0;
     std::vector<pb::StashRange> h_stash; pb::StashRange* d_stash = nullptr;

@@ -203,6 +203,20 @@ def tiny_cnn(seed=11, ticks=24, flags=FLAG_SC | FLAG_LWP):
                     0.02, 0.9, ticks, seed, flags)
 
 
+def tail_cnn(seed=14, ticks=40, flags=FLAG_SC | FLAG_LWP):
+    """The tail of a VGG-style net in small: 3x3 convolutions on 4x4 and 2x2 images with
+    32..64 channels (a handful of output pixels per weight: weight-streaming stages)."""
+    b = _Builder()
+    b.conv(3, 32, 3, 1, 1, 8, pool=(2, 2, 0))         # 8x8 -> 4x4
+    b.conv(32, 64, 3, 1, 1, 8)                        # 4x4
+    b.conv(64, 64, 3, 1, 1, 16, pool=(2, 2, 0))       # 4x4 -> 2x2
+    b.conv(64, 32, 3, 1, 1, 4)                        # 2x2
+    b.conv(32, 32, 3, 1, 1, 8, pool=(2, 2, 0))        # 2x2 -> 1x1
+    b.fc(32, 6, relu=False, loss=True)
+    return Workload("tail_cnn", b.layers, b.stage_of, (3, 8, 8), 6,
+                    0.01, 0.9, ticks, seed, flags)
+
+
 def tiny_resnet(seed=12, ticks=40, flags=FLAG_SC | FLAG_LWP, bottleneck=False, relu=True):
     """Small residual nets that reach every skip form the big ones use."""
     if bottleneck:

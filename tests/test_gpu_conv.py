@@ -2,7 +2,7 @@
 import numpy as np
 import pytest
 
-from pb_workloads import tall_bottleneck, tiny_cnn, tiny_resnet, workload
+from pb_workloads import tail_cnn, tall_bottleneck, tiny_cnn, tiny_resnet, workload
 from tests.parity import compare_ticks
 
 pytestmark = pytest.mark.gpu
@@ -26,6 +26,17 @@ def test_tiny_cnn(flags):
     wl = tiny_cnn(flags=flags)
     w = compare_ticks(wl, 2 * (wl.n_stages - 1) + 24, TOL)
     assert w["ticks"] == 2 * (wl.n_stages - 1) + 24
+
+
+@pytest.mark.parametrize("flags", [3, 0, 1, 2])
+def test_weight_streaming_conv_stages_on_tiny_images(flags):
+    # 3x3 stages on 4x4 and 2x2 images run as ONE fused pass over (w, v) per tick (forward with
+    # the predicted weights, data gradient, weight gradient, update), like FC stages
+    wl = tail_cnn(flags=flags)
+    n = 2 * (wl.n_stages - 1) + 24
+    w = compare_ticks(wl, n, TOL, **FRAGILE)
+    assert w["ticks"] == n and w["min_updates"] >= 24
+    assert w["fragile_tick"] is None or w["fragile_tick"] >= wl.n_stages
 
 
 def test_tiny_resnet_skips_and_subsampled_shortcut():
