@@ -42,7 +42,8 @@ constexpr int kTcChunk = 64;                  // K elements per shared-memory st
 constexpr int kTcBM = 128;
 constexpr int kTcStageBytes = 16384 * 2;      // A tile + B tile
 constexpr int kTcStages = 3;                  // shared-memory stages of the operand pipeline (97 KB: two blocks per SM)
-constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + 1024;
+constexpr int kTcEpiBufFloats = 32 * 17;      // per epilogue warp: a 32 x 16 piece of D, padded, on its way to coalesced stores
+constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + 4 * kTcEpiBufFloats * 4 + 1024;
 constexpr int kTcEpiWarps = 4;                // warps 0-3: quarter q of the tensor-memory lanes belongs to warp q
 constexpr int kTcProdWarps = 4;               // warps 4-7
 constexpr int kTcProducers = 32 * kTcProdWarps;
@@ -56,7 +57,8 @@ constexpr int kTcThreads = 32 * (kTcMmaWarp + 1);
 constexpr int kTcTmemCols = 256;              // two accumulators of 128 columns
 constexpr long long kTcWaitNs = 200LL * 1000 * 1000;   // a barrier wait gives up after 0.2 s
 constexpr int kTcMaxK = 3072;                 // longest K loop of one dgrad / wgrad tile before K is sliced
-constexpr int kTcMaxKFprop = 8192;            // ... of a forward tile (a single slice lets the epilogue finish the stage's statistics)
+constexpr int kTcMaxKFprop = 1152;            // ... of a forward tile: the few deep stages with a longer K (3x3 on 256 or 512 channels, 1x1 on 2048)
+                                              // would otherwise be the tail of the whole launch; their statistics then come from the first normalisation step
 
 struct ConvGemmTC {
     int mode, M, N, K;
@@ -178,6 +180,7 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
                             const CUtensorMap* __restrict__ tmaps, const TickState* ts, long long t, int S,
                             unsigned char* smem, TcShared& sh) {
     const int ptid = threadIdx.x - 32 * kTcEpiWarps;          // 0 .. kTcProducers - 1
+    const int lane = threadIdx.x & 31;
     int it = 0;                                               // chunks issued so far (all tiles)
     bool ok_all = true;
     for (int q = q0; q < q1 && ok_all; ++q) {
@@ -234,7 +237,8 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
 
         for (int c = 0; c < nchunks; ++c, ++it) {
             const int stg = it % kTcStages;
-            if (it >= kTcStages && !mbar_wait(smem_u32(&sh.empty[stg]), (uint32_t)(((it / kTcStages) & 1) ^ 1), &sh.fail)) { ok_all = false; break; }
+            // (the verdict is taken by the whole warp, so that its lanes stay together for the warp-level arrival below)
+            if (it >= kTcStages && !__all_sync(0xffffffffu, mbar_wait(smem_u32(&sh.empty[stg]), (uint32_t)(((it / kTcStages) & 1) ^ 1), &sh.fail))) { ok_all = false; break; }
             unsigned char* sA = smem + stg * kTcStageBytes;
             unsigned char* sB = sA + 16384;
             const int k0 = kb + c * kTcChunk;
@@ -338,12 +342,14 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
             // this thread's copies of the chunk issued kTcLag iterations ago have landed: make them
-            // visible to the tensor core (async proxy) and count in at that chunk's barrier; the
-            // copies of the kTcLag chunks issued since stay in flight meanwhile
+            // visible to the tensor core (async proxy); once the whole warp has done so, one lane
+            // counts the warp in at that chunk's barrier.  The copies of the kTcLag chunks issued
+            // since stay in flight meanwhile.
             if (it >= kTcLag) {
                 asm volatile("cp.async.wait_group %0;" ::"n"(kTcLag) : "memory");
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_arrive(smem_u32(&sh.full[(it - kTcLag) % kTcStages]));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh.full[(it - kTcLag) % kTcStages]));
             }
         }
     }
@@ -351,7 +357,9 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
     if (ok_all) {
         // the chunks still owed an arrival, oldest first
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        for (int c = max(0, it - kTcLag); c < it; ++c) mbar_arrive(smem_u32(&sh.full[c % kTcStages]));
+        __syncwarp();
+        if (lane == 0)
+            for (int c = max(0, it - kTcLag); c < it; ++c) mbar_arrive(smem_u32(&sh.full[c % kTcStages]));
     }
     if (!ok_all) sh.fail = 1;
 }
@@ -408,9 +416,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 
 __device__ void tc_epilogue(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, int q0, int q1,
-                            const TickState* ts, long long t, int S, TcShared& sh) {
+                            const TickState* ts, long long t, int S, unsigned char* smem, TcShared& sh) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;      // warp = quarter of the tensor-memory lanes
     const uint32_t tmem = sh.tmem_base;
+    // A thread holds one ROW of D (32 consecutive columns per load).  Stored as they are, a warp's
+    // store instruction would touch 32 rows at once (32 half-used sectors); instead 16 columns at a
+    // time go through a padded shared-memory buffer, so that half a warp writes 64 contiguous bytes of one row.
+    float* tb = reinterpret_cast<float*>(smem + kTcStages * kTcStageBytes) + warp * kTcEpiBufFloats;
+    const int sub = lane >> 4, col = lane & 15;
     int lt = 0;
     for (int q = q0; q < q1; ++q) {
         const GemmTile tl = tiles[q];
@@ -429,19 +442,22 @@ __device__ void tc_epilogue(const ConvGemmTC* __restrict__ gemms, const GemmTile
             if (tl.n0 + c0 >= N) break;                             // uniform
             uint32_t r[32];
             tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * 128 + c0), r);
-            if (m < M) {
-                float* dst = Cp + (size_t)m * N + tl.n0 + c0;
-                const int nleft = min(N - (tl.n0 + c0), BN - c0);      // columns of this tile that exist (a tile may be narrower than 32 k)
-                if (nleft >= 32 && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+            const int nleft = min(N - (tl.n0 + c0), BN - c0);          // columns of this tile that exist (a tile may be narrower than 32 k)
 #pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        reinterpret_cast<float4*>(dst)[u] = make_float4(__uint_as_float(r[4 * u]), __uint_as_float(r[4 * u + 1]),
-                                                                        __uint_as_float(r[4 * u + 2]), __uint_as_float(r[4 * u + 3]));
-                } else {
+            for (int half = 0; half < 2; ++half) {
+                __syncwarp();
 #pragma unroll
-                    for (int u = 0; u < 32; ++u)
-                        if (u < nleft) dst[u] = __uint_as_float(r[u]);
+                for (int u = 0; u < 16; ++u) tb[lane * 17 + u] = __uint_as_float(r[half * 16 + u]);
+                __syncwarp();
+                const int cg = half * 16 + col;
+                if (cg < nleft) {
+                    float* dst = Cp + (size_t)(tl.m0 + warp * 32 + sub) * N + tl.n0 + c0 + cg;
+#pragma unroll
+                    for (int rr = 0; rr < 16; ++rr)
+                        if (tl.m0 + warp * 32 + 2 * rr + sub < M) dst[(size_t)(2 * rr) * N] = tb[(2 * rr + sub) * 17 + col];
                 }
+            }
+            if (m < M) {
                 if (G.fuse) {
                     // count / mean / M2 of these (up to) 32 values, merged into the row's running triple
                     const int nv = min(32, nleft);
@@ -486,7 +502,7 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, TcLaunch L, const CUtensorM
     }
     if (tid == 32) {
         for (int q = 0; q < kTcStages; ++q) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh.full[q])), "r"(kTcProducers + 1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&sh.full[q])), "r"(kTcProdWarps + 1) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sh.empty[q])) : "memory");
         }
         for (int q = 0; q < 2; ++q) {
@@ -500,7 +516,7 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, TcLaunch L, const CUtensorM
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const long long t = ts->cnt[par];
-    if (warp < kTcEpiWarps) tc_epilogue(gemms, L.tiles, q0, q1, ts, t, S, sh);
+    if (warp < kTcEpiWarps) tc_epilogue(gemms, L.tiles, q0, q1, ts, t, S, smem, sh);
     else if (warp < kTcMmaWarp) tc_producer(gemms, L.tiles, q0, q1, tmaps, ts, t, S, smem, sh);
     else if (tid == 32 * kTcMmaWarp) tc_mma(gemms, L.tiles, q0, q1, ts, t, S, smem, sh);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
