@@ -42,7 +42,8 @@ constexpr int kTcChunk = 64;                  // K elements per shared-memory st
 constexpr int kTcBM = 128;
 constexpr int kTcStageBytes = 16384 * 2;      // A tile + B tile
 constexpr int kTcStages = 3;                  // shared-memory stages of the operand pipeline (97 KB: two blocks per SM)
-constexpr int kTcEpiBufFloats = 32 * 17;      // per epilogue warp: a 32 x 16 piece of D, padded, on its way to coalesced stores
+constexpr int kTcEpiPitch = 20;               // floats between rows of an epilogue warp's staging buffer (16-byte aligned, conflict-free 128-bit writes)
+constexpr int kTcEpiBufFloats = 32 * kTcEpiPitch;   // per epilogue warp: a 32 x 16 piece of D on its way to coalesced stores
 constexpr int kTcSmemBytes = kTcStages * kTcStageBytes + 4 * kTcEpiBufFloats * 4 + 1024;
 constexpr int kTcEpiWarps = 4;                // warps 0-3: quarter q of the tensor-memory lanes belongs to warp q
 constexpr int kTcProdWarps = 4;               // warps 4-7
@@ -53,7 +54,8 @@ constexpr int kTcKStep = kTcProducers / 16;   // MN-major tiles of width 128: k 
 constexpr int kTcKIters = kTcChunk / kTcKStep;
 constexpr int kTcLag = 1;                     // chunks a producer thread keeps in flight behind the one it is issuing (< kTcStages - 1)
 constexpr int kTcMmaWarp = kTcEpiWarps + kTcProdWarps;
-constexpr int kTcThreads = 32 * (kTcMmaWarp + 1);
+constexpr int kTcTmaWarp = kTcMmaWarp + 1;    // one thread of it issues every bulk tensor copy
+constexpr int kTcThreads = 32 * (kTcTmaWarp + 1);
 constexpr int kTcTmemCols = 256;              // two accumulators of 128 columns
 constexpr long long kTcWaitNs = 200LL * 1000 * 1000;   // a barrier wait gives up after 0.2 s
 constexpr int kTcMaxK = 3072;                 // longest K loop of one dgrad / wgrad tile before K is sliced
@@ -163,7 +165,7 @@ __device__ __forceinline__ void cp_async16(unsigned char* dst, const __nv_bfloat
 }
 
 struct TcShared {
-    uint64_t full[kTcStages];     // a stage's operands have landed (one arrival per producer thread + 1 with the bulk copies' bytes)
+    uint64_t full[kTcStages];     // a stage's operands have landed (one arrival per producer warp + 1 with the bulk copies' bytes)
     uint64_t empty[kTcStages];    // the MMAs that read a stage have completed
     uint64_t acc_full[2];         // a tile's accumulator is complete
     uint64_t acc_empty[2];        // the epilogue warps have drained an accumulator
@@ -177,8 +179,7 @@ __device__ __forceinline__ long long tc_sample(const ConvGemmTC& G, long long t,
 
 // ------------------------------------------------------------------ producer warps
 __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, int q0, int q1,
-                            const CUtensorMap* __restrict__ tmaps, const TickState* ts, long long t, int S,
-                            unsigned char* smem, TcShared& sh) {
+                            const TickState* ts, long long t, int S, unsigned char* smem, TcShared& sh) {
     const int ptid = threadIdx.x - 32 * kTcEpiWarps;          // 0 .. kTcProducers - 1
     const int lane = threadIdx.x & 31;
     int it = 0;                                               // chunks issued so far (all tiles)
@@ -195,14 +196,7 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
         const __nv_bfloat16* __restrict__ A = G.a + (size_t)(smp % G.a_slots) * G.a_elems;
         const __nv_bfloat16* __restrict__ B = G.b + (size_t)slot * G.b_elems;
         const int CI = G.ci, CO = G.co, ksz = G.k, st = G.stride, pad = G.pad, ih = G.ih, iw = G.iw, oh = G.oh, ow = G.ow;
-        const CUtensorMap* tmA = G.a_tmap >= 0 ? tmaps + G.a_tmap : nullptr;
-        const CUtensorMap* tmB = G.b_tmap >= 0 ? tmaps + G.b_tmap : nullptr;
-        // MN-major tiles arrive as boxes of 64 columns: a second box that would lie wholly outside
-        // the matrix is not fetched (its rows / columns of D are never stored)
-        const bool a2 = mode != kFprop && tl.m0 + 64 < M;
-        const bool b2 = mode == kWgrad && BN == 128 && tl.n0 + 64 < N;
-        const uint32_t tx_bytes = (tmA ? (mode == kFprop ? 16384u : (a2 ? 16384u : 8192u)) : 0u) +
-                                  (tmB ? (mode == kWgrad ? (b2 ? 16384u : 8192u) : (uint32_t)G.b_bytes) : 0u);
+        const bool tmA = G.a_tmap >= 0, tmB = G.b_tmap >= 0;      // operands the bulk-copy thread fetches
         // the gathers divide by these for every 16-byte unit: reciprocals once per tile
         const float inv_ci = 1.f / (float)CI, inv_co = 1.f / (float)CO, inv_ksz = 1.f / (float)ksz,
                     inv_st = 1.f / (float)st, inv_ow = 1.f / (float)ow;
@@ -242,42 +236,6 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
             unsigned char* sA = smem + stg * kTcStageBytes;
             unsigned char* sB = sA + 16384;
             const int k0 = kb + c * kTcChunk;
-            const uint32_t fullb = smem_u32(&sh.full[stg]);
-            if (ptid == 0) {
-                // the extra arrival of the stage, carrying the bytes of this chunk's bulk copies
-                if (tx_bytes) mbar_arrive_tx(fullb, tx_bytes); else mbar_arrive(fullb);
-                if (tmA) {
-                    if (mode == kFprop) {
-                        tma_2d(smem_u32(sA), tmA, k0, tl.m0, fullb);
-                    } else if (mode == kDgrad) {
-                        const int rs = k0 / CO, co0 = k0 - rs * CO;       // a chunk is 64 output channels of one tap
-                        tma_3d(smem_u32(sA), tmA, tl.m0, rs, co0, fullb);
-                        if (a2) tma_3d(smem_u32(sA) + 8192, tmA, tl.m0 + 64, rs, co0, fullb);
-                    } else {
-                        tma_2d(smem_u32(sA), tmA, tl.m0, k0, fullb);
-                        if (a2) tma_2d(smem_u32(sA) + 8192, tmA, tl.m0 + 64, k0, fullb);
-                    }
-                }
-                if (tmB) {
-                    if (G.b_rect) {
-                        // 3x3, stride 1: the chunk is 64 channels of ONE tap (r, s); the tile's pixels are whole
-                        // image rows, so its operand is the same box of the image shifted by the tap
-                        // (rows and columns outside the image arrive as zeros)
-                        const int C = mode == kFprop ? CI : CO;
-                        const int rs = k0 / C, c0 = k0 - rs * C, r = rs / ksz, sx = rs - r * ksz;
-                        const int row0 = tl.n0 / G.b_rect;
-                        if (mode == kFprop) tma_4d(smem_u32(sB), tmB, c0, sx - pad, row0 + r - pad, slot, fullb);
-                        else tma_3d(smem_u32(sB), tmB, c0, pad - sx, row0 + pad - r, fullb);
-                    } else if (mode == kFprop) {
-                        tma_3d(smem_u32(sB), tmB, k0, tl.n0, slot, fullb);
-                    } else if (mode == kDgrad) {
-                        tma_2d(smem_u32(sB), tmB, k0, tl.n0, fullb);
-                    } else {
-                        tma_3d(smem_u32(sB), tmB, tl.n0, k0, slot, fullb);
-                        if (b2) tma_3d(smem_u32(sB) + 8192, tmB, tl.n0 + 64, k0, slot, fullb);
-                    }
-                }
-            }
             // ---------------- gathered A tile
             if (!tmA) {
                 if (mode == kFprop) {
@@ -364,6 +322,79 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
     if (!ok_all) sh.fail = 1;
 }
 
+// ------------------------------------------------------------------ bulk-copy thread
+// Issues every bulk tensor copy of the block's tiles, chunk by chunk, as soon as the chunk's stage
+// is free, and counts in at the stage's barrier with the bytes to expect.  It runs apart from the
+// gathering warps: a thread that follows its copies with a proxy fence waits for them to land,
+// which would bring the pipeline down to one chunk per memory latency.
+__device__ void tc_tma(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, int q0, int q1,
+                       const CUtensorMap* __restrict__ tmaps, const TickState* ts, long long t, int S,
+                       unsigned char* smem, TcShared& sh) {
+    int it = 0;
+    for (int q = q0; q < q1; ++q) {
+        const GemmTile tl = tiles[q];
+        const ConvGemmTC& G = gemms[tl.gemm];
+        const long long smp = tc_sample(G, t, S);
+        if (!sample_live(ts, smp)) continue;
+        const int mode = G.mode, M = G.M, N = G.N, BN = G.bn;
+        const int kb = tl.split * G.k_per_split, ke = min(G.K, kb + G.k_per_split);
+        const int nchunks = (ke - kb + kTcChunk - 1) / kTcChunk;
+        const int slot = (int)(smp % G.b_slots);
+        const int CI = G.ci, CO = G.co, ksz = G.k, pad = G.pad, b_rect = G.b_rect;
+        const CUtensorMap* tmA = G.a_tmap >= 0 ? tmaps + G.a_tmap : nullptr;
+        const CUtensorMap* tmB = G.b_tmap >= 0 ? tmaps + G.b_tmap : nullptr;
+        // MN-major tiles arrive as boxes of 64 columns: a second box that would lie wholly outside
+        // the matrix is not fetched (its rows / columns of D are never stored)
+        const bool a2 = mode != kFprop && tl.m0 + 64 < M;
+        const bool b2 = mode == kWgrad && BN == 128 && tl.n0 + 64 < N;
+        const uint32_t tx_bytes = (tmA ? (mode == kFprop ? 16384u : (a2 ? 16384u : 8192u)) : 0u) +
+                                  (tmB ? (mode == kWgrad ? (b2 ? 16384u : 8192u) : (uint32_t)G.b_bytes) : 0u);
+        for (int c = 0; c < nchunks; ++c, ++it) {
+            const int stg = it % kTcStages;
+            if (it >= kTcStages && !mbar_wait(smem_u32(&sh.empty[stg]), (uint32_t)(((it / kTcStages) & 1) ^ 1), &sh.fail)) { sh.fail = 1; return; }
+            unsigned char* sA = smem + stg * kTcStageBytes;
+            unsigned char* sB = sA + 16384;
+            const int k0 = kb + c * kTcChunk;
+            const uint32_t fullb = smem_u32(&sh.full[stg]);
+            {
+                // the extra arrival of the stage, carrying the bytes of this chunk's bulk copies
+                if (tx_bytes) mbar_arrive_tx(fullb, tx_bytes); else mbar_arrive(fullb);
+                if (tmA) {
+                    if (mode == kFprop) {
+                        tma_2d(smem_u32(sA), tmA, k0, tl.m0, fullb);
+                    } else if (mode == kDgrad) {
+                        const int rs = k0 / CO, co0 = k0 - rs * CO;       // a chunk is 64 output channels of one tap
+                        tma_3d(smem_u32(sA), tmA, tl.m0, rs, co0, fullb);
+                        if (a2) tma_3d(smem_u32(sA) + 8192, tmA, tl.m0 + 64, rs, co0, fullb);
+                    } else {
+                        tma_2d(smem_u32(sA), tmA, tl.m0, k0, fullb);
+                        if (a2) tma_2d(smem_u32(sA) + 8192, tmA, tl.m0 + 64, k0, fullb);
+                    }
+                }
+                if (tmB) {
+                    if (b_rect) {
+                        // 3x3, stride 1: the chunk is 64 channels of ONE tap (r, s); the tile's pixels are whole
+                        // image rows, so its operand is the same box of the image shifted by the tap
+                        // (rows and columns outside the image arrive as zeros)
+                        const int C = mode == kFprop ? CI : CO;
+                        const int rs = k0 / C, c0 = k0 - rs * C, r = rs / ksz, sx = rs - r * ksz;
+                        const int row0 = tl.n0 / b_rect;
+                        if (mode == kFprop) tma_4d(smem_u32(sB), tmB, c0, sx - pad, row0 + r - pad, slot, fullb);
+                        else tma_3d(smem_u32(sB), tmB, c0, pad - sx, row0 + pad - r, fullb);
+                    } else if (mode == kFprop) {
+                        tma_3d(smem_u32(sB), tmB, k0, tl.n0, slot, fullb);
+                    } else if (mode == kDgrad) {
+                        tma_2d(smem_u32(sB), tmB, k0, tl.n0, fullb);
+                    } else {
+                        tma_3d(smem_u32(sB), tmB, tl.n0, k0, slot, fullb);
+                        if (b2) tma_3d(smem_u32(sB) + 8192, tmB, tl.n0 + 64, k0, slot, fullb);
+                    }
+                }
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------ MMA warp (one thread)
 __device__ void tc_mma(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, int q0, int q1,
                        const TickState* ts, long long t, int S, unsigned char* smem, TcShared& sh) {
@@ -421,9 +452,12 @@ __device__ void tc_epilogue(const ConvGemmTC* __restrict__ gemms, const GemmTile
     const uint32_t tmem = sh.tmem_base;
     // A thread holds one ROW of D (32 consecutive columns per load).  Stored as they are, a warp's
     // store instruction would touch 32 rows at once (32 half-used sectors); instead 16 columns at a
-    // time go through a padded shared-memory buffer, so that half a warp writes 64 contiguous bytes of one row.
+    // time go through a shared-memory buffer, from which four lanes write the 64 contiguous bytes of
+    // one row with 128-bit stores (eight rows per instruction), or, where rows of D do not start on
+    // 16-byte boundaries (N not a multiple of 4), half a warp writes them with 32-bit stores.
     float* tb = reinterpret_cast<float*>(smem + kTcStages * kTcStageBytes) + warp * kTcEpiBufFloats;
     const int sub = lane >> 4, col = lane & 15;
+    const int rsub = lane >> 2, c4 = (lane & 3) * 4;
     int lt = 0;
     for (int q = q0; q < q1; ++q) {
         const GemmTile tl = tiles[q];
@@ -437,6 +471,7 @@ __device__ void tc_epilogue(const ConvGemmTC* __restrict__ gemms, const GemmTile
         float* __restrict__ Cp = G.fuse ? G.c + (size_t)(smp % G.c_slots) * ((size_t)M * N)
                                         : G.c + ((size_t)(smp % G.c_slots) * G.nsplit + tl.split) * ((size_t)M * N);
         const int m = tl.m0 + warp * 32 + lane;                     // row of D held by this thread
+        const bool vec = (N & 3) == 0;
         float cnt = 0.f, mean = 0.f, m2 = 0.f;                      // statistics of this row's columns (forward, fused)
         for (int c0 = 0; c0 < BN; c0 += 32) {
             if (tl.n0 + c0 >= N) break;                             // uniform
@@ -446,15 +481,30 @@ __device__ void tc_epilogue(const ConvGemmTC* __restrict__ gemms, const GemmTile
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 __syncwarp();
+                float4* trow = reinterpret_cast<float4*>(tb + lane * kTcEpiPitch);
 #pragma unroll
-                for (int u = 0; u < 16; ++u) tb[lane * 17 + u] = __uint_as_float(r[half * 16 + u]);
+                for (int j = 0; j < 4; ++j)
+                    trow[j] = make_float4(__uint_as_float(r[half * 16 + 4 * j]), __uint_as_float(r[half * 16 + 4 * j + 1]),
+                                          __uint_as_float(r[half * 16 + 4 * j + 2]), __uint_as_float(r[half * 16 + 4 * j + 3]));
                 __syncwarp();
-                const int cg = half * 16 + col;
-                if (cg < nleft) {
-                    float* dst = Cp + (size_t)(tl.m0 + warp * 32 + sub) * N + tl.n0 + c0 + cg;
+                if (vec) {
+                    // n0, c0 and the tile widths are multiples of 16, so nleft is a multiple of 4 here
+                    const int cg = half * 16 + c4;
+                    if (cg < nleft) {
+                        float* dst = Cp + (size_t)(tl.m0 + warp * 32 + rsub) * N + tl.n0 + c0 + cg;
 #pragma unroll
-                    for (int rr = 0; rr < 16; ++rr)
-                        if (tl.m0 + warp * 32 + 2 * rr + sub < M) dst[(size_t)(2 * rr) * N] = tb[(2 * rr + sub) * 17 + col];
+                        for (int i = 0; i < 4; ++i)
+                            if (tl.m0 + warp * 32 + 8 * i + rsub < M)
+                                *reinterpret_cast<float4*>(dst + (size_t)(8 * i) * N) = *reinterpret_cast<const float4*>(tb + (8 * i + rsub) * kTcEpiPitch + c4);
+                    }
+                } else {
+                    const int cg = half * 16 + col;
+                    if (cg < nleft) {
+                        float* dst = Cp + (size_t)(tl.m0 + warp * 32 + sub) * N + tl.n0 + c0 + cg;
+#pragma unroll
+                        for (int rr = 0; rr < 16; ++rr)
+                            if (tl.m0 + warp * 32 + 2 * rr + sub < M) dst[(size_t)(2 * rr) * N] = tb[(2 * rr + sub) * kTcEpiPitch + col];
+                    }
                 }
             }
             if (m < M) {
@@ -517,8 +567,9 @@ conv_tc_kernel(const ConvGemmTC* __restrict__ gemms, TcLaunch L, const CUtensorM
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const long long t = ts->cnt[par];
     if (warp < kTcEpiWarps) tc_epilogue(gemms, L.tiles, q0, q1, ts, t, S, smem, sh);
-    else if (warp < kTcMmaWarp) tc_producer(gemms, L.tiles, q0, q1, tmaps, ts, t, S, smem, sh);
+    else if (warp < kTcMmaWarp) tc_producer(gemms, L.tiles, q0, q1, ts, t, S, smem, sh);
     else if (tid == 32 * kTcMmaWarp) tc_mma(gemms, L.tiles, q0, q1, ts, t, S, smem, sh);
+    else if (tid == 32 * kTcTmaWarp) tc_tma(gemms, L.tiles, q0, q1, tmaps, ts, t, S, smem, sh);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (sh.fail) {
