@@ -10,7 +10,8 @@
 // blocks fit on an SM) and the per-channel sums cross the cluster through
 // distributed shared memory:
 //   forward   merge the (channel, column tile) statistics that the GEMM epilogue
-//             left -> group mean and 1/std -> normalise, add the skip input,
+//             left (or, where the GEMM left K slices, sum them and take the
+//             statistics of the sum) -> group mean and 1/std -> normalise, add the skip input,
 //             ReLU -> float32 output (only where somebody reads it), ReLU mask,
 //             and the bfloat16 copy, transposed through shared memory;
 //   backward  gradient at the normalised activation (consumers' partial rows
@@ -31,7 +32,8 @@ namespace pb {
 constexpr int kGroupThreads = 256;
 constexpr int kGroupWarps = kGroupThreads / 32;
 constexpr int kGroupMaxElems = 25088;          // elements of a bundle that stay in shared memory (98 KB as float32)
-constexpr int kGroupMaxChannels = 64;
+constexpr int kGroupMaxChannels = 256;        // channels of a bundle
+constexpr int kGroupTargetElems = 12544;       // small groups are bundled up to about this many elements (one block then has a few thousand)
 constexpr int kGroupSplit = 4;                 // blocks (one cluster) that share a bundle's pixels
 
 // One block's bundle: groups [grp0, grp0 + ngrp) of one stage.
@@ -59,49 +61,78 @@ __device__ void group_forward(const ConvStage& st, const GroupBlock gb, int rank
     const int slot = slot_of(i, st.slots);
     const int hw = st.oh * st.ow, cpg = st.cpg, c0 = gb.grp0 * cpg, nch = gb.ngrp * cpg;
     const size_t zelems = (size_t)st.co * hw;
-    // ---- group statistics from the GEMM epilogue's partials (count, mean, M2 per channel and column
-    // tile): every thread folds the entries k = tid, tid + 256, ... of a group into one triple (all its
-    // loads are independent: one memory latency), then the triples are merged along a fixed tree
-    for (int g = 0; g < gb.ngrp; ++g) {
-        const int grp = gb.grp0 + g, nidx = st.fstat_stride;
-        const float* f = st.fstat + (size_t)grp * nidx * 3;
-        float n = 0.f, mean = 0.f, m2 = 0.f;
-        for (int k = tid; k < nidx; k += kGroupThreads) {
-            const float nb = f[3 * k], mb = f[3 * k + 1], qb = f[3 * k + 2];
-            const float tot = n + nb, dl = mb - mean;
-            if (tot > 0.f) { mean += dl * (nb / tot); m2 += qb + dl * dl * (n * nb / tot); }
-            n = tot;
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float nb = __shfl_xor_sync(0xffffffffu, n, o), mb = __shfl_xor_sync(0xffffffffu, mean, o), qb = __shfl_xor_sync(0xffffffffu, m2, o);
-            // (both partners compute the same merged triple: a and b enter symmetrically up to the sign of dl)
-            const bool low = (lane & o) == 0;
-            const float na = low ? n : nb, ma = low ? mean : mb, qa = low ? m2 : qb;
-            const float nc = low ? nb : n, mc = low ? mb : mean, qc = low ? qb : m2;
-            const float tot = na + nc, dl = mc - ma;
-            if (tot > 0.f) { mean = ma + dl * (nc / tot); m2 = qa + qc + dl * dl * (na * nc / tot); } else { mean = 0.f; m2 = 0.f; }
-            n = tot;
-        }
-        if (lane == 0) { sh.s1[warp] = n; sh.s2[warp] = mean; sh.t1[warp] = m2; }
-        __syncthreads();
-        if (tid == 0) {
-            float na = sh.s1[0], ma = sh.s2[0], qa = sh.t1[0];
-            for (int w = 1; w < kGroupWarps; ++w) {
-                const float nc = sh.s1[w], mc = sh.s2[w], qc = sh.t1[w];
-                const float tot = na + nc, dl = mc - ma;
-                if (tot > 0.f) { ma += dl * (nc / tot); qa += qc + dl * dl * (na * nc / tot); }
-                na = tot;
+    const int npu = hw / VEC;
+    int u_lo, u_hi;
+    group_range(npu, rank, u_lo, u_hi);
+    const int p_lo = u_lo * VEC, np = (u_hi - u_lo) * VEC;               // this block's pixels
+    // ---- group statistics, a warp per group (every block of the bundle computes the same numbers)
+    for (int g = warp; g < gb.ngrp; g += kGroupWarps) {
+        const int grp = gb.grp0 + g;
+        float mean, rstd;
+        if (st.fused) {
+            // from the GEMM epilogue's partials (count, mean, M2 per channel and column tile): a lane folds
+            // the entries k = lane, lane + 32, ... into one triple (independent loads), then the triples
+            // are merged along a fixed tree
+            const int nidx = st.fstat_stride;
+            const float* f = st.fstat + (size_t)grp * nidx * 3;
+            float n = 0.f, m2 = 0.f;
+            mean = 0.f;
+            for (int k = lane; k < nidx; k += 32) {
+                const float nb = f[3 * k], mb = f[3 * k + 1], qb = f[3 * k + 2];
+                const float tot = n + nb, dl = mb - mean;
+                if (tot > 0.f) { mean += dl * (nb / tot); m2 += qb + dl * dl * (n * nb / tot); }
+                n = tot;
             }
-            const float rstd = rsqrtf(qa / na + kGnEps);
-            sh.m1[g] = ma; sh.m2[g] = rstd;
-            if (rank == 0) {                   // (every block of the bundle computes the same numbers)
-                st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0] = ma;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float nb = __shfl_xor_sync(0xffffffffu, n, o), mb = __shfl_xor_sync(0xffffffffu, mean, o), qb = __shfl_xor_sync(0xffffffffu, m2, o);
+                // (both partners compute the same merged triple: a and b enter symmetrically up to the sign of dl)
+                const bool low = (lane & o) == 0;
+                const float na = low ? n : nb, ma = low ? mean : mb, qa = low ? m2 : qb;
+                const float nc = low ? nb : n, mc = low ? mb : mean, qc = low ? qb : m2;
+                const float tot = na + nc, dl = mc - ma;
+                if (tot > 0.f) { mean = ma + dl * (nc / tot); m2 = qa + qc + dl * dl * (na * nc / tot); } else { mean = 0.f; m2 = 0.f; }
+                n = tot;
+            }
+            rstd = rsqrtf(m2 / n + kGnEps);
+        } else {
+            // the forward GEMM left K slices: the conv output is their sum in slice order (this block
+            // files its own pixels in the ring for the backward); mean, then squared deviations
+            const size_t gbase = (size_t)grp * cpg * hw;
+            const int ne = cpg * hw;
+            const float inv_hw = 1.f / (float)hw;
+            float* __restrict__ zr = st.z_ring + (size_t)slot * zelems;
+            float s1 = 0.f;
+            for (int e = lane; e < ne; e += 32) {
+                float v = 0.f;
+                for (int q = 0; q < st.z_nsplit; ++q) v += st.zpart[(size_t)q * zelems + gbase + e];
+                s1 += v;
+                const int p = e - quot(e, inv_hw) * hw;
+                if (p >= p_lo && p < p_lo + np) zr[gbase + e] = v;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+            mean = s1 / (float)ne;
+            float s2 = 0.f;
+            for (int e = lane; e < ne; e += 32) {
+                float v = 0.f;
+                for (int q = 0; q < st.z_nsplit; ++q) v += st.zpart[(size_t)q * zelems + gbase + e];
+                const float d = v - mean;
+                s2 = fmaf(d, d, s2);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+            rstd = rsqrtf(s2 / (float)ne + kGnEps);
+        }
+        if (lane == 0) {
+            sh.m1[g] = mean; sh.m2[g] = rstd;
+            if (rank == 0) {
+                st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0] = mean;
                 st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 1] = rstd;
             }
         }
-        __syncthreads();
     }
+    __syncthreads();          // (also orders this block's ring writes before its reads below)
     for (int cl = tid; cl < nch; cl += kGroupThreads) {
         const int g = cl / cpg, c = c0 + cl;
         sh.gs[cl] = st.wh[st.nw + c] * sh.m2[g];
@@ -114,10 +145,6 @@ __device__ void group_forward(const ConvStage& st, const GroupBlock gb, int rank
         ? st.skip_ring + (size_t)slot_of(i, st.skip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
     unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems;
     float* __restrict__ out = st.out_ring + (size_t)slot * zelems;
-    const int npu = hw / VEC;
-    int u_lo, u_hi;
-    group_range(npu, rank, u_lo, u_hi);
-    const int p_lo = u_lo * VEC, np = (u_hi - u_lo) * VEC;               // this block's pixels
     __nv_bfloat16* t16 = reinterpret_cast<__nv_bfloat16*>(buf);          // [nch][np + 2]
     const int rs = np + 2;
     // ---- normalise, skip, ReLU: the bundle's (channel, pixel unit) pairs spread flat over the

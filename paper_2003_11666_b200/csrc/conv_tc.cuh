@@ -325,8 +325,8 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
 // ------------------------------------------------------------------ bulk-copy thread
 // Issues every bulk tensor copy of the block's tiles, chunk by chunk, as soon as the chunk's stage
 // is free, and counts in at the stage's barrier with the bytes to expect.  It runs apart from the
-// gathering warps: a thread that follows its copies with a proxy fence waits for them to land,
-// which would bring the pipeline down to one chunk per memory latency.
+// gathering warps, whose every iteration waits for their own copies of the chunk before: issued
+// from there, the bulk copies of a chunk would start one memory latency after those of the last.
 __device__ void tc_tma(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, int q0, int q1,
                        const CUtensorMap* __restrict__ tmaps, const TickState* ts, long long t, int S,
                        unsigned char* smem, TcShared& sh) {

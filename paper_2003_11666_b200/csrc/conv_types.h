@@ -56,6 +56,7 @@ struct ConvStage {
     float* z_ring;               // [slots][co*oh*ow] conv output, kept for the backward
     float* stat_ring;            // [slots][2*groups] mean, rstd
     float* fstat; int fstat_stride;      // forward chunk partials [groups][fstat_stride][3]: count, mean, M2
+    int fused;                           // the forward GEMM wrote z_ring and fstat itself (one K slice)
     float* bsum; int npieces;            // backward channel partials [co][npieces][2]
     float* gsum;                 // backward group means [groups][2] (of d*gamma and d*gamma*zhat)
     unsigned char* code_ring;    // [slots][co*oh*ow] bit0: ReLU passed

@@ -617,7 +617,7 @@ bool fill_conv_tables(pb_handle* h) {
         for (int q : x.consumers_skip) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dskip, y.dskip_slots, 1}; }
         c.dz = x.dz;
         c.gstash = x.gstash; c.gstash_slots = x.stash_slots;
-        c.fstat = x.fstat; c.fstat_stride = x.fstat_stride; c.bsum = x.bsum; c.npieces = x.npieces; c.gsum = x.gsum;
+        c.fstat = x.fstat; c.fstat_stride = x.fstat_stride; c.fused = x.fuse_stats ? 1 : 0; c.bsum = x.bsum; c.npieces = x.npieces; c.gsum = x.gsum;
         {
             // Chunks of the first step: whole channels while they fit, else pieces of one channel.
             // Tiles of the second step: (a multiple of 8 channels) x pixels, up to kPostChunk
@@ -636,14 +636,17 @@ bool fill_conv_tables(pb_handle* h) {
             // one block per bundle, forward and backward (conv_group.cuh), and leaves the lists below.
             // (a bundle spans whole 8-channel units: groups of 1, 2, 4 channels are bundled, groups of 8, 16, ... stand alone)
             const bool units_ok = x.tc && L.c_out % 8 == 0 && (cpg < 8 ? 8 % cpg == 0 : cpg % 8 == 0);
-            const bool resident = x.fuse_stats && units_ok && !x.has_pool && !x.avgpool && x.gn_groups % gpb == 0 &&
-                                  gpb * cpg <= kGroupMaxChannels && (long long)gpb * cpg * hw <= kGroupMaxElems;
+            // small groups are bundled further (a block pays its chain of memory latencies whatever its size)
+            int rgpb = gpb;
+            while (x.gn_groups % (2 * rgpb) == 0 && 2 * rgpb * cpg <= kGroupMaxChannels && 2LL * rgpb * cpg * hw <= kGroupTargetElems) rgpb *= 2;
+            const bool resident = x.tc && !h->post_fuse && units_ok && !x.has_pool && !x.avgpool && x.gn_groups % rgpb == 0 &&
+                                  rgpb * cpg <= kGroupMaxChannels && (long long)rgpb * cpg * hw <= kGroupMaxElems;
             if (resident) {
-                for (int g0 = 0; g0 < x.gn_groups; g0 += gpb) h->h_gblocks.push_back(GroupBlock{stage_idx, g0, gpb});
+                for (int g0 = 0; g0 < x.gn_groups; g0 += rgpb) h->h_gblocks.push_back(GroupBlock{stage_idx, g0, rgpb});
                 // each of the kGroupSplit blocks of a bundle holds a quarter of the pixels (rounded up to whole units of 4)
                 const size_t np = (size_t)(ceil_div(ceil_div(hw, 4), kGroupSplit) + 1) * 4;
-                h->group_smem_fwd = std::max(h->group_smem_fwd, (size_t)gpb * cpg * (np + 2) * 2);
-                h->group_smem_bwd = std::max(h->group_smem_bwd, (size_t)2 * gpb * cpg * (np + 4) * 4);      // dn and zhat
+                h->group_smem_fwd = std::max(h->group_smem_fwd, (size_t)rgpb * cpg * (np + 2) * 2);
+                h->group_smem_bwd = std::max(h->group_smem_bwd, (size_t)2 * rgpb * cpg * (np + 4) * 4);      // dn and zhat
             }
             if (!resident) {
             const bool pooled = x.has_pool || x.avgpool;
