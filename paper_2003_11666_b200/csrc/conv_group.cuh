@@ -34,6 +34,9 @@ constexpr int kGroupWarps = kGroupThreads / 32;
 constexpr int kGroupMaxElems = 25088;          // elements of a bundle that stay in shared memory (98 KB as float32)
 constexpr int kGroupMaxChannels = 256;        // channels of a bundle
 constexpr int kGroupTargetElems = 12544;       // small groups are bundled up to about this many elements (one block then has a few thousand)
+constexpr int kGroupSliceElems = 6272;         // a bundle whose forward GEMM left K slices also keeps their float32 sum in shared memory: at most this many elements
+constexpr int kGroupSliceTarget = 3136;        // ... and such groups are bundled only up to this many
+constexpr int kGroupMaxRows = kMaxDeltaSrc * 16;   // partial rows of all consumers of one stage (a consumer's dgrad has at most 16 K slices)
 constexpr int kGroupSplit = 4;                 // blocks (one cluster) that share a bundle's pixels
 
 // One block's bundle: groups [grp0, grp0 + ngrp) of one stage.
@@ -45,6 +48,9 @@ struct GroupShared {
     float s1[kGroupMaxChannels], s2[kGroupMaxChannels];       // per channel sums of dn and dn * zhat
     float m1[kGroupMaxChannels], m2[kGroupMaxChannels];       // per channel copy of its group's means
     float t1[kGroupMaxChannels], t2[kGroupMaxChannels];       // the sums over the whole cluster
+    const float* rows[kGroupMaxRows];                         // backward: the consumers' partial rows for this sample, in summation order
+    int nrows;
+    float part[kGroupWarps][3];                               // forward: a warp's share of a group's statistics
 };
 
 // Pixel units [lo, hi) of block `rank` of a bundle's cluster (npu units of VEC pixels per channel).
@@ -65,23 +71,30 @@ __device__ void group_forward(const ConvStage& st, const GroupBlock gb, int rank
     int u_lo, u_hi;
     group_range(npu, rank, u_lo, u_hi);
     const int p_lo = u_lo * VEC, np = (u_hi - u_lo) * VEC;               // this block's pixels
-    // ---- group statistics, a warp per group (every block of the bundle computes the same numbers)
-    for (int g = warp; g < gb.ngrp; g += kGroupWarps) {
-        const int grp = gb.grp0 + g;
-        float mean, rstd;
-        if (st.fused) {
-            // from the GEMM epilogue's partials (count, mean, M2 per channel and column tile): a lane folds
-            // the entries k = lane, lane + 32, ... into one triple (independent loads), then the triples
-            // are merged along a fixed tree
-            const int nidx = st.fstat_stride;
-            const float* f = st.fstat + (size_t)grp * nidx * 3;
-            float n = 0.f, m2 = 0.f;
-            mean = 0.f;
-            for (int k = lane; k < nidx; k += 32) {
-                const float nb = f[3 * k], mb = f[3 * k + 1], qb = f[3 * k + 2];
-                const float tot = n + nb, dl = mb - mean;
-                if (tot > 0.f) { mean += dl * (nb / tot); m2 += qb + dl * dl * (n * nb / tot); }
-                n = tot;
+    // ---- group statistics (every block of the bundle computes the same numbers)
+    __nv_bfloat16* t16 = reinterpret_cast<__nv_bfloat16*>(buf);          // [nch][np + 2]
+    const int rs = np + 2;
+    float* zs = buf + ((nch * rs * 2 + 15) / 16) * 4;                    // [nch][hw]: sum of the K slices (only where the GEMM left slices)
+    if (st.fused) {
+        // From the GEMM epilogue's partials (count, mean, M2 per channel and column tile).  A bundle
+        // of few groups gives each group several warps: wpg warps fold the entries k = sub * 32 + lane,
+        // + 32 wpg, ... of a group into one triple per lane (independent loads), merge them along a
+        // fixed shuffle tree, and one thread merges the warps' triples in warp order.
+        int wpg = 1;
+        while (2 * wpg * gb.ngrp <= kGroupWarps) wpg *= 2;
+        const int gpp = kGroupWarps / wpg;                               // groups per pass
+        const int nidx = st.fstat_stride;
+        for (int g0 = 0; g0 < gb.ngrp; g0 += gpp) {
+            const int g = g0 + warp / wpg, sub = warp % wpg;
+            float n = 0.f, mean = 0.f, m2 = 0.f;
+            if (g < gb.ngrp) {
+                const float* f = st.fstat + (size_t)(gb.grp0 + g) * nidx * 3;
+                for (int k = sub * 32 + lane; k < nidx; k += 32 * wpg) {
+                    const float nb = f[3 * k], mb = f[3 * k + 1], qb = f[3 * k + 2];
+                    const float tot = n + nb, dl = mb - mean;
+                    if (tot > 0.f) { mean += dl * (nb / tot); m2 += qb + dl * dl * (n * nb / tot); }
+                    n = tot;
+                }
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
@@ -94,45 +107,67 @@ __device__ void group_forward(const ConvStage& st, const GroupBlock gb, int rank
                 if (tot > 0.f) { mean = ma + dl * (nc / tot); m2 = qa + qc + dl * dl * (na * nc / tot); } else { mean = 0.f; m2 = 0.f; }
                 n = tot;
             }
-            rstd = rsqrtf(m2 / n + kGnEps);
-        } else {
-            // the forward GEMM left K slices: the conv output is their sum in slice order (this block
-            // files its own pixels in the ring for the backward); mean, then squared deviations
-            const size_t gbase = (size_t)grp * cpg * hw;
-            const int ne = cpg * hw;
-            const float inv_hw = 1.f / (float)hw;
-            float* __restrict__ zr = st.z_ring + (size_t)slot * zelems;
-            float s1 = 0.f;
-            for (int e = lane; e < ne; e += 32) {
-                float v = 0.f;
-                for (int q = 0; q < st.z_nsplit; ++q) v += st.zpart[(size_t)q * zelems + gbase + e];
-                s1 += v;
-                const int p = e - quot(e, inv_hw) * hw;
-                if (p >= p_lo && p < p_lo + np) zr[gbase + e] = v;
+            if (lane == 0) { sh.part[warp][0] = n; sh.part[warp][1] = mean; sh.part[warp][2] = m2; }
+            __syncthreads();
+            if (tid < gpp && g0 + tid < gb.ngrp) {
+                float na = sh.part[tid * wpg][0], ma = sh.part[tid * wpg][1], qa = sh.part[tid * wpg][2];
+                for (int w = 1; w < wpg; ++w) {
+                    const float nc = sh.part[tid * wpg + w][0], mc = sh.part[tid * wpg + w][1], qc = sh.part[tid * wpg + w][2];
+                    const float tot = na + nc, dl = mc - ma;
+                    if (tot > 0.f) { ma += dl * (nc / tot); qa += qc + dl * dl * (na * nc / tot); }
+                    na = tot;
+                }
+                const float rstd = rsqrtf(qa / na + kGnEps);
+                const int gg = g0 + tid, grp = gb.grp0 + gg;
+                sh.m1[gg] = ma; sh.m2[gg] = rstd;
+                if (rank == 0) {
+                    st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0] = ma;
+                    st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 1] = rstd;
+                }
             }
+            __syncthreads();
+        }
+    } else {
+        // The forward GEMM left K slices: the conv output is their sum in slice order, kept in shared
+        // memory for the whole bundle (this block files its own pixels in the ring for the backward);
+        // then mean and squared deviations of every group, a warp per group.
+        const int ne = nch * hw;
+        const float inv_hw = 1.f / (float)hw;
+        const float* __restrict__ zp = st.zpart + (size_t)c0 * hw;
+        float* __restrict__ zr = st.z_ring + (size_t)slot * zelems + (size_t)c0 * hw;
+#pragma unroll 4
+        for (int e = tid; e < ne; e += kGroupThreads) {
+            float v = 0.f;
+            for (int q = 0; q < st.z_nsplit; ++q) v += zp[(size_t)q * zelems + e];
+            zs[e] = v;
+            const int p = e - quot(e, inv_hw) * hw;
+            if (p >= p_lo && p < p_lo + np) zr[e] = v;
+        }
+        __syncthreads();
+        const int gne = cpg * hw;
+        for (int g = warp; g < gb.ngrp; g += kGroupWarps) {
+            const float* zg = zs + g * gne;
+            float s1 = 0.f;
+            for (int e = lane; e < gne; e += 32) s1 += zg[e];
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) s1 += __shfl_xor_sync(0xffffffffu, s1, o);
-            mean = s1 / (float)ne;
+            const float mean = s1 / (float)gne;
             float s2 = 0.f;
-            for (int e = lane; e < ne; e += 32) {
-                float v = 0.f;
-                for (int q = 0; q < st.z_nsplit; ++q) v += st.zpart[(size_t)q * zelems + gbase + e];
-                const float d = v - mean;
-                s2 = fmaf(d, d, s2);
-            }
+            for (int e = lane; e < gne; e += 32) { const float d = zg[e] - mean; s2 = fmaf(d, d, s2); }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) s2 += __shfl_xor_sync(0xffffffffu, s2, o);
-            rstd = rsqrtf(s2 / (float)ne + kGnEps);
-        }
-        if (lane == 0) {
-            sh.m1[g] = mean; sh.m2[g] = rstd;
-            if (rank == 0) {
-                st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0] = mean;
-                st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 1] = rstd;
+            if (lane == 0) {
+                const float rstd = rsqrtf(s2 / (float)gne + kGnEps);
+                const int grp = gb.grp0 + g;
+                sh.m1[g] = mean; sh.m2[g] = rstd;
+                if (rank == 0) {
+                    st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 0] = mean;
+                    st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 1] = rstd;
+                }
             }
         }
+        __syncthreads();
     }
-    __syncthreads();          // (also orders this block's ring writes before its reads below)
     for (int cl = tid; cl < nch; cl += kGroupThreads) {
         const int g = cl / cpg, c = c0 + cl;
         sh.gs[cl] = st.wh[st.nw + c] * sh.m2[g];
@@ -145,8 +180,6 @@ __device__ void group_forward(const ConvStage& st, const GroupBlock gb, int rank
         ? st.skip_ring + (size_t)slot_of(i, st.skip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
     unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems;
     float* __restrict__ out = st.out_ring + (size_t)slot * zelems;
-    __nv_bfloat16* t16 = reinterpret_cast<__nv_bfloat16*>(buf);          // [nch][np + 2]
-    const int rs = np + 2;
     // ---- normalise, skip, ReLU: the bundle's (channel, pixel unit) pairs spread flat over the
     // block, four units of a thread in flight at a time (a channel's share of the pixels can be
     // a dozen pixels: per-channel loops would wait one memory latency per channel)
@@ -160,7 +193,12 @@ __device__ void group_forward(const ConvStage& st, const GroupBlock gb, int rank
         const size_t base = (size_t)c * hw;
         float zv[VEC], sv[VEC], a[VEC];
         unsigned char cd[VEC];
-        vload<VEC>(zv, z + base + p);
+        if (st.fused) {
+            vload<VEC>(zv, z + base + p);
+        } else {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) zv[e] = zs[cl * hw + p + e];
+        }
         if (!sk) {
 #pragma unroll
             for (int e = 0; e < VEC; ++e) sv[e] = 0.f;
@@ -245,16 +283,17 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
         sh.rstd[cl] = st.stat_ring[((size_t)slot * st.groups + grp) * 2 + 1];
         sh.gs[cl] = gam[c0 + cl];
     }
-    __syncthreads();
-    // where each consumer's partial rows for this sample start (the same for the whole block)
-    const float* dptr[kMaxDeltaSrc];
-    int dnp[kMaxDeltaSrc];
-#pragma unroll
-    for (int q = 0; q < kMaxDeltaSrc; ++q) {
-        const bool on = q < st.n_dsrc;
-        dnp[q] = on ? st.dsrc[q].nparts : 0;
-        dptr[q] = on ? st.dsrc[q].ptr + (size_t)slot_of(j, st.dsrc[q].slots) * st.dsrc[q].nparts * zelems : nullptr;
+    // the consumers' partial rows for this sample, flat and in summation order (consumer, then K slice)
+    if (tid == 0) {
+        int nr = 0;
+        for (int q = 0; q < st.n_dsrc; ++q) {
+            const float* p0 = st.dsrc[q].ptr + (size_t)slot_of(j, st.dsrc[q].slots) * st.dsrc[q].nparts * zelems;
+            for (int kp = 0; kp < st.dsrc[q].nparts && nr < kGroupMaxRows; ++kp) sh.rows[nr++] = p0 + (size_t)kp * zelems;
+        }
+        sh.nrows = nr;
     }
+    __syncthreads();
+    const int nrows = sh.nrows;
     // ---- gradient at the normalised activation, and the normalised conv output, into shared
     // memory: the bundle's (channel, pixel unit) pairs spread flat over the block, several units
     // of a thread in flight at a time
@@ -272,15 +311,15 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
         for (int e = 0; e < VEC; ++e) d[e] = 0.f;
         vload<VEC>(zv, z + base + p);
         ldb<VEC>(cd, code + base + p);
+        // four rows in flight at a time (a row beyond the list re-reads row 0 and counts as zero)
+        for (int r0 = 0; r0 < nrows; r0 += 4) {
+            float r[4][VEC];
 #pragma unroll
-        for (int q = 0; q < kMaxDeltaSrc; ++q) {
-            const float* bp = dptr[q] + base + p;
-            for (int kp = 0; kp < dnp[q]; ++kp, bp += zelems) {
-                float r[VEC];
-                vload<VEC>(r, bp);
+            for (int k = 0; k < 4; ++k) vload<VEC>(r[k], sh.rows[r0 + k < nrows ? r0 + k : 0] + base + p);
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) d[e] += r[e];
-            }
+            for (int k = 0; k < 4; ++k)
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) d[e] += (r0 + k < nrows) ? r[k][e] : 0.f;
         }
 #pragma unroll
         for (int e = 0; e < VEC; ++e) {
@@ -289,17 +328,27 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
         }
     }
     __syncthreads();
-    // ---- per-channel sums of dn and dn * zhat over this block's pixels: a warp per channel, from shared memory
-    for (int cl = warp; cl < nch; cl += kGroupWarps) {
-        float a1 = 0.f, a2 = 0.f;
-        for (int p = lane; p < np; p += 32) {
-            const float d = dn[cl * rs + p];
-            a1 += d;
-            a2 = fmaf(d, zh[cl * rs + p], a2);
+    // ---- per-channel sums of dn and dn * zhat over this block's pixels, from shared memory: `width`
+    // lanes per channel (the power of two that covers the pixels, at least 4), 32 / width channels per warp
+    {
+        int width = 32;
+        while (width > 4 && (width >> 1) >= np) width >>= 1;
+        const int cpw = 32 / width, sub = lane / width, l = lane - sub * width;
+        for (int cl0 = warp * cpw; cl0 < nch; cl0 += kGroupWarps * cpw) {
+            const int cl = cl0 + sub;
+            float a1 = 0.f, a2 = 0.f;
+            if (cl < nch)
+                for (int p = l; p < np; p += width) {
+                    const float d = dn[cl * rs + p];
+                    a1 += d;
+                    a2 = fmaf(d, zh[cl * rs + p], a2);
+                }
+            for (int o = width >> 1; o > 0; o >>= 1) {
+                a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+                a2 += __shfl_xor_sync(0xffffffffu, a2, o);
+            }
+            if (l == 0 && cl < nch) { sh.s1[cl] = a1; sh.s2[cl] = a2; }   // this block's pixels only
         }
-        a1 = warp_sum(a1);
-        a2 = warp_sum(a2);
-        if (lane == 0) { sh.s1[cl] = a1; sh.s2[cl] = a2; }   // this block's pixels only
     }
     // ---- the cluster's blocks add their sums up in rank order (distributed shared memory)
     cluster.sync();

@@ -638,14 +638,17 @@ bool fill_conv_tables(pb_handle* h) {
             const bool units_ok = x.tc && L.c_out % 8 == 0 && (cpg < 8 ? 8 % cpg == 0 : cpg % 8 == 0);
             // small groups are bundled further (a block pays its chain of memory latencies whatever its size)
             int rgpb = gpb;
-            while (x.gn_groups % (2 * rgpb) == 0 && 2 * rgpb * cpg <= kGroupMaxChannels && 2LL * rgpb * cpg * hw <= kGroupTargetElems) rgpb *= 2;
+            const long long target = x.fuse_stats ? kGroupTargetElems : kGroupSliceTarget;
+            while (x.gn_groups % (2 * rgpb) == 0 && 2 * rgpb * cpg <= kGroupMaxChannels && 2LL * rgpb * cpg * hw <= target) rgpb *= 2;
+            // (a stage whose forward GEMM left K slices keeps the float32 sum of a bundle in shared memory)
             const bool resident = x.tc && !h->post_fuse && units_ok && !x.has_pool && !x.avgpool && x.gn_groups % rgpb == 0 &&
-                                  rgpb * cpg <= kGroupMaxChannels && (long long)rgpb * cpg * hw <= kGroupMaxElems;
+                                  rgpb * cpg <= kGroupMaxChannels && (long long)rgpb * cpg * hw <= (x.fuse_stats ? kGroupMaxElems : kGroupSliceElems);
             if (resident) {
                 for (int g0 = 0; g0 < x.gn_groups; g0 += rgpb) h->h_gblocks.push_back(GroupBlock{stage_idx, g0, rgpb});
                 // each of the kGroupSplit blocks of a bundle holds a quarter of the pixels (rounded up to whole units of 4)
                 const size_t np = (size_t)(ceil_div(ceil_div(hw, 4), kGroupSplit) + 1) * 4;
-                h->group_smem_fwd = std::max(h->group_smem_fwd, (size_t)rgpb * cpg * (np + 2) * 2);
+                const size_t t16_bytes = align_up((size_t)rgpb * cpg * (np + 2) * 2, 16);
+                h->group_smem_fwd = std::max(h->group_smem_fwd, t16_bytes + (x.fuse_stats ? 0 : (size_t)rgpb * cpg * hw * 4));
                 h->group_smem_bwd = std::max(h->group_smem_bwd, (size_t)2 * rgpb * cpg * (np + 4) * 4);      // dn and zhat
             }
             if (!resident) {
