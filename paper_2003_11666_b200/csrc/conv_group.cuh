@@ -135,13 +135,23 @@ __device__ void group_forward(const ConvStage& st, const GroupBlock gb, int rank
         const float inv_hw = 1.f / (float)hw;
         const float* __restrict__ zp = st.zpart + (size_t)c0 * hw;
         float* __restrict__ zr = st.z_ring + (size_t)slot * zelems + (size_t)c0 * hw;
-#pragma unroll 4
-        for (int e = tid; e < ne; e += kGroupThreads) {
-            float v = 0.f;
-            for (int q = 0; q < st.z_nsplit; ++q) v += zp[(size_t)q * zelems + e];
-            zs[e] = v;
-            const int p = e - quot(e, inv_hw) * hw;
-            if (p >= p_lo && p < p_lo + np) zr[e] = v;
+        for (int e0 = tid; e0 < ne; e0 += 4 * kGroupThreads) {
+            float v[4] = {0.f, 0.f, 0.f, 0.f};                  // four elements of a thread in flight (loads before any store)
+            for (int q = 0; q < st.z_nsplit; ++q)
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int e = e0 + k * kGroupThreads;
+                    if (e < ne) v[k] += zp[(size_t)q * zelems + e];
+                }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int e = e0 + k * kGroupThreads;
+                if (e < ne) {
+                    zs[e] = v[k];
+                    const int p = e - quot(e, inv_hw) * hw;
+                    if (p >= p_lo && p < p_lo + np) zr[e] = v[k];
+                }
+            }
         }
         __syncthreads();
         const int gne = cpg * hw;
@@ -185,7 +195,7 @@ __device__ void group_forward(const ConvStage& st, const GroupBlock gb, int rank
     // a dozen pixels: per-channel loops would wait one memory latency per channel)
     const int upc = u_hi - u_lo, total = nch * upc;
     const float inv_upc = 1.f / (float)max(upc, 1);
-#pragma unroll 4
+#pragma unroll(VEC == 4 ? 4 : 8)
     for (int idx = tid; idx < total; idx += kGroupThreads) {
         const int cl = quot(idx, inv_upc), u = u_lo + idx - cl * upc;
         const int c = c0 + cl, p = u * VEC;
@@ -275,7 +285,7 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
     int u_lo, u_hi;
     group_range(npu, rank, u_lo, u_hi);
     const int p_lo = u_lo * VEC, np = (u_hi - u_lo) * VEC;   // this block's pixels
-    const int rs = np + 4;                                   // row pitch of dn and zhat in shared memory
+    const int rs = np <= 16 ? ((np + 4) | 1) : np + 4;       // row pitch of dn and zhat in shared memory (odd where a thread walks a row)
     float* zh = dn + (size_t)nch * rs;                       // normalised conv output, kept beside dn
     for (int cl = tid; cl < nch; cl += kGroupThreads) {
         const int grp = (c0 + cl) / cpg;
@@ -299,7 +309,7 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
     // of a thread in flight at a time
     const int upc = u_hi - u_lo, total = nch * upc;
     const float inv_upc = 1.f / (float)max(upc, 1);
-#pragma unroll 2
+#pragma unroll(VEC == 4 ? 2 : 8)
     for (int idx = tid; idx < total; idx += kGroupThreads) {
         const int cl = quot(idx, inv_upc), u = u_lo + idx - cl * upc;
         const int p = u * VEC;
@@ -328,26 +338,30 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
         }
     }
     __syncthreads();
-    // ---- per-channel sums of dn and dn * zhat over this block's pixels, from shared memory: `width`
-    // lanes per channel (the power of two that covers the pixels, at least 4), 32 / width channels per warp
-    {
-        int width = 32;
-        while (width > 4 && (width >> 1) >= np) width >>= 1;
-        const int cpw = 32 / width, sub = lane / width, l = lane - sub * width;
-        for (int cl0 = warp * cpw; cl0 < nch; cl0 += kGroupWarps * cpw) {
-            const int cl = cl0 + sub;
+    // ---- per-channel sums of dn and dn * zhat over this block's pixels, from shared memory: a thread
+    // per channel where a block has at most 16 pixels of each (odd pitch: no bank conflicts), else a
+    // warp per channel
+    if (np <= 16) {
+        for (int cl = tid; cl < nch; cl += kGroupThreads) {
             float a1 = 0.f, a2 = 0.f;
-            if (cl < nch)
-                for (int p = l; p < np; p += width) {
-                    const float d = dn[cl * rs + p];
-                    a1 += d;
-                    a2 = fmaf(d, zh[cl * rs + p], a2);
-                }
-            for (int o = width >> 1; o > 0; o >>= 1) {
-                a1 += __shfl_xor_sync(0xffffffffu, a1, o);
-                a2 += __shfl_xor_sync(0xffffffffu, a2, o);
+            for (int p = 0; p < np; ++p) {
+                const float d = dn[cl * rs + p];
+                a1 += d;
+                a2 = fmaf(d, zh[cl * rs + p], a2);
             }
-            if (l == 0 && cl < nch) { sh.s1[cl] = a1; sh.s2[cl] = a2; }   // this block's pixels only
+            sh.s1[cl] = a1; sh.s2[cl] = a2;                  // this block's pixels only
+        }
+    } else {
+        for (int cl = warp; cl < nch; cl += kGroupWarps) {
+            float a1 = 0.f, a2 = 0.f;
+            for (int p = lane; p < np; p += 32) {
+                const float d = dn[cl * rs + p];
+                a1 += d;
+                a2 = fmaf(d, zh[cl * rs + p], a2);
+            }
+            a1 = warp_sum(a1);
+            a2 = warp_sum(a2);
+            if (lane == 0) { sh.s1[cl] = a1; sh.s2[cl] = a2; }
         }
     }
     // ---- the cluster's blocks add their sums up in rank order (distributed shared memory)
@@ -379,7 +393,7 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
     // ---- gradient at the conv output (kept in place of dn), gradient of the skip input
     float* __restrict__ dsk = st.dskip
         ? st.dskip + (size_t)slot_of(j, st.dskip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
-#pragma unroll 2
+#pragma unroll(VEC == 4 ? 2 : 8)
     for (int idx = tid; idx < total; idx += kGroupThreads) {
         const int cl = quot(idx, inv_upc), u = u_lo + idx - cl * upc;
         const int c = c0 + cl, p = u * VEC;

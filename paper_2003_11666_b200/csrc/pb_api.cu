@@ -649,7 +649,7 @@ bool fill_conv_tables(pb_handle* h) {
                 const size_t np = (size_t)(ceil_div(ceil_div(hw, 4), kGroupSplit) + 1) * 4;
                 const size_t t16_bytes = align_up((size_t)rgpb * cpg * (np + 2) * 2, 16);
                 h->group_smem_fwd = std::max(h->group_smem_fwd, t16_bytes + (x.fuse_stats ? 0 : (size_t)rgpb * cpg * hw * 4));
-                h->group_smem_bwd = std::max(h->group_smem_bwd, (size_t)2 * rgpb * cpg * (np + 4) * 4);      // dn and zhat
+                h->group_smem_bwd = std::max(h->group_smem_bwd, (size_t)2 * rgpb * cpg * (np + 5) * 4);      // dn and zhat (pitch np + 4, made odd for short rows)
             }
             if (!resident) {
             const bool pooled = x.has_pool || x.avgpool;
