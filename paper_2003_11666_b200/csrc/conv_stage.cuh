@@ -735,10 +735,17 @@ update_kernel(const UpdRange* __restrict__ ranges, const UpdChunk* __restrict__ 
     if (vec) {
         // four parameters per thread and step (kUpdChunk and ch.start are multiples of 4)
         for (int e = ch.start + 4 * threadIdx.x; e < end; e += 4 * 256) {
-            float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int q = 0; q < R.nparts; ++q) {
-                const float4 p = *reinterpret_cast<const float4*>(R.g + (size_t)q * R.part_stride + e);
-                g.x += p.x; g.y += p.y; g.z += p.z; g.w += p.w;
+            // the K slices of the gradient, summed in slice order, four loads in flight at a time
+            // (a slice beyond the last re-reads slice 0 and counts as zero)
+            float4 g = *reinterpret_cast<const float4*>(R.g + e);
+            for (int q0 = 1; q0 < R.nparts; q0 += 4) {
+                float4 p[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    p[k] = *reinterpret_cast<const float4*>(R.g + (size_t)(q0 + k < R.nparts ? q0 + k : 0) * R.part_stride + e);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (q0 + k < R.nparts) { g.x += p[k].x; g.y += p[k].y; g.z += p[k].z; g.w += p[k].w; }
             }
             g.x *= gsc; g.y *= gsc; g.z *= gsc; g.w *= gsc;
             const float4 w = *reinterpret_cast<const float4*>(R.w + e), v = *reinterpret_cast<const float4*>(R.v + e);
