@@ -330,6 +330,13 @@ __device__ void tc_producer(const ConvGemmTC* __restrict__ gemms, const GemmTile
 __device__ void tc_tma(const ConvGemmTC* __restrict__ gemms, const GemmTile* __restrict__ tiles, int q0, int q1,
                        const CUtensorMap* __restrict__ tmaps, const TickState* ts, long long t, int S,
                        unsigned char* smem, TcShared& sh) {
+    // the descriptors of all this block's tiles on their way into the descriptor cache (a tile
+    // switch would otherwise wait for them, one memory latency each)
+    for (int q = q0; q < q1; ++q) {
+        const ConvGemmTC& G = gemms[tiles[q].gemm];
+        if (G.a_tmap >= 0) asm volatile("prefetch.tensormap [%0];" ::"l"(tmaps + G.a_tmap) : "memory");
+        if (G.b_tmap >= 0) asm volatile("prefetch.tensormap [%0];" ::"l"(tmaps + G.b_tmap) : "memory");
+    }
     int it = 0;
     for (int q = q0; q < q1; ++q) {
         const GemmTile tl = tiles[q];

@@ -765,6 +765,11 @@ bool fill_conv_tables(pb_handle* h) {
             add(h->d_wh + x.dev_off + nw, x.gstash, 4, L.c_out, x.gstash_stride);
         }
     }
+    // Data-gradient and weight-gradient GEMMs both start from dz and write different buffers: one
+    // launch takes the tiles of both (one start-up and one tail instead of two, and the long K loops
+    // of the data gradients balance against the many short tiles of the weight gradients).
+    h->h_tctiles[1].insert(h->h_tctiles[1].end(), h->h_tctiles[2].begin(), h->h_tctiles[2].end());
+    h->h_tctiles[2].clear();
     for (int q = 0; q < 3; ++q) balance_tc_tiles(h, h->h_tc, h->h_tctiles[q], h->h_tcbegin[q]);
     // the first forward normalisation step skips the stages whose GEMM epilogue has done it
     {
