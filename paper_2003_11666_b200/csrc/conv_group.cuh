@@ -195,39 +195,54 @@ __device__ void group_forward(const ConvStage& st, const GroupBlock gb, int rank
     // a dozen pixels: per-channel loops would wait one memory latency per channel)
     const int upc = u_hi - u_lo, total = nch * upc;
     const float inv_upc = 1.f / (float)max(upc, 1);
-#pragma unroll(VEC == 4 ? 4 : 8)
-    for (int idx = tid; idx < total; idx += kGroupThreads) {
-        const int cl = quot(idx, inv_upc), u = u_lo + idx - cl * upc;
-        const int c = c0 + cl, p = u * VEC;
-        const float gs = sh.gs[cl], bb = sh.bb[cl], mean = sh.mean[cl];
-        const size_t base = (size_t)c * hw;
-        float zv[VEC], sv[VEC], a[VEC];
-        unsigned char cd[VEC];
-        if (st.fused) {
-            vload<VEC>(zv, z + base + p);
-        } else {
+    // (explicit batches of U units: all loads of a batch are issued before any is used, whatever the
+    //  branches on the kind of skip input do to the compiler's own unrolling)
+    constexpr int U = VEC == 4 ? 4 : 8;
+    const bool fused = st.fused != 0, relu = st.relu != 0, out32 = st.need_out32 != 0;
+    const int skip_kind = !sk ? 0 : (st.skip_mode == 0 ? 1 : 2);
+    for (int i0 = tid; i0 < total; i0 += U * kGroupThreads) {
+        int cl[U], p[U];
+        float zv[U][VEC], sv[U][VEC];
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) zv[e] = zs[cl * hw + p + e];
+        for (int k = 0; k < U; ++k) {
+            const int idx = min(i0 + k * kGroupThreads, total - 1);      // (a unit beyond the end repeats the last one and is not stored)
+            cl[k] = quot(idx, inv_upc);
+            p[k] = (u_lo + idx - cl[k] * upc) * VEC;
+            const size_t base = (size_t)(c0 + cl[k]) * hw;
+            if (fused) {
+                vload<VEC>(zv[k], z + base + p[k]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) zv[k][e] = zs[cl[k] * hw + p[k] + e];
+            }
+            if (skip_kind == 1) {
+                vload<VEC>(sv[k], sk + base + p[k]);
+            } else if (skip_kind == 2) {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) sv[k][e] = skip_value(st, sk, c0 + cl[k], (p[k] + e) / st.ow, (p[k] + e) % st.ow);
+            } else {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) sv[k][e] = 0.f;
+            }
         }
-        if (!sk) {
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) sv[e] = 0.f;
-        } else if (st.skip_mode == 0) {
-            vload<VEC>(sv, sk + base + p);
-        } else {
+        for (int k = 0; k < U; ++k) {
+            if (i0 + k * kGroupThreads >= total) break;
+            const float gs = sh.gs[cl[k]], bb = sh.bb[cl[k]], mean = sh.mean[cl[k]];
+            const size_t base = (size_t)(c0 + cl[k]) * hw;
+            float a[VEC];
+            unsigned char cd[VEC];
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) sv[e] = skip_value(st, sk, c, (p + e) / st.ow, (p + e) % st.ow);
+            for (int e = 0; e < VEC; ++e) {
+                const float v = fmaf(gs, zv[k][e] - mean, bb) + sv[k][e];
+                const bool pass = relu ? v > 0.f : true;
+                cd[e] = pass ? 1 : 0;
+                a[e] = pass ? v : 0.f;
+                t16[cl[k] * rs + p[k] - p_lo + e] = __float2bfloat16_rn(a[e]);
+            }
+            stb<VEC>(code + base + p[k], cd);
+            if (out32) vstore<VEC>(out + base + p[k], a);
         }
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) {
-            const float v = fmaf(gs, zv[e] - mean, bb) + sv[e];
-            const bool pass = st.relu ? v > 0.f : true;
-            cd[e] = pass ? 1 : 0;
-            a[e] = pass ? v : 0.f;
-            t16[cl * rs + p - p_lo + e] = __float2bfloat16_rn(a[e]);
-        }
-        stb<VEC>(code + base + p, cd);
-        if (st.need_out32) vstore<VEC>(out + base + p, a);
     }
     __syncthreads();
     // ---- bfloat16 [pixel][channel] copy: 16-byte runs of 8 channels (bundles span multiples of 8 channels)
@@ -309,32 +324,50 @@ __device__ void group_backward(const ConvStage& st, const GroupBlock gb, long lo
     // of a thread in flight at a time
     const int upc = u_hi - u_lo, total = nch * upc;
     const float inv_upc = 1.f / (float)max(upc, 1);
-#pragma unroll(VEC == 4 ? 2 : 8)
-    for (int idx = tid; idx < total; idx += kGroupThreads) {
-        const int cl = quot(idx, inv_upc), u = u_lo + idx - cl * upc;
-        const int p = u * VEC;
-        const size_t base = (size_t)(c0 + cl) * hw;
-        const float mean = sh.mean[cl], rstd = sh.rstd[cl];
-        float d[VEC], zv[VEC];
-        unsigned char cd[VEC];
+    // (explicit batches of U units x 4 rows: all loads of a batch are issued before any is used)
+    constexpr int U = VEC == 4 ? 2 : 4;
+    for (int i0 = tid; i0 < total; i0 += U * kGroupThreads) {
+        int cl[U], p[U];
+        size_t off[U];
+        float d[U][VEC], zv[U][VEC];
+        unsigned char cd[U][VEC];
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) d[e] = 0.f;
-        vload<VEC>(zv, z + base + p);
-        ldb<VEC>(cd, code + base + p);
-        // four rows in flight at a time (a row beyond the list re-reads row 0 and counts as zero)
+        for (int k = 0; k < U; ++k) {
+            const int idx = min(i0 + k * kGroupThreads, total - 1);      // (a unit beyond the end repeats the last one and is not stored)
+            cl[k] = quot(idx, inv_upc);
+            p[k] = (u_lo + idx - cl[k] * upc) * VEC;
+            off[k] = (size_t)(c0 + cl[k]) * hw + p[k];
+            vload<VEC>(zv[k], z + off[k]);
+            ldb<VEC>(cd[k], code + off[k]);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) d[k][e] = 0.f;
+        }
+        // the consumers' rows in summation order, four rows in flight per unit (a row beyond the list
+        // re-reads row 0 and counts as zero)
         for (int r0 = 0; r0 < nrows; r0 += 4) {
-            float r[4][VEC];
+            float r[U][4][VEC];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) vload<VEC>(r[k], sh.rows[r0 + k < nrows ? r0 + k : 0] + base + p);
+            for (int j = 0; j < 4; ++j) {
+                const float* rp = sh.rows[r0 + j < nrows ? r0 + j : 0];
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
+                for (int k = 0; k < U; ++k) vload<VEC>(r[k][j], rp + off[k]);
+            }
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) d[e] += (r0 + k < nrows) ? r[k][e] : 0.f;
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int k = 0; k < U; ++k)
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) d[k][e] += (r0 + j < nrows) ? r[k][j][e] : 0.f;
         }
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) {
-            dn[cl * rs + p - p_lo + e] = cd[e] ? d[e] : 0.f;
-            zh[cl * rs + p - p_lo + e] = (zv[e] - mean) * rstd;
+        for (int k = 0; k < U; ++k) {
+            if (i0 + k * kGroupThreads >= total) break;
+            const float mean = sh.mean[cl[k]], rstd = sh.rstd[cl[k]];
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+                dn[cl[k] * rs + p[k] - p_lo + e] = cd[k][e] ? d[k][e] : 0.f;
+                zh[cl[k] * rs + p[k] - p_lo + e] = (zv[k][e] - mean) * rstd;
+            }
         }
     }
     __syncthreads();
