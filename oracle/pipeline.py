@@ -48,7 +48,7 @@ class _Stage:
         self.index = index
         self.head = None          # the FC / CONV2D layer record
         self.gn_groups = 0
-        self.skip = None          # (source stage, mode)
+        self.skip = None          # (source stage, mode, joins before the normalisation)
         self.relu = False
         self.maxpool = None       # (k, stride, pad)
         self.avgpool = False
@@ -75,16 +75,23 @@ class _Stage:
     margins = False           # record how close the ReLU / max-pool decisions were
 
     def forward(self, theta_hat, x, skip_in):
+        """Returns (stage output, what the backward needs, convolution output after a
+        pre-normalisation skip addition: the residual sum later stages may add to theirs)."""
         h = self.head
         W, b, gamma, beta = self.split(theta_hat)
         st = {"x": x}
+        res = None
         if h.op == OP_FC:
             n = L.fc_forward(W, b, x.ravel()).reshape(-1, 1, 1)
         else:
             n = L.conv2d_forward(W, x, h.stride, h.pad, self.rnd)
+            if self.skip is not None and self.skip[2]:
+                # pre-activation residual network: the running sum joins here, before the normalisation
+                n = n + L.skip_forward(skip_in, self.skip[1], n.shape)
+            res = n
             if self.gn_groups:
                 n, st["zhat"], st["rstd"] = L.groupnorm_forward(gamma, beta, n, self.gn_groups)
-        if self.skip is not None:
+        if self.skip is not None and not self.skip[2]:
             n = n + L.skip_forward(skip_in, self.skip[1], n.shape)
         st["pre"] = n
         a = L.relu_forward(n) if self.relu else n
@@ -101,10 +108,12 @@ class _Stage:
                 a, st["arg"] = L.maxpool_forward(a, *self.maxpool)
         if self.avgpool:
             a = L.avgpool_forward(a)
-        return a, st
+        return a, st, res
 
-    def backward(self, theta, st, dy, need_dx, skip_shape):
-        """Returns (g flat like theta, dx or None, dskip or None)."""
+    def backward(self, theta, st, dy, need_dx, skip_shape, dres=None):
+        """Returns (g flat like theta, dx or None, dskip or None).  dres: gradient that later
+        stages sent straight to this stage's convolution output (they added it to theirs
+        before their normalisation), or None."""
         h = self.head
         W, b, gamma, beta = self.split(theta)
         pre = st["pre"]
@@ -116,7 +125,7 @@ class _Stage:
         if self.relu:
             d = L.relu_backward(pre, d)
         dskip = None
-        if self.skip is not None:
+        if self.skip is not None and not self.skip[2]:
             dskip = L.skip_backward(d, self.skip[1], skip_shape)
         g = np.zeros_like(theta)
         if h.op == OP_FC:
@@ -131,6 +140,10 @@ class _Stage:
                 d, gg, gbeta = L.groupnorm_backward(gamma, st["zhat"], st["rstd"], d, self.gn_groups)
                 g[nw:nw + h.c_out] = gg
                 g[nw + h.c_out:] = gbeta
+            if dres is not None:
+                d = d + dres
+            if self.skip is not None and self.skip[2]:
+                dskip = L.skip_backward(d, self.skip[1], skip_shape)
             dx, gW = L.conv2d_backward(W, st["x"], d, h.stride, h.pad, self.rnd)
             g[:nw] = gW.ravel()
             if not need_dx:
@@ -171,7 +184,9 @@ def build_stages(layer_list, stage_of_layer, in_shape):
             st.gn_groups = lay.groups
             st.n_params += 2 * st.head.c_out
         elif op == OP_ADD_SKIP:
-            st.skip = (lay.src, lay.skip_mode)
+            st.skip = (lay.src, lay.skip_mode & 1, bool(lay.skip_mode & 2))
+            if st.skip[2] and (st.head.op != OP_CONV2D or stages[lay.src].head.op != OP_CONV2D):
+                raise ValueError("a pre-normalisation skip joins two convolution stages")
         elif op == OP_RELU:
             st.relu = True
         elif op == OP_MAXPOOL:
@@ -222,6 +237,8 @@ class PBOracle:
         self.opt = None
         self.t = 0
         self.out, self.stash, self.dsum, self.labels = {}, {}, {}, {}
+        self.res, self.dres = {}, {}      # residual sums (forward) and the gradients sent straight to them (backward)
+        self.res_sources = {st.skip[0] for st in self.stages if st.skip is not None and st.skip[2]}
         self.weight_stash = bool(weight_stash)
         self.wstash = {}          # (stage, sample) -> weights of that sample's forward pass
         self.record = record
@@ -298,9 +315,13 @@ class PBOracle:
             s, i = st.index, t - st.index
             if not self.live(i):
                 continue
-            skip_in = self.out[(st.skip[0], i)] if st.skip is not None else None
-            y, stash = st.forward(theta_hat[s], self.out[(st.src, i)], skip_in)
+            skip_in = None
+            if st.skip is not None:
+                skip_in = (self.res if st.skip[2] else self.out)[(st.skip[0], i)]
+            y, stash, res = st.forward(theta_hat[s], self.out[(st.src, i)], skip_in)
             self.out[(s, i)], self.stash[(s, i)] = y, stash
+            if s in self.res_sources:
+                self.res[(s, i)] = res
             if self.weight_stash:
                 self.wstash[(s, i)] = theta_hat[s]
             if st.margins:
@@ -323,14 +344,22 @@ class PBOracle:
             if not self.live(j):
                 continue
             dy = self.dsum.pop((s, j))
-            skip_shape = self.stages[st.skip[0]].out_shape if st.skip is not None else None
+            skip_shape = None
+            if st.skip is not None:
+                src_stage = self.stages[st.skip[0]]
+                skip_shape = src_stage.z_shape if st.skip[2] else src_stage.out_shape
             theta_b = self.wstash.pop((s, j)) if self.weight_stash else self.opt[s].w
             g, dx, dskip = st.backward(theta_b, self.stash.pop((s, j)), dy,
-                                       st.src >= 0, skip_shape)
+                                       st.src >= 0, skip_shape, self.dres.pop((s, j), None))
             if dx is not None:
                 self._accumulate((st.src, j), dx)
             if dskip is not None:
-                self._accumulate((st.skip[0], j), dskip)
+                if st.skip[2]:
+                    key = (st.skip[0], j)
+                    self.dres[key] = self.dres[key] + dskip if key in self.dres else dskip
+                else:
+                    self._accumulate((st.skip[0], j), dskip)
+            self.res.pop((s, j), None)
             grads[s] = g
             del self.out[(s, j)]
             if s == 0:

@@ -10,9 +10,9 @@ from .gen import (splitmix64, uniform01, normal, labels, he_normal_weights,
                   make_inputs)
 from .configs import (OP, Layer, Workload, workload, WORKLOAD_NAMES,
                       param_sizes, infer_shapes, work_per_tick, mlp, tiny_cnn, tiny_resnet,
-                      tall_bottleneck, tail_cnn)
+                      tall_bottleneck, tail_cnn, preact_resnet, SKIP_PRENORM)
 
 __all__ = ["splitmix64", "uniform01", "normal", "labels", "he_normal_weights",
            "make_inputs", "OP", "Layer", "Workload", "workload",
            "WORKLOAD_NAMES", "param_sizes", "infer_shapes", "work_per_tick", "mlp", "tiny_cnn",
-           "tiny_resnet", "tall_bottleneck", "tail_cnn"]
+           "tiny_resnet", "tall_bottleneck", "tail_cnn", "preact_resnet", "SKIP_PRENORM"]

@@ -26,6 +26,9 @@ class OP(IntEnum):
 
 SKIP_IDENTITY = 0      # same shape
 SKIP_SUBSAMPLE_PAD = 1  # every second pixel, new channels filled with zeros
+SKIP_PRENORM = 2        # flag, added to one of the above: the skip input joins the convolution output BEFORE the
+                        # normalisation, and it is the source stage's own convolution output after ITS such
+                        # addition (the running sum of a pre-activation residual network)
 
 FLAG_SC = 1
 FLAG_LWP = 2
@@ -100,8 +103,10 @@ class _Builder:
              skip=None, skip_mode=SKIP_IDENTITY, pool=None, avgpool=False):
         s = self.new_stage()
         self.add(Layer(OP.CONV2D, c_in, c_out, k, stride, pad, src=src))
+        if skip is not None and skip_mode & SKIP_PRENORM:
+            self.add(Layer(OP.ADD_SKIP, src=skip, skip_mode=skip_mode))
         self.add(Layer(OP.GROUPNORM, c_out, c_out, groups=groups))
-        if skip is not None:
+        if skip is not None and not skip_mode & SKIP_PRENORM:
             self.add(Layer(OP.ADD_SKIP, src=skip, skip_mode=skip_mode))
         if relu:
             self.add(Layer(OP.RELU))
@@ -225,6 +230,30 @@ def tiny_resnet(seed=12, ticks=40, flags=FLAG_SC | FLAG_LWP, bottleneck=False, r
                          flags=flags, relu=relu)
     return _resnet20(widths=(4, 8), blocks=1, groups=2, hw=8, n_classes=5,
                      name="tiny_resnet", lr=0.02, ticks=ticks, seed=seed)
+
+
+def preact_resnet(widths=(8, 16), blocks=2, groups=4, hw=16, n_classes=10, name="preact_resnet",
+                  lr=0.01, ticks=48, seed=15, flags=FLAG_SC | FLAG_LWP):
+    """Pre-activation residual network (normalisation and ReLU BEFORE each convolution, the layout the
+    paper trains: Section 4, Experiment Details) in stages of convolution -> (+ running sum) ->
+    normalisation -> ReLU: a stage's normalisation and ReLU are the pre-activation of the next
+    convolution, and the residual sum runs along the convolution outputs.  Basic blocks of two 3x3
+    convolutions; parameter-free shortcut (every second pixel, zero channels) where the width changes."""
+    b = _Builder()
+    prev = b.conv(3, widths[0], 3, 1, 1, groups)                 # stem; its output sum starts the residual stream
+    c_in = widths[0]
+    n_blocks, done = len(widths) * blocks, 0
+    for g, c in enumerate(widths):
+        for q in range(blocks):
+            down = g > 0 and q == 0
+            b.conv(c_in, c, 3, 2 if down else 1, 1, groups)
+            done += 1
+            prev = b.conv(c, c, 3, 1, 1, groups, skip=prev,
+                          skip_mode=(SKIP_SUBSAMPLE_PAD if down else SKIP_IDENTITY) | SKIP_PRENORM,
+                          avgpool=(done == n_blocks))
+            c_in = c
+    b.fc(c_in, n_classes, relu=False, loss=True)
+    return Workload(name, b.layers, b.stage_of, (3, hw, hw), n_classes, lr, 0.9, ticks, seed, flags)
 
 
 def tall_bottleneck(seed=13, ticks=48, lr=0.001, flags=FLAG_SC | FLAG_LWP | FLAG_CONV_BF16, relu=True):

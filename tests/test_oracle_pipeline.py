@@ -11,7 +11,7 @@ import torch
 
 from oracle import PBOracle, sc_coefficients
 from pb_workloads import (he_normal_weights, make_inputs, mlp, tiny_cnn, tiny_resnet,
-                          workload, Layer, OP, Workload)
+                          workload, Layer, OP, Workload, preact_resnet)
 from tests import torch_ref
 
 
@@ -55,7 +55,7 @@ def test_single_stage_is_plain_sgdm():
 
 
 @pytest.mark.parametrize("make", [lambda: mlp([10, 8, 6, 4]), tiny_cnn, tiny_resnet,
-                                  lambda: tiny_resnet(bottleneck=True)])
+                                  lambda: tiny_resnet(bottleneck=True), preact_resnet])
 def test_latency_and_frozen_forward(make):
     # A sample takes 2S-1 steps; its loss appears S-1 ticks after it enters.
     # With lr = 0 the weights never move, so the loss at tick t is an ordinary
@@ -107,7 +107,7 @@ def test_staleness_equals_stage_delay(make):
 @pytest.mark.parametrize("make,flags", [
     (lambda: mlp([9, 7, 6, 5], lr=0.05), 3), (tiny_cnn, 3), (tiny_resnet, 3),
     (lambda: tiny_resnet(bottleneck=True), 3), (tiny_cnn, 0), (tiny_cnn, 1), (tiny_cnn, 2),
-    (tiny_resnet, 7)])
+    (tiny_resnet, 7), (preact_resnet, 3), (preact_resnet, 0)])
 def test_per_sample_replay(make, flags):
     """Recompute every sample's gradient with torch autograd from the logged
     weight versions: forward values from the predicted weights of the forward
@@ -158,7 +158,7 @@ def test_per_sample_replay(make, flags):
 
 @pytest.mark.parametrize("make,flags", [
     (lambda: mlp([9, 7, 6, 5], lr=0.05), 0), (tiny_cnn, 0), (tiny_resnet, 0),
-    (lambda: tiny_resnet(bottleneck=True), 3), (tiny_cnn, 2)])
+    (lambda: tiny_resnet(bottleneck=True), 3), (tiny_cnn, 2), (preact_resnet, 3)])
 def test_weight_stashing_gives_the_true_gradient_at_the_forward_weights(make, flags):
     """Eq. "W_{i+1} = W_i - eta grad L(x_i; F_i)": with stashing every sample's
     gradient is an ORDINARY backward pass (plain torch autograd, nothing mixed)

@@ -60,45 +60,53 @@ def _mix(value_with_fwd, same_with_bwd):
     return same_with_bwd + (value_with_fwd - same_with_bwd).detach()
 
 
+def _shortcut(sk, mode, channels):
+    if mode & 1:
+        sub = sk[:, ::2, ::2]
+        sk = torch.cat([sub, torch.zeros(channels - sub.shape[0], *sub.shape[1:], dtype=sk.dtype)], 0)
+    return sk
+
+
 def stage_forward(st, theta_fwd, x, skip_in, theta_bwd=None):
-    """Output of one stage for input x [C,H,W].  With theta_bwd given, values
-    come from theta_fwd while every derivative is taken as if the linear maps
-    held theta_bwd (the stored activations stay those of the forward)."""
+    """(output, convolution output after a pre-normalisation shortcut) of one stage for input
+    x [C,H,W].  With theta_bwd given, values come from theta_fwd while every derivative is taken
+    as if the linear maps held theta_bwd (the stored activations stay those of the forward)."""
     tb = theta_fwd if theta_bwd is None else theta_bwd
     Wf, bf, gf, betaf = split(st, theta_fwd)
     Wb, bb, gb, betab = split(st, tb)
     h = st.head
+    res = None
     if h.op == OP.FC:
         xf = x.reshape(-1)
         n = _mix(Wf @ xf + bf, Wb @ xf + bb).view(-1, 1, 1)
     else:
         conv = lambda W: F.conv2d(x[None], W, stride=h.stride, padding=h.pad)[0]
         n = _mix(conv(Wf), conv(Wb))
+        if st.skip is not None and st.skip[1] & 2:
+            n = n + _shortcut(skip_in, st.skip[1], n.shape[0])      # pre-activation network: the running sum
+        res = n
         if st.gn:
             zhat = F.group_norm(n[None], st.gn, eps=1e-5)[0]
             n = _mix(gf[:, None, None] * zhat + betaf[:, None, None],
                      gb[:, None, None] * zhat + betab[:, None, None])
-    if st.skip is not None:
-        sk = skip_in
-        if st.skip[1] == 1:
-            sub = sk[:, ::2, ::2]
-            sk = torch.cat([sub, torch.zeros(n.shape[0] - sub.shape[0], *sub.shape[1:],
-                                             dtype=n.dtype)], 0)
-        n = n + sk
+    if st.skip is not None and not st.skip[1] & 2:
+        n = n + _shortcut(skip_in, st.skip[1], n.shape[0])
     a = F.relu(n) if st.relu else n
     if st.pool is not None:
         k, s, p = st.pool
         a = F.max_pool2d(a[None], k, s, p)[0]
     if st.avg:
         a = a.mean(dim=(1, 2), keepdim=True)
-    return a
+    return a, res
 
 
 def network_loss(stages, thetas_fwd, x, label, thetas_bwd=None):
-    outs = {-1: x}
+    outs, sums = {-1: x}, {}
     for st in stages:
         tb = None if thetas_bwd is None else thetas_bwd[st.index]
-        skip_in = outs[st.skip[0]] if st.skip is not None else None
-        outs[st.index] = stage_forward(st, thetas_fwd[st.index], outs[st.src], skip_in, tb)
+        skip_in = None
+        if st.skip is not None:
+            skip_in = (sums if st.skip[1] & 2 else outs)[st.skip[0]]
+        outs[st.index], sums[st.index] = stage_forward(st, thetas_fwd[st.index], outs[st.src], skip_in, tb)
     logits = outs[len(stages) - 1].reshape(1, -1)
     return F.cross_entropy(logits, torch.tensor([int(label)]))
