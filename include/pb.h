@@ -69,7 +69,16 @@ typedef struct {
                           before, or the network input for stage 0);
                           ADD_SKIP: stage whose output is added                  */
     int32_t skip_mode; /* ADD_SKIP: 0 identity, 1 every second pixel + zero
-                          channels appended up to c_out                          */
+                          channels appended up to c_out.  + 2 (pre-activation
+                          residual networks, Section "Experiments" / Experiment
+                          Details): the input joins the convolution output
+                          BEFORE the normalisation, and it is the source
+                          stage's own convolution output after ITS such
+                          addition (the running residual sum) instead of that
+                          stage's output; such an ADD_SKIP is listed before the
+                          stage's GROUPNORM, joins two CONV2D stages and runs on
+                          the float32 convolution path only (with PB_CONV_BF16:
+                          PB_E_UNSUPPORTED)                                      */
 } pb_layer;
 
 /* Mitigation switches (Section "Methods").  PB_SC: a = m^D, b = (1-m^D)/(1-m),

@@ -113,6 +113,27 @@ __device__ void conv_stats_chunk(const ConvStage& st, const PostChunk& ch, long 
             }
         }
     }
+    if (st.skip_ring && st.skip_pre) {
+        // pre-activation network: the source stage's running sum (its own conv output after such an
+        // addition, same sample) joins before the statistics are taken
+        const float* __restrict__ sk = st.skip_ring + (size_t)slot_of(i, st.skip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int unit = u * kPostThreads + tid;
+            if (unit >= cg.nunits) continue;
+            const int flat = cg.base + unit * VEC;              // index in this stage's [channel][pixel] tensor
+            if (st.skip_mode == 0) {
+                float r[VEC];
+                vload<VEC>(r, sk + flat);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) vals[u][e] += r[e];
+            } else {
+                const int c = flat / cg.hw, p = flat - c * cg.hw;
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) vals[u][e] += skip_value(st, sk, c, (p + e) / st.ow, (p + e) % st.ow);
+            }
+        }
+    }
     float sum = 0.f;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -173,7 +194,7 @@ __device__ void conv_apply_fwd_chunk(const ConvStage& st, const PostChunk& ch, l
     const float* __restrict__ gam = st.wh + st.nw;
     const float* __restrict__ bet = gam + st.co;
     const float* stat = st.stat_ring + (size_t)slot * st.groups * 2;     // may have been written by this very block
-    const float* __restrict__ sk = st.skip_ring
+    const float* __restrict__ sk = (st.skip_ring && !st.skip_pre)      // (a pre-normalisation skip is already part of z)
         ? st.skip_ring + (size_t)slot_of(i, st.skip_slots) * ((size_t)st.skip_c * st.skip_h * st.skip_w) : nullptr;
     unsigned char* __restrict__ code = st.code_ring + (size_t)slot * zelems;
     const bool pooled = st.pool_k > 0 || st.avgpool;
@@ -487,10 +508,27 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
         if (!ok[u]) continue;
         const int c = cc[u], p = pp[u];
         const size_t idx = (size_t)c * hw + p;
-        // the skip input joined after the normalisation: it receives dn itself
+        float dd[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            const float zh = (zv[u][e] - mean[u]) * rstd[u];
+            dd[e] = rstd[u] * (fmaf(dnv[u][e], gv[u], -m1[u]) - zh * m2[u]);
+        }
+        // later stages that added this stage's pre-normalisation sum to theirs send their gradient straight here
+        for (int q = 0; q < st.n_rsrc; ++q) {
+            float r[VEC];
+            vload<VEC>(r, st.rsrc[q].ptr + (size_t)slot_of(j, st.rsrc[q].slots) * zelems + idx);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) dd[e] += r[e];
+        }
+        // a skip input that joined after the normalisation receives dn itself, one that joined before it dz
         if (dsk) {
+            const float* src = st.skip_pre ? dd : dnv[u];
             if (st.skip_mode == 0) {
-                vstore<VEC>(dsk + idx, dnv[u]);
+                float tmp[VEC];
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) tmp[e] = src[e];
+                vstore<VEC>(dsk + idx, tmp);
             } else if (c < st.skip_c) {
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) {
@@ -499,16 +537,10 @@ __device__ void conv_bwd_dz_chunk(const ConvStage& st, const PostChunk& ch, long
                         for (int dx = 0; dx < 2; ++dx) {
                             const int ys = 2 * y + dy, xs = 2 * x + dx;
                             if (ys < st.skip_h && xs < st.skip_w)
-                                dsk[((size_t)c * st.skip_h + ys) * st.skip_w + xs] = (dy | dx) ? 0.f : dnv[u][e];
+                                dsk[((size_t)c * st.skip_h + ys) * st.skip_w + xs] = (dy | dx) ? 0.f : src[e];
                         }
                 }
             }
-        }
-        float dd[VEC];
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) {
-            const float zh = (zv[u][e] - mean[u]) * rstd[u];
-            dd[e] = rstd[u] * (fmaf(dnv[u][e], gv[u], -m1[u]) - zh * m2[u]);
         }
         vstore<VEC>(dz + idx, dd);
         if (transposed) {

@@ -70,6 +70,9 @@ struct ConvStage {
     int nw;                      // number of conv weights (offset of gamma)
     // skip input
     const float* skip_ring; int skip_slots, skip_mode, skip_c, skip_h, skip_w;   // skip_ring == nullptr: none
+    int skip_pre;                // the skip input joins the convolution output BEFORE the normalisation and is the source
+                                 // stage's own such sum (skip_ring is then that stage's z_ring): pre-activation networks
+    int n_rsrc; DeltaSrc rsrc[kMaxDeltaSrc];   // later stages that added this stage's sum to theirs: their gradients join dz
     float* dskip; int dskip_slots;       // gradient handed to the skip source [slots][skip elems]
     // backward
     int n_dsrc; DeltaSrc dsrc[kMaxDeltaSrc];

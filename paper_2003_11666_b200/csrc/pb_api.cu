@@ -79,10 +79,15 @@ int parse_layers(pb_handle* h, const pb_layer* layers, int n_layers, const int32
                 break;
             case PB_ADD_SKIP:
                 if (L.src < 0 || L.src >= s) return fail(nullptr, PB_E_ARG, "ADD_SKIP needs an earlier stage");
-                x.has_skip = true; x.skip_src = L.src; x.skip_mode = L.skip_mode;
+                if (L.skip_mode < 0 || L.skip_mode > 3) return fail(nullptr, PB_E_ARG, "unknown skip mode");
+                x.has_skip = true; x.skip_src = L.src; x.skip_mode = L.skip_mode & 1; x.skip_pre = (L.skip_mode & 2) != 0;
+                if (x.skip_pre && (x.head_op != PB_CONV2D || st[L.src].head_op != PB_CONV2D))
+                    return fail(nullptr, PB_E_ARG, "a pre-normalisation skip joins two CONV2D stages");
+                if (x.skip_pre && x.gn_groups > 0)
+                    return fail(nullptr, PB_E_ARG, "a pre-normalisation ADD_SKIP comes before the stage's GROUPNORM in the layer list");
                 {
-                    const Shape& sk = st[L.src].out;
-                    bool ok = L.skip_mode == 0 ? (sk.c == x.z.c && sk.h == x.z.h && sk.w == x.z.w)
+                    const Shape& sk = x.skip_pre ? st[L.src].z : st[L.src].out;
+                    bool ok = x.skip_mode == 0 ? (sk.c == x.z.c && sk.h == x.z.h && sk.w == x.z.w)
                                                : (sk.c <= x.z.c && (sk.h + 1) / 2 == x.z.h && (sk.w + 1) / 2 == x.z.w);
                     if (!ok) return fail(nullptr, PB_E_SHAPE, "ADD_SKIP shapes do not match at stage " + std::to_string(s));
                 }
@@ -149,7 +154,7 @@ void schedule_constants(pb_handle* h) {
         dev_off += align_up(x.n_params, 64);
         if (x.head_op != PB_FC) h->all_fc = false;
         if (x.src >= 0) h->stages[x.src].consumers_main.push_back(x.index);
-        if (x.has_skip) h->stages[x.skip_src].consumers_skip.push_back(x.index);
+        if (x.has_skip) (x.skip_pre ? h->stages[x.skip_src].consumers_res : h->stages[x.skip_src].consumers_skip).push_back(x.index);
     }
     h->dev_params = dev_off;
 }
@@ -350,7 +355,7 @@ void plan_conv(pb_handle* h) {
         // tick kernel of conv_gemv.cuh (forward, both gradients and the update in one pass over w, v)
         x.gemv = x.head.k == 3 && x.head.stride == 1 && x.head.pad == 1 && x.src >= 0 && x.in.h == x.in.w &&
                  (x.in.h == 4 || x.in.h == 2) && x.z.h == x.in.h && x.head.c_in % 32 == 0 &&
-                 !(h->flags & (PB_LWP_WFORM | PB_WEIGHT_STASH));
+                 !(h->flags & (PB_LWP_WFORM | PB_WEIGHT_STASH)) && !x.skip_pre && x.consumers_res.empty();
         if (x.gemv) {
             x.split_f = 1; x.kps_f = ceil_div(x.head.c_in * k2, kBK) * kBK;
             x.split_w = 1; x.kps_w = ceil_div(x.z.h * x.z.w, kBK) * kBK;
@@ -608,13 +613,17 @@ bool fill_conv_tables(pb_handle* h) {
         c.wh = h->d_wh + x.dev_off; c.w = h->d_w + x.dev_off; c.g = h->d_g + x.dev_off; c.nw = nw;
         if (x.has_skip) {
             const StageHost& y = h->stages[x.skip_src];
-            c.skip_ring = y.out_ring; c.skip_slots = y.out_slots; c.skip_mode = x.skip_mode;
-            c.skip_c = y.out.c; c.skip_h = y.out.h; c.skip_w = y.out.w;
+            c.skip_ring = x.skip_pre ? y.z_ring : y.out_ring; c.skip_slots = y.out_slots; c.skip_mode = x.skip_mode;
+            c.skip_pre = x.skip_pre ? 1 : 0;
+            const Shape& ys = x.skip_pre ? y.z : y.out;
+            c.skip_c = ys.c; c.skip_h = ys.h; c.skip_w = ys.w;
             c.dskip = x.dskip; c.dskip_slots = x.dskip_slots;
         }
         c.n_dsrc = 0;
         for (int q : x.consumers_main) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dx, y.dx_slots, y.dx_nparts}; }
         for (int q : x.consumers_skip) { const StageHost& y = h->stages[q]; c.dsrc[c.n_dsrc++] = DeltaSrc{y.dskip, y.dskip_slots, 1}; }
+        c.n_rsrc = 0;
+        for (int q : x.consumers_res) { const StageHost& y = h->stages[q]; c.rsrc[c.n_rsrc++] = DeltaSrc{y.dskip, y.dskip_slots, 1}; }
         c.dz = x.dz;
         c.gstash = x.gstash; c.gstash_slots = x.stash_slots;
         c.fstat = x.fstat; c.fstat_stride = x.fstat_stride; c.fused = x.fuse_stats ? 1 : 0; c.bsum = x.bsum; c.npieces = x.npieces; c.gsum = x.gsum;
@@ -788,6 +797,9 @@ int validate_conv(pb_handle* h) {
         if (x.has_pool && x.avgpool) return fail(nullptr, PB_E_UNSUPPORTED, "max-pool and average pool in one stage");
         if (x.avgpool && x.z.h * x.z.w > kPostChunk) return fail(nullptr, PB_E_UNSUPPORTED, "global average pool over more than 2048 pixels");
         if ((int)(x.consumers_main.size() + x.consumers_skip.size()) > kMaxDeltaSrc) return fail(nullptr, PB_E_UNSUPPORTED, "too many consumers of one stage");
+        if ((int)x.consumers_res.size() > kMaxDeltaSrc) return fail(nullptr, PB_E_UNSUPPORTED, "too many stages add one stage's pre-normalisation sum");
+        if ((x.skip_pre || !x.consumers_res.empty()) && (h->flags & PB_CONV_BF16))
+            return fail(nullptr, PB_E_UNSUPPORTED, "pre-normalisation skips run on the float32 convolution path only");
     }
     for (const StageHost& x : h->stages)
         if (x.head_op == PB_FC && (x.has_skip || x.has_pool || x.avgpool || x.gn_groups)) return fail(nullptr, PB_E_UNSUPPORTED, "FC stages take only RELU or SOFTMAX_CE");
@@ -868,7 +880,7 @@ size_t layout(pb_handle* h, char* base, size_t* zero_from) {
         }
         if (x.has_skip) {
             x.dskip_slots = x.index - x.skip_src + 1;
-            x.dskip = c.take<float>((size_t)x.dskip_slots * h->stages[x.skip_src].out.elems());
+            x.dskip = c.take<float>((size_t)x.dskip_slots * (x.skip_pre ? h->stages[x.skip_src].z.elems() : h->stages[x.skip_src].out.elems()));
         }
         if (x.head_op == PB_CONV2D) {
             const size_t ze = x.z.elems(), nw = (size_t)x.head.c_out * x.head.c_in * x.head.k * x.head.k;

@@ -22,6 +22,7 @@ struct StageHost {
     pb_layer head{};
     int gn_groups = 0;
     int skip_src = -1, skip_mode = 0;
+    bool skip_pre = false;                                          // the skip joins before the normalisation (and reads the source's pre-normalisation sum)
     bool has_skip = false, relu = false, avgpool = false, loss = false;
     bool has_pool = false;
     int pool_k = 0, pool_stride = 0, pool_pad = 0;
@@ -37,6 +38,7 @@ struct StageHost {
     float* dx = nullptr; int dx_slots = 0, dx_nparts = 1;          // gradient w.r.t. main input
     float* dskip = nullptr; int dskip_slots = 0;                   // gradient w.r.t. skip input
     std::vector<int> consumers_main, consumers_skip;               // stages reading this output
+    std::vector<int> consumers_res;                                 // stages adding this stage's pre-normalisation sum to theirs
     // convolution stages only
     float *z_ring = nullptr, *stat_ring = nullptr, *zpart = nullptr, *dz = nullptr, *gpart = nullptr;
     unsigned char *code_ring = nullptr, *arg_ring = nullptr;

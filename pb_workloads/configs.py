@@ -233,22 +233,22 @@ def tiny_resnet(seed=12, ticks=40, flags=FLAG_SC | FLAG_LWP, bottleneck=False, r
 
 
 def preact_resnet(widths=(8, 16), blocks=2, groups=4, hw=16, n_classes=10, name="preact_resnet",
-                  lr=0.01, ticks=48, seed=15, flags=FLAG_SC | FLAG_LWP):
+                  lr=0.01, ticks=48, seed=15, flags=FLAG_SC | FLAG_LWP, relu=True):
     """Pre-activation residual network (normalisation and ReLU BEFORE each convolution, the layout the
     paper trains: Section 4, Experiment Details) in stages of convolution -> (+ running sum) ->
     normalisation -> ReLU: a stage's normalisation and ReLU are the pre-activation of the next
     convolution, and the residual sum runs along the convolution outputs.  Basic blocks of two 3x3
     convolutions; parameter-free shortcut (every second pixel, zero channels) where the width changes."""
     b = _Builder()
-    prev = b.conv(3, widths[0], 3, 1, 1, groups)                 # stem; its output sum starts the residual stream
+    prev = b.conv(3, widths[0], 3, 1, 1, groups, relu=relu)      # stem; its output sum starts the residual stream
     c_in = widths[0]
     n_blocks, done = len(widths) * blocks, 0
     for g, c in enumerate(widths):
         for q in range(blocks):
             down = g > 0 and q == 0
-            b.conv(c_in, c, 3, 2 if down else 1, 1, groups)
+            b.conv(c_in, c, 3, 2 if down else 1, 1, groups, relu=relu)
             done += 1
-            prev = b.conv(c, c, 3, 1, 1, groups, skip=prev,
+            prev = b.conv(c, c, 3, 1, 1, groups, relu=relu, skip=prev,
                           skip_mode=(SKIP_SUBSAMPLE_PAD if down else SKIP_IDENTITY) | SKIP_PRENORM,
                           avgpool=(done == n_blocks))
             c_in = c

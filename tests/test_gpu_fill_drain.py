@@ -12,7 +12,7 @@ import math
 import numpy as np
 import pytest
 
-from pb_workloads import make_inputs, mlp, tail_cnn, tiny_cnn, tiny_resnet
+from pb_workloads import make_inputs, mlp, tail_cnn, tiny_cnn, tiny_resnet, preact_resnet
 from tests.parity import make_engine, make_oracle, rel_err
 
 pytestmark = pytest.mark.gpu
@@ -69,7 +69,7 @@ def _run(wl, N, n_cycles, tol, tol_v=None, use_run=False):
                                     (lambda: mlp([48, 40, 33, 24, 5], lr=0.02, seed=42), 1),
                                     (lambda: mlp([2048, 300, 10], lr=0.01, seed=43), 3),
                                     (tiny_cnn, 5), (tiny_resnet, 3), (tail_cnn, 4),
-                                    (lambda: tiny_resnet(bottleneck=True), 4)])
+                                    (lambda: tiny_resnet(bottleneck=True), 4), (preact_resnet, 3)])
 def test_fill_and_drain_matches_minibatch_sgdm(make, N):
     _run(make(), N, 4, TOL)
 

@@ -3,7 +3,7 @@ weight-difference form of LWP (with and without SC), over-compensation
 (SC_2D, LWP_2D) and horizons T = alpha D."""
 import pytest
 
-from pb_workloads import mlp, tiny_cnn, tiny_resnet
+from pb_workloads import mlp, tiny_cnn, tiny_resnet, preact_resnet
 from tests.parity import compare_ticks
 
 pytestmark = pytest.mark.gpu
@@ -90,7 +90,7 @@ def _stashed(wl):
     (lambda: mlp([64, 48, 32, 6], lr=0.003, seed=34, flags=0), TOL),
     (tiny_cnn, TOL), (lambda: tiny_cnn(flags=0), TOL), (lambda: _resnet(3), TOL),
     (lambda: tiny_resnet(bottleneck=True, flags=3), TOL),
-    (lambda: tiny_resnet(bottleneck=True, flags=3 | 8, relu=False), 2e-2)])
+    (lambda: tiny_resnet(bottleneck=True, flags=3 | 8, relu=False), 2e-2), (preact_resnet, TOL)])
 def test_weight_stashing(make, tol):
     # the comparison mode of the paper's appendix (PipeDream's rule): the backward pass of a
     # sample uses the weights of its own forward pass; FC stages, CUDA-core and tensor-core
